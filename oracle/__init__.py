@@ -1,0 +1,8 @@
+"""fp64 CPU oracle of the filtered convolution backward pass.
+
+TEST INFRASTRUCTURE, NOT THE PRODUCT: imported only by tests, the smoke check
+and the benchmark's CPU-baseline leg.
+"""
+from .gf_oracle import (backward, exact_backward, expand, grid, kernel_sum,  # noqa: F401
+                        literal_backward, num_threads, patch_mean, patch_sum,
+                        reduced_gw, reduced_gx, stash_forward, stash_num_values)
