@@ -1,0 +1,123 @@
+/*
+ * gf.h -- C ABI of the filtered convolution backward pass of gradient filtering
+ * (Yang, Li, Marculescu, "Efficient On-device Training via Gradient Filtering",
+ * CVPR 2023), implemented as CUDA kernels for sm_100a.
+ *
+ * The method (paper Section 3): the forward pass keeps, instead of the input
+ * feature map x, its r x r patch sums x~ (Section 3.4, text after Eq. (grad_w);
+ * memory analysis in Section 4.3).  The backward pass replaces g_y by its r x r
+ * patch means g~_y (Section 3.3), sums the kernel over its taps (theta~', text
+ * under Eq. (grad_x)), and computes
+ *     g~_theta[c_o,c_i,u,v] = sum_{n,patches} x~ * g~_y          (Eq. (grad_w))
+ *     g~_x[n,c_i,h,w]       = sum_{c_o} g~_y[n,c_o,h,w] theta~'[c_o,c_i]  (Eq. (grad_x))
+ * the latter expanded back to full resolution.  A patch size of 1 means exact
+ * ("vanilla") convolution backward (Section 4.2).
+ *
+ * General conventions
+ *  - Every data pointer is a DEVICE pointer unless its name starts with "h_".
+ *    The caller owns all buffers; the library allocates and frees nothing.
+ *  - Device data pointers must be 16-byte aligned (GF_ERR_ALIGN otherwise) and
+ *    dense in the stated layout.  Inputs are read-only, outputs are overwritten
+ *    (never accumulated into) and must not alias inputs.
+ *  - Tensors: x [N,C_in,H,W], g_y [N,C_out,H,W], W [C_out,C_in/groups,KH,KW],
+ *    g_X like x, g_W like W but ALWAYS fp32.  x, g_y, W, the stash and g_X have
+ *    the descriptor's dtype; all sums are accumulated in fp32.
+ *  - Supported geometry: stride 1, odd KH and KW, pad_h = (KH-1)/2,
+ *    pad_w = (KW-1)/2 (so g_y has the resolution of x, as Eq. (grad_x)
+ *    requires), groups dividing C_in and C_out, any r >= 1 (r need not divide
+ *    H or W: there are ceil(H/r) x ceil(W/r) patches and an edge patch averages
+ *    over the elements it has).  NCHW only.  Anything else: GF_ERR_UNSUPPORTED.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Work
+ *    is enqueued on it and the call returns without synchronising.  Errors that
+ *    the host can detect are returned before anything is launched.
+ *  - Functions return a gf_status; none aborts, throws, or traps the GPU.
+ */
+#ifndef GF_H_
+#define GF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum gf_status {
+    GF_OK = 0,
+    GF_ERR_NULL = 1,        /* a required pointer is NULL */
+    GF_ERR_BAD_DESC = 2,    /* non-positive size, groups not dividing channels, bad enum */
+    GF_ERR_UNSUPPORTED = 3, /* geometry outside the supported set (see above) */
+    GF_ERR_WORKSPACE = 4,   /* workspace smaller than gf_backward_workspace_bytes */
+    GF_ERR_ALIGN = 5,       /* a device pointer is not 16-byte aligned */
+    GF_ERR_CUDA = 6,        /* a CUDA runtime call failed (launch, copy) */
+    GF_ERR_TIMEOUT = 7      /* a bounded device-side wait expired (async status) */
+} gf_status;
+
+typedef enum gf_dtype { GF_F32 = 0, GF_BF16 = 1 } gf_dtype;
+typedef enum gf_layout { GF_NCHW = 0, GF_NHWC = 1 } gf_layout;
+
+/* One convolution layer and the patch size r used for its backward pass. */
+typedef struct gf_conv_desc {
+    int32_t N, C_in, C_out, H, W;
+    int32_t KH, KW;
+    int32_t stride;         /* must be 1 */
+    int32_t pad_h, pad_w;   /* must be (KH-1)/2, (KW-1)/2 */
+    int32_t groups;
+    int32_t r;              /* patch size, >= 1; 1 = exact backward */
+    int32_t dtype;          /* gf_dtype */
+    int32_t layout;         /* gf_layout; only GF_NCHW */
+} gf_conv_desc;
+
+/* Logical shape [N, C_in, ceil(H/r), ceil(W/r)] of the stash (Section 3.3: one
+ * unique value per patch).  For r == 1 it is the shape of x. */
+gf_status gf_stash_dims(const gf_conv_desc* desc, int64_t dims[4]);
+
+/* Bytes of the stash: product of gf_stash_dims times the element size.  The
+ * physical layout is the dense NCHW array of that shape. */
+gf_status gf_stash_bytes(const gf_conv_desc* desc, size_t* bytes);
+
+/* Bytes of device scratch gf_backward needs for this descriptor (always > 0). */
+gf_status gf_backward_workspace_bytes(const gf_conv_desc* desc, size_t* bytes);
+
+/* Forward-side step (Section 3.4 / Section 4.3): stash[n,c,a,b] = sum of x over
+ * patch (a,b); for r == 1 a plain copy of x.  x and stash are device pointers. */
+gf_status gf_stash_forward(const gf_conv_desc* desc, const void* x, void* stash,
+                           void* stream);
+
+/* Backward of one layer (Sections 3.3-3.4): from g_y, the stash written by
+ * gf_stash_forward and the kernel W, write g_W (fp32, all KH*KW taps of an
+ * input/output channel pair carry the same value when r >= 2) and g_X.  Either
+ * output may be NULL and is then skipped (a first trained layer needs no g_X).
+ * `workspace` is device scratch of at least gf_backward_workspace_bytes; its
+ * contents are undefined afterwards, and two calls that overlap in time must
+ * not share it. */
+gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* stash,
+                      const void* W, float* g_W, void* g_X, void* workspace,
+                      size_t workspace_bytes, void* stream);
+
+/* Reads the error word that device-side bounded waits of the last gf_backward
+ * on `workspace` may have set.  Synchronises `stream` (blocking).  GF_OK if no
+ * wait expired. */
+gf_status gf_last_async_status(const void* workspace, void* stream);
+
+/* One training-side step for a layer with every tensor in HOST memory
+ * (pinned memory recommended): copies h_x, h_gy, h_W to the device arena, runs
+ * gf_stash_forward and gf_backward there, and copies g_W (fp32) and g_X back to
+ * h_gW / h_gX (each nullable).  All on `stream`, no synchronisation: the host
+ * buffers are valid for reading after the caller synchronises the stream.
+ * `arena` is device scratch of at least gf_host_step_arena_bytes. */
+gf_status gf_host_step_arena_bytes(const gf_conv_desc* desc, size_t* bytes);
+gf_status gf_layer_step_host(const gf_conv_desc* desc, const void* h_x, const void* h_gy,
+                             const void* h_W, float* h_gW, void* h_gX, void* arena,
+                             size_t arena_bytes, void* stream);
+
+/* Number of kernels this library has launched in this process so far. */
+uint64_t gf_kernel_launch_count(void);
+
+/* Static, human-readable name of a status code. */
+const char* gf_status_string(gf_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GF_H_ */

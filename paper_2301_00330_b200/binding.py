@@ -1,0 +1,203 @@
+"""ctypes binding over the C ABI declared in include/gf.h.
+
+Argument marshalling only: every step of the method runs in the CUDA kernels
+of libgf_b200.so.  torch is used for device memory and streams.  There is no
+CPU fallback: if the library is missing or cannot be loaded, every entry point
+raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+from . import build as _build
+
+GF_OK, GF_ERR_NULL, GF_ERR_BAD_DESC, GF_ERR_UNSUPPORTED = 0, 1, 2, 3
+GF_ERR_WORKSPACE, GF_ERR_ALIGN, GF_ERR_CUDA, GF_ERR_TIMEOUT = 4, 5, 6, 7
+GF_F32, GF_BF16 = 0, 1
+GF_NCHW, GF_NHWC = 0, 1
+
+EXPORTS = (
+    "gf_stash_dims", "gf_stash_bytes", "gf_backward_workspace_bytes", "gf_stash_forward",
+    "gf_backward", "gf_last_async_status", "gf_host_step_arena_bytes", "gf_layer_step_host",
+    "gf_kernel_launch_count", "gf_status_string",
+)
+
+
+class gf_conv_desc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("N", "C_in", "C_out", "H", "W", "KH", "KW", "stride", "pad_h", "pad_w",
+                 "groups", "r", "dtype", "layout")]
+
+
+class GfError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)}")
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def build_library(force: bool = False) -> str:
+    """Compile libgf_b200.so for sm_100a if it is missing or stale."""
+    return _build.build(force=force)
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        path = library_path()
+        if not os.path.exists(path):
+            raise RuntimeError(
+                f"{path} is missing: build it with `python -m paper_2301_00330_b200.build` "
+                "(there is no fallback path)")
+        L = ctypes.CDLL(path)
+        vp, sz = ctypes.c_void_p, ctypes.c_size_t
+        dp = ctypes.POINTER(gf_conv_desc)
+        L.gf_stash_dims.argtypes = [dp, ctypes.POINTER(ctypes.c_int64 * 4)]
+        L.gf_stash_bytes.argtypes = [dp, ctypes.POINTER(sz)]
+        L.gf_backward_workspace_bytes.argtypes = [dp, ctypes.POINTER(sz)]
+        L.gf_stash_forward.argtypes = [dp, vp, vp, vp]
+        L.gf_backward.argtypes = [dp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.gf_last_async_status.argtypes = [vp, vp]
+        L.gf_host_step_arena_bytes.argtypes = [dp, ctypes.POINTER(sz)]
+        L.gf_layer_step_host.argtypes = [dp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.gf_kernel_launch_count.argtypes = []
+        L.gf_kernel_launch_count.restype = ctypes.c_uint64
+        L.gf_status_string.argtypes = [ctypes.c_int]
+        L.gf_status_string.restype = ctypes.c_char_p
+        for name in ("gf_stash_dims", "gf_stash_bytes", "gf_backward_workspace_bytes", "gf_stash_forward",
+                     "gf_backward", "gf_last_async_status", "gf_host_step_arena_bytes", "gf_layer_step_host"):
+            getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().gf_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != GF_OK:
+        raise GfError(status, where)
+
+
+def make_desc(N, C_in, C_out, H, W, KH, KW=None, *, r, groups=1, stride=1, pad_h=None, pad_w=None,
+              dtype=GF_F32, layout=GF_NCHW) -> gf_conv_desc:
+    KW = KH if KW is None else KW
+    pad_h = (KH - 1) // 2 if pad_h is None else pad_h
+    pad_w = (KW - 1) // 2 if pad_w is None else pad_w
+    if isinstance(dtype, torch.dtype):
+        dtype = {torch.float32: GF_F32, torch.bfloat16: GF_BF16}[dtype]
+    return gf_conv_desc(N, C_in, C_out, H, W, KH, KW, stride, pad_h, pad_w, groups, r, dtype, layout)
+
+
+def desc_for(layer) -> gf_conv_desc:
+    """Descriptor of a workloads.Layer."""
+    return make_desc(layer.N, layer.C_in, layer.C_out, layer.H, layer.W, layer.K, r=layer.r,
+                     groups=layer.groups, dtype=GF_F32 if layer.dtype == "f32" else GF_BF16)
+
+
+def _ptr(t) -> ctypes.c_void_p:
+    if t is None:
+        return ctypes.c_void_p(0)
+    if isinstance(t, torch.Tensor):
+        if not t.is_contiguous():
+            raise ValueError("tensors passed to the gf_* calls must be contiguous")
+        return ctypes.c_void_p(t.data_ptr())
+    return ctypes.c_void_p(int(t))
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    if isinstance(stream, torch.cuda.Stream):
+        return ctypes.c_void_p(stream.cuda_stream)
+    return ctypes.c_void_p(int(stream))
+
+
+# ---- the C calls, same names ----------------------------------------------------
+
+def gf_stash_dims(desc: gf_conv_desc) -> tuple[int, int, int, int]:
+    dims = (ctypes.c_int64 * 4)()
+    _check(lib().gf_stash_dims(ctypes.byref(desc), ctypes.byref(dims)), "gf_stash_dims")
+    return tuple(int(v) for v in dims)
+
+
+def gf_stash_bytes(desc: gf_conv_desc) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().gf_stash_bytes(ctypes.byref(desc), ctypes.byref(out)), "gf_stash_bytes")
+    return int(out.value)
+
+
+def gf_backward_workspace_bytes(desc: gf_conv_desc) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().gf_backward_workspace_bytes(ctypes.byref(desc), ctypes.byref(out)),
+           "gf_backward_workspace_bytes")
+    return int(out.value)
+
+
+def gf_stash_forward(desc: gf_conv_desc, x, stash, stream=None) -> None:
+    _check(lib().gf_stash_forward(ctypes.byref(desc), _ptr(x), _ptr(stash), _stream(stream)),
+           "gf_stash_forward")
+
+
+def gf_backward(desc: gf_conv_desc, g_y, stash, W, g_W, g_X, workspace, workspace_bytes=None,
+                stream=None) -> None:
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    _check(lib().gf_backward(ctypes.byref(desc), _ptr(g_y), _ptr(stash), _ptr(W), _ptr(g_W), _ptr(g_X),
+                             _ptr(workspace), ctypes.c_size_t(workspace_bytes), _stream(stream)),
+           "gf_backward")
+
+
+def gf_last_async_status(workspace, stream=None) -> int:
+    return int(lib().gf_last_async_status(_ptr(workspace), _stream(stream)))
+
+
+def gf_host_step_arena_bytes(desc: gf_conv_desc) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().gf_host_step_arena_bytes(ctypes.byref(desc), ctypes.byref(out)), "gf_host_step_arena_bytes")
+    return int(out.value)
+
+
+def gf_layer_step_host(desc: gf_conv_desc, h_x, h_gy, h_W, h_gW, h_gX, arena, arena_bytes=None,
+                       stream=None) -> None:
+    if arena_bytes is None:
+        arena_bytes = arena.numel() * arena.element_size()
+    _check(lib().gf_layer_step_host(ctypes.byref(desc), _ptr(h_x), _ptr(h_gy), _ptr(h_W), _ptr(h_gW),
+                                    _ptr(h_gX), _ptr(arena), ctypes.c_size_t(arena_bytes), _stream(stream)),
+           "gf_layer_step_host")
+
+
+def gf_kernel_launch_count() -> int:
+    return int(lib().gf_kernel_launch_count())
+
+
+# ---- conveniences that only allocate ---------------------------------------------
+
+@dataclass
+class LayerBuffers:
+    desc: gf_conv_desc
+    stash: torch.Tensor
+    g_W: torch.Tensor
+    g_X: torch.Tensor
+    workspace: torch.Tensor
+
+
+def alloc_layer(desc: gf_conv_desc, device="cuda") -> LayerBuffers:
+    dt = torch.float32 if desc.dtype == GF_F32 else torch.bfloat16
+    stash = torch.empty(gf_stash_dims(desc), dtype=dt, device=device)
+    g_W = torch.empty((desc.C_out, desc.C_in // desc.groups, desc.KH, desc.KW), dtype=torch.float32,
+                      device=device)
+    g_X = torch.empty((desc.N, desc.C_in, desc.H, desc.W), dtype=dt, device=device)
+    ws = torch.empty(gf_backward_workspace_bytes(desc), dtype=torch.uint8, device=device)
+    return LayerBuffers(desc, stash, g_W, g_X, ws)

@@ -1,0 +1,257 @@
+// C ABI of the library: argument validation, workspace planning and dispatch.
+// Every step of the method runs in the kernels of this directory; this file
+// only checks arguments and enqueues launches.
+#include <atomic>
+
+#include "gf_common.cuh"
+
+namespace gf {
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+Geo make_geo(const gf_conv_desc& d) {
+    Geo g;
+    g.N = d.N; g.C_in = d.C_in; g.C_out = d.C_out; g.H = d.H; g.W = d.W;
+    g.KH = d.KH; g.KW = d.KW; g.G = d.groups; g.r = d.r;
+    g.Hp = (d.H + d.r - 1) / d.r; g.Wp = (d.W + d.r - 1) / d.r;
+    g.C_ig = d.C_in / d.groups; g.C_og = d.C_out / d.groups;
+    g.dtype = d.dtype; g.esize = d.dtype == GF_F32 ? 4 : 2;
+    return g;
+}
+
+static gf_status validate(const gf_conv_desc* d) {
+    if (!d) return GF_ERR_NULL;
+    if (d->N < 1 || d->C_in < 1 || d->C_out < 1 || d->H < 1 || d->W < 1 || d->KH < 1 || d->KW < 1 ||
+        d->groups < 1 || d->r < 1 || d->stride < 1 || d->pad_h < 0 || d->pad_w < 0)
+        return GF_ERR_BAD_DESC;
+    if (d->C_in % d->groups != 0 || d->C_out % d->groups != 0) return GF_ERR_BAD_DESC;
+    if (d->dtype != GF_F32 && d->dtype != GF_BF16) return GF_ERR_BAD_DESC;
+    if (d->layout != GF_NCHW && d->layout != GF_NHWC) return GF_ERR_BAD_DESC;
+    if (d->layout != GF_NCHW) return GF_ERR_UNSUPPORTED;
+    if (d->stride != 1) return GF_ERR_UNSUPPORTED;
+    if (d->KH % 2 == 0 || d->KW % 2 == 0) return GF_ERR_UNSUPPORTED;
+    if (d->pad_h != (d->KH - 1) / 2 || d->pad_w != (d->KW - 1) / 2) return GF_ERR_UNSUPPORTED;
+    // index arithmetic inside the kernels is 32-bit per plane and per tile
+    if ((int64_t)d->H * d->W > (int64_t)1 << 30) return GF_ERR_UNSUPPORTED;
+    if ((int64_t)d->N * d->C_in > (int64_t)1 << 30 || (int64_t)d->N * d->C_out > (int64_t)1 << 30)
+        return GF_ERR_UNSUPPORTED;
+    if ((int64_t)d->C_out * (d->C_in / d->groups) * d->KH * d->KW > (int64_t)1 << 30) return GF_ERR_UNSUPPORTED;
+    return GF_OK;
+}
+
+static bool is_depthwise(const Geo& g) { return g.G == g.C_in && g.G == g.C_out; }
+
+static int dense_splits(const Geo& g) {
+    const long long tiles = (long long)((g.C_og + 63) / 64) * ((g.C_ig + 63) / 64) * g.G;
+    long long s = (592 + tiles - 1) / tiles;
+    if (s < 1) s = 1;
+    if (s > g.N) s = g.N;
+    if (s * g.G > 65535) s = 65535 / g.G > 0 ? 65535 / g.G : 1;
+    return (int)s;
+}
+
+Workspace plan_workspace(const Geo& g) {
+    Workspace w;
+    w.off_err = 0;
+    size_t off = 256;
+    if (g.r == 1) { w.off_tsum = w.off_gbar = w.off_part = off; w.splits = 0; w.total = off; return w; }
+    w.off_tsum = off; off += align_up((size_t)g.C_out * g.C_ig * 4, 256);
+    w.off_gbar = off; off += align_up((size_t)g.N * g.C_out * g.Hp * g.Wp * 4, 256);
+    int s = dense_splits(g);
+    if (is_depthwise(g)) { const int ds = depthwise_splits(g); if (ds > s) s = ds; }
+    w.splits = s;
+    w.off_part = off; off += align_up((size_t)s * g.C_out * g.C_ig * 4, 256);
+    w.total = off;
+    return w;
+}
+
+static bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+}  // namespace gf
+
+using namespace gf;
+
+extern "C" {
+
+gf_status gf_stash_dims(const gf_conv_desc* desc, int64_t dims[4]) {
+    if (!dims) return GF_ERR_NULL;
+    gf_status st = validate(desc);
+    if (st != GF_OK) return st;
+    dims[0] = desc->N; dims[1] = desc->C_in;
+    dims[2] = (desc->H + desc->r - 1) / desc->r;
+    dims[3] = (desc->W + desc->r - 1) / desc->r;
+    return GF_OK;
+}
+
+gf_status gf_stash_bytes(const gf_conv_desc* desc, size_t* bytes) {
+    if (!bytes) return GF_ERR_NULL;
+    int64_t d[4];
+    gf_status st = gf_stash_dims(desc, d);
+    if (st != GF_OK) return st;
+    *bytes = (size_t)d[0] * d[1] * d[2] * d[3] * (desc->dtype == GF_F32 ? 4 : 2);
+    return GF_OK;
+}
+
+gf_status gf_backward_workspace_bytes(const gf_conv_desc* desc, size_t* bytes) {
+    if (!bytes) return GF_ERR_NULL;
+    gf_status st = validate(desc);
+    if (st != GF_OK) return st;
+    *bytes = plan_workspace(make_geo(*desc)).total;
+    return GF_OK;
+}
+
+gf_status gf_stash_forward(const gf_conv_desc* desc, const void* x, void* stash, void* stream) {
+    if (!desc || !x || !stash) return GF_ERR_NULL;
+    gf_status st = validate(desc);
+    if (st != GF_OK) return st;
+    if (misaligned(x) || misaligned(stash)) return GF_ERR_ALIGN;
+    const Geo g = make_geo(*desc);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int64_t planes = (int64_t)g.N * g.C_in;
+    if (g.r == 1) return launch_copy(x, stash, (size_t)planes * g.H * g.W * g.esize, s);
+    return launch_pool(x, g.dtype, stash, g.dtype, /*mean=*/false, planes, g.H, g.W, g.r, s);
+}
+
+gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* stash, const void* W,
+                      float* g_W, void* g_X, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!desc || !g_y || !W || !workspace) return GF_ERR_NULL;
+    if (g_W && !stash) return GF_ERR_NULL;
+    gf_status st = validate(desc);
+    if (st != GF_OK) return st;
+    if (misaligned(g_y) || misaligned(W) || misaligned(workspace) || (stash && misaligned(stash)) ||
+        (g_W && misaligned(g_W)) || (g_X && misaligned(g_X)))
+        return GF_ERR_ALIGN;
+    const Geo g = make_geo(*desc);
+    const Workspace ws = plan_workspace(g);
+    if (workspace_bytes < ws.total) return GF_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    char* base = static_cast<char*>(workspace);
+    uint32_t* err = reinterpret_cast<uint32_t*>(base + ws.off_err);
+    if (!g_W && !g_X) return GF_OK;
+
+    if (g.r == 1) {
+        GF_CUDA_TRY(cudaMemsetAsync(err, 0, sizeof(uint32_t), s));
+        return launch_exact(g_y, stash, W, g_W, g_X, g, s);
+    }
+
+    float* tsum = reinterpret_cast<float*>(base + ws.off_tsum);
+    float* gbar = reinterpret_cast<float*>(base + ws.off_gbar);
+    float* part = reinterpret_cast<float*>(base + ws.off_part);
+
+    if (is_depthwise(g) && depthwise_splits(g) > 0) {
+        int splits = 0;
+        st = launch_depthwise(g_y, stash, W, g_W ? part : nullptr, g_X, err, g, &splits, s);
+        if (st != GF_OK) return st;
+        if (g_W) return launch_gw_finish(part, splits, g_W, g, s);
+        return GF_OK;
+    }
+
+    // kernel sums (also clears the error word), then the gradient filter:
+    // patch means of g_y, read once
+    st = launch_ksum(W, g, tsum, err, s);
+    if (st != GF_OK) return st;
+    st = launch_pool(g_y, g.dtype, gbar, GF_F32, /*mean=*/true, (int64_t)g.N * g.C_out, g.H, g.W, g.r, s);
+    if (st != GF_OK) return st;
+    if (g_X) {
+        st = launch_gx_mix(gbar, tsum, g_X, g, s);
+        if (st != GF_OK) return st;
+    }
+    if (g_W) {
+        st = launch_gw_partial(gbar, stash, part, ws.splits, g, s);
+        if (st != GF_OK) return st;
+        st = launch_gw_finish(part, ws.splits, g_W, g, s);
+        if (st != GF_OK) return st;
+    }
+    return GF_OK;
+}
+
+gf_status gf_last_async_status(const void* workspace, void* stream) {
+    if (!workspace) return GF_ERR_NULL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint32_t word = 0;
+    GF_CUDA_TRY(cudaMemcpyAsync(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost, s));
+    GF_CUDA_TRY(cudaStreamSynchronize(s));
+    return word == 0 ? GF_OK : GF_ERR_TIMEOUT;
+}
+
+// ---- host-buffer step ---------------------------------------------------------
+namespace {
+struct Arena { size_t x, gy, w, stash, gw, gx, ws, ws_bytes, total; };
+gf_status plan_arena(const gf_conv_desc* desc, Arena* a) {
+    gf_status st = validate(desc);
+    if (st != GF_OK) return st;
+    const Geo g = make_geo(*desc);
+    size_t stash_bytes = 0;
+    st = gf_stash_bytes(desc, &stash_bytes);
+    if (st != GF_OK) return st;
+    size_t off = 0;
+    a->x = off; off += align_up((size_t)g.N * g.C_in * g.H * g.W * g.esize, 256);
+    a->gy = off; off += align_up((size_t)g.N * g.C_out * g.H * g.W * g.esize, 256);
+    a->w = off; off += align_up((size_t)g.C_out * g.C_ig * g.KH * g.KW * g.esize, 256);
+    a->stash = off; off += align_up(stash_bytes, 256);
+    a->gw = off; off += align_up((size_t)g.C_out * g.C_ig * g.KH * g.KW * 4, 256);
+    a->gx = off; off += align_up((size_t)g.N * g.C_in * g.H * g.W * g.esize, 256);
+    a->ws_bytes = plan_workspace(g).total;
+    a->ws = off; off += align_up(a->ws_bytes, 256);
+    a->total = off;
+    return GF_OK;
+}
+}  // namespace
+
+gf_status gf_host_step_arena_bytes(const gf_conv_desc* desc, size_t* bytes) {
+    if (!bytes) return GF_ERR_NULL;
+    Arena a;
+    gf_status st = plan_arena(desc, &a);
+    if (st != GF_OK) return st;
+    *bytes = a.total;
+    return GF_OK;
+}
+
+gf_status gf_layer_step_host(const gf_conv_desc* desc, const void* h_x, const void* h_gy, const void* h_W,
+                             float* h_gW, void* h_gX, void* arena, size_t arena_bytes, void* stream) {
+    if (!desc || !h_x || !h_gy || !h_W || !arena) return GF_ERR_NULL;
+    Arena a;
+    gf_status st = plan_arena(desc, &a);
+    if (st != GF_OK) return st;
+    if (misaligned(arena)) return GF_ERR_ALIGN;
+    if (arena_bytes < a.total) return GF_ERR_WORKSPACE;
+    const Geo g = make_geo(*desc);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    char* base = static_cast<char*>(arena);
+    const size_t x_bytes = (size_t)g.N * g.C_in * g.H * g.W * g.esize;
+    const size_t gy_bytes = (size_t)g.N * g.C_out * g.H * g.W * g.esize;
+    const size_t w_elems = (size_t)g.C_out * g.C_ig * g.KH * g.KW;
+    GF_CUDA_TRY(cudaMemcpyAsync(base + a.x, h_x, x_bytes, cudaMemcpyHostToDevice, s));
+    GF_CUDA_TRY(cudaMemcpyAsync(base + a.gy, h_gy, gy_bytes, cudaMemcpyHostToDevice, s));
+    GF_CUDA_TRY(cudaMemcpyAsync(base + a.w, h_W, w_elems * g.esize, cudaMemcpyHostToDevice, s));
+    st = gf_stash_forward(desc, base + a.x, base + a.stash, stream);
+    if (st != GF_OK) return st;
+    st = gf_backward(desc, base + a.gy, base + a.stash, base + a.w,
+                     h_gW ? reinterpret_cast<float*>(base + a.gw) : nullptr, h_gX ? base + a.gx : nullptr,
+                     base + a.ws, a.ws_bytes, stream);
+    if (st != GF_OK) return st;
+    if (h_gW) GF_CUDA_TRY(cudaMemcpyAsync(h_gW, base + a.gw, w_elems * 4, cudaMemcpyDeviceToHost, s));
+    if (h_gX) GF_CUDA_TRY(cudaMemcpyAsync(h_gX, base + a.gx, x_bytes, cudaMemcpyDeviceToHost, s));
+    return GF_OK;
+}
+
+uint64_t gf_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* gf_status_string(gf_status s) {
+    switch (s) {
+        case GF_OK: return "GF_OK";
+        case GF_ERR_NULL: return "GF_ERR_NULL: a required pointer is NULL";
+        case GF_ERR_BAD_DESC: return "GF_ERR_BAD_DESC: invalid descriptor";
+        case GF_ERR_UNSUPPORTED: return "GF_ERR_UNSUPPORTED: geometry or layout not supported";
+        case GF_ERR_WORKSPACE: return "GF_ERR_WORKSPACE: workspace too small";
+        case GF_ERR_ALIGN: return "GF_ERR_ALIGN: device pointer not 16-byte aligned";
+        case GF_ERR_CUDA: return "GF_ERR_CUDA: a CUDA runtime call failed";
+        case GF_ERR_TIMEOUT: return "GF_ERR_TIMEOUT: a bounded device-side wait expired";
+    }
+    return "unknown gf_status";
+}
+
+}  // extern "C"

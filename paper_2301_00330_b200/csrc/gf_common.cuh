@@ -1,0 +1,137 @@
+// Shared device/host helpers of the CUDA library (not used by the CPU checker).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "gf.h"
+
+namespace gf {
+
+// ---- launch accounting -----------------------------------------------------
+void count_launch(int n = 1);
+
+#define GF_CUDA_TRY(expr)                         \
+    do {                                          \
+        cudaError_t e__ = (expr);                 \
+        if (e__ != cudaSuccess) return GF_ERR_CUDA; \
+    } while (0)
+
+// Checks the launch that was just made and counts it.
+static inline gf_status after_launch() {
+    count_launch();
+    return cudaPeekAtLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
+}
+
+static inline int64_t cdiv64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// ---- division by a runtime constant ---------------------------------------
+// q = n / d for any 32-bit n via one multiply-high, an add and two shifts.
+struct FastDiv {
+    uint32_t mul, shr, d;
+    FastDiv() : mul(0), shr(0), d(1) {}
+    explicit FastDiv(uint32_t div) : d(div) {
+        if (div == 1) { mul = 0; shr = 0; return; }
+        uint32_t l = 0;
+        while ((1u << l) < div) ++l;                       // ceil(log2 d)
+        uint64_t m = ((uint64_t(1) << 32) * ((uint64_t(1) << l) - div)) / div + 1;
+        mul = (uint32_t)m;
+        shr = l;
+    }
+    __host__ __device__ __forceinline__ uint32_t div(uint32_t n) const {
+#ifdef __CUDA_ARCH__
+        if (d == 1) return n;
+        uint32_t t = __umulhi(n, mul);
+        return (t + ((n - t) >> 1)) >> (shr - 1);
+#else
+        return n / d;
+#endif
+    }
+    __host__ __device__ __forceinline__ void divmod(uint32_t n, uint32_t& q, uint32_t& rem) const {
+        q = div(n);
+        rem = n - q * d;
+    }
+};
+
+// ---- element access --------------------------------------------------------
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) {
+    return __float2bfloat16_rn(v);
+}
+
+// Sum of CNT consecutive shared-memory elements starting at `p` (CNT is 2, 4 or
+// 8 and p is aligned to min(CNT elements, 16 bytes)).
+template <int CNT> __device__ __forceinline__ float sum_run(const float* p) {
+    if constexpr (CNT == 2) { float2 v = *reinterpret_cast<const float2*>(p); return v.x + v.y; }
+    else if constexpr (CNT == 4) { float4 v = *reinterpret_cast<const float4*>(p); return (v.x + v.y) + (v.z + v.w); }
+    else { float4 a = *reinterpret_cast<const float4*>(p); float4 b = *reinterpret_cast<const float4*>(p + 4);
+           return ((a.x + a.y) + (a.z + a.w)) + ((b.x + b.y) + (b.z + b.w)); }
+}
+template <int CNT> __device__ __forceinline__ float sum_run(const __nv_bfloat16* p) {
+    if constexpr (CNT == 2) {
+        float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(p));
+        return f.x + f.y;
+    } else if constexpr (CNT == 4) {
+        uint2 raw = *reinterpret_cast<const uint2*>(p);
+        float2 a = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&raw.x));
+        float2 b = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&raw.y));
+        return (a.x + a.y) + (b.x + b.y);
+    } else {
+        uint4 raw = *reinterpret_cast<const uint4*>(p);
+        float2 a = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&raw.x));
+        float2 b = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&raw.y));
+        float2 c = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&raw.z));
+        float2 d = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&raw.w));
+        return ((a.x + a.y) + (b.x + b.y)) + ((c.x + c.y) + (d.x + d.y));
+    }
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// ---- geometry shared by the kernels ----------------------------------------
+struct Geo {
+    int N, C_in, C_out, H, W, KH, KW, G, r;
+    int Hp, Wp;           // ceil(H/r), ceil(W/r)
+    int C_ig, C_og;       // channels per group
+    int dtype;
+    size_t esize;
+};
+
+Geo make_geo(const gf_conv_desc& d);
+
+// ---- workspace layout of gf_backward ---------------------------------------
+// [ error word (256 B) | theta sum fp32 [C_out,C_ig] | gbar fp32 [N,C_out,Hp,Wp] |
+//   split partials fp32 [S, C_out, C_ig] ]
+struct Workspace {
+    size_t off_err, off_tsum, off_gbar, off_part, total;
+    int splits;           // S: number of partial g_W matrices
+};
+Workspace plan_workspace(const Geo& g);
+
+// ---- kernel entry points (host launchers) ----------------------------------
+// pool: out[plane, a, b] = sum (or mean) of in[plane] over patch (a,b)
+gf_status launch_pool(const void* in, int in_dtype, void* out, int out_dtype, bool mean,
+                      int64_t planes, int H, int W, int r, cudaStream_t s);
+gf_status launch_copy(const void* in, void* out, size_t bytes, cudaStream_t s);
+
+gf_status launch_ksum(const void* W, const Geo& g, float* tsum, uint32_t* err_word, cudaStream_t s);
+gf_status launch_gx_mix(const float* gbar, const float* tsum, void* gX, const Geo& g, cudaStream_t s);
+gf_status launch_gw_partial(const float* gbar, const void* stash, float* part, int splits,
+                            const Geo& g, cudaStream_t s);
+gf_status launch_gw_finish(const float* part, int splits, float* gW, const Geo& g, cudaStream_t s);
+gf_status launch_depthwise(const void* gy, const void* stash, const void* W, float* part,
+                           void* gX, uint32_t* err_word, const Geo& g, int* splits_out, cudaStream_t s);
+int depthwise_splits(const Geo& g);
+gf_status launch_exact(const void* gy, const void* x, const void* W, float* gW, void* gX,
+                       const Geo& g, cudaStream_t s);
+
+}  // namespace gf

@@ -1,0 +1,101 @@
+// r == 1: the method is off and the backward is the exact ("vanilla")
+// convolution backward of Section 3.1, stride 1, zero padding.  Plain direct
+// kernels, not tuned: this path exists so that a patch size of 1 has the
+// meaning the paper gives it.
+//   g_W[c_o,c_l,u,v] = sum_{n,i,j} x[n,c_i,i+u-ph,j+v-pw] g_y[n,c_o,i,j]
+//   g_X[n,c_i,h,w]   = sum_{c_o,u,v} W[c_o,c_l,u,v] g_y[n,c_o,h-u+ph,w-v+pw]
+#include "gf_common.cuh"
+
+namespace gf {
+
+template <typename T>
+__global__ void __launch_bounds__(256) exact_gx_kernel(const T* __restrict__ gy, const T* __restrict__ Wt,
+                                                       T* __restrict__ gX, int N, int C_in, int C_out, int G,
+                                                       int H, int W, int KH, int KW) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long total = (long long)N * C_in * H * W;
+    if (idx >= total) return;
+    const int w = (int)(idx % W), h = (int)((idx / W) % H);
+    const int ci = (int)((idx / ((long long)W * H)) % C_in), n = (int)(idx / ((long long)W * H * C_in));
+    const int C_ig = C_in / G, C_og = C_out / G, q = ci / C_ig, cl = ci - q * C_ig;
+    const int ph = (KH - 1) / 2, pw = (KW - 1) / 2;
+    float s = 0.f;
+    for (int co = q * C_og; co < (q + 1) * C_og; ++co)
+        for (int u = 0; u < KH; ++u) {
+            const int i = h - u + ph;
+            if (i < 0 || i >= H) continue;
+            for (int v = 0; v < KW; ++v) {
+                const int j = w - v + pw;
+                if (j < 0 || j >= W) continue;
+                s = fmaf(to_f32(Wt[(((size_t)co * C_ig + cl) * KH + u) * KW + v]),
+                         to_f32(gy[(((size_t)n * C_out + co) * H + i) * W + j]), s);
+            }
+        }
+    gX[idx] = from_f32<T>(s);
+}
+
+// One block per (c_o, c_l, u, v): strided sum over (n, i, j), block reduction.
+template <typename T>
+__global__ void __launch_bounds__(256) exact_gw_kernel(const T* __restrict__ gy, const T* __restrict__ x,
+                                                       float* __restrict__ gW, int N, int C_in, int C_out, int G,
+                                                       int H, int W, int KH, int KW) {
+    __shared__ float warp_part[8];
+    const int taps = KH * KW;
+    const int C_ig = C_in / G, C_og = C_out / G;
+    const long long o = blockIdx.x;
+    const int t = (int)(o % taps), cl = (int)((o / taps) % C_ig), co = (int)(o / ((long long)taps * C_ig));
+    const int u = t / KW, v = t - u * KW;
+    const int ci = (co / C_og) * C_ig + cl;
+    const int ph = (KH - 1) / 2, pw = (KW - 1) / 2;
+    const long long per = (long long)H * W, total = (long long)N * per;
+    float s = 0.f;
+    for (long long e = threadIdx.x; e < total; e += 256) {
+        const int n = (int)(e / per), rem = (int)(e - n * per);
+        const int i = rem / W, j = rem - i * W;
+        const int h = i + u - ph, w = j + v - pw;
+        if (h < 0 || h >= H || w < 0 || w >= W) continue;
+        s = fmaf(to_f32(x[(((size_t)n * C_in + ci) * H + h) * W + w]),
+                 to_f32(gy[(((size_t)n * C_out + co) * H + i) * W + j]), s);
+    }
+    s = warp_sum(s);
+    if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        float r = threadIdx.x < 8 ? warp_part[threadIdx.x] : 0.f;
+        r = warp_sum(r);
+        if (threadIdx.x == 0) gW[o] = r;
+    }
+}
+
+gf_status launch_exact(const void* gy, const void* x, const void* W, float* gW, void* gX,
+                       const Geo& g, cudaStream_t s) {
+    if (gX) {
+        const long long total = (long long)g.N * g.C_in * g.H * g.W;
+        const long long blocks = (total + 255) / 256;
+        if (blocks > 0x7fffffffLL) return GF_ERR_UNSUPPORTED;
+        if (g.dtype == GF_F32)
+            exact_gx_kernel<float><<<(unsigned)blocks, 256, 0, s>>>((const float*)gy, (const float*)W, (float*)gX,
+                                                                     g.N, g.C_in, g.C_out, g.G, g.H, g.W, g.KH, g.KW);
+        else
+            exact_gx_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, s>>>(
+                (const __nv_bfloat16*)gy, (const __nv_bfloat16*)W, (__nv_bfloat16*)gX, g.N, g.C_in, g.C_out, g.G,
+                g.H, g.W, g.KH, g.KW);
+        gf_status st = after_launch();
+        if (st != GF_OK) return st;
+    }
+    if (gW) {
+        const long long blocks = (long long)g.C_out * g.C_ig * g.KH * g.KW;
+        if (blocks > 0x7fffffffLL) return GF_ERR_UNSUPPORTED;
+        if (g.dtype == GF_F32)
+            exact_gw_kernel<float><<<(unsigned)blocks, 256, 0, s>>>((const float*)gy, (const float*)x, gW, g.N,
+                                                                     g.C_in, g.C_out, g.G, g.H, g.W, g.KH, g.KW);
+        else
+            exact_gw_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, s>>>(
+                (const __nv_bfloat16*)gy, (const __nv_bfloat16*)x, gW, g.N, g.C_in, g.C_out, g.G, g.H, g.W, g.KH,
+                g.KW);
+        return after_launch();
+    }
+    return GF_OK;
+}
+
+}  // namespace gf
