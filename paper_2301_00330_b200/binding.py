@@ -23,7 +23,8 @@ GF_NCHW, GF_NHWC = 0, 1
 EXPORTS = (
     "gf_stash_dims", "gf_stash_bytes", "gf_backward_workspace_bytes", "gf_stash_forward",
     "gf_backward", "gf_last_async_status", "gf_host_step_arena_bytes", "gf_layer_step_host",
-    "gf_kernel_launch_count", "gf_status_string",
+    "gf_kernel_launch_count", "gf_status_string", "gf_profile_configure", "gf_profile_read",
+    "gf_kernel_name", "gf_kernel_id_count",
 )
 
 
@@ -31,6 +32,10 @@ class gf_conv_desc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("N", "C_in", "C_out", "H", "W", "KH", "KW", "stride", "pad_h", "pad_w",
                  "groups", "r", "dtype", "layout")]
+
+
+class gf_kernel_time(ctypes.Structure):
+    _fields_ = [("kernel_id", ctypes.c_int32), ("launches", ctypes.c_int32), ("total_ms", ctypes.c_double)]
 
 
 class GfError(RuntimeError):
@@ -72,6 +77,14 @@ def lib() -> ctypes.CDLL:
         L.gf_layer_step_host.argtypes = [dp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.gf_kernel_launch_count.argtypes = []
         L.gf_kernel_launch_count.restype = ctypes.c_uint64
+        L.gf_profile_configure.argtypes = [ctypes.c_int32, ctypes.c_int32]
+        L.gf_profile_configure.restype = ctypes.c_int
+        L.gf_profile_read.argtypes = [ctypes.POINTER(gf_kernel_time), ctypes.c_int32]
+        L.gf_profile_read.restype = ctypes.c_int32
+        L.gf_kernel_name.argtypes = [ctypes.c_int32]
+        L.gf_kernel_name.restype = ctypes.c_char_p
+        L.gf_kernel_id_count.argtypes = []
+        L.gf_kernel_id_count.restype = ctypes.c_int32
         L.gf_status_string.argtypes = [ctypes.c_int]
         L.gf_status_string.restype = ctypes.c_char_p
         for name in ("gf_stash_dims", "gf_stash_bytes", "gf_backward_workspace_bytes", "gf_stash_forward",
@@ -180,6 +193,36 @@ def gf_layer_step_host(desc: gf_conv_desc, h_x, h_gy, h_W, h_gW, h_gX, arena, ar
 
 def gf_kernel_launch_count() -> int:
     return int(lib().gf_kernel_launch_count())
+
+
+def gf_kernel_id_count() -> int:
+    return int(lib().gf_kernel_id_count())
+
+
+def gf_kernel_name(kernel_id: int) -> str | None:
+    n = lib().gf_kernel_name(int(kernel_id))
+    return n.decode() if n else None
+
+
+def kernel_id(name: str) -> int:
+    for k in range(gf_kernel_id_count()):
+        if gf_kernel_name(k) == name:
+            return k
+    raise KeyError(name)
+
+
+def gf_profile_configure(mode: int, kernel_id: int = -1) -> None:
+    _check(lib().gf_profile_configure(int(mode), int(kernel_id)), "gf_profile_configure")
+
+
+def gf_profile_read() -> dict[str, tuple[int, float]]:
+    """{kernel name: (timed launches, total ms)} since the last read."""
+    n = gf_kernel_id_count()
+    buf = (gf_kernel_time * n)()
+    got = lib().gf_profile_read(buf, n)
+    if got < 0:
+        raise GfError(GF_ERR_CUDA, "gf_profile_read")
+    return {gf_kernel_name(buf[i].kernel_id): (int(buf[i].launches), float(buf[i].total_ms)) for i in range(got)}
 
 
 # ---- conveniences that only allocate ---------------------------------------------

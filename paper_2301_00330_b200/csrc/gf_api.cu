@@ -2,6 +2,7 @@
 // Every step of the method runs in the kernels of this directory; this file
 // only checks arguments and enqueues launches.
 #include <atomic>
+#include <mutex>
 
 #include "gf_common.cuh"
 
@@ -9,6 +10,38 @@ namespace gf {
 
 static std::atomic<uint64_t> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+// ---- optional event timing ----------------------------------------------------
+namespace {
+constexpr int kProfPairs = 8192;
+std::mutex g_prof_mu;
+int g_prof_mode = 0, g_prof_kid = -1;
+cudaEvent_t g_prof_ev[kProfPairs][2];
+int g_prof_created = 0;          // event pairs that exist
+int g_prof_used = 0;             // event pairs recorded since the last read
+int g_prof_slot_kid[kProfPairs];
+const char* const kKernelNames[K_COUNT] = {
+    "stash_pool", "ksum", "gy_pool", "gx_mix", "gw_partial", "gw_finish", "dw_fused", "exact_gx", "exact_gw"};
+}  // namespace
+
+ProfScope::ProfScope(int kernel_id, cudaStream_t s) : slot(-1), stream(s) {
+    if (g_prof_mode == 0) return;
+    std::lock_guard<std::mutex> lock(g_prof_mu);
+    if (g_prof_mode == 1 && kernel_id != g_prof_kid) return;
+    if (g_prof_used >= kProfPairs) return;
+    if (g_prof_used >= g_prof_created) {
+        if (cudaEventCreate(&g_prof_ev[g_prof_created][0]) != cudaSuccess) return;
+        if (cudaEventCreate(&g_prof_ev[g_prof_created][1]) != cudaSuccess) return;
+        ++g_prof_created;
+    }
+    slot = g_prof_used++;
+    g_prof_slot_kid[slot] = kernel_id;
+    cudaEventRecord(g_prof_ev[slot][0], stream);
+}
+
+ProfScope::~ProfScope() {
+    if (slot >= 0) cudaEventRecord(g_prof_ev[slot][1], stream);
+}
 
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -112,7 +145,7 @@ gf_status gf_stash_forward(const gf_conv_desc* desc, const void* x, void* stash,
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int64_t planes = (int64_t)g.N * g.C_in;
     if (g.r == 1) return launch_copy(x, stash, (size_t)planes * g.H * g.W * g.esize, s);
-    return launch_pool(x, g.dtype, stash, g.dtype, /*mean=*/false, planes, g.H, g.W, g.r, s);
+    return launch_pool(K_STASH_POOL, x, g.dtype, stash, g.dtype, /*mean=*/false, planes, g.H, g.W, g.r, s);
 }
 
 gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* stash, const void* W,
@@ -153,7 +186,7 @@ gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* sta
     // patch means of g_y, read once
     st = launch_ksum(W, g, tsum, err, s);
     if (st != GF_OK) return st;
-    st = launch_pool(g_y, g.dtype, gbar, GF_F32, /*mean=*/true, (int64_t)g.N * g.C_out, g.H, g.W, g.r, s);
+    st = launch_pool(K_GY_POOL, g_y, g.dtype, gbar, GF_F32, /*mean=*/true, (int64_t)g.N * g.C_out, g.H, g.W, g.r, s);
     if (st != GF_OK) return st;
     if (g_X) {
         st = launch_gx_mix(gbar, tsum, g_X, g, s);
@@ -237,6 +270,39 @@ gf_status gf_layer_step_host(const gf_conv_desc* desc, const void* h_x, const vo
     if (h_gX) GF_CUDA_TRY(cudaMemcpyAsync(h_gX, base + a.gx, x_bytes, cudaMemcpyDeviceToHost, s));
     return GF_OK;
 }
+
+gf_status gf_profile_configure(int32_t mode, int32_t kernel_id) {
+    if (mode < 0 || mode > 2) return GF_ERR_BAD_DESC;
+    if (mode == 1 && (kernel_id < 0 || kernel_id >= K_COUNT)) return GF_ERR_BAD_DESC;
+    std::lock_guard<std::mutex> lock(g_prof_mu);
+    g_prof_mode = mode;
+    g_prof_kid = kernel_id;
+    return GF_OK;
+}
+
+int32_t gf_profile_read(gf_kernel_time* out, int32_t max_entries) {
+    std::lock_guard<std::mutex> lock(g_prof_mu);
+    double total[K_COUNT] = {};
+    int launches[K_COUNT] = {};
+    for (int i = 0; i < g_prof_used; ++i) {
+        if (cudaEventSynchronize(g_prof_ev[i][1]) != cudaSuccess) return -1;
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, g_prof_ev[i][0], g_prof_ev[i][1]) != cudaSuccess) return -1;
+        total[g_prof_slot_kid[i]] += ms;
+        launches[g_prof_slot_kid[i]] += 1;
+    }
+    g_prof_used = 0;
+    int32_t n = 0;
+    for (int k = 0; k < K_COUNT && out && n < max_entries; ++k)
+        if (launches[k] > 0) { out[n].kernel_id = k; out[n].launches = launches[k]; out[n].total_ms = total[k]; ++n; }
+    return n;
+}
+
+const char* gf_kernel_name(int32_t kernel_id) {
+    return (kernel_id >= 0 && kernel_id < K_COUNT) ? kKernelNames[kernel_id] : nullptr;
+}
+
+int32_t gf_kernel_id_count(void) { return K_COUNT; }
 
 uint64_t gf_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

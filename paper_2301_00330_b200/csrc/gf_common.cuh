@@ -9,8 +9,22 @@
 
 namespace gf {
 
-// ---- launch accounting -----------------------------------------------------
+// ---- launch accounting and optional event timing -----------------------------
 void count_launch(int n = 1);
+
+enum KernelId {
+    K_STASH_POOL = 0, K_KSUM, K_GY_POOL, K_GX_MIX, K_GW_PARTIAL, K_GW_FINISH, K_DW_FUSED,
+    K_EXACT_GX, K_EXACT_GW, K_COUNT
+};
+
+// Brackets the launches made during its lifetime with a pair of events when
+// timing of this kernel id is switched on; otherwise does nothing.
+struct ProfScope {
+    int slot;
+    cudaStream_t stream;
+    ProfScope(int kernel_id, cudaStream_t s);
+    ~ProfScope();
+};
 
 #define GF_CUDA_TRY(expr)                         \
     do {                                          \
@@ -119,7 +133,7 @@ Workspace plan_workspace(const Geo& g);
 
 // ---- kernel entry points (host launchers) ----------------------------------
 // pool: out[plane, a, b] = sum (or mean) of in[plane] over patch (a,b)
-gf_status launch_pool(const void* in, int in_dtype, void* out, int out_dtype, bool mean,
+gf_status launch_pool(int kernel_id, const void* in, int in_dtype, void* out, int out_dtype, bool mean,
                       int64_t planes, int H, int W, int r, cudaStream_t s);
 gf_status launch_copy(const void* in, void* out, size_t bytes, cudaStream_t s);
 

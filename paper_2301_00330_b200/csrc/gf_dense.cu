@@ -20,6 +20,7 @@ __global__ void ksum_kernel(const T* __restrict__ W, float* __restrict__ tsum, i
 }
 
 gf_status launch_ksum(const void* W, const Geo& g, float* tsum, uint32_t* err_word, cudaStream_t s) {
+    ProfScope prof(K_KSUM, s);
     const int n_pairs = g.C_out * g.C_ig, taps = g.KH * g.KW;
     const int grid = (n_pairs + 255) / 256;
     if (g.dtype == GF_F32) ksum_kernel<float><<<grid, 256, 0, s>>>((const float*)W, tsum, n_pairs, taps, err_word);
@@ -108,6 +109,7 @@ __global__ void __launch_bounds__(256) gx_mix_kernel(const GxParams p) {
 }
 
 gf_status launch_gx_mix(const float* gbar, const float* tsum, void* gX, const Geo& g, cudaStream_t s) {
+    ProfScope prof(K_GX_MIX, s);
     GxParams p;
     p.gbar = gbar; p.tsum = tsum; p.gX = gX;
     p.N = g.N; p.C_in = g.C_in; p.C_out = g.C_out; p.G = g.G; p.C_ig = g.C_ig; p.C_og = g.C_og;
@@ -181,6 +183,7 @@ __global__ void __launch_bounds__(256) gw_partial_kernel(const GwParams p) {
 
 gf_status launch_gw_partial(const float* gbar, const void* stash, float* part, int splits,
                             const Geo& g, cudaStream_t s) {
+    ProfScope prof(K_GW_PARTIAL, s);
     GwParams p;
     p.gbar = gbar; p.stash = stash; p.part = part;
     p.N = g.N; p.C_in = g.C_in; p.C_out = g.C_out; p.G = g.G; p.C_ig = g.C_ig; p.C_og = g.C_og;
@@ -205,6 +208,7 @@ __global__ void gw_finish_kernel(const float* __restrict__ part, int S, size_t n
 }
 
 gf_status launch_gw_finish(const float* part, int splits, float* gW, const Geo& g, cudaStream_t s) {
+    ProfScope prof(K_GW_FINISH, s);
     const size_t n_pairs = (size_t)g.C_out * g.C_ig;
     const int taps = g.KH * g.KW;
     const size_t total = n_pairs * taps;

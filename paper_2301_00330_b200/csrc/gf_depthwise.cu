@@ -166,6 +166,7 @@ gf_status launch_depthwise(const void* gy, const void* stash, const void* W, flo
                            void* gX, uint32_t* err_word, const Geo& g, int* splits_out, cudaStream_t s) {
     const DwPlan d = dw_plan(g);
     if (!d.ok) return GF_ERR_UNSUPPORTED;
+    ProfScope prof(K_DW_FUSED, s);
     DwParams p;
     p.gy = gy; p.stash = stash; p.W = W; p.part = part; p.gX = gX; p.err_word = err_word;
     p.planes = (long long)g.N * g.C_in; p.total_elems = p.planes * g.H * g.W;

@@ -70,6 +70,7 @@ __global__ void __launch_bounds__(256) exact_gw_kernel(const T* __restrict__ gy,
 gf_status launch_exact(const void* gy, const void* x, const void* W, float* gW, void* gX,
                        const Geo& g, cudaStream_t s) {
     if (gX) {
+        ProfScope prof(K_EXACT_GX, s);
         const long long total = (long long)g.N * g.C_in * g.H * g.W;
         const long long blocks = (total + 255) / 256;
         if (blocks > 0x7fffffffLL) return GF_ERR_UNSUPPORTED;
@@ -84,6 +85,7 @@ gf_status launch_exact(const void* gy, const void* x, const void* W, float* gW, 
         if (st != GF_OK) return st;
     }
     if (gW) {
+        ProfScope prof(K_EXACT_GW, s);
         const long long blocks = (long long)g.C_out * g.C_ig * g.KH * g.KW;
         if (blocks > 0x7fffffffLL) return GF_ERR_UNSUPPORTED;
         if (g.dtype == GF_F32)

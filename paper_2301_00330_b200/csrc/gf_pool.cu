@@ -139,8 +139,9 @@ static gf_status pool_dispatch(const PoolParams& p, long long tiles, bool big, c
     return after_launch();
 }
 
-gf_status launch_pool(const void* in, int in_dtype, void* out, int out_dtype, bool mean,
+gf_status launch_pool(int kernel_id, const void* in, int in_dtype, void* out, int out_dtype, bool mean,
                       int64_t planes, int H, int W, int r, cudaStream_t s) {
+    ProfScope prof(kernel_id, s);
     PoolParams p;
     p.in = in; p.out = out; p.planes = planes; p.total_elems = planes * H * W;
     p.H = H; p.W = W; p.r = r;

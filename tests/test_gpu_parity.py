@@ -1,0 +1,121 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 CPU
+oracle on the same seeded inputs.  Small cases are compared element by element;
+the full-size benchmark configurations on sampled outputs and on properties."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2301_00330_b200 import workloads
+from paper_2301_00330_b200.workloads import Layer
+
+from parity_util import TOL, check_layer_full, check_layer_sampled, f64, relerr, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+def L(name, N, Cin, Cout, H, W, K, G, r, dtype="f32", x_dist="relu", gy_std=1e-2, idx=0):
+    return Layer(name, 0, idx, N, Cin, Cout, H, W, K, G, r, dtype, x_dist, gy_std)
+
+
+SMALL = [
+    L("tile_multi", 3, 24, 40, 14, 14, 3, 1, 2),
+    L("partial_patches_r4", 3, 24, 40, 14, 14, 3, 1, 4),
+    L("odd_map_7x7", 2, 8, 8, 7, 7, 3, 1, 2),
+    L("ragged_channels", 2, 70, 130, 9, 11, 3, 1, 2),
+    L("ragged_channels_1x1", 2, 130, 70, 12, 20, 1, 1, 4),
+    L("r_gt_H", 1, 6, 4, 5, 5, 1, 2, 8),
+    L("r3_generic", 2, 16, 16, 12, 9, 3, 1, 3),
+    L("r7", 2, 16, 24, 32, 32, 3, 1, 7),
+    L("k5", 2, 8, 12, 16, 16, 5, 1, 4),
+    L("groups2", 2, 16, 24, 10, 10, 3, 2, 2),
+    L("groups4_ragged", 3, 20, 12, 9, 9, 3, 4, 2),
+    L("dw_r2", 2, 12, 12, 28, 28, 3, 12, 2),
+    L("dw_r4", 2, 12, 12, 28, 28, 3, 12, 4),
+    L("dw_r7", 2, 12, 12, 20, 20, 3, 12, 7),
+    L("dw_odd", 3, 5, 5, 7, 9, 3, 5, 2),
+    L("band_mode", 1, 3, 2, 160, 120, 3, 1, 2),
+    L("band_mode_r8_ragged", 1, 2, 3, 100, 120, 3, 1, 8),
+    L("dw_band_mode", 1, 4, 4, 160, 120, 3, 4, 4),
+    L("big_patch", 1, 2, 2, 16, 600, 3, 1, 8),
+    L("dw_big_patch", 1, 3, 3, 40, 4100, 3, 3, 40),
+    L("n1", 1, 32, 32, 16, 16, 3, 1, 2),
+    L("wide_map", 1, 8, 8, 6, 200, 3, 1, 2),
+]
+
+
+@pytest.mark.parametrize("layer", SMALL, ids=lambda l: l.name)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_small_shapes_element_by_element(gf, layer, dtype):
+    check_layer_full(gf, layer.with_(dtype=dtype))
+
+
+def test_config1_r2_and_r1_exact(gf):
+    (l2,) = workloads.config1(2)
+    check_layer_full(gf, l2)
+    (l1,) = workloads.config1(1)
+    errs = check_layer_full(gf, l1)
+    assert errs["stash"] == 0.0          # r == 1: the stash is x itself
+
+
+def test_r1_exact_other_shapes(gf):
+    for layer in (L("r1_groups", 2, 8, 12, 9, 7, 3, 2, 1), L("r1_k5", 1, 4, 4, 8, 8, 5, 1, 1),
+                  L("r1_dw", 2, 6, 6, 8, 8, 3, 6, 1), L("r1_bf16", 2, 8, 8, 8, 8, 3, 1, 1, "bf16")):
+        check_layer_full(gf, layer)
+
+
+def test_nullable_outputs_and_repeatability(gf):
+    layer = L("nullable", 2, 24, 40, 14, 14, 3, 1, 2)
+    x, gy, w = workloads.make_inputs(layer)
+    _, gW_a, gX_a = run_gpu(gf, layer, x, gy, w)
+    _, gW_b, _ = run_gpu(gf, layer, x, gy, w, need_gx=False)
+    _, _, gX_c = run_gpu(gf, layer, x, gy, w, need_gw=False)
+    assert relerr(f64(gW_b), f64(gW_a)) <= TOL["f32"]
+    assert torch.equal(gX_a, gX_c)
+    for _ in range(2):
+        _, gW_d, gX_d = run_gpu(gf, layer, x, gy, w)
+        assert relerr(f64(gW_d), f64(gW_a)) <= TOL["f32"] and torch.equal(gX_d, gX_a)
+
+
+def test_host_buffer_step_matches_device_path(gf):
+    layer = L("host_step", 2, 24, 40, 14, 14, 3, 1, 2, "bf16")
+    x, gy, w = workloads.make_inputs(layer)
+    desc = gf.desc_for(layer)
+    _, gW_dev, gX_dev = run_gpu(gf, layer, x, gy, w)
+    hx, hgy, hw = x.pin_memory(), gy.pin_memory(), w.pin_memory()
+    h_gW = torch.empty(gW_dev.shape, dtype=torch.float32).pin_memory()
+    h_gX = torch.empty(gX_dev.shape, dtype=torch.bfloat16).pin_memory()
+    arena = torch.empty(gf.gf_host_step_arena_bytes(desc), dtype=torch.uint8, device="cuda")
+    gf.gf_layer_step_host(desc, hx, hgy, hw, h_gW, h_gX, arena)
+    torch.cuda.synchronize()
+    assert relerr(f64(h_gW), f64(gW_dev)) <= 1e-6
+    assert torch.equal(h_gX, gX_dev.cpu())
+
+
+# ---- the benchmark configurations at full size, in the launch configuration bench.py times ----
+FULL = (workloads.config2() + workloads.config3(2) + workloads.config3(4) + workloads.config4()
+        + [l for dt in ("f32", "bf16") for r in (2, 4, 8) for l in workloads.config5(r, dt)])
+
+
+@pytest.mark.parametrize("layer", FULL, ids=lambda l: f"{l.name}_r{l.r}_{l.dtype}")
+def test_full_size_configs_sampled(gf, layer):
+    check_layer_sampled(gf, layer)
+
+
+def test_ondevice_table_shapes_sampled(gf):
+    """The seven layer shapes of the paper's on-device latency table (batch 32,
+    3x3, stride 1, pad 1); 14x14 with r = 4 has partial patches."""
+    for layer in workloads.ondevice_table(r=4, N=8):
+        check_layer_sampled(gf, layer, n_ch=4, n_img=1)
+
+
+def test_oracle_disagrees_when_a_mistake_is_planted(gf):
+    """The comparison is sharp enough to see a wrong patch divisor planted on the
+    CPU side: the zero-padded average (divide by r^2 on partial patches)."""
+    layer = L("planted", 2, 8, 8, 7, 7, 3, 1, 2)
+    x, gy, w = workloads.make_inputs(layer)
+    _, _, gX = run_gpu(gf, layer, x, gy, w)
+    gsum = oracle.patch_sum(f64(gy), 2)
+    wrong_mean = gsum / 4.0
+    gx_wrong = oracle.reduced_gx(wrong_mean, oracle.kernel_sum(f64(w)), 1, 7, 7, 2)
+    assert relerr(f64(gX), gx_wrong) > 100 * TOL["f32"]
