@@ -1,0 +1,384 @@
+#!/usr/bin/env python
+"""Benchmark of the filtered convolution backward pass (gradient filtering).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = one pass of the whole hot path over one batch of one layer:
+gf_stash_forward (patch-summed activations) + gf_backward (gradient filter,
+reduced g_W, reduced g_X with expansion), on the ResNet-style layer
+3x3, 256->256, N=64, 28x28, r=2, bf16 inputs with fp32 accumulation.
+Prints ONE JSON line (rank 0).  The metric is microseconds per layer backward
+(lower is better).  N > 1: independent replicas, one per GPU, no collective on
+the data path; the value is time divided by the layers all ranks processed.
+
+--impl reference times the fp64 CPU checker (oracle/) on the host cores on a
+bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "filtered_conv_backward_us_per_layer"
+UNIT = "us"
+FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # SMs x FMA lanes x 2 flop x max SM clock
+
+# DRAM bytes per launch of a kernel from one ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum), keyed by kernel name, with the sha1 of the source file
+# at capture time; a changed source makes the entry stale (reported as null).
+NCU_TRAFFIC: dict[str, dict] = {}
+
+KERNEL_SOURCE = {
+    "stash_pool": "gf_pool.cu", "gy_pool": "gf_pool.cu", "ksum": "gf_dense.cu", "gx_mix": "gf_dense.cu",
+    "gw_partial": "gf_dense.cu", "gw_finish": "gf_dense.cu", "dw_fused": "gf_depthwise.cu",
+}
+
+
+def measured_peaks() -> tuple[dict, str]:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return ({"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                 "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"]))}, "measured")
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, "fallback"
+
+
+def workload():
+    from paper_2301_00330_b200 import workloads
+    (layer,) = workloads.config2()
+    return layer
+
+
+def workload_config(layer, extra=None) -> dict:
+    cfg = {
+        "workload": "configs[1]: ResNet-style 3x3 conv backward, stride 1, pad 1, N=64, 256->256, 28x28, r=2",
+        "layer": layer.name, "N": layer.N, "C_in": layer.C_in, "C_out": layer.C_out, "H": layer.H,
+        "W": layer.W, "K": layer.K, "groups": layer.groups, "r": layer.r,
+        "step": "gf_stash_forward + gf_backward (g_W and g_X)",
+    }
+    if extra:
+        cfg.update(extra)
+    return cfg
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the GPU works."""
+
+    def __init__(self, index: int):
+        self.samples = []
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def sample(self):
+        if not self.nv:
+            return
+        try:
+            mhz = self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM)
+            reasons = self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.h) \
+                if hasattr(self.nv, "nvmlDeviceGetCurrentClocksEventReasons") \
+                else self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+            self.samples.append((mhz, int(reasons)))
+        except Exception:
+            pass
+
+    def _run(self):
+        while not self._stop.is_set():
+            self.sample()
+            time.sleep(0.01)
+
+    def start(self):
+        self.samples = []
+        self._stop.clear()
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
+
+    def stop(self) -> dict:
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"]}
+        mhz = sorted(s[0] for s in self.samples)
+        bits = 0
+        for _, r in self.samples:
+            bits |= r
+        names = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+                 0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+                 0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+        reasons = [n for b, n in names.items() if bits & b and n != "gpu_idle"]
+        return {"sm_mhz": mhz[len(mhz) // 2], "sm_max_mhz": self.max_mhz, "reasons": reasons,
+                "samples": len(mhz)}
+
+
+# --------------------------------------------------------------------------- roofline
+def kernel_cost(name: str, L, splits: int) -> tuple[float, float]:
+    """(algorithmic bytes, flops) of one launch of kernel `name` on layer L."""
+    e = L.elem_bytes
+    gbar = 4 * L.N * L.C_out * L.Hp * L.Wp
+    pairs = L.C_out * L.C_ig
+    M = L.N * L.Hp * L.Wp
+    mix = 2.0 * M * L.C_out * L.C_ig
+    table = {
+        "stash_pool": (e * (L.numel_x() + L.numel_stash()), L.numel_x()),
+        "gy_pool": (e * L.numel_gy() + gbar, L.numel_gy()),
+        "ksum": (e * L.numel_w() + 4 * pairs, L.numel_w()),
+        "gx_mix": (gbar + 4 * pairs + e * L.numel_x(), mix),
+        "gw_partial": (gbar + e * L.numel_stash() + 4 * splits * pairs, mix),
+        "gw_finish": (4 * splits * pairs + 4 * L.numel_w(), splits * pairs),
+        "dw_fused": (e * (L.numel_gy() + L.numel_stash() + L.numel_x() + L.numel_w()), 3 * L.numel_gy()),
+    }
+    return table[name]
+
+
+def traffic_for(name: str):
+    ent = NCU_TRAFFIC.get(name)
+    src = KERNEL_SOURCE.get(name)
+    if not ent or not src:
+        return None
+    path = os.path.join(ROOT, "paper_2301_00330_b200", "csrc", src)
+    with open(path, "rb") as f:
+        sha = hashlib.sha1(f.read()).hexdigest()
+    return ent["bytes"] if sha == ent.get("sha1") else None
+
+
+def roofline(name: str, avg_ms: float, L, splits: int) -> dict:
+    peaks, which = measured_peaks()
+    nbytes, flops = kernel_cost(name, L, splits)
+    t = avg_ms * 1e-3
+    t_mem = nbytes / (peaks["hbm_gbs"] * 1e9)
+    t_alu = flops / (FP32_ALU_TFLOPS * 1e12)
+    if t_alu > t_mem and name in ("gx_mix", "gw_partial"):
+        ach = flops / t / 1e12
+        return {"kernel": name, "bound": "alu", "achieved": ach, "peak": FP32_ALU_TFLOPS, "unit": "TFLOP/s",
+                "frac": ach / FP32_ALU_TFLOPS, "traffic": traffic_for(name), "peak_source": "derived: 148 SM x 128 FMA x 2 x 1.965 GHz",
+                "avg_launch_us": avg_ms * 1e3}
+    ach = nbytes / t / 1e9
+    return {"kernel": name, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": ach / peaks["hbm_gbs"], "traffic": traffic_for(name), "peak_source": f"of {which}",
+            "avg_launch_us": avg_ms * 1e3}
+
+
+# --------------------------------------------------------------------------- CPU checker timing
+def time_oracle(layer, n_sample: int, steps: int, warmup: int) -> dict:
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2301_00330_b200 import workloads
+    L = layer.with_(N=n_sample)
+    x, gy, w = workloads.make_inputs(L)
+    x64, gy64, w64 = (t.to(torch.float64).numpy() for t in (x, gy, w))
+
+    def one():
+        stash = oracle.stash_forward(x64, L.r)
+        return oracle.backward(gy64, stash, w64, L.r, groups=L.groups)
+
+    for _ in range(warmup):
+        one()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        gw, gx = one()
+    dt = (time.perf_counter() - t0) / steps
+    assert np.isfinite(gw).all() and np.isfinite(gx).all()
+    scale = layer.N / n_sample
+    return {"value": dt * 1e6 * scale, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{n_sample} of {layer.N} images of the same layer, fp64, time scaled x{scale:g} "
+                      f"(every step is linear in the batch); {steps} timed passes",
+            "seconds_per_pass": dt}
+
+
+def run_reference(args) -> None:
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    layer = workload()
+    base = time_oracle(layer, layer.N, max(1, args.steps), max(0, args.warmup))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": base["value"] / 1e3,
+        "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": workload_config(layer, {"dtype_in": "bf16 values widened to f64"}),
+        "cpu_baseline": base,
+        "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------- GPU arm
+def run_ours(args) -> None:
+    import torch
+    import paper_2301_00330_b200 as gf
+    from paper_2301_00330_b200 import workloads
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    gf.build_library()
+
+    layer = workload()
+    desc = gf.desc_for(layer)
+    dt = workloads.torch_dtype(layer.dtype)
+    x0, gy0, w0 = workloads.make_inputs(layer)
+    n_sets = 4   # rotating input/output sets: 4 x ~106 MB > 3 x the 126 MB L2
+    sets = []
+    for i in range(n_sets):
+        buf = gf.alloc_layer(desc)
+        sets.append((torch.roll(x0, i, 0).cuda().contiguous(), torch.roll(gy0, i, 0).cuda().contiguous(), buf))
+    w = w0.cuda()
+    ws_bytes = gf.gf_backward_workspace_bytes(desc)
+    set_bytes = sum(t.numel() * t.element_size() for t in (sets[0][0], sets[0][1], sets[0][2].stash,
+                                                            sets[0][2].g_X, sets[0][2].g_W, sets[0][2].workspace))
+    stream = torch.cuda.current_stream()
+
+    def step(i: int):
+        x, gy, b = sets[i % n_sets]
+        gf.gf_stash_forward(desc, x, b.stash, stream)
+        gf.gf_backward(desc, gy, b.stash, w, b.g_W, b.g_X, b.workspace, ws_bytes, stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- warm-up; its first steps bracket every kernel to find the dominant one ----
+    warm = max(3, args.warmup)
+    diag_steps = min(warm, 8)
+    gf.gf_profile_configure(2)
+    for i in range(diag_steps):
+        step(i)
+    torch.cuda.synchronize()
+    diag = gf.gf_profile_read()
+    gf.gf_profile_configure(0)
+    for i in range(warm - diag_steps):
+        step(i)
+    torch.cuda.synchronize()
+    total_diag = sum(ms for _, ms in diag.values()) or 1.0
+    breakdown = {k: {"launches_per_step": n / diag_steps, "avg_us": ms / n * 1e3, "share": ms / total_diag}
+                 for k, (n, ms) in diag.items()}
+    dominant = max(diag.items(), key=lambda kv: kv[1][1])[0]
+
+    # ---- timed region: K steps; only the dominant kernel carries event pairs ----
+    sampler = ClockSampler(local_rank)
+    gf.gf_profile_configure(1, gf.kernel_id(dominant))
+    launches0 = gf.gf_kernel_launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.start()
+    ev0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    ev1.record(stream)
+    sampler.sample()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    barrier()
+    launches = gf.gf_kernel_launch_count() - launches0
+    ms_total = ev0.elapsed_time(ev1)
+    dom = gf.gf_profile_read()
+    gf.gf_profile_configure(0)
+    assert gf.gf_last_async_status(sets[0][2].workspace) == gf.GF_OK
+    if dist is not None:
+        t = torch.tensor([ms_total], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    value = ms_total * 1e3 / (args.steps * world)      # us per layer over all ranks' layers
+
+    # ---- end to end: host buffers in, host buffers out, through the C ABI ----
+    hx, hgy, hw = x0.pin_memory(), gy0.pin_memory(), w0.pin_memory()
+    h_gW = torch.empty((layer.C_out, layer.C_ig, layer.K, layer.K), dtype=torch.float32).pin_memory()
+    h_gX = torch.empty(tuple(x0.shape), dtype=dt).pin_memory()
+    arena = torch.empty(gf.gf_host_step_arena_bytes(desc), dtype=torch.uint8, device="cuda")
+    e2e_steps = max(1, min(args.steps, 30))
+    for _ in range(2):
+        gf.gf_layer_step_host(desc, hx, hgy, hw, h_gW, h_gX, arena, stream=stream)
+    barrier()
+    ev0.record(stream)
+    for _ in range(e2e_steps):
+        gf.gf_layer_step_host(desc, hx, hgy, hw, h_gW, h_gX, arena, stream=stream)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = ev0.elapsed_time(ev1)
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    h2d = sum(t.numel() * t.element_size() for t in (hx, hgy, hw))
+    d2h = sum(t.numel() * t.element_size() for t in (h_gW, h_gX))
+    e2e = {"value": e2e_ms * 1e3 / (e2e_steps * world), "unit": UNIT, "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": d2h, "steps": e2e_steps, "api": "gf_layer_step_host (pinned host buffers)"}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # split count of the reduced g_W contraction, needed for its byte count
+    tiles = ((layer.C_out // layer.groups + 63) // 64) * ((layer.C_ig + 63) // 64) * layer.groups
+    splits = max(1, min(layer.N, -(-592 // tiles)))
+    n_dom, ms_dom = dom.get(dominant, (0, 0.0))
+    roof = roofline(dominant, ms_dom / max(n_dom, 1), layer, splits)
+    roof["timed_launches"] = n_dom
+    peaks, which = measured_peaks()
+    step_bytes = layer.backward_bytes() + layer.stash_bytes_moved()
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": workload_config(layer, {
+            "l2": f"inputs and outputs rotate over {n_sets} sets of {set_bytes / 1e6:.0f} MB (> 3x the 126 MB L2)",
+            "parallelism": "replicas only" if world > 1 else "single GPU"}),
+        "step_algorithmic_bytes": step_bytes,
+        "step_gbs": step_bytes / (ms_per_step * 1e-3) / 1e9,
+        "step_frac_of_hbm": step_bytes / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
+        "peaks": {"hbm_gbs": peaks["hbm_gbs"], "source": which},
+        "roofline": roof, "kernels": breakdown, "clocks": clocks, "e2e": e2e,
+        "gpu_launches": int(launches),
+    }
+    if world == 1:
+        line["cpu_baseline"] = time_oracle(layer, layer.N, 5, 1)
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
