@@ -96,8 +96,9 @@ gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* sta
                       size_t workspace_bytes, void* stream);
 
 /* Reads the error word that device-side bounded waits of the last gf_backward
- * on `workspace` may have set.  Synchronises `stream` (blocking).  GF_OK if no
- * wait expired. */
+ * on `workspace` may have set, and the library-wide word that gf_stash_forward
+ * reports to (cleared by this call).  Synchronises `stream` (blocking).  GF_OK
+ * if no wait expired. */
 gf_status gf_last_async_status(const void* workspace, void* stream);
 
 /* One training-side step for a layer with every tensor in HOST memory

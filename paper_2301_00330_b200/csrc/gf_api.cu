@@ -43,6 +43,23 @@ ProfScope::~ProfScope() {
     if (slot >= 0) cudaEventRecord(g_prof_ev[slot][1], stream);
 }
 
+// ---- error word for kernels that run without a workspace ---------------------------
+// Device-side bounded waits report here when the call has no workspace of its own
+// (gf_stash_forward).  The address is looked up once per device.
+static __device__ uint32_t g_err_word_dev;
+
+static uint32_t* global_err_word() {
+    static uint32_t* cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!cached[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_err_word_dev) != cudaSuccess) return nullptr;
+        cached[dev] = static_cast<uint32_t*>(ptr);
+    }
+    return cached[dev];
+}
+
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 Geo make_geo(const gf_conv_desc& d) {
@@ -145,7 +162,9 @@ gf_status gf_stash_forward(const gf_conv_desc* desc, const void* x, void* stash,
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int64_t planes = (int64_t)g.N * g.C_in;
     if (g.r == 1) return launch_copy(x, stash, (size_t)planes * g.H * g.W * g.esize, s);
-    return launch_pool(K_STASH_POOL, x, g.dtype, stash, g.dtype, /*mean=*/false, planes, g.H, g.W, g.r, s);
+    uint32_t* err = global_err_word();
+    if (!err) return GF_ERR_CUDA;
+    return launch_pool(K_STASH_POOL, x, g.dtype, stash, g.dtype, /*mean=*/false, planes, g.H, g.W, g.r, err, s);
 }
 
 gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* stash, const void* W,
@@ -186,7 +205,7 @@ gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* sta
     // patch means of g_y, read once
     st = launch_ksum(W, g, tsum, err, s);
     if (st != GF_OK) return st;
-    st = launch_pool(K_GY_POOL, g_y, g.dtype, gbar, GF_F32, /*mean=*/true, (int64_t)g.N * g.C_out, g.H, g.W, g.r, s);
+    st = launch_pool(K_GY_POOL, g_y, g.dtype, gbar, GF_F32, /*mean=*/true, (int64_t)g.N * g.C_out, g.H, g.W, g.r, err, s);
     if (st != GF_OK) return st;
     if (g_X) {
         st = launch_gx_mix(gbar, tsum, g_X, g, s);
@@ -204,10 +223,17 @@ gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* sta
 gf_status gf_last_async_status(const void* workspace, void* stream) {
     if (!workspace) return GF_ERR_NULL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    uint32_t word = 0;
+    uint32_t* gerr = global_err_word();
+    if (!gerr) return GF_ERR_CUDA;
+    uint32_t word = 0, gword = 0;
     GF_CUDA_TRY(cudaMemcpyAsync(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost, s));
+    GF_CUDA_TRY(cudaMemcpyAsync(&gword, gerr, sizeof(gword), cudaMemcpyDeviceToHost, s));
     GF_CUDA_TRY(cudaStreamSynchronize(s));
-    return word == 0 ? GF_OK : GF_ERR_TIMEOUT;
+    if (gword != 0) {   // sticky until read: clear it for the next call
+        GF_CUDA_TRY(cudaMemsetAsync(gerr, 0, sizeof(uint32_t), s));
+        GF_CUDA_TRY(cudaStreamSynchronize(s));
+    }
+    return (word | gword) == 0 ? GF_OK : GF_ERR_TIMEOUT;
 }
 
 // ---- host-buffer step ---------------------------------------------------------

@@ -134,7 +134,7 @@ Workspace plan_workspace(const Geo& g);
 // ---- kernel entry points (host launchers) ----------------------------------
 // pool: out[plane, a, b] = sum (or mean) of in[plane] over patch (a,b)
 gf_status launch_pool(int kernel_id, const void* in, int in_dtype, void* out, int out_dtype, bool mean,
-                      int64_t planes, int H, int W, int r, cudaStream_t s);
+                      int64_t planes, int H, int W, int r, uint32_t* err_word, cudaStream_t s);
 gf_status launch_copy(const void* in, void* out, size_t bytes, cudaStream_t s);
 
 gf_status launch_ksum(const void* W, const Geo& g, float* tsum, uint32_t* err_word, cudaStream_t s);

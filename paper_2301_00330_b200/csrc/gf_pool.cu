@@ -2,76 +2,259 @@
 // Section 3.4 / 4.3) and the gradient filter (patch MEAN of g_y, Section 3.3).
 //
 // A tile is one contiguous range of global memory: either P whole planes (small
-// maps) or a band of whole patch-rows of one plane (large maps).  The range is
-// staged in shared memory with 128-bit streaming loads, the patches are reduced
-// from there in fp32, and the outputs of a tile are one contiguous range too.
+// maps) or a band of whole patch-rows of one plane (large maps); its outputs are
+// one contiguous range too.
+//
+//  pool_stream_kernel   r in {2,4,8} dividing W: persistent CTAs, one per SM.  The
+//                       copy engine (cp.async.bulk) fills a ring of shared-memory
+//                       tiles several tiles ahead; threads reduce G adjacent
+//                       patches each from 8/16-byte shared loads and write vectors.
+//  pool_tile_kernel     any r, any alignment: one tile per CTA, staged with
+//                       128-bit loads.
+//  pool_bigpatch_kernel patches too large for a tile: one CTA per output value.
 #include "gf_common.cuh"
+#include "gf_pipe.cuh"
 
 namespace gf {
 
 constexpr int kPoolThreads = 256;
 constexpr int kPoolTileBytes = 16384;
 
+constexpr int kStreamThreads = 512;
+constexpr int kStreamTileBytes = 32768;
+constexpr int kStreamStages = 4;
+
 struct PoolParams {
     const void* in;
     void* out;
-    long long planes, total_elems;
+    uint32_t* err_word;
+    long long planes, total_elems, tiles;
     int H, W, r, Hp, Wp;
     int P;       // planes per tile
     int BR;      // patch rows per tile (== Hp when P > 1)
     int bands;   // tiles along the patch rows of one plane (1 when P > 1)
+    int mean;    // 1: patch mean, 0: patch sum
     FastDiv div_bands, div_plane_out /* Hp*Wp */, div_Wp;
     float inv_full;  // 1 / r^2
 };
 
-template <typename TIn, typename TOut, int R, bool MEAN>
-__global__ void __launch_bounds__(kPoolThreads) pool_tile_kernel(const PoolParams p) {
-    constexpr int VE = 16 / (int)sizeof(TIn);
-    __shared__ uint4 smem_v[kPoolTileBytes / 16 + 1];
-    TIn* smem = reinterpret_cast<TIn*>(smem_v);
-    const TIn* __restrict__ in = static_cast<const TIn*>(p.in);
-    TOut* __restrict__ out = static_cast<TOut*>(p.out);
+// ---- NE consecutive shared-memory elements as floats -----------------------------
+template <int NE> __device__ __forceinline__ void load_span(const float* p, float (&v)[NE]) {
+    if constexpr (NE >= 4) {
+#pragma unroll
+        for (int i = 0; i < NE / 4; ++i) {
+            const float4 t = reinterpret_cast<const float4*>(p)[i];
+            v[4 * i] = t.x; v[4 * i + 1] = t.y; v[4 * i + 2] = t.z; v[4 * i + 3] = t.w;
+        }
+    } else {
+        const float2 t = *reinterpret_cast<const float2*>(p);
+        v[0] = t.x; v[1] = t.y;
+    }
+}
+__device__ __forceinline__ void unpack_bf16x2(uint32_t u, float& lo, float& hi) {
+    lo = __uint_as_float(u << 16);
+    hi = __uint_as_float(u & 0xffff0000u);
+}
+template <int NE> __device__ __forceinline__ void load_span(const __nv_bfloat16* p, float (&v)[NE]) {
+    if constexpr (NE >= 8) {
+#pragma unroll
+        for (int i = 0; i < NE / 8; ++i) {
+            const uint4 t = reinterpret_cast<const uint4*>(p)[i];
+            unpack_bf16x2(t.x, v[8 * i], v[8 * i + 1]); unpack_bf16x2(t.y, v[8 * i + 2], v[8 * i + 3]);
+            unpack_bf16x2(t.z, v[8 * i + 4], v[8 * i + 5]); unpack_bf16x2(t.w, v[8 * i + 6], v[8 * i + 7]);
+        }
+    } else if constexpr (NE == 4) {
+        const uint2 t = *reinterpret_cast<const uint2*>(p);
+        unpack_bf16x2(t.x, v[0], v[1]); unpack_bf16x2(t.y, v[2], v[3]);
+    } else {
+        unpack_bf16x2(*reinterpret_cast<const uint32_t*>(p), v[0], v[1]);
+    }
+}
 
+// ---- G consecutive outputs ---------------------------------------------------------
+template <int G> __device__ __forceinline__ void store_vec(float* dst, const float (&a)[G]) {
+    if constexpr (G == 4) *reinterpret_cast<float4*>(dst) = make_float4(a[0], a[1], a[2], a[3]);
+    else if constexpr (G == 2) *reinterpret_cast<float2*>(dst) = make_float2(a[0], a[1]);
+    else *dst = a[0];
+}
+template <int G> __device__ __forceinline__ void store_vec(__nv_bfloat16* dst, const float (&a)[G]) {
+    if constexpr (G == 4) {
+        __nv_bfloat162 lo = __floats2bfloat162_rn(a[0], a[1]), hi = __floats2bfloat162_rn(a[2], a[3]);
+        uint2 t;
+        t.x = *reinterpret_cast<uint32_t*>(&lo); t.y = *reinterpret_cast<uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(dst) = t;
+    } else if constexpr (G == 2) {
+        *reinterpret_cast<__nv_bfloat162*>(dst) = __floats2bfloat162_rn(a[0], a[1]);
+    } else {
+        *dst = __float2bfloat16_rn(a[0]);
+    }
+}
+
+// ---- tile geometry (shared by the two tiled kernels) ------------------------------
+struct Tile { long long g0, out_base; int len, np, a0, na; };
+__device__ __forceinline__ Tile tile_of(const PoolParams& p, long long t) {
+    Tile g;
     uint32_t pg, band;
-    p.div_bands.divmod(blockIdx.x, pg, band);
+    p.div_bands.divmod((uint32_t)t, pg, band);
     const long long p0 = (long long)pg * p.P;
-    const int np = (int)min((long long)p.P, p.planes - p0);
-    const int a0 = band * p.BR;
-    const int na = min(p.BR, p.Hp - a0);
-    const int i0 = a0 * p.r;
-    const int i1 = min((a0 + na) * p.r, p.H);
+    g.np = (int)min((long long)p.P, p.planes - p0);
+    g.a0 = band * p.BR;
+    g.na = min(p.BR, p.Hp - g.a0);
+    const int i0 = g.a0 * p.r;
+    const int i1 = min((g.a0 + g.na) * p.r, p.H);
     const long long plane_elems = (long long)p.H * p.W;
-    const long long g0 = p0 * plane_elems + (long long)i0 * p.W;
-    const int len = (np - 1) * (int)plane_elems + (i1 - i0) * p.W;
+    g.g0 = p0 * plane_elems + (long long)i0 * p.W;
+    g.len = (g.np - 1) * (int)plane_elems + (i1 - i0) * p.W;
+    g.out_base = p0 * (long long)(p.Hp * p.Wp) + (long long)g.a0 * p.Wp;
+    return g;
+}
 
-    // ---- stage the range [g0, g0 + len) ----
+// Stages [g0, g0+len) with 128-bit loads; element k of the range lands at
+// smem[shift + k], shift = g0 mod (elements per 16 bytes).  Returns shift.
+template <typename TIn, int THREADS>
+__device__ __forceinline__ int stage_plain(const TIn* __restrict__ in, long long total_elems, long long g0, int len,
+                                           uint4* smem_v) {
+    constexpr int VE = 16 / (int)sizeof(TIn);
+    TIn* smem = reinterpret_cast<TIn*>(smem_v);
     const long long v0 = g0 / VE;
     const int shift = (int)(g0 - v0 * VE);
     const int nvec = (shift + len + VE - 1) / VE;
-    const long long full_vecs = p.total_elems / VE;
+    const long long full_vecs = total_elems / VE;
+    const int nfast = (int)min((long long)nvec, full_vecs - v0);   // vectors wholly inside the tensor
     const uint4* gv = reinterpret_cast<const uint4*>(in) + v0;
-    for (int v = threadIdx.x; v < nvec; v += kPoolThreads) {
-        if (v0 + v < full_vecs) {
-            smem_v[v] = __ldcs(gv + v);
-        } else {
-            for (int e = 0; e < VE; ++e) {
-                const long long idx = (v0 + v) * VE + e;
-                smem[v * VE + e] = idx < p.total_elems ? in[idx] : from_f32<TIn>(0.f);
+    for (int v = threadIdx.x; v < nfast; v += 4 * THREADS) {
+        uint4 t[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (v + u * THREADS < nfast) t[u] = __ldcs(gv + v + u * THREADS);
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (v + u * THREADS < nfast) smem_v[v + u * THREADS] = t[u];
+    }
+    for (int v = nfast + threadIdx.x; v < nvec; v += THREADS)
+        for (int e = 0; e < VE; ++e) {
+            const long long idx = (v0 + v) * VE + e;
+            smem[v * VE + e] = idx < total_elems ? in[idx] : from_f32<TIn>(0.f);
+        }
+    return shift;
+}
+
+// ---- streamed kernel ------------------------------------------------------------------
+template <typename TIn, typename TOut, int R, int G>
+__device__ __forceinline__ void reduce_tile_vec(const PoolParams& p, const Tile& g, const TIn* buf,
+                                                TOut* __restrict__ out) {
+    const int nitems = g.np * g.na * p.Wp / G;
+    for (int q = threadIdx.x; q < nitems; q += kStreamThreads) {
+        const uint32_t o = q * G;
+        uint32_t pl = 0, rem = o;
+        if (p.P > 1) p.div_plane_out.divmod(o, pl, rem);
+        uint32_t al, b;
+        p.div_Wp.divmod(rem, al, b);
+        const int nr = min(R, p.H - (g.a0 + (int)al) * R);
+        const TIn* src = buf + ((int)pl * p.H + (int)al * R) * p.W + (int)b * R;
+        float acc[G];
+#pragma unroll
+        for (int k = 0; k < G; ++k) acc[k] = 0.f;
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+            if (i < nr) {
+                float v[G * R];
+                load_span<G * R>(src + i * p.W, v);
+#pragma unroll
+                for (int k = 0; k < G; ++k) {
+                    float s = v[k * R];
+#pragma unroll
+                    for (int j = 1; j < R; ++j) s += v[k * R + j];
+                    acc[k] += s;
+                }
             }
         }
+        if (p.mean) {
+            const float sc = nr == R ? p.inv_full : 1.0f / (float)(nr * R);
+#pragma unroll
+            for (int k = 0; k < G; ++k) acc[k] *= sc;
+        }
+        store_vec<G>(out + g.out_base + o, acc);
+    }
+}
+
+template <typename TIn, typename TOut, int R, int G>
+__global__ void __launch_bounds__(kStreamThreads, 1) pool_stream_kernel(const PoolParams p) {
+    extern __shared__ __align__(128) unsigned char dyn_smem[];
+    __shared__ uint64_t full[kStreamStages];
+    const TIn* __restrict__ in = static_cast<const TIn*>(p.in);
+    TOut* __restrict__ out = static_cast<TOut*>(p.out);
+    const long long first = blockIdx.x, stride = gridDim.x;
+    const int n_my = first < p.tiles ? (int)((p.tiles - first + stride - 1) / stride) : 0;
+    auto buf = [&](int s) { return reinterpret_cast<TIn*>(dyn_smem + (size_t)s * kStreamTileBytes); };
+    // copy-engine load of my it-th tile into its ring slot (tiles whose byte count
+    // is not a multiple of 16 -- only the last tile of the tensor -- are staged by
+    // the threads instead)
+    auto issue = [&](int it) {
+        const Tile g = tile_of(p, first + (long long)it * stride);
+        const uint32_t bytes = (uint32_t)g.len * (uint32_t)sizeof(TIn);
+        if ((bytes & 15u) == 0) {
+            const int s = it % kStreamStages;
+            mbar_expect_tx(&full[s], bytes);
+            bulk_g2s(buf(s), in + g.g0, bytes, &full[s]);
+        }
+    };
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStreamStages; ++s) mbar_init(&full[s], 1);
+        mbar_fence_init();
     }
     __syncthreads();
+    if (threadIdx.x == 0)
+        for (int it = 0; it < kStreamStages && it < n_my; ++it) issue(it);
 
-    // ---- reduce the patches; output o of the tile is out[out_base + o] ----
-    const int plane_out = p.Hp * p.Wp;
-    const int nout = np * na * p.Wp;
-    const long long out_base = p0 * plane_out + (long long)a0 * p.Wp;
+    int done = 0;
+    bool failed = false;
+    for (int it = 0; it < n_my; ++it) {
+        const int s = it % kStreamStages;
+        const Tile g = tile_of(p, first + (long long)it * stride);
+        const uint32_t bytes = (uint32_t)g.len * (uint32_t)sizeof(TIn);
+        bool ok = true;
+        if ((bytes & 15u) == 0) {
+            ok = mbar_wait_bounded(&full[s], (uint32_t)(it / kStreamStages) & 1u);
+        } else {
+            stage_plain<TIn, kStreamThreads>(in, p.total_elems, g.g0, g.len, reinterpret_cast<uint4*>(buf(s)));
+            __syncthreads();
+        }
+        if (ok) reduce_tile_vec<TIn, TOut, R, G>(p, g, buf(s), out);
+        failed = __syncthreads_or(!ok);     // also: every thread is done reading slot s
+        done = it + 1;
+        if (failed) break;
+        if (threadIdx.x == 0 && it + kStreamStages < n_my) issue(it + kStreamStages);
+    }
+    if (failed && threadIdx.x == 0) {
+        atomicOr(p.err_word, 1u);
+        // copies still in flight target this CTA's shared memory: wait for them (bounded)
+        for (int it = done; it < n_my && it < done + kStreamStages - 1; ++it) {
+            const Tile g = tile_of(p, first + (long long)it * stride);
+            if ((((uint32_t)g.len * (uint32_t)sizeof(TIn)) & 15u) == 0)
+                mbar_wait_bounded(&full[it % kStreamStages], (uint32_t)(it / kStreamStages) & 1u);
+        }
+    }
+}
+
+// ---- generic tiled kernel -----------------------------------------------------------------
+template <typename TIn, typename TOut, int R>
+__global__ void __launch_bounds__(kPoolThreads) pool_tile_kernel(const PoolParams p) {
+    __shared__ uint4 smem_v[kPoolTileBytes / 16 + 1];
+    const TIn* __restrict__ in = static_cast<const TIn*>(p.in);
+    TOut* __restrict__ out = static_cast<TOut*>(p.out);
+    const Tile g = tile_of(p, blockIdx.x);
+    const int shift = stage_plain<TIn, kPoolThreads>(in, p.total_elems, g.g0, g.len, smem_v);
+    const TIn* smem = reinterpret_cast<const TIn*>(smem_v);
+    __syncthreads();
+
+    const int nout = g.np * g.na * p.Wp;
     for (int o = threadIdx.x; o < nout; o += kPoolThreads) {
         uint32_t pl = 0, rem = o;
         if (p.P > 1) p.div_plane_out.divmod(o, pl, rem);
         uint32_t al, b;
         p.div_Wp.divmod(rem, al, b);
-        const int nr = min(p.r, p.H - (a0 + (int)al) * p.r);
+        const int nr = min(p.r, p.H - (g.a0 + (int)al) * p.r);
         const TIn* src = smem + shift + ((int)pl * p.H + (int)al * p.r) * p.W + (int)b * p.r;
         float s = 0.f;
         int cnt;
@@ -87,14 +270,14 @@ __global__ void __launch_bounds__(kPoolThreads) pool_tile_kernel(const PoolParam
             }
             cnt = nr * nc;
         }
-        if constexpr (MEAN) s *= (cnt == p.r * p.r) ? p.inv_full : 1.0f / (float)cnt;
-        out[out_base + o] = from_f32<TOut>(s);
+        if (p.mean) s *= (cnt == p.r * p.r) ? p.inv_full : 1.0f / (float)cnt;
+        out[g.out_base + o] = from_f32<TOut>(s);
     }
 }
 
 // One block per output value, for patches so large that not even one patch-row
 // band fits the tile: strided loads, warp-shuffle + shared-memory reduction.
-template <typename TIn, typename TOut, bool MEAN>
+template <typename TIn, typename TOut>
 __global__ void __launch_bounds__(kPoolThreads) pool_bigpatch_kernel(const PoolParams p) {
     __shared__ float warp_part[kPoolThreads / 32];
     const TIn* __restrict__ in = static_cast<const TIn*>(p.in);
@@ -118,37 +301,84 @@ __global__ void __launch_bounds__(kPoolThreads) pool_bigpatch_kernel(const PoolP
         float t = threadIdx.x < kPoolThreads / 32 ? warp_part[threadIdx.x] : 0.f;
         t = warp_sum(t);
         if (threadIdx.x == 0) {
-            if constexpr (MEAN) t /= (float)(nr * nc);
+            if (p.mean) t /= (float)(nr * nc);
             out[o] = from_f32<TOut>(t);
         }
     }
 }
 
-template <typename TIn, typename TOut, bool MEAN>
-static gf_status pool_dispatch(const PoolParams& p, long long tiles, bool big, cudaStream_t s) {
-    if (big) {
-        pool_bigpatch_kernel<TIn, TOut, MEAN><<<(unsigned)(p.planes * p.Hp * p.Wp), kPoolThreads, 0, s>>>(p);
-        return after_launch();
+// ---- host side ---------------------------------------------------------------------------------
+static int gcd_int(int a, int b) { while (b) { int t = a % b; a = b; b = t; } return a; }
+
+// Tiling for the streamed kernel: every tile but the last of the tensor must
+// start on a 16-byte boundary and span a multiple of 16 bytes.
+static bool plan_stream(PoolParams& p, size_t e) {
+    if (!(p.r == 2 || p.r == 4 || p.r == 8) || p.W % p.r != 0) return false;
+    const long long plane_bytes = (long long)p.H * p.W * (long long)e;
+    const long long band_bytes = (long long)p.r * p.W * (long long)e;
+    if (plane_bytes <= kStreamTileBytes) {
+        const int q = 16 / gcd_int(16, (int)(plane_bytes % 16 == 0 ? 16 : plane_bytes % 16));
+        int P = (int)(kStreamTileBytes / plane_bytes) / q * q;
+        if (P < 1) return false;
+        // no more planes per tile than keeps every SM busy for a few tiles
+        while (P > q && cdiv64(p.planes, P) < 4 * 148) P -= q;
+        p.P = P; p.BR = p.Hp; p.bands = 1;
+        return true;
     }
-    const bool vec = (p.W % p.r == 0);
-    const unsigned grid = (unsigned)tiles;
-    if (vec && p.r == 2) pool_tile_kernel<TIn, TOut, 2, MEAN><<<grid, kPoolThreads, 0, s>>>(p);
-    else if (vec && p.r == 4) pool_tile_kernel<TIn, TOut, 4, MEAN><<<grid, kPoolThreads, 0, s>>>(p);
-    else if (vec && p.r == 8) pool_tile_kernel<TIn, TOut, 8, MEAN><<<grid, kPoolThreads, 0, s>>>(p);
-    else pool_tile_kernel<TIn, TOut, 0, MEAN><<<grid, kPoolThreads, 0, s>>>(p);
+    if (plane_bytes % 16 != 0 || band_bytes > kStreamTileBytes) return false;
+    const int q = 16 / gcd_int(16, (int)(band_bytes % 16 == 0 ? 16 : band_bytes % 16));
+    const int BR = (int)(kStreamTileBytes / band_bytes) / q * q;
+    if (BR < 1) return false;
+    p.P = 1; p.BR = BR < p.Hp ? BR : p.Hp; p.bands = (p.Hp + p.BR - 1) / p.BR;
+    return true;
+}
+
+static int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = 148;
+    }
+    return n;
+}
+
+template <typename TIn, typename TOut, int R, int G>
+static gf_status launch_stream_inst(const PoolParams& p, cudaStream_t s) {
+    constexpr size_t smem = (size_t)kStreamStages * kStreamTileBytes;
+    static bool configured = false;
+    if (!configured) {
+        GF_CUDA_TRY(cudaFuncSetAttribute(pool_stream_kernel<TIn, TOut, R, G>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        configured = true;
+    }
+    const long long grid = p.tiles < sm_count() ? p.tiles : sm_count();
+    pool_stream_kernel<TIn, TOut, R, G><<<(unsigned)grid, kStreamThreads, smem, s>>>(p);
     return after_launch();
 }
 
-gf_status launch_pool(int kernel_id, const void* in, int in_dtype, void* out, int out_dtype, bool mean,
-                      int64_t planes, int H, int W, int r, cudaStream_t s) {
-    ProfScope prof(kernel_id, s);
-    PoolParams p;
-    p.in = in; p.out = out; p.planes = planes; p.total_elems = planes * H * W;
-    p.H = H; p.W = W; p.r = r;
-    p.Hp = (H + r - 1) / r; p.Wp = (W + r - 1) / r;
-    const size_t e = in_dtype == GF_F32 ? 4 : 2;
-    const long long plane_bytes = (long long)H * W * e;
-    const long long band_bytes = (long long)(r < H ? r : H) * W * e;   // one patch row
+template <typename TIn, typename TOut>
+static gf_status launch_stream(const PoolParams& p, cudaStream_t s) {
+    const int G = p.Wp % 4 == 0 ? 4 : (p.Wp % 2 == 0 ? 2 : 1);
+#define GF_STREAM_CASE(RR, GG) \
+    if (p.r == RR && G == GG) return launch_stream_inst<TIn, TOut, RR, GG>(p, s);
+    GF_STREAM_CASE(2, 4) GF_STREAM_CASE(2, 2) GF_STREAM_CASE(2, 1)
+    GF_STREAM_CASE(4, 4) GF_STREAM_CASE(4, 2) GF_STREAM_CASE(4, 1)
+    GF_STREAM_CASE(8, 4) GF_STREAM_CASE(8, 2) GF_STREAM_CASE(8, 1)
+#undef GF_STREAM_CASE
+    return GF_ERR_UNSUPPORTED;
+}
+
+template <typename TIn, typename TOut>
+static gf_status pool_dispatch(PoolParams& p, size_t e, cudaStream_t s) {
+    if (plan_stream(p, e)) {
+        p.div_bands = FastDiv(p.bands);
+        p.tiles = cdiv64(p.planes, p.P) * p.bands;
+        if (p.tiles > 0x7fffffffLL) return GF_ERR_UNSUPPORTED;
+        return launch_stream<TIn, TOut>(p, s);
+    }
+    const long long plane_bytes = (long long)p.H * p.W * (long long)e;
+    const long long band_bytes = (long long)(p.r < p.H ? p.r : p.H) * p.W * (long long)e;   // one patch row
     bool big = false;
     if (plane_bytes <= kPoolTileBytes) {
         p.P = (int)(kPoolTileBytes / plane_bytes); p.BR = p.Hp; p.bands = 1;
@@ -158,21 +388,36 @@ gf_status launch_pool(int kernel_id, const void* in, int in_dtype, void* out, in
         p.P = 1; p.BR = 1; p.bands = p.Hp; big = true;
     }
     p.div_bands = FastDiv(p.bands);
+    p.tiles = cdiv64(p.planes, p.P) * p.bands;
+    if (p.tiles > 0x7fffffffLL || p.planes * p.Hp * p.Wp > 0x7fffffffLL) return GF_ERR_UNSUPPORTED;
+    if (big) {
+        pool_bigpatch_kernel<TIn, TOut><<<(unsigned)(p.planes * p.Hp * p.Wp), kPoolThreads, 0, s>>>(p);
+        return after_launch();
+    }
+    const bool vec = (p.W % p.r == 0);
+    const unsigned grid = (unsigned)p.tiles;
+    if (vec && p.r == 2) pool_tile_kernel<TIn, TOut, 2><<<grid, kPoolThreads, 0, s>>>(p);
+    else if (vec && p.r == 4) pool_tile_kernel<TIn, TOut, 4><<<grid, kPoolThreads, 0, s>>>(p);
+    else if (vec && p.r == 8) pool_tile_kernel<TIn, TOut, 8><<<grid, kPoolThreads, 0, s>>>(p);
+    else pool_tile_kernel<TIn, TOut, 0><<<grid, kPoolThreads, 0, s>>>(p);
+    return after_launch();
+}
+
+gf_status launch_pool(int kernel_id, const void* in, int in_dtype, void* out, int out_dtype, bool mean,
+                      int64_t planes, int H, int W, int r, uint32_t* err_word, cudaStream_t s) {
+    ProfScope prof(kernel_id, s);
+    PoolParams p;
+    p.in = in; p.out = out; p.err_word = err_word; p.planes = planes; p.total_elems = planes * H * W;
+    p.H = H; p.W = W; p.r = r; p.mean = mean ? 1 : 0;
+    p.Hp = (H + r - 1) / r; p.Wp = (W + r - 1) / r;
     p.div_plane_out = FastDiv(p.Hp * p.Wp);
     p.div_Wp = FastDiv(p.Wp);
     p.inv_full = 1.0f / ((float)r * (float)r);
-    const long long tiles = cdiv64(planes, p.P) * p.bands;
-    if (tiles > 0x7fffffffLL || planes * p.Hp * p.Wp > 0x7fffffffLL) return GF_ERR_UNSUPPORTED;
     if (planes == 0) return GF_OK;
-    if (in_dtype == GF_F32 && out_dtype == GF_F32)
-        return mean ? pool_dispatch<float, float, true>(p, tiles, big, s)
-                    : pool_dispatch<float, float, false>(p, tiles, big, s);
-    if (in_dtype == GF_BF16 && out_dtype == GF_BF16)
-        return mean ? pool_dispatch<__nv_bfloat16, __nv_bfloat16, true>(p, tiles, big, s)
-                    : pool_dispatch<__nv_bfloat16, __nv_bfloat16, false>(p, tiles, big, s);
-    if (in_dtype == GF_BF16 && out_dtype == GF_F32)
-        return mean ? pool_dispatch<__nv_bfloat16, float, true>(p, tiles, big, s)
-                    : pool_dispatch<__nv_bfloat16, float, false>(p, tiles, big, s);
+    const size_t e = in_dtype == GF_F32 ? 4 : 2;
+    if (in_dtype == GF_F32 && out_dtype == GF_F32) return pool_dispatch<float, float>(p, e, s);
+    if (in_dtype == GF_BF16 && out_dtype == GF_BF16) return pool_dispatch<__nv_bfloat16, __nv_bfloat16>(p, e, s);
+    if (in_dtype == GF_BF16 && out_dtype == GF_F32) return pool_dispatch<__nv_bfloat16, float>(p, e, s);
     return GF_ERR_UNSUPPORTED;
 }
 

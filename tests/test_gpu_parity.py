@@ -41,6 +41,10 @@ SMALL = [
     L("dw_big_patch", 1, 3, 3, 40, 4100, 3, 3, 40),
     L("n1", 1, 32, 32, 16, 16, 3, 1, 2),
     L("wide_map", 1, 8, 8, 6, 200, 3, 1, 2),
+    L("odd_planes", 1, 3, 5, 14, 14, 3, 1, 2),
+    L("many_small_planes", 5, 33, 47, 6, 6, 3, 1, 2),
+    L("r8_16x16", 3, 20, 36, 16, 16, 3, 1, 8),
+    L("r4_32x32", 2, 20, 12, 32, 32, 1, 1, 4),
 ]
 
 
