@@ -22,7 +22,7 @@ constexpr int kPoolTileBytes = 16384;
 
 constexpr int kStreamThreads = 512;
 constexpr int kStreamTileBytes = 32768;
-constexpr int kStreamStages = 4;
+constexpr int kStreamStages = 6;
 
 struct PoolParams {
     const void* in;
@@ -34,6 +34,8 @@ struct PoolParams {
     int BR;      // patch rows per tile (== Hp when P > 1)
     int bands;   // tiles along the patch rows of one plane (1 when P > 1)
     int mean;    // 1: patch mean, 0: patch sum
+    long long strips;   // streamed kernel: planes * H / r strips of r rows
+    int S;              // streamed kernel: strips per tile
     FastDiv div_bands, div_plane_out /* Hp*Wp */, div_Wp;
     float inv_full;  // 1 / r^2
 };
@@ -140,42 +142,36 @@ __device__ __forceinline__ int stage_plain(const TIn* __restrict__ in, long long
 }
 
 // ---- streamed kernel ------------------------------------------------------------------
+// Requires r in {2,4,8}, r | W and r | H.  Then the whole tensor is a sequence of
+// "strips": strip s is the R image rows [s*R, s*R+R) of the [planes*H, W] matrix,
+// R*W contiguous elements that produce the Wp contiguous outputs s*Wp .. s*Wp+Wp-1.
+// A tile is S consecutive strips (plane boundaries do not matter).
 template <typename TIn, typename TOut, int R, int G>
-__device__ __forceinline__ void reduce_tile_vec(const PoolParams& p, const Tile& g, const TIn* buf,
-                                                TOut* __restrict__ out) {
-    const int nitems = g.np * g.na * p.Wp / G;
-    for (int q = threadIdx.x; q < nitems; q += kStreamThreads) {
-        const uint32_t o = q * G;
-        uint32_t pl = 0, rem = o;
-        if (p.P > 1) p.div_plane_out.divmod(o, pl, rem);
-        uint32_t al, b;
-        p.div_Wp.divmod(rem, al, b);
-        const int nr = min(R, p.H - (g.a0 + (int)al) * R);
-        const TIn* src = buf + ((int)pl * p.H + (int)al * R) * p.W + (int)b * R;
-        float acc[G];
+__device__ __forceinline__ void reduce_item(const PoolParams& p, const TIn* buf, TOut* dst, uint32_t q) {
+    const uint32_t o = q * G;
+    uint32_t A, b;
+    p.div_Wp.divmod(o, A, b);
+    const TIn* src = buf + (int)(A * R) * p.W + (int)b * R;
+    float acc[G];
 #pragma unroll
-        for (int k = 0; k < G; ++k) acc[k] = 0.f;
+    for (int k = 0; k < G; ++k) acc[k] = 0.f;
 #pragma unroll
-        for (int i = 0; i < R; ++i) {
-            if (i < nr) {
-                float v[G * R];
-                load_span<G * R>(src + i * p.W, v);
+    for (int i = 0; i < R; ++i) {
+        float v[G * R];
+        load_span<G * R>(src + i * p.W, v);
 #pragma unroll
-                for (int k = 0; k < G; ++k) {
-                    float s = v[k * R];
+        for (int k = 0; k < G; ++k) {
+            float s = v[k * R];
 #pragma unroll
-                    for (int j = 1; j < R; ++j) s += v[k * R + j];
-                    acc[k] += s;
-                }
-            }
+            for (int j = 1; j < R; ++j) s += v[k * R + j];
+            acc[k] += s;
         }
-        if (p.mean) {
-            const float sc = nr == R ? p.inv_full : 1.0f / (float)(nr * R);
-#pragma unroll
-            for (int k = 0; k < G; ++k) acc[k] *= sc;
-        }
-        store_vec<G>(out + g.out_base + o, acc);
     }
+    if (p.mean) {
+#pragma unroll
+        for (int k = 0; k < G; ++k) acc[k] *= p.inv_full;
+    }
+    store_vec<G>(dst + o, acc);
 }
 
 template <typename TIn, typename TOut, int R, int G>
@@ -186,17 +182,19 @@ __global__ void __launch_bounds__(kStreamThreads, 1) pool_stream_kernel(const Po
     TOut* __restrict__ out = static_cast<TOut*>(p.out);
     const long long first = blockIdx.x, stride = gridDim.x;
     const int n_my = first < p.tiles ? (int)((p.tiles - first + stride - 1) / stride) : 0;
+    const int strip_elems = R * p.W;
     auto buf = [&](int s) { return reinterpret_cast<TIn*>(dyn_smem + (size_t)s * kStreamTileBytes); };
-    // copy-engine load of my it-th tile into its ring slot (tiles whose byte count
-    // is not a multiple of 16 -- only the last tile of the tensor -- are staged by
+    auto strips_of = [&](long long tile) { return (int)min((long long)p.S, p.strips - tile * p.S); };
+    // copy-engine load of my it-th tile into its ring slot (a tile whose byte count is
+    // not a multiple of 16 -- only the last tile of the tensor can be -- is staged by
     // the threads instead)
     auto issue = [&](int it) {
-        const Tile g = tile_of(p, first + (long long)it * stride);
-        const uint32_t bytes = (uint32_t)g.len * (uint32_t)sizeof(TIn);
+        const long long tile = first + (long long)it * stride;
+        const uint32_t bytes = (uint32_t)(strips_of(tile) * strip_elems) * (uint32_t)sizeof(TIn);
         if ((bytes & 15u) == 0) {
             const int s = it % kStreamStages;
             mbar_expect_tx(&full[s], bytes);
-            bulk_g2s(buf(s), in + g.g0, bytes, &full[s]);
+            bulk_g2s(buf(s), in + tile * p.S * strip_elems, bytes, &full[s]);
         }
     };
     if (threadIdx.x == 0) {
@@ -211,16 +209,28 @@ __global__ void __launch_bounds__(kStreamThreads, 1) pool_stream_kernel(const Po
     bool failed = false;
     for (int it = 0; it < n_my; ++it) {
         const int s = it % kStreamStages;
-        const Tile g = tile_of(p, first + (long long)it * stride);
-        const uint32_t bytes = (uint32_t)g.len * (uint32_t)sizeof(TIn);
+        const long long tile = first + (long long)it * stride;
+        const int ns = strips_of(tile);
+        const uint32_t bytes = (uint32_t)(ns * strip_elems) * (uint32_t)sizeof(TIn);
         bool ok = true;
         if ((bytes & 15u) == 0) {
             ok = mbar_wait_bounded(&full[s], (uint32_t)(it / kStreamStages) & 1u);
         } else {
-            stage_plain<TIn, kStreamThreads>(in, p.total_elems, g.g0, g.len, reinterpret_cast<uint4*>(buf(s)));
+            stage_plain<TIn, kStreamThreads>(in, p.total_elems, tile * p.S * strip_elems, ns * strip_elems,
+                                             reinterpret_cast<uint4*>(buf(s)));
             __syncthreads();
         }
-        if (ok) reduce_tile_vec<TIn, TOut, R, G>(p, g, buf(s), out);
+        if (ok) {
+            const uint32_t nitems = (uint32_t)(ns * p.Wp) / G;
+            TOut* dst = out + tile * p.S * p.Wp;
+            const TIn* b = buf(s);
+            uint32_t q = threadIdx.x;
+            for (; q + kStreamThreads < nitems; q += 2 * kStreamThreads) {   // two independent items in flight
+                reduce_item<TIn, TOut, R, G>(p, b, dst, q);
+                reduce_item<TIn, TOut, R, G>(p, b, dst, q + kStreamThreads);
+            }
+            if (q < nitems) reduce_item<TIn, TOut, R, G>(p, b, dst, q);
+        }
         failed = __syncthreads_or(!ok);     // also: every thread is done reading slot s
         done = it + 1;
         if (failed) break;
@@ -230,8 +240,8 @@ __global__ void __launch_bounds__(kStreamThreads, 1) pool_stream_kernel(const Po
         atomicOr(p.err_word, 1u);
         // copies still in flight target this CTA's shared memory: wait for them (bounded)
         for (int it = done; it < n_my && it < done + kStreamStages - 1; ++it) {
-            const Tile g = tile_of(p, first + (long long)it * stride);
-            if ((((uint32_t)g.len * (uint32_t)sizeof(TIn)) & 15u) == 0)
+            const long long tile = first + (long long)it * stride;
+            if ((((uint32_t)(strips_of(tile) * strip_elems) * (uint32_t)sizeof(TIn)) & 15u) == 0)
                 mbar_wait_bounded(&full[it % kStreamStages], (uint32_t)(it / kStreamStages) & 1u);
         }
     }
@@ -310,27 +320,26 @@ __global__ void __launch_bounds__(kPoolThreads) pool_bigpatch_kernel(const PoolP
 // ---- host side ---------------------------------------------------------------------------------
 static int gcd_int(int a, int b) { while (b) { int t = a % b; a = b; b = t; } return a; }
 
-// Tiling for the streamed kernel: every tile but the last of the tensor must
-// start on a 16-byte boundary and span a multiple of 16 bytes.
+// Tiling for the streamed kernel: S strips per tile, a multiple of the count that
+// makes a tile a multiple of 16 bytes (so that every tile starts 16-byte aligned),
+// sized so that every CTA of the persistent grid gets the same number of tiles.
+static int sm_count();
 static bool plan_stream(PoolParams& p, size_t e) {
-    if (!(p.r == 2 || p.r == 4 || p.r == 8) || p.W % p.r != 0) return false;
-    const long long plane_bytes = (long long)p.H * p.W * (long long)e;
-    const long long band_bytes = (long long)p.r * p.W * (long long)e;
-    if (plane_bytes <= kStreamTileBytes) {
-        const int q = 16 / gcd_int(16, (int)(plane_bytes % 16 == 0 ? 16 : plane_bytes % 16));
-        int P = (int)(kStreamTileBytes / plane_bytes) / q * q;
-        if (P < 1) return false;
-        // no more planes per tile than keeps every SM busy for a few tiles
-        while (P > q && cdiv64(p.planes, P) < 4 * 148) P -= q;
-        p.P = P; p.BR = p.Hp; p.bands = 1;
-        return true;
-    }
-    if (plane_bytes % 16 != 0 || band_bytes > kStreamTileBytes) return false;
-    const int q = 16 / gcd_int(16, (int)(band_bytes % 16 == 0 ? 16 : band_bytes % 16));
-    const int BR = (int)(kStreamTileBytes / band_bytes) / q * q;
-    if (BR < 1) return false;
-    p.P = 1; p.BR = BR < p.Hp ? BR : p.Hp; p.bands = (p.Hp + p.BR - 1) / p.BR;
-    return true;
+    if (!(p.r == 2 || p.r == 4 || p.r == 8) || p.W % p.r != 0 || p.H % p.r != 0) return false;
+    const long long strip_bytes = (long long)p.r * p.W * (long long)e;
+    if (strip_bytes > kStreamTileBytes) return false;
+    const int q = 16 / gcd_int(16, (int)(strip_bytes % 16 == 0 ? 16 : strip_bytes % 16));
+    const int s_max = (int)(kStreamTileBytes / strip_bytes) / q * q;
+    if (s_max < 1) return false;
+    p.strips = p.planes * (p.H / p.r);
+    const long long ctas = sm_count();
+    const long long per_cta = cdiv64(p.strips, ctas);                 // strips per CTA
+    const long long tiles_per_cta = cdiv64(per_cta, s_max);
+    long long S = cdiv64(cdiv64(per_cta, tiles_per_cta), q) * q;      // even split, rounded up to q
+    if (S > s_max) S = s_max;
+    p.S = (int)S;
+    p.tiles = cdiv64(p.strips, p.S);
+    return p.tiles <= 0x7fffffffLL;
 }
 
 static int sm_count() {
@@ -371,12 +380,7 @@ static gf_status launch_stream(const PoolParams& p, cudaStream_t s) {
 
 template <typename TIn, typename TOut>
 static gf_status pool_dispatch(PoolParams& p, size_t e, cudaStream_t s) {
-    if (plan_stream(p, e)) {
-        p.div_bands = FastDiv(p.bands);
-        p.tiles = cdiv64(p.planes, p.P) * p.bands;
-        if (p.tiles > 0x7fffffffLL) return GF_ERR_UNSUPPORTED;
-        return launch_stream<TIn, TOut>(p, s);
-    }
+    if (plan_stream(p, e)) return launch_stream<TIn, TOut>(p, s);
     const long long plane_bytes = (long long)p.H * p.W * (long long)e;
     const long long band_bytes = (long long)(p.r < p.H ? p.r : p.H) * p.W * (long long)e;   // one patch row
     bool big = false;
