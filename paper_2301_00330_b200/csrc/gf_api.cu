@@ -21,7 +21,7 @@ int g_prof_created = 0;          // event pairs that exist
 int g_prof_used = 0;             // event pairs recorded since the last read
 int g_prof_slot_kid[kProfPairs];
 const char* const kKernelNames[K_COUNT] = {
-    "stash_pool", "ksum", "gy_pool", "gx_mix", "gw_partial", "gw_finish", "dw_fused", "exact_gx", "exact_gw"};
+    "stash_pool", "ksum", "gy_pool", "gx_mix", "gw_partial", "gw_finish", "dw_fused", "exact_gx", "exact_gw", "gx_tc", "gw_tc"};
 }  // namespace
 
 ProfScope::ProfScope(int kernel_id, cudaStream_t s) : slot(-1), stream(s) {
@@ -111,6 +111,7 @@ Workspace plan_workspace(const Geo& g) {
     w.off_tsum = off; off += align_up((size_t)g.C_out * g.C_ig * 4, 256);
     w.off_gbar = off; off += align_up((size_t)g.N * g.C_out * g.Hp * g.Wp * 4, 256);
     int s = dense_splits(g);
+    if (tc_eligible(g)) { const int ts = tc_gw_splits(g); if (ts > s) s = ts; }
     if (is_depthwise(g)) { const int ds = depthwise_splits(g); if (ds > s) s = ds; }
     w.splits = s;
     w.off_part = off; off += align_up((size_t)s * g.C_out * g.C_ig * 4, 256);
@@ -198,6 +199,30 @@ gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* sta
         st = launch_depthwise(g_y, stash, W, g_W ? part : nullptr, g_X, err, g, &splits, s);
         if (st != GF_OK) return st;
         if (g_W) return launch_gw_finish(part, splits, g_W, g, s);
+        return GF_OK;
+    }
+
+    if (tc_eligible(g)) {
+        // tensor-core path: theta sums (transposed, bf16; clears the error word), patch
+        // means of g_y as bf16, then the two contractions on tcgen05
+        __nv_bfloat16* thetaT = reinterpret_cast<__nv_bfloat16*>(tsum);
+        __nv_bfloat16* gbar16 = reinterpret_cast<__nv_bfloat16*>(gbar);
+        st = launch_ksum_t(W, g, thetaT, err, s);
+        if (st != GF_OK) return st;
+        st = launch_pool(K_GY_POOL, g_y, g.dtype, gbar16, GF_BF16, /*mean=*/true, (int64_t)g.N * g.C_out, g.H, g.W,
+                         g.r, err, s);
+        if (st != GF_OK) return st;
+        if (g_X) {
+            st = launch_gx_tc(gbar16, thetaT, g_X, err, g, s);
+            if (st != GF_OK) return st;
+        }
+        if (g_W) {
+            const int splits = tc_gw_splits(g);
+            st = launch_gw_tc(gbar16, static_cast<const __nv_bfloat16*>(stash), part, splits, err, g, s);
+            if (st != GF_OK) return st;
+            st = launch_gw_finish(part, splits, g_W, g, s);
+            if (st != GF_OK) return st;
+        }
         return GF_OK;
     }
 

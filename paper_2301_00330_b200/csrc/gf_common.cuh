@@ -14,7 +14,7 @@ void count_launch(int n = 1);
 
 enum KernelId {
     K_STASH_POOL = 0, K_KSUM, K_GY_POOL, K_GX_MIX, K_GW_PARTIAL, K_GW_FINISH, K_DW_FUSED,
-    K_EXACT_GX, K_EXACT_GW, K_COUNT
+    K_EXACT_GX, K_EXACT_GW, K_GX_TC, K_GW_TC, K_COUNT
 };
 
 // Brackets the launches made during its lifetime with a pair of events when
@@ -145,6 +145,15 @@ gf_status launch_gw_finish(const float* part, int splits, float* gW, const Geo& 
 gf_status launch_depthwise(const void* gy, const void* stash, const void* W, float* part,
                            void* gX, uint32_t* err_word, const Geo& g, int* splits_out, cudaStream_t s);
 int depthwise_splits(const Geo& g);
+
+// tensor-core path (bf16 operands, dense layers)
+bool tc_eligible(const Geo& g);
+int tc_gw_splits(const Geo& g);
+gf_status launch_ksum_t(const void* W, const Geo& g, __nv_bfloat16* thetaT, uint32_t* err_word, cudaStream_t s);
+gf_status launch_gx_tc(const __nv_bfloat16* gbar, const __nv_bfloat16* thetaT, void* gX, uint32_t* err_word,
+                       const Geo& g, cudaStream_t s);
+gf_status launch_gw_tc(const __nv_bfloat16* gbar, const __nv_bfloat16* stash, float* part, int splits,
+                       uint32_t* err_word, const Geo& g, cudaStream_t s);
 gf_status launch_exact(const void* gy, const void* x, const void* W, float* gW, void* gX,
                        const Geo& g, cudaStream_t s);
 
