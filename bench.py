@@ -40,6 +40,7 @@ NCU_TRAFFIC: dict[str, dict] = {}
 KERNEL_SOURCE = {
     "stash_pool": "gf_pool.cu", "gy_pool": "gf_pool.cu", "ksum": "gf_dense.cu", "gx_mix": "gf_dense.cu",
     "gw_partial": "gf_dense.cu", "gw_finish": "gf_dense.cu", "dw_fused": "gf_depthwise.cu",
+    "gx_tc": "gf_tc.cu", "gw_tc": "gf_tc.cu",
 }
 
 
@@ -134,13 +135,17 @@ class ClockSampler:
 def kernel_cost(name: str, L, splits: int) -> tuple[float, float]:
     """(algorithmic bytes, flops) of one launch of kernel `name` on layer L."""
     e = L.elem_bytes
-    gbar = 4 * L.N * L.C_out * L.Hp * L.Wp
+    gbar = 4 * L.N * L.C_out * L.Hp * L.Wp          # fp32 patch means (CUDA-core path)
+    gbar16 = gbar // 2                              # bf16 patch means (tensor-core path)
     pairs = L.C_out * L.C_ig
     M = L.N * L.Hp * L.Wp
     mix = 2.0 * M * L.C_out * L.C_ig
+    tc = L.dtype == "bf16" and L.groups == 1
     table = {
+        "gx_tc": (gbar16 + 2 * pairs + e * L.numel_x(), mix),
+        "gw_tc": (gbar16 + e * L.numel_stash() + 4 * splits * pairs, mix),
         "stash_pool": (e * (L.numel_x() + L.numel_stash()), L.numel_x()),
-        "gy_pool": (e * L.numel_gy() + gbar, L.numel_gy()),
+        "gy_pool": (e * L.numel_gy() + (gbar16 if tc else gbar), L.numel_gy()),
         "ksum": (e * L.numel_w() + 4 * pairs, L.numel_w()),
         "gx_mix": (gbar + 4 * pairs + e * L.numel_x(), mix),
         "gw_partial": (gbar + e * L.numel_stash() + 4 * splits * pairs, mix),
@@ -380,8 +385,13 @@ def run_ours(args) -> None:
         return
 
     # split count of the reduced g_W contraction, needed for its byte count
-    tiles = ((layer.C_out // layer.groups + 63) // 64) * ((layer.C_ig + 63) // 64) * layer.groups
-    splits = max(1, min(layer.N, -(-592 // tiles)))
+    if layer.dtype == "bf16" and layer.groups == 1:      # tensor-core path: 128 x 128 tiles, one wave of CTAs
+        tiles = ((layer.C_out + 127) // 128) * ((layer.C_in + 127) // 128)
+        chunks = -(-(layer.N * layer.Hp * layer.Wp) // 64)
+        splits = max(1, min(chunks, -(-148 // tiles)))
+    else:
+        tiles = ((layer.C_out // layer.groups + 63) // 64) * ((layer.C_ig + 63) // 64) * layer.groups
+        splits = max(1, min(layer.N, -(-592 // tiles)))
     n_dom, ms_dom = dom.get(dominant, (0, 0.0))
     roof = roofline(dominant, ms_dom / max(n_dom, 1), layer, splits)
     roof["timed_launches"] = n_dom

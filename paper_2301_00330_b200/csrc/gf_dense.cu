@@ -202,9 +202,15 @@ __global__ void gw_finish_kernel(const float* __restrict__ part, int S, size_t n
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n_pairs * taps) return;
     const uint32_t pair = div_taps.div((uint32_t)i);
-    float s = 0.f;
-    for (int k = 0; k < S; ++k) s += part[(size_t)k * n_pairs + pair];
-    gW[i] = s;
+    // eight independent loads in flight; the order of the sum stays fixed
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    int k = 0;
+    for (; k + 8 <= S; k += 8) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) acc[u] += part[(size_t)(k + u) * n_pairs + pair];
+    }
+    for (; k < S; ++k) acc[0] += part[(size_t)k * n_pairs + pair];
+    gW[i] = ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
 }
 
 gf_status launch_gw_finish(const float* part, int splits, float* gW, const Geo& g, cudaStream_t s) {

@@ -115,6 +115,46 @@ __device__ __forceinline__ void load_mnmajor(unsigned char* tile, const FlatSrc&
     }
 }
 
+// ---- the same tiles filled by asynchronous copies (cp.async, V >= 2) ------------------------
+// The copies of a stage are issued back to back without waiting; out-of-range pieces
+// are zero-filled (source size 0).
+__device__ __forceinline__ void cp_async_piece(uint32_t dst, const void* src, int V, bool valid) {
+    const uint32_t n = valid ? (uint32_t)(V * 2) : 0u;
+    if (V == 8) asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
+    else if (V == 4) asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
+    else asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+template <int ROWS>
+__device__ __forceinline__ void issue_kmajor(uint32_t tile, const FlatSrc& s, int c0, long long k0, int tid) {
+    const int lpr = 6 - s.logV;
+    const int total = ROWS << lpr;
+#pragma unroll 4
+    for (int id = tid; id < total; id += kTcLoaders) {
+        const int row = id >> lpr, k = (id & ((1 << lpr) - 1)) << s.logV;
+        const bool valid = c0 + row < s.C && k0 + k < s.k_total;
+        cp_async_piece(tile + kmajor_off(row, k), valid ? flat_ptr(s, c0 + row, k0 + k) : s.base, s.V, valid);
+    }
+}
+
+template <int NT>
+__device__ __forceinline__ void issue_mnmajor(uint32_t tile, const FlatSrc& s, int c0, long long j0, int tid) {
+    int lnt = 0;
+    while ((1 << lnt) < NT) ++lnt;
+    const int lpr = lnt - s.logV;
+    const int total = kTcBK << lpr;
+#pragma unroll 4
+    for (int id = tid; id < total; id += kTcLoaders) {
+        const int krow = id >> lpr, j = (id & ((1 << lpr) - 1)) << s.logV;
+        const bool valid = c0 + krow < s.C && j0 + j < s.k_total;
+        cp_async_piece(tile + mnmajor_off(krow, j), valid ? flat_ptr(s, c0 + krow, j0 + j) : s.base, s.V, valid);
+    }
+}
+
 // ---- pipeline state shared by the two kernels ----------------------------------------------
 struct TcShared {
     uint64_t full[kTcStages];    // loaders -> MMA   (count = loader threads)
@@ -202,15 +242,37 @@ __global__ void __launch_bounds__(kTcThreads) gx_tc_kernel(const GxTcParams p) {
 
     if (warp < 4) {
         // ---- loaders ----
-        for (int kc = 0; kc < n_chunks && ok; ++kc) {
-            const int s = kc % kTcStages;
-            if (kc >= kTcStages) ok = mbar_wait_bounded(&sh.empty[s], (uint32_t)((kc / kTcStages) - 1) & 1u);
-            if (!ok) break;
-            unsigned char* a_tile = dyn + (size_t)s * kStageBytes;
-            load_kmajor<128>(a_tile, p.thetaT, ci0, (long long)kc * kTcBK, tid);
-            load_mnmajor<NT>(a_tile + kABytes, p.gbar, kc * kTcBK, col0, tid);
-            fence_proxy_async_smem();
-            mbar_arrive(&sh.full[s]);
+        if (p.gbar.V >= 2) {
+            // asynchronous copies, kTcStages-1 chunks in flight; a chunk is published
+            // (proxy fence + arrive) once this thread's copies of it have landed
+            for (int kc = 0; kc < n_chunks + kTcStages - 1; ++kc) {
+                if (kc < n_chunks) {
+                    const int s = kc % kTcStages;
+                    if (kc >= kTcStages) ok = mbar_wait_bounded(&sh.empty[s], (uint32_t)((kc / kTcStages) - 1) & 1u);
+                    if (!ok) break;
+                    const uint32_t a_tile = smem_u32(dyn + (size_t)s * kStageBytes);
+                    issue_kmajor<128>(a_tile, p.thetaT, ci0, (long long)kc * kTcBK, tid);
+                    issue_mnmajor<NT>(a_tile + kABytes, p.gbar, kc * kTcBK, col0, tid);
+                }
+                cp_async_commit();
+                if (kc >= kTcStages - 1) {
+                    cp_async_wait<kTcStages - 1>();
+                    fence_proxy_async_smem();
+                    mbar_arrive(&sh.full[(kc - (kTcStages - 1)) % kTcStages]);
+                }
+            }
+            cp_async_wait<0>();
+        } else {
+            for (int kc = 0; kc < n_chunks && ok; ++kc) {
+                const int s = kc % kTcStages;
+                if (kc >= kTcStages) ok = mbar_wait_bounded(&sh.empty[s], (uint32_t)((kc / kTcStages) - 1) & 1u);
+                if (!ok) break;
+                unsigned char* a_tile = dyn + (size_t)s * kStageBytes;
+                load_kmajor<128>(a_tile, p.thetaT, ci0, (long long)kc * kTcBK, tid);
+                load_mnmajor<NT>(a_tile + kABytes, p.gbar, kc * kTcBK, col0, tid);
+                fence_proxy_async_smem();
+                mbar_arrive(&sh.full[s]);
+            }
         }
         // patch offsets of this tile's columns (used by the expansion below)
         for (int j = tid; j < NT; j += kTcLoaders) {
@@ -328,16 +390,37 @@ __global__ void __launch_bounds__(kTcThreads) gw_tc_kernel(const GwTcParams p) {
     bool ok = true;
 
     if (warp < 4) {
-        for (int it = 0; it < n_chunks && ok; ++it) {
-            const int s = it % kTcStages;
-            if (it >= kTcStages) ok = mbar_wait_bounded(&sh.empty[s], (uint32_t)((it / kTcStages) - 1) & 1u);
-            if (!ok) break;
-            unsigned char* a_tile = dyn + (size_t)s * kStageBytes;
-            const long long k0 = (long long)(kc_begin + it) * kTcBK;
-            load_kmajor<128>(a_tile, p.gbar, co0, k0, tid);
-            load_kmajor<NT>(a_tile + kABytes, p.stash, ci0, k0, tid);
-            fence_proxy_async_smem();
-            mbar_arrive(&sh.full[s]);
+        if (p.gbar.V >= 2) {
+            for (int it = 0; it < n_chunks + kTcStages - 1; ++it) {
+                if (it < n_chunks) {
+                    const int s = it % kTcStages;
+                    if (it >= kTcStages) ok = mbar_wait_bounded(&sh.empty[s], (uint32_t)((it / kTcStages) - 1) & 1u);
+                    if (!ok) break;
+                    const uint32_t a_tile = smem_u32(dyn + (size_t)s * kStageBytes);
+                    const long long k0 = (long long)(kc_begin + it) * kTcBK;
+                    issue_kmajor<128>(a_tile, p.gbar, co0, k0, tid);
+                    issue_kmajor<NT>(a_tile + kABytes, p.stash, ci0, k0, tid);
+                }
+                cp_async_commit();
+                if (it >= kTcStages - 1) {
+                    cp_async_wait<kTcStages - 1>();
+                    fence_proxy_async_smem();
+                    mbar_arrive(&sh.full[(it - (kTcStages - 1)) % kTcStages]);
+                }
+            }
+            cp_async_wait<0>();
+        } else {
+            for (int it = 0; it < n_chunks && ok; ++it) {
+                const int s = it % kTcStages;
+                if (it >= kTcStages) ok = mbar_wait_bounded(&sh.empty[s], (uint32_t)((it / kTcStages) - 1) & 1u);
+                if (!ok) break;
+                unsigned char* a_tile = dyn + (size_t)s * kStageBytes;
+                const long long k0 = (long long)(kc_begin + it) * kTcBK;
+                load_kmajor<128>(a_tile, p.gbar, co0, k0, tid);
+                load_kmajor<NT>(a_tile + kABytes, p.stash, ci0, k0, tid);
+                fence_proxy_async_smem();
+                mbar_arrive(&sh.full[s]);
+            }
         }
         if (ok && n_chunks > 0) ok = mbar_wait_bounded(&sh.accum, 0);
         tc_fence_after_sync();
