@@ -207,7 +207,7 @@ gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* sta
         // means of g_y as bf16, then the two contractions on tcgen05
         __nv_bfloat16* thetaT = reinterpret_cast<__nv_bfloat16*>(tsum);
         __nv_bfloat16* gbar16 = reinterpret_cast<__nv_bfloat16*>(gbar);
-        st = launch_ksum_t(W, g, thetaT, err, s);
+        st = launch_ksum_t(W, g, thetaT, g_W ? part : nullptr, err, s);
         if (st != GF_OK) return st;
         st = launch_pool(K_GY_POOL, g_y, g.dtype, gbar16, GF_BF16, /*mean=*/true, (int64_t)g.N * g.C_out, g.H, g.W,
                          g.r, err, s);
@@ -220,7 +220,7 @@ gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* sta
             const int splits = tc_gw_splits(g);
             st = launch_gw_tc(gbar16, static_cast<const __nv_bfloat16*>(stash), part, splits, err, g, s);
             if (st != GF_OK) return st;
-            st = launch_gw_finish(part, splits, g_W, g, s);
+            st = launch_gw_finish(part, 1, g_W, g, s);
             if (st != GF_OK) return st;
         }
         return GF_OK;

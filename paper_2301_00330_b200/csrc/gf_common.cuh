@@ -149,10 +149,11 @@ int depthwise_splits(const Geo& g);
 // tensor-core path (bf16 operands, dense layers)
 bool tc_eligible(const Geo& g);
 int tc_gw_splits(const Geo& g);
-gf_status launch_ksum_t(const void* W, const Geo& g, __nv_bfloat16* thetaT, uint32_t* err_word, cudaStream_t s);
+gf_status launch_ksum_t(const void* W, const Geo& g, __nv_bfloat16* thetaT, float* gwu, uint32_t* err_word,
+                        cudaStream_t s);
 gf_status launch_gx_tc(const __nv_bfloat16* gbar, const __nv_bfloat16* thetaT, void* gX, uint32_t* err_word,
                        const Geo& g, cudaStream_t s);
-gf_status launch_gw_tc(const __nv_bfloat16* gbar, const __nv_bfloat16* stash, float* part, int splits,
+gf_status launch_gw_tc(const __nv_bfloat16* gbar, const __nv_bfloat16* stash, float* gwu, int splits,
                        uint32_t* err_word, const Geo& g, cudaStream_t s);
 gf_status launch_exact(const void* gy, const void* x, const void* W, float* gW, void* gX,
                        const Geo& g, cudaStream_t s);

@@ -5,34 +5,45 @@
 //           col = flattened (image, patch); the epilogue expands every value to its
 //           r x r block of g_X.
 //   gw_tc   Eq. (grad_w):  D[c_o, c_i] = sum_{k} gbar[c_o, k] * stash[c_i, k],
-//           k = flattened (image, patch), split over the batch; the slices are summed
-//           and broadcast to the KH*KW taps by gw_finish.
+//           k = flattened (image, patch), split over the batch; every CTA adds its
+//           slice to g_W's unique-value matrix, which gw_finish broadcasts to the taps.
 //
-// One CTA computes one 128-row output tile.  Warps 0-7 stage the operand tiles
-// (asynchronous copies into 128-byte-swizzled shared memory) through a ring of stages
-// guarded by mbarriers, then drain the accumulator from tensor memory; one thread of
-// warp 8 issues the tcgen05.mma instructions.  Every wait is bounded: on expiry the
-// CTA sets the error word, frees its tensor memory and returns.
+// gx_tc is persistent (one CTA per SM loops over output tiles) and warp-specialised:
+// warps 0-7 stage the operand tiles (asynchronous copies into 128-byte-swizzled shared
+// memory, a ring of stages guarded by mbarriers), one thread of warp 16 issues the
+// tcgen05.mma instructions into one of two accumulators in tensor memory, and warps
+// 8-15 drain the other accumulator and write the expanded tile, so loading, the
+// contraction and the stores of consecutive tiles overlap.  gw_tc computes one
+// 128 x 128 tile of one batch slice per CTA and adds it to the unique-value matrix
+// with vector reductions (the order of the additions is not fixed).
+// Every wait is bounded: on expiry the CTA sets the error word, frees its tensor memory
+// and returns.
 #include "gf_common.cuh"
 #include "gf_tc.cuh"
 
 namespace gf {
 
-constexpr int kTcLoaders = 256;     // 8 loader / epilogue warps
-constexpr int kTcThreads = 288;     // + 1 MMA warp
-constexpr int kTcStages = 3;
 constexpr int kTcBK = 64;           // K elements per stage (one 128-byte swizzled row)
+constexpr int kGwLoaders = 256;     // gw_tc: 8 loader / epilogue warps + 1 MMA warp
+constexpr int kGwThreads = 288;
+constexpr int kGwStages = 3;
+constexpr int kGxLoaders = 256;     // gx_tc: 8 loader warps, 8 epilogue warps, 1 MMA warp
+constexpr int kGxEpi = 256;
+constexpr int kGxThreads = kGxLoaders + kGxEpi + 32;
+constexpr int kGxMmaWarp = (kGxLoaders + kGxEpi) / 32;
+constexpr int kGxStages = 4;
 
 // Source of an operand: a [n][C][P] bf16 array read along the flattened index
 // k = n*P + p (row c is a channel).  A plain [rows][pitch] matrix is the case P = pitch,
-// k < pitch.
+// k < pitch.  Pieces of V = 2^logV elements never straddle an image (V | P) and are
+// V*2-byte aligned.
 struct FlatSrc {
     const __nv_bfloat16* base;
     int C;              // channels per image
     int P;              // elements per (image, channel)
     long long k_total;  // N*P
     FastDiv div_P;
-    int V, logV;        // piece width in elements: V | P, pieces are V*2-byte aligned
+    int logV;
 };
 
 __device__ __forceinline__ const __nv_bfloat16* flat_ptr(const FlatSrc& s, int c, long long k) {
@@ -41,14 +52,13 @@ __device__ __forceinline__ const __nv_bfloat16* flat_ptr(const FlatSrc& s, int c
     return s.base + ((size_t)n * s.C + c) * s.P + p;
 }
 
-// ---- tiles filled by asynchronous copies (cp.async, V >= 2) ------------------------------------
-// A thread owns one piece position along the contiguous direction and walks over the
-// rows, so its source pointer advances by a constant and no division is needed per
-// piece.  Out-of-range pieces are zero-filled (source size 0).
-__device__ __forceinline__ void cp_async_piece(uint32_t dst, const void* src, int V, bool valid) {
-    const uint32_t n = valid ? (uint32_t)(V * 2) : 0u;
-    if (V == 8) asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
-    else if (V == 4) asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
+// ---- asynchronous copies ----------------------------------------------------------------------
+template <int LOGV>
+__device__ __forceinline__ void cp_async_piece(uint32_t dst, const void* src, bool valid) {
+    static_assert(LOGV >= 1 && LOGV <= 3, "pieces of 4, 8 or 16 bytes");
+    const uint32_t n = valid ? (uint32_t)(2 << LOGV) : 0u;     // source bytes; 0 = fill with zeros
+    if constexpr (LOGV == 3) asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
+    else if constexpr (LOGV == 2) asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
     else asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
@@ -56,46 +66,66 @@ template <int N> __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
-// K-major tile [ROWS][64]: rows = channels c0.., k range [k0, k0+64).
-template <int ROWS>
-__device__ __forceinline__ void issue_kmajor(uint32_t tile, const FlatSrc& s, int c0, long long k0, int tid) {
-    const int lpr = 6 - s.logV;                       // log2(pieces per row)
-    const int k = (tid & ((1 << lpr) - 1)) << s.logV;
-    const int row_step = kTcLoaders >> lpr;
-    const long long kk = k0 + k;
-    const bool k_ok = kk < s.k_total;
-    const __nv_bfloat16* src = flat_ptr(s, c0 + (tid >> lpr), k_ok ? kk : 0);
-    const size_t src_step = (size_t)row_step * s.P;
-#pragma unroll 4
-    for (int row = tid >> lpr; row < ROWS; row += row_step, src += src_step) {
-        const bool valid = k_ok && (c0 + row < s.C);
-        cp_async_piece(tile + kmajor_off(row, k), valid ? src : s.base, s.V, valid);
+// A thread's share of a K-major tile [ROWS][64]: one piece position k along the row and
+// the rows row0, row0 + ROW_STEP, ...  The shared-memory offsets are the same for every
+// chunk, so they are computed once; per chunk only the source pointer moves.
+template <int ROWS, int NTHR, int LOGV>
+struct KMajorPieces {
+    static constexpr int LPR = 6 - LOGV;                  // log2(pieces per row)
+    static constexpr int ROW_STEP = NTHR >> LPR;
+    static constexpr int NP = ROWS / ROW_STEP;
+    uint32_t soff[NP];
+    int k, row0;
+    __device__ __forceinline__ void init(int tid) {
+        k = (tid & ((1 << LPR) - 1)) << LOGV;
+        row0 = tid >> LPR;
+#pragma unroll
+        for (int i = 0; i < NP; ++i) soff[i] = kmajor_off(row0 + i * ROW_STEP, k);
     }
-}
-
-// MN-major tile [64 k][NT]: k = channel c0 + krow, columns = flattened index j0 + j.
-template <int NT>
-__device__ __forceinline__ void issue_mnmajor(uint32_t tile, const FlatSrc& s, int c0, long long j0, int tid) {
-    int lnt = 0;
-    while ((1 << lnt) < NT) ++lnt;
-    const int lpr = lnt - s.logV;                     // log2(pieces per k row)
-    const int j = (tid & ((1 << lpr) - 1)) << s.logV;
-    const int k_step = kTcLoaders >> lpr;
-    const long long col = j0 + j;
-    const bool c_ok = col < s.k_total;
-    const __nv_bfloat16* src = flat_ptr(s, c0 + (tid >> lpr), c_ok ? col : 0);
-    const size_t src_step = (size_t)k_step * s.P;
-#pragma unroll 4
-    for (int krow = tid >> lpr; krow < kTcBK; krow += k_step, src += src_step) {
-        const bool valid = c_ok && (c0 + krow < s.C);
-        cp_async_piece(tile + mnmajor_off(krow, j), valid ? src : s.base, s.V, valid);
+    // src: element (first row of this thread, this thread's k); pitch = elements between rows;
+    // rows_valid = rows of the source from the thread's first row on; ok = the k position exists.
+    __device__ __forceinline__ void issue(uint32_t tile, const __nv_bfloat16* src, size_t pitch, int rows_valid,
+                                          bool ok, const void* safe) const {
+        const size_t step = (size_t)ROW_STEP * pitch;
+#pragma unroll
+        for (int i = 0; i < NP; ++i) {
+            const bool valid = ok && (i * ROW_STEP < rows_valid);
+            cp_async_piece<LOGV>(tile + soff[i], valid ? (const void*)(src + i * step) : safe, valid);
+        }
     }
-}
+};
 
-// ---- the same tiles through registers (V == 1: 2-byte pieces cannot be copied asynchronously) ----
-template <int ROWS>
+// A thread's share of an MN-major tile [64 k][NT]: one piece position j along the
+// contiguous (M/N) direction and the k rows krow0, krow0 + K_STEP, ...
+template <int NT, int NTHR, int LOGV>
+struct MNMajorPieces {
+    static constexpr int LNT = NT == 32 ? 5 : NT == 64 ? 6 : NT == 128 ? 7 : 8;
+    static constexpr int LPR = LNT - LOGV;
+    static constexpr int K_STEP = NTHR >> LPR;
+    static constexpr int NP = kTcBK / K_STEP;
+    uint32_t soff[NP];
+    int j, krow0;
+    __device__ __forceinline__ void init(int tid) {
+        j = (tid & ((1 << LPR) - 1)) << LOGV;
+        krow0 = tid >> LPR;
+#pragma unroll
+        for (int i = 0; i < NP; ++i) soff[i] = mnmajor_off(krow0 + i * K_STEP, j);
+    }
+    __device__ __forceinline__ void issue(uint32_t tile, const __nv_bfloat16* src, size_t pitch, int rows_valid,
+                                          bool ok, const void* safe) const {
+        const size_t step = (size_t)K_STEP * pitch;
+#pragma unroll
+        for (int i = 0; i < NP; ++i) {
+            const bool valid = ok && (i * K_STEP < rows_valid);
+            cp_async_piece<LOGV>(tile + soff[i], valid ? (const void*)(src + i * step) : safe, valid);
+        }
+    }
+};
+
+// ---- the same tiles through registers (LOGV == 0: 2-byte pieces cannot be copied asynchronously) ----
+template <int ROWS, int NTHR>
 __device__ __forceinline__ void load_kmajor_scalar(unsigned char* tile, const FlatSrc& s, int c0, long long k0, int tid) {
-    for (int id = tid; id < ROWS * kTcBK; id += kTcLoaders) {
+    for (int id = tid; id < ROWS * kTcBK; id += NTHR) {
         const int row = id >> 6, k = id & 63;
         unsigned short v = 0;
         if (c0 + row < s.C && k0 + k < s.k_total)
@@ -103,9 +133,9 @@ __device__ __forceinline__ void load_kmajor_scalar(unsigned char* tile, const Fl
         *reinterpret_cast<unsigned short*>(tile + kmajor_off(row, k)) = v;
     }
 }
-template <int NT>
+template <int NT, int NTHR>
 __device__ __forceinline__ void load_mnmajor_scalar(unsigned char* tile, const FlatSrc& s, int c0, long long j0, int tid) {
-    for (int id = tid; id < kTcBK * NT; id += kTcLoaders) {
+    for (int id = tid; id < kTcBK * NT; id += NTHR) {
         const int krow = id / NT, j = id - krow * NT;
         unsigned short v = 0;
         if (c0 + krow < s.C && j0 + j < s.k_total)
@@ -114,86 +144,68 @@ __device__ __forceinline__ void load_mnmajor_scalar(unsigned char* tile, const F
     }
 }
 
-// ---- pipeline state shared by the two kernels ----------------------------------------------
-struct TcShared {
-    uint64_t full[kTcStages];    // loaders -> MMA   (count = loader threads)
-    uint64_t empty[kTcStages];   // MMA -> loaders   (count = 1, by tcgen05.commit)
-    uint64_t accum;              // MMA -> epilogue  (count = 1)
-    uint32_t tmem_base;
-};
-
+// ---- pipeline pieces shared by the two kernels -----------------------------------------------
 __device__ __forceinline__ unsigned char* align1024(unsigned char* p) {
     return reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(p) + 1023) & ~uintptr_t(1023));
 }
 
-__device__ __forceinline__ void tc_setup(TcShared& sh, int tid, int warp, uint32_t tmem_cols) {
-    if (tid == 0) {
-        for (int s = 0; s < kTcStages; ++s) { mbar_init(&sh.full[s], kTcLoaders); mbar_init(&sh.empty[s], 1); }
-        mbar_init(&sh.accum, 1);
-        mbar_fence_init();
-    }
-    if (warp == 8) { tmem_alloc(&sh.tmem_base, tmem_cols); tmem_relinquish(); }
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-}
-
-// The loaders' side of the ring: issue(kc, stage_smem_addr) enqueues the asynchronous
-// copies of chunk kc; kTcStages-1 chunks are in flight; a chunk is published (proxy
-// fence + arrive) once this thread's copies of it have landed.
-template <typename Issue>
-__device__ __forceinline__ bool run_async_loaders(TcShared& sh, unsigned char* dyn, int stage_bytes, int n_chunks,
-                                                  Issue issue) {
+// The loaders' side of a ring of STAGES stages over `total` chunks: issue(q, smem addr of the
+// stage) enqueues the asynchronous copies of chunk q; STAGES-1 chunks are in flight; a
+// chunk is published (proxy fence + arrive on full[stage]) once this thread's copies of
+// it have landed.
+template <int STAGES, typename Issue>
+__device__ __forceinline__ bool run_async_loaders(uint64_t* full, uint64_t* empty, unsigned char* dyn, int stage_bytes,
+                                                  int total, Issue issue) {
     bool ok = true;
-    for (int kc = 0; kc < n_chunks + kTcStages - 1; ++kc) {
-        if (kc < n_chunks) {
-            const int s = kc % kTcStages;
-            if (kc >= kTcStages) ok = mbar_wait_bounded(&sh.empty[s], (uint32_t)((kc / kTcStages) - 1) & 1u);
+    for (int q = 0; q < total + STAGES - 1; ++q) {
+        if (q < total) {
+            const int s = q % STAGES;
+            if (q >= STAGES) ok = mbar_wait_bounded(&empty[s], (uint32_t)((q / STAGES) - 1) & 1u);
             if (!ok) break;
-            issue(kc, smem_u32(dyn + (size_t)s * stage_bytes));
+            issue(q, smem_u32(dyn + (size_t)s * stage_bytes));
         }
         cp_async_commit();
-        if (kc >= kTcStages - 1) {
-            cp_async_wait<kTcStages - 1>();
+        if (q >= STAGES - 1) {
+            cp_async_wait<STAGES - 1>();
             fence_proxy_async_smem();
-            mbar_arrive(&sh.full[(kc - (kTcStages - 1)) % kTcStages]);
+            mbar_arrive(&full[(q - (STAGES - 1)) % STAGES]);
         }
     }
     cp_async_wait<0>();
     return ok;
 }
-template <typename Load>
-__device__ __forceinline__ bool run_sync_loaders(TcShared& sh, unsigned char* dyn, int stage_bytes, int n_chunks,
-                                                 Load load) {
-    for (int kc = 0; kc < n_chunks; ++kc) {
-        const int s = kc % kTcStages;
-        if (kc >= kTcStages && !mbar_wait_bounded(&sh.empty[s], (uint32_t)((kc / kTcStages) - 1) & 1u)) return false;
-        load(kc, dyn + (size_t)s * stage_bytes);
+template <int STAGES, typename Load>
+__device__ __forceinline__ bool run_sync_loaders(uint64_t* full, uint64_t* empty, unsigned char* dyn, int stage_bytes,
+                                                 int total, Load load) {
+    for (int q = 0; q < total; ++q) {
+        const int s = q % STAGES;
+        if (q >= STAGES && !mbar_wait_bounded(&empty[s], (uint32_t)((q / STAGES) - 1) & 1u)) return false;
+        load(q, dyn + (size_t)s * stage_bytes);
         fence_proxy_async_smem();
-        mbar_arrive(&sh.full[s]);
+        mbar_arrive(&full[s]);
     }
     return true;
 }
 
-// The MMA thread's side: per chunk, four K = 16 steps; b_step = start-address advance of
-// the B descriptor per step (32 bytes K-major, 2048 bytes MN-major).
-__device__ __forceinline__ bool run_mma(TcShared& sh, unsigned char* dyn, int stage_bytes, int a_bytes, int n_chunks,
-                                        uint32_t tmem, uint32_t idesc, uint32_t b_step, uint32_t b_lbo) {
-    for (int kc = 0; kc < n_chunks; ++kc) {
-        const int s = kc % kTcStages;
-        if (!mbar_wait_bounded(&sh.full[s], (uint32_t)(kc / kTcStages) & 1u)) return false;
-        tc_fence_after_sync();
-        const uint32_t a_addr = smem_u32(dyn + (size_t)s * stage_bytes);
-        const uint32_t b_addr = a_addr + a_bytes;
+// One chunk of the MMA thread's work: wait for the stage, four K = 16 steps, release it.
+// b_step = start-address advance of the B descriptor per step (32 bytes K-major, 2048
+// bytes MN-major); b_lbo = its leading byte offset.
+template <int STAGES>
+__device__ __forceinline__ bool mma_chunk(uint64_t* full, uint64_t* empty, unsigned char* dyn, int stage_bytes,
+                                          int a_bytes, int q, bool first, uint32_t d_tmem, uint32_t idesc,
+                                          uint32_t b_step, uint32_t b_lbo) {
+    const int s = q % STAGES;
+    if (!mbar_wait_bounded(&full[s], (uint32_t)(q / STAGES) & 1u)) return false;
+    tc_fence_after_sync();
+    const uint32_t a_addr = smem_u32(dyn + (size_t)s * stage_bytes);
+    const uint32_t b_addr = a_addr + a_bytes;
 #pragma unroll
-        for (int ks = 0; ks < kTcBK / 16; ++ks) {
-            const uint64_t adesc = umma_smem_desc(a_addr + ks * 32, 16, 1024);
-            const uint64_t bdesc = umma_smem_desc(b_addr + ks * b_step, b_lbo, 1024);
-            umma_bf16(tmem, adesc, bdesc, idesc, (kc | ks) != 0);
-        }
-        umma_commit(&sh.empty[s]);
+    for (int ks = 0; ks < kTcBK / 16; ++ks) {
+        const uint64_t adesc = umma_smem_desc(a_addr + ks * 32, 16, 1024);
+        const uint64_t bdesc = umma_smem_desc(b_addr + ks * b_step, b_lbo, 1024);
+        umma_bf16(d_tmem, adesc, bdesc, idesc, !(first && ks == 0));
     }
-    if (n_chunks > 0) umma_commit(&sh.accum);
+    umma_commit(&empty[s]);
     return true;
 }
 
@@ -204,7 +216,8 @@ struct GxTcParams {
     void* gX;
     uint32_t* err_word;
     int N, C_in, C_out, H, W, r, Hp, Wp, P;
-    FastDiv div_Wp;
+    int n_ci_tiles, items;
+    FastDiv div_Wp, div_ci_tiles;
 };
 
 // R consecutive copies of v
@@ -221,134 +234,215 @@ template <int R> __device__ __forceinline__ void store_rep(__nv_bfloat16* dst, f
     else *reinterpret_cast<uint4*>(dst) = make_uint4(w, w, w, w);
 }
 
+struct GxShared {
+    uint64_t full[kGxStages], empty[kGxStages];
+    uint64_t acc_full[2], acc_empty[2];
+    uint32_t tmem_base;
+};
+
 // R > 0: r == R and r | W (every patch row segment is a whole, aligned vector);
 // R == 0: any r, element-wise stores clipped at the right and bottom edges.
-template <typename TOut, int NT, int R>
-__global__ void __launch_bounds__(kTcThreads) gx_tc_kernel(const GxTcParams p) {
+// LOGV: log2 of the piece width of gbar (0: 2-byte pieces through registers).
+template <typename TOut, int NT, int R, int LOGV>
+__global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p) {
     constexpr int kABytes = 128 * kTcBK * 2;             // 16 KB
     constexpr int kBBytes = kTcBK * NT * 2;              // 64 k x NT columns
     constexpr int kStageBytes = kABytes + kBBytes;
+    constexpr int kColsPerLane = NT / 32;
     constexpr uint32_t kIdesc = umma_idesc_bf16(128, NT, /*A K-major*/ 0, /*B MN-major*/ 1);
     extern __shared__ unsigned char dyn_raw[];
-    __shared__ TcShared sh;
+    __shared__ GxShared sh;
     __shared__ long long col_off[NT];     // g_X offset of a column's patch | rows inside the map << 56; -1: no column
     __shared__ int col_cols[NT];          // columns of the patch inside the map (R == 0 only)
     unsigned char* dyn = align1024(dyn_raw);
+    float* D = reinterpret_cast<float*>(dyn + (size_t)kGxStages * kStageBytes);   // [128][NT+1]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const long long col0 = (long long)blockIdx.x * NT;
-    const int ci0 = blockIdx.y * 128;
     const int n_chunks = (p.C_out + kTcBK - 1) / kTcBK;
+    const int first = blockIdx.x, stride = gridDim.x;
+    const int n_my = first < p.items ? (p.items - first + stride - 1) / stride : 0;
 
-    tc_setup(sh, tid, warp, NT);
+    if (tid == 0) {
+        for (int s = 0; s < kGxStages; ++s) { mbar_init(&sh.full[s], kGxLoaders); mbar_init(&sh.empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&sh.acc_full[b], 1); mbar_init(&sh.acc_empty[b], 1); }
+        mbar_fence_init();
+    }
+    if (warp == kGxMmaWarp) { tmem_alloc(&sh.tmem_base, 2 * NT); tmem_relinquish(); }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
     const uint32_t tmem = sh.tmem_base;
     bool ok = true;
+    auto item_of = [&](int it, int& ci0, long long& col0) {
+        uint32_t ct, cit;
+        p.div_ci_tiles.divmod((uint32_t)(first + it * stride), ct, cit);
+        ci0 = (int)cit * 128;
+        col0 = (long long)ct * NT;
+    };
 
-    if (warp < 8) {
-        // ---- loaders ----
-        if (p.gbar.V >= 2) {
-            ok = run_async_loaders(sh, dyn, kStageBytes, n_chunks, [&](int kc, uint32_t tile) {
-                issue_kmajor<128>(tile, p.thetaT, ci0, (long long)kc * kTcBK, tid);
-                issue_mnmajor<NT>(tile + kABytes, p.gbar, kc * kTcBK, col0, tid);
+    if (warp < kGxLoaders / 32) {
+        // ---- loaders: chunk q of this CTA = chunk q % n_chunks of its item q / n_chunks ----
+        if constexpr (LOGV > 0) {
+            KMajorPieces<128, kGxLoaders, 3> pa;          // thetaT rows are 16-byte aligned (C_out % 8 == 0)
+            MNMajorPieces<NT, kGxLoaders, LOGV> pb;
+            pa.init(tid);
+            pb.init(tid);
+            int cur_it = -1, ci0 = 0;
+            const __nv_bfloat16 *a_src = nullptr, *b_src = nullptr;
+            bool b_ok = false;
+            ok = run_async_loaders<kGxStages>(sh.full, sh.empty, dyn, kStageBytes, n_my * n_chunks,
+                                              [&](int q, uint32_t tile) {
+                const int it = q / n_chunks, kc = q - it * n_chunks;
+                if (it != cur_it) {                        // per item: this thread's first source elements
+                    long long col0;
+                    item_of(it, ci0, col0);
+                    cur_it = it;
+                    a_src = p.thetaT.base + (size_t)(ci0 + pa.row0) * p.C_out + pa.k;
+                    const long long col = col0 + pb.j;
+                    b_ok = col < p.gbar.k_total;
+                    b_src = flat_ptr(p.gbar, pb.krow0, b_ok ? col : 0);
+                }
+                const int k0 = kc * kTcBK;
+                pa.issue(tile, a_src + k0, (size_t)p.C_out, p.C_in - ci0 - pa.row0, k0 + pa.k < p.C_out, p.thetaT.base);
+                pb.issue(tile + kABytes, b_src + (size_t)k0 * p.P, (size_t)p.P, p.C_out - k0 - pb.krow0, b_ok,
+                         p.gbar.base);
             });
         } else {
-            ok = run_sync_loaders(sh, dyn, kStageBytes, n_chunks, [&](int kc, unsigned char* tile) {
-                load_kmajor_scalar<128>(tile, p.thetaT, ci0, (long long)kc * kTcBK, tid);
-                load_mnmajor_scalar<NT>(tile + kABytes, p.gbar, kc * kTcBK, col0, tid);
+            ok = run_sync_loaders<kGxStages>(sh.full, sh.empty, dyn, kStageBytes, n_my * n_chunks,
+                                             [&](int q, unsigned char* tile) {
+                const int it = q / n_chunks, kc = q - it * n_chunks;
+                int ci0; long long col0;
+                item_of(it, ci0, col0);
+                load_kmajor_scalar<128, kGxLoaders>(tile, p.thetaT, ci0, (long long)kc * kTcBK, tid);
+                load_mnmajor_scalar<NT, kGxLoaders>(tile + kABytes, p.gbar, kc * kTcBK, col0, tid);
             });
         }
-        // patch offsets of this tile's columns (used by the expansion below)
-        for (int j = tid; j < NT; j += kTcLoaders) {
-            const long long c = col0 + j;
-            long long off = -1;
-            int ncols = 0;
-            if (c < p.gbar.k_total) {
-                const uint32_t n = p.gbar.div_P.div((uint32_t)c), pp = (uint32_t)c - n * (uint32_t)p.P;
-                uint32_t a, b;
-                p.div_Wp.divmod(pp, a, b);
-                off = (long long)n * p.C_in * p.H * p.W + (long long)a * p.r * p.W + (long long)b * p.r;
-                const int nrows = min(p.r, p.H - (int)a * p.r);
-                ncols = min(p.r, p.W - (int)b * p.r);
-                if constexpr (R > 0) off |= (long long)nrows << 56;
-                else ncols |= nrows << 16;
+    } else if (warp == kGxMmaWarp) {
+        // ---- MMA issuer: accumulator it & 1 ----
+        if (lane == 0) {
+            for (int it = 0; it < n_my && ok; ++it) {
+                const int buf = it & 1;
+                if (it >= 2) ok = mbar_wait_bounded(&sh.acc_empty[buf], (uint32_t)((it >> 1) - 1) & 1u);
+                for (int kc = 0; kc < n_chunks && ok; ++kc)
+                    ok = mma_chunk<kGxStages>(sh.full, sh.empty, dyn, kStageBytes, kABytes, it * n_chunks + kc, kc == 0,
+                                              tmem + (uint32_t)(buf * NT), kIdesc, 2048, 8192);
+                if (ok) umma_commit(&sh.acc_full[buf]);
             }
-            col_off[j] = off;
-            if constexpr (R == 0) col_cols[j] = ncols;
         }
-        // ---- epilogue: accumulator -> shared memory (fp32 [128][NT+1]) ----
-        if (ok) ok = mbar_wait_bounded(&sh.accum, 0);
-        tc_fence_after_sync();
-        float* D = reinterpret_cast<float*>(dyn);
-        if (ok) {
-            const int row = (warp & 3) * 32 + lane;
-            const int c_base = (warp >> 2) * (NT / 2);
+    } else {
+        // ---- epilogue warps: lane quarter warp & 3, column half ew >> 2 ----
+        const int et = tid - kGxLoaders, ew = et >> 5;
+        TOut* gx = static_cast<TOut*>(p.gX);
+        const size_t plane = (size_t)p.H * p.W;
+        for (int it = 0; it < n_my; ++it) {
+            const int buf = it & 1;
+            int ci0; long long col0;
+            item_of(it, ci0, col0);
+            for (int j = et; j < NT; j += kGxEpi) {      // patch offsets of this tile's columns
+                const long long c = col0 + j;
+                long long off = -1;
+                int ncols = 0;
+                if (c < p.gbar.k_total) {
+                    const uint32_t n = p.gbar.div_P.div((uint32_t)c), pp = (uint32_t)c - n * (uint32_t)p.P;
+                    uint32_t a, b;
+                    p.div_Wp.divmod(pp, a, b);
+                    off = (long long)n * p.C_in * p.H * p.W + (long long)a * p.r * p.W + (long long)b * p.r;
+                    const int nrows = min(p.r, p.H - (int)a * p.r);
+                    ncols = min(p.r, p.W - (int)b * p.r);
+                    if constexpr (R > 0) off |= (long long)nrows << 56;
+                    else ncols |= nrows << 16;
+                }
+                col_off[j] = off;
+                if constexpr (R == 0) col_cols[j] = ncols;
+            }
+            if (ok) ok = mbar_wait_bounded(&sh.acc_full[buf], (uint32_t)(it >> 1) & 1u);
+            tc_fence_after_sync();
+            if (ok) {                                     // accumulator -> shared memory, fp32 [128][NT+1]
+                const int row = (warp & 3) * 32 + lane;
+                const int c_base = (ew >> 2) * (NT / 2);
 #pragma unroll 1
-            for (int c = c_base; c < c_base + NT / 2; c += 32) {
-                uint32_t v[32];
-                tmem_ld32(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)c, v);
-                tmem_ld_wait();
+                for (int c = c_base; c < c_base + NT / 2; c += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(buf * NT + c), v);
+                    tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) D[row * (NT + 1) + c + i] = __uint_as_float(v[i]);
+                    for (int i = 0; i < 32; ++i) D[row * (NT + 1) + c + i] = __uint_as_float(v[i]);
+                }
             }
-        }
-        tc_fence_before_sync();
-        asm volatile("bar.sync 1, 256;" ::: "memory");      // the eight epilogue warps
-        // ---- expansion: value (m, column j) -> r consecutive pixels on each of r rows ----
-        if (ok) {
-            TOut* gx = static_cast<TOut*>(p.gX);
-            const size_t plane = (size_t)p.H * p.W;
-            const int m_cnt = min(128, p.C_in - ci0);
-            for (int m = warp; m < m_cnt; m += 8) {
-                TOut* base = gx + (size_t)(ci0 + m) * plane;
-                const float* drow = D + m * (NT + 1);
+            tc_fence_before_sync();
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            if (et == 0) mbar_arrive(&sh.acc_empty[buf]);   // the accumulator may be overwritten
+            if (ok) {
+                // expansion: a lane owns the columns lane, lane+32, ...; value (m, j) goes to r
+                // consecutive pixels on each of r rows of plane c_i0 + m
+                const int m_cnt = min(128, p.C_in - ci0);
+                TOut* base = gx + (size_t)ci0 * plane;
 #pragma unroll
-                for (int j = lane; j < NT; j += 32) {
+                for (int t = 0; t < kColsPerLane; ++t) {
+                    const int j = lane + 32 * t;
                     const long long info = col_off[j];
                     if (info < 0) continue;
-                    const float v = drow[j];
                     if constexpr (R > 0) {
-                        TOut* dst = base + (info & 0x00ffffffffffffffLL);
+                        TOut* dst0 = base + (info & 0x00ffffffffffffffLL);
                         const int nrows = (int)(info >> 56);
+#pragma unroll 4
+                        for (int m = ew; m < m_cnt; m += 8) {
+                            const float v = D[m * (NT + 1) + j];
+                            TOut* dst = dst0 + (size_t)m * plane;
 #pragma unroll
-                        for (int dr = 0; dr < R; ++dr)
-                            if (dr < nrows) store_rep<R>(dst + (size_t)dr * p.W, v);
+                            for (int dr = 0; dr < R; ++dr)
+                                if (dr < nrows) store_rep<R>(dst + (size_t)dr * p.W, v);
+                        }
                     } else {
-                        TOut* dst = base + info;
                         const int ext = col_cols[j], ncols = ext & 0xffff, nrows = ext >> 16;
-                        const TOut o = from_f32<TOut>(v);
-                        for (int dr = 0; dr < nrows; ++dr)
-                            for (int dc = 0; dc < ncols; ++dc) dst[(size_t)dr * p.W + dc] = o;
+                        for (int m = ew; m < m_cnt; m += 8) {
+                            const TOut o = from_f32<TOut>(D[m * (NT + 1) + j]);
+                            TOut* dst = base + info + (size_t)m * plane;
+                            for (int dr = 0; dr < nrows; ++dr)
+                                for (int dc = 0; dc < ncols; ++dc) dst[(size_t)dr * p.W + dc] = o;
+                        }
                     }
                 }
             }
+            asm volatile("bar.sync 1, 256;" ::: "memory");   // D and the offsets are free again
         }
-    } else if (lane == 0) {
-        ok = run_mma(sh, dyn, kStageBytes, kABytes, n_chunks, tmem, kIdesc, 2048, 8192);
     }
     if (!ok) atomicOr(p.err_word, 2u);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    if (warp == 8) tmem_dealloc(tmem, NT);
+    if (warp == kGxMmaWarp) tmem_dealloc(tmem, 2 * NT);
 }
 
 // ================================================================== gw_tc
 struct GwTcParams {
     FlatSrc gbar;        // [N][C_out][P]   rows of A
     FlatSrc stash;       // [N][C_in][P]    rows of B
-    float* part;         // [S][C_out][C_in]
+    float* gwu;          // [C_out][C_in] fp32, zeroed beforehand; every CTA adds its slice
     uint32_t* err_word;
     int C_in, C_out, S, chunks_total;
 };
 
-template <int NT>
-__global__ void __launch_bounds__(kTcThreads) gw_tc_kernel(const GwTcParams p) {
+struct GwShared {
+    uint64_t full[kGwStages], empty[kGwStages];
+    uint64_t accum;
+    uint32_t tmem_base;
+};
+
+__device__ __forceinline__ void red_add_v4(float* dst, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(__uint_as_float(a)),
+                 "f"(__uint_as_float(b)), "f"(__uint_as_float(c)), "f"(__uint_as_float(d))
+                 : "memory");
+}
+
+template <int NT, int LOGV>
+__global__ void __launch_bounds__(kGwThreads) gw_tc_kernel(const GwTcParams p) {
     constexpr int kABytes = 128 * kTcBK * 2;
     constexpr int kBBytes = NT * kTcBK * 2;
     constexpr int kStageBytes = kABytes + kBBytes;
     constexpr uint32_t kIdesc = umma_idesc_bf16(128, NT, 0, 0);
     extern __shared__ unsigned char dyn_raw[];
-    __shared__ TcShared sh;
+    __shared__ GwShared sh;
     unsigned char* dyn = align1024(dyn_raw);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -357,56 +451,70 @@ __global__ void __launch_bounds__(kTcThreads) gw_tc_kernel(const GwTcParams p) {
     const int kc_end = (int)((long long)p.chunks_total * (split + 1) / p.S);
     const int n_chunks = kc_end - kc_begin;
 
-    tc_setup(sh, tid, warp, NT);
+    if (tid == 0) {
+        for (int s = 0; s < kGwStages; ++s) { mbar_init(&sh.full[s], kGwLoaders); mbar_init(&sh.empty[s], 1); }
+        mbar_init(&sh.accum, 1);
+        mbar_fence_init();
+    }
+    if (warp == 8) { tmem_alloc(&sh.tmem_base, NT); tmem_relinquish(); }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
     const uint32_t tmem = sh.tmem_base;
     bool ok = true;
 
     if (warp < 8) {
-        if (p.gbar.V >= 2) {
-            ok = run_async_loaders(sh, dyn, kStageBytes, n_chunks, [&](int it, uint32_t tile) {
-                const long long k0 = (long long)(kc_begin + it) * kTcBK;
-                issue_kmajor<128>(tile, p.gbar, co0, k0, tid);
-                issue_kmajor<NT>(tile + kABytes, p.stash, ci0, k0, tid);
+        if constexpr (LOGV > 0) {
+            KMajorPieces<128, kGwLoaders, LOGV> pa;
+            KMajorPieces<NT, kGwLoaders, LOGV> pb;
+            pa.init(tid);
+            pb.init(tid);
+            ok = run_async_loaders<kGwStages>(sh.full, sh.empty, dyn, kStageBytes, n_chunks, [&](int it, uint32_t tile) {
+                // this thread's k position of the chunk: one (image, patch) pair for all its rows
+                const long long kk = (long long)(kc_begin + it) * kTcBK + pa.k;
+                const bool k_ok = kk < p.gbar.k_total;
+                const uint32_t n = p.gbar.div_P.div((uint32_t)(k_ok ? kk : 0));
+                const uint32_t pp = (uint32_t)(k_ok ? kk : 0) - n * (uint32_t)p.gbar.P;
+                const __nv_bfloat16* a_src = p.gbar.base + ((size_t)n * p.C_out + co0 + pa.row0) * p.gbar.P + pp;
+                const __nv_bfloat16* b_src = p.stash.base + ((size_t)n * p.C_in + ci0 + pb.row0) * p.gbar.P + pp;
+                pa.issue(tile, a_src, (size_t)p.gbar.P, p.C_out - co0 - pa.row0, k_ok, p.gbar.base);
+                pb.issue(tile + kABytes, b_src, (size_t)p.gbar.P, p.C_in - ci0 - pb.row0, k_ok, p.stash.base);
             });
         } else {
-            ok = run_sync_loaders(sh, dyn, kStageBytes, n_chunks, [&](int it, unsigned char* tile) {
+            ok = run_sync_loaders<kGwStages>(sh.full, sh.empty, dyn, kStageBytes, n_chunks, [&](int it, unsigned char* tile) {
                 const long long k0 = (long long)(kc_begin + it) * kTcBK;
-                load_kmajor_scalar<128>(tile, p.gbar, co0, k0, tid);
-                load_kmajor_scalar<NT>(tile + kABytes, p.stash, ci0, k0, tid);
+                load_kmajor_scalar<128, kGwLoaders>(tile, p.gbar, co0, k0, tid);
+                load_kmajor_scalar<NT, kGwLoaders>(tile + kABytes, p.stash, ci0, k0, tid);
             });
         }
         if (ok && n_chunks > 0) ok = mbar_wait_bounded(&sh.accum, 0);
         tc_fence_after_sync();
-        if (ok) {
+        if (ok && n_chunks > 0) {
             const int co = co0 + (warp & 3) * 32 + lane;
             const int c_base = (warp >> 2) * (NT / 2);
-            float* out = p.part + ((size_t)split * p.C_out + co) * p.C_in + ci0;
+            float* out = p.gwu + (size_t)co * p.C_in + ci0;
             const bool vec_ok = (p.C_in % 4 == 0);
 #pragma unroll 1
             for (int c = c_base; c < c_base + NT / 2; c += 32) {
                 uint32_t v[32];
-                if (n_chunks > 0) {
-                    tmem_ld32(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)c, v);
-                    tmem_ld_wait();
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = 0u;
-                }
+                tmem_ld32(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)c, v);
+                tmem_ld_wait();
                 if (co < p.C_out) {
                     if (vec_ok && ci0 + c + 32 <= p.C_in) {
 #pragma unroll
-                        for (int i = 0; i < 32; i += 4)
-                            *reinterpret_cast<uint4*>(out + c + i) = make_uint4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                        for (int i = 0; i < 32; i += 4) red_add_v4(out + c + i, v[i], v[i + 1], v[i + 2], v[i + 3]);
                     } else {
 #pragma unroll
                         for (int i = 0; i < 32; ++i)
-                            if (ci0 + c + i < p.C_in) out[c + i] = __uint_as_float(v[i]);
+                            if (ci0 + c + i < p.C_in) atomicAdd(out + c + i, __uint_as_float(v[i]));
                     }
                 }
             }
         }
     } else if (lane == 0) {
-        ok = run_mma(sh, dyn, kStageBytes, kABytes, n_chunks, tmem, kIdesc, 32, 16);
+        for (int it = 0; it < n_chunks && ok; ++it)
+            ok = mma_chunk<kGwStages>(sh.full, sh.empty, dyn, kStageBytes, kABytes, it, it == 0, tmem, kIdesc, 32, 16);
+        if (ok && n_chunks > 0) umma_commit(&sh.accum);
     }
     if (!ok) atomicOr(p.err_word, 4u);
     tc_fence_before_sync();
@@ -416,17 +524,30 @@ __global__ void __launch_bounds__(kTcThreads) gw_tc_kernel(const GwTcParams p) {
 }
 
 // ================================================================== theta sum, transposed bf16
+// thetaT[c_i][c_o] = sum_taps W[c_o][c_i][:], a 32 x 32 tile per block through shared
+// memory so that both the reads (along c_i, taps) and the writes (along c_o) are
+// contiguous.  Also clears the error word and g_W's unique-value accumulator.
 template <typename T>
-__global__ void ksum_t_kernel(const T* __restrict__ W, __nv_bfloat16* __restrict__ thetaT, int C_in, int C_out,
-                              int taps, uint32_t* err_word) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;       // i = ci * C_out + co
-    if (i == 0 && err_word) *err_word = 0u;
-    if (i >= C_in * C_out) return;
-    const int ci = i / C_out, co = i - ci * C_out;
-    const T* w = W + ((size_t)co * C_in + ci) * taps;
-    float s = 0.f;
-    for (int t = 0; t < taps; ++t) s += to_f32(w[t]);
-    thetaT[i] = __float2bfloat16_rn(s);
+__global__ void __launch_bounds__(1024) ksum_t_kernel(const T* __restrict__ W, __nv_bfloat16* __restrict__ thetaT,
+                                                      float* __restrict__ gwu, int C_in, int C_out, int taps,
+                                                      uint32_t* err_word) {
+    __shared__ float tile[32][33];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const int co0 = blockIdx.y * 32, ci0 = blockIdx.x * 32;
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0 && err_word) *err_word = 0u;
+    {
+        const int co = co0 + ty, ci = ci0 + tx;
+        float s = 0.f;
+        if (co < C_out && ci < C_in) {
+            const T* w = W + ((size_t)co * C_in + ci) * taps;
+            for (int t = 0; t < taps; ++t) s += to_f32(w[t]);
+            if (gwu) gwu[(size_t)co * C_in + ci] = 0.f;
+        }
+        tile[ty][tx] = s;
+    }
+    __syncthreads();
+    const int ci = ci0 + ty, co = co0 + tx;
+    if (ci < C_in && co < C_out) thetaT[(size_t)ci * C_out + co] = __float2bfloat16_rn(tile[tx][ty]);
 }
 
 // ================================================================== host side
@@ -434,8 +555,7 @@ static FlatSrc make_flat(const void* base, int C, int P, long long k_total) {
     FlatSrc s;
     s.base = static_cast<const __nv_bfloat16*>(base);
     s.C = C; s.P = P; s.k_total = k_total; s.div_P = FastDiv((uint32_t)P);
-    s.V = (P % 8 == 0) ? 8 : (P % 4 == 0) ? 4 : (P % 2 == 0) ? 2 : 1;
-    s.logV = s.V == 8 ? 3 : s.V == 4 ? 2 : s.V == 2 ? 1 : 0;
+    s.logV = (P % 8 == 0) ? 3 : (P % 4 == 0) ? 2 : (P % 2 == 0) ? 1 : 0;
     return s;
 }
 
@@ -455,31 +575,54 @@ int tc_gw_splits(const Geo& g) {
     return s;
 }
 
-gf_status launch_ksum_t(const void* W, const Geo& g, __nv_bfloat16* thetaT, uint32_t* err_word, cudaStream_t s) {
+gf_status launch_ksum_t(const void* W, const Geo& g, __nv_bfloat16* thetaT, float* gwu, uint32_t* err_word,
+                        cudaStream_t s) {
     ProfScope prof(K_KSUM, s);
-    const int n = g.C_in * g.C_out, taps = g.KH * g.KW;
-    const int grid = (n + 255) / 256;
-    if (g.dtype == GF_F32) ksum_t_kernel<float><<<grid, 256, 0, s>>>((const float*)W, thetaT, g.C_in, g.C_out, taps, err_word);
-    else ksum_t_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16*)W, thetaT, g.C_in, g.C_out, taps, err_word);
+    const int taps = g.KH * g.KW;
+    dim3 grid((g.C_in + 31) / 32, (g.C_out + 31) / 32, 1);
+    if (grid.y > 65535) return GF_ERR_UNSUPPORTED;
+    if (g.dtype == GF_F32) ksum_t_kernel<float><<<grid, 1024, 0, s>>>((const float*)W, thetaT, gwu, g.C_in, g.C_out, taps, err_word);
+    else ksum_t_kernel<__nv_bfloat16><<<grid, 1024, 0, s>>>((const __nv_bfloat16*)W, thetaT, gwu, g.C_in, g.C_out, taps, err_word);
+    return after_launch();
+}
+
+static int sm_count_tc() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = 148;
+    }
+    return n;
+}
+
+template <typename TOut, int NT, int R, int LOGV>
+static gf_status launch_gx_tc_inst(const GxTcParams& p, cudaStream_t s) {
+    constexpr size_t smem = (size_t)kGxStages * (128 * kTcBK * 2 + kTcBK * NT * 2) + (size_t)128 * (NT + 1) * 4 + 1024;
+    static bool configured = false;
+    if (!configured) {
+        GF_CUDA_TRY(cudaFuncSetAttribute(gx_tc_kernel<TOut, NT, R, LOGV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        configured = true;
+    }
+    const int grid = p.items < sm_count_tc() ? p.items : sm_count_tc();
+    gx_tc_kernel<TOut, NT, R, LOGV><<<grid, kGxThreads, smem, s>>>(p);
     return after_launch();
 }
 
 template <typename TOut, int NT, int R>
-static gf_status launch_gx_tc_inst(const GxTcParams& p, dim3 grid, cudaStream_t s) {
-    constexpr size_t smem = (size_t)kTcStages * (128 * kTcBK * 2 + kTcBK * NT * 2) + 1024;
-    static bool configured = false;
-    if (!configured) {
-        GF_CUDA_TRY(cudaFuncSetAttribute(gx_tc_kernel<TOut, NT, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        configured = true;
+static gf_status launch_gx_tc_v(const GxTcParams& p, cudaStream_t s) {
+    switch (p.gbar.logV) {
+        case 3: return launch_gx_tc_inst<TOut, NT, R, 3>(p, s);
+        case 2: return launch_gx_tc_inst<TOut, NT, R, 2>(p, s);
+        case 1: return launch_gx_tc_inst<TOut, NT, R, 1>(p, s);
+        default: return launch_gx_tc_inst<TOut, NT, R, 0>(p, s);
     }
-    gx_tc_kernel<TOut, NT, R><<<grid, kTcThreads, smem, s>>>(p);
-    return after_launch();
 }
 
 gf_status launch_gx_tc(const __nv_bfloat16* gbar, const __nv_bfloat16* thetaT, void* gX, uint32_t* err_word,
                        const Geo& g, cudaStream_t s) {
     ProfScope prof(K_GX_TC, s);
-    constexpr int NT = 128;
+    constexpr int NT = 64;
     GxTcParams p;
     const int P = g.Hp * g.Wp;
     p.gbar = make_flat(gbar, g.C_out, P, (long long)g.N * P);
@@ -487,17 +630,33 @@ gf_status launch_gx_tc(const __nv_bfloat16* gbar, const __nv_bfloat16* thetaT, v
     p.gX = gX; p.err_word = err_word;
     p.N = g.N; p.C_in = g.C_in; p.C_out = g.C_out; p.H = g.H; p.W = g.W; p.r = g.r; p.Hp = g.Hp; p.Wp = g.Wp; p.P = P;
     p.div_Wp = FastDiv((uint32_t)g.Wp);
+    p.n_ci_tiles = (g.C_in + 127) / 128;
+    p.div_ci_tiles = FastDiv((uint32_t)p.n_ci_tiles);
     const long long col_tiles = ((long long)g.N * P + NT - 1) / NT;
-    if (col_tiles > 0x7fffffffLL || (g.C_in + 127) / 128 > 65535) return GF_ERR_UNSUPPORTED;
-    dim3 grid((unsigned)col_tiles, (g.C_in + 127) / 128, 1);
+    const long long items = col_tiles * p.n_ci_tiles;
+    const int n_chunks = (g.C_out + kTcBK - 1) / kTcBK;
+    if (items * n_chunks > 0x7fffffffLL) return GF_ERR_UNSUPPORTED;
+    p.items = (int)items;
     const int R = (g.W % g.r == 0 && (g.r == 2 || g.r == 4 || g.r == 8)) ? g.r : 0;
-    if (R == 2) return launch_gx_tc_inst<__nv_bfloat16, NT, 2>(p, grid, s);
-    if (R == 4) return launch_gx_tc_inst<__nv_bfloat16, NT, 4>(p, grid, s);
-    if (R == 8) return launch_gx_tc_inst<__nv_bfloat16, NT, 8>(p, grid, s);
-    return launch_gx_tc_inst<__nv_bfloat16, NT, 0>(p, grid, s);
+    if (R == 2) return launch_gx_tc_v<__nv_bfloat16, NT, 2>(p, s);
+    if (R == 4) return launch_gx_tc_v<__nv_bfloat16, NT, 4>(p, s);
+    if (R == 8) return launch_gx_tc_v<__nv_bfloat16, NT, 8>(p, s);
+    return launch_gx_tc_v<__nv_bfloat16, NT, 0>(p, s);
 }
 
-gf_status launch_gw_tc(const __nv_bfloat16* gbar, const __nv_bfloat16* stash, float* part, int splits,
+template <int NT, int LOGV>
+static gf_status launch_gw_tc_inst(const GwTcParams& p, dim3 grid, cudaStream_t s) {
+    constexpr size_t smem = (size_t)kGwStages * (128 * kTcBK * 2 + NT * kTcBK * 2) + 1024;
+    static bool configured = false;
+    if (!configured) {
+        GF_CUDA_TRY(cudaFuncSetAttribute(gw_tc_kernel<NT, LOGV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        configured = true;
+    }
+    gw_tc_kernel<NT, LOGV><<<grid, kGwThreads, smem, s>>>(p);
+    return after_launch();
+}
+
+gf_status launch_gw_tc(const __nv_bfloat16* gbar, const __nv_bfloat16* stash, float* gwu, int splits,
                        uint32_t* err_word, const Geo& g, cudaStream_t s) {
     ProfScope prof(K_GW_TC, s);
     constexpr int NT = 128;
@@ -506,18 +665,16 @@ gf_status launch_gw_tc(const __nv_bfloat16* gbar, const __nv_bfloat16* stash, fl
     const long long K = (long long)g.N * P;
     p.gbar = make_flat(gbar, g.C_out, P, K);
     p.stash = make_flat(stash, g.C_in, P, K);
-    p.part = part; p.err_word = err_word; p.C_in = g.C_in; p.C_out = g.C_out; p.S = splits;
+    p.gwu = gwu; p.err_word = err_word; p.C_in = g.C_in; p.C_out = g.C_out; p.S = splits;
     p.chunks_total = (int)((K + kTcBK - 1) / kTcBK);
-    constexpr size_t smem = (size_t)kTcStages * (128 * kTcBK * 2 + NT * kTcBK * 2) + 1024;
-    static bool configured = false;
-    if (!configured) {
-        GF_CUDA_TRY(cudaFuncSetAttribute(gw_tc_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        configured = true;
-    }
     if ((g.C_out + 127) / 128 > 65535 || splits > 65535) return GF_ERR_UNSUPPORTED;
     dim3 grid((g.C_in + NT - 1) / NT, (g.C_out + 127) / 128, splits);
-    gw_tc_kernel<NT><<<grid, kTcThreads, smem, s>>>(p);
-    return after_launch();
+    switch (p.gbar.logV) {
+        case 3: return launch_gw_tc_inst<NT, 3>(p, grid, s);
+        case 2: return launch_gw_tc_inst<NT, 2>(p, grid, s);
+        case 1: return launch_gw_tc_inst<NT, 1>(p, grid, s);
+        default: return launch_gw_tc_inst<NT, 0>(p, grid, s);
+    }
 }
 
 }  // namespace gf
