@@ -134,11 +134,12 @@ __device__ __forceinline__ void load_kmajor_scalar(unsigned char* tile, const Fl
     }
 }
 template <int NT, int NTHR>
-__device__ __forceinline__ void load_mnmajor_scalar(unsigned char* tile, const FlatSrc& s, int c0, long long j0, int tid) {
+__device__ __forceinline__ void load_mnmajor_scalar(unsigned char* tile, const FlatSrc& s, int c0, long long j0,
+                                                    int ncols, int tid) {
     for (int id = tid; id < kTcBK * NT; id += NTHR) {
         const int krow = id / NT, j = id - krow * NT;
         unsigned short v = 0;
-        if (c0 + krow < s.C && j0 + j < s.k_total)
+        if (c0 + krow < s.C && j < ncols)
             v = __ldg(reinterpret_cast<const unsigned short*>(flat_ptr(s, c0 + krow, j0 + j)));
         *reinterpret_cast<unsigned short*>(tile + mnmajor_off(krow, j)) = v;
     }
@@ -217,7 +218,8 @@ struct GxTcParams {
     uint32_t* err_word;
     int N, C_in, C_out, H, W, r, Hp, Wp, P;
     int n_ci_tiles, items;
-    FastDiv div_Wp, div_ci_tiles;
+    int tile_cols;                      // flattened columns per tile: whole patch rows (R > 0) or NT
+    FastDiv div_Wp, div_Hp, div_RWp, div_ci_tiles;
 };
 
 // R consecutive copies of v
@@ -240,8 +242,10 @@ struct GxShared {
     uint32_t tmem_base;
 };
 
-// R > 0: r == R and r | W (every patch row segment is a whole, aligned vector);
-// R == 0: any r, element-wise stores clipped at the right and bottom edges.
+// R > 0: r == R, r | W and Wp <= NT.  A tile is a run of whole patch rows (of consecutive
+//        images), so its part of a g_X plane is made of whole pixel rows and the stores
+//        follow memory order: consecutive lanes write consecutive R-element vectors.
+// R == 0: any r; a tile is NT flattened patches, element-wise stores clipped at the edges.
 // LOGV: log2 of the piece width of gbar (0: 2-byte pieces through registers).
 template <typename TOut, int NT, int R, int LOGV>
 __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p) {
@@ -249,11 +253,15 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
     constexpr int kBBytes = kTcBK * NT * 2;              // 64 k x NT columns
     constexpr int kStageBytes = kABytes + kBBytes;
     constexpr int kColsPerLane = NT / 32;
+    constexpr int kUnits = R > 0 ? NT * R : 1;           // R-element vectors of a tile's part of one plane
+    constexpr int kColTab = R == 0 ? NT : 1;
     constexpr uint32_t kIdesc = umma_idesc_bf16(128, NT, /*A K-major*/ 0, /*B MN-major*/ 1);
     extern __shared__ unsigned char dyn_raw[];
     __shared__ GxShared sh;
-    __shared__ long long col_off[NT];     // g_X offset of a column's patch | rows inside the map << 56; -1: no column
-    __shared__ int col_cols[NT];          // columns of the patch inside the map (R == 0 only)
+    __shared__ long long unit_off[kUnits];        // R > 0: g_X offset of a vector (plane 0 of its image's c_i0), -1: none
+    __shared__ unsigned short unit_src[kUnits];   //        column of the tile it replicates
+    __shared__ long long col_off[kColTab];        // R == 0: g_X offset of a column's patch, -1: no column
+    __shared__ int col_cols[kColTab];             //         columns | rows << 16 of the patch inside the map
     unsigned char* dyn = align1024(dyn_raw);
     float* D = reinterpret_cast<float*>(dyn + (size_t)kGxStages * kStageBytes);   // [128][NT+1]
 
@@ -273,11 +281,12 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
     tc_fence_after_sync();
     const uint32_t tmem = sh.tmem_base;
     bool ok = true;
-    auto item_of = [&](int it, int& ci0, long long& col0) {
+    auto item_of = [&](int it, int& ci0, long long& col0, int& ncols) {
         uint32_t ct, cit;
         p.div_ci_tiles.divmod((uint32_t)(first + it * stride), ct, cit);
         ci0 = (int)cit * 128;
-        col0 = (long long)ct * NT;
+        col0 = (long long)ct * p.tile_cols;
+        ncols = (int)min((long long)p.tile_cols, p.gbar.k_total - col0);
     };
 
     if (warp < kGxLoaders / 32) {
@@ -295,12 +304,12 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
                 const int it = q / n_chunks, kc = q - it * n_chunks;
                 if (it != cur_it) {                        // per item: this thread's first source elements
                     long long col0;
-                    item_of(it, ci0, col0);
+                    int ncols;
+                    item_of(it, ci0, col0, ncols);
                     cur_it = it;
                     a_src = p.thetaT.base + (size_t)(ci0 + pa.row0) * p.C_out + pa.k;
-                    const long long col = col0 + pb.j;
-                    b_ok = col < p.gbar.k_total;
-                    b_src = flat_ptr(p.gbar, pb.krow0, b_ok ? col : 0);
+                    b_ok = pb.j < ncols;
+                    b_src = flat_ptr(p.gbar, pb.krow0, b_ok ? col0 + pb.j : 0);
                 }
                 const int k0 = kc * kTcBK;
                 pa.issue(tile, a_src + k0, (size_t)p.C_out, p.C_in - ci0 - pa.row0, k0 + pa.k < p.C_out, p.thetaT.base);
@@ -311,10 +320,10 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
             ok = run_sync_loaders<kGxStages>(sh.full, sh.empty, dyn, kStageBytes, n_my * n_chunks,
                                              [&](int q, unsigned char* tile) {
                 const int it = q / n_chunks, kc = q - it * n_chunks;
-                int ci0; long long col0;
-                item_of(it, ci0, col0);
+                int ci0, ncols; long long col0;
+                item_of(it, ci0, col0, ncols);
                 load_kmajor_scalar<128, kGxLoaders>(tile, p.thetaT, ci0, (long long)kc * kTcBK, tid);
-                load_mnmajor_scalar<NT, kGxLoaders>(tile + kABytes, p.gbar, kc * kTcBK, col0, tid);
+                load_mnmajor_scalar<NT, kGxLoaders>(tile + kABytes, p.gbar, kc * kTcBK, col0, ncols, tid);
             });
         }
     } else if (warp == kGxMmaWarp) {
@@ -336,24 +345,37 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
         const size_t plane = (size_t)p.H * p.W;
         for (int it = 0; it < n_my; ++it) {
             const int buf = it & 1;
-            int ci0; long long col0;
-            item_of(it, ci0, col0);
-            for (int j = et; j < NT; j += kGxEpi) {      // patch offsets of this tile's columns
-                const long long c = col0 + j;
-                long long off = -1;
-                int ncols = 0;
-                if (c < p.gbar.k_total) {
-                    const uint32_t n = p.gbar.div_P.div((uint32_t)c), pp = (uint32_t)c - n * (uint32_t)p.P;
-                    uint32_t a, b;
-                    p.div_Wp.divmod(pp, a, b);
-                    off = (long long)n * p.C_in * p.H * p.W + (long long)a * p.r * p.W + (long long)b * p.r;
-                    const int nrows = min(p.r, p.H - (int)a * p.r);
-                    ncols = min(p.r, p.W - (int)b * p.r);
-                    if constexpr (R > 0) off |= (long long)nrows << 56;
-                    else ncols |= nrows << 16;
+            int ci0, ncols; long long col0;
+            item_of(it, ci0, col0, ncols);
+            if constexpr (R > 0) {
+                // vector u of the tile's part of a plane, in memory order: patch row ta of the tile,
+                // pixel row dr of that patch row, patch jb of the row
+                const uint32_t A0 = p.div_Wp.div((uint32_t)col0);          // first global patch row
+                for (int u = et; u < ncols * R; u += kGxEpi) {
+                    uint32_t ta, rem, dr, jb, n, a;
+                    p.div_RWp.divmod((uint32_t)u, ta, rem);
+                    p.div_Wp.divmod(rem, dr, jb);
+                    p.div_Hp.divmod(A0 + ta, n, a);
+                    const int row = (int)a * R + (int)dr;
+                    unit_off[u] = row < p.H ? (long long)n * p.C_in * p.H * p.W + (long long)row * p.W + (long long)jb * R
+                                            : -1;
+                    unit_src[u] = (unsigned short)(ta * p.Wp + jb);
                 }
-                col_off[j] = off;
-                if constexpr (R == 0) col_cols[j] = ncols;
+            } else {
+                for (int j = et; j < NT; j += kGxEpi) {      // patch offsets of this tile's columns
+                    long long off = -1;
+                    int ext = 0;
+                    if (j < ncols) {
+                        const long long c = col0 + j;
+                        const uint32_t n = p.gbar.div_P.div((uint32_t)c), pp = (uint32_t)c - n * (uint32_t)p.P;
+                        uint32_t a, b;
+                        p.div_Wp.divmod(pp, a, b);
+                        off = (long long)n * p.C_in * p.H * p.W + (long long)a * p.r * p.W + (long long)b * p.r;
+                        ext = min(p.r, p.W - (int)b * p.r) | (min(p.r, p.H - (int)a * p.r) << 16);
+                    }
+                    col_off[j] = off;
+                    col_cols[j] = ext;
+                }
             }
             if (ok) ok = mbar_wait_bounded(&sh.acc_full[buf], (uint32_t)(it >> 1) & 1u);
             tc_fence_after_sync();
@@ -373,33 +395,31 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
             asm volatile("bar.sync 1, 256;" ::: "memory");
             if (et == 0) mbar_arrive(&sh.acc_empty[buf]);   // the accumulator may be overwritten
             if (ok) {
-                // expansion: a lane owns the columns lane, lane+32, ...; value (m, j) goes to r
-                // consecutive pixels on each of r rows of plane c_i0 + m
                 const int m_cnt = min(128, p.C_in - ci0);
                 TOut* base = gx + (size_t)ci0 * plane;
-#pragma unroll
-                for (int t = 0; t < kColsPerLane; ++t) {
-                    const int j = lane + 32 * t;
-                    const long long info = col_off[j];
-                    if (info < 0) continue;
-                    if constexpr (R > 0) {
-                        TOut* dst0 = base + (info & 0x00ffffffffffffffLL);
-                        const int nrows = (int)(info >> 56);
+                if constexpr (R > 0) {
+                    // expansion in memory order: lane l writes the vectors l, l+32, ... of every plane
+                    const int n_units = ncols * R;
+                    for (int u = lane; u < n_units; u += 32) {
+                        const long long off = unit_off[u];
+                        if (off < 0) continue;
+                        const float* dcol = D + unit_src[u];
+                        TOut* dst0 = base + off;
 #pragma unroll 4
-                        for (int m = ew; m < m_cnt; m += 8) {
-                            const float v = D[m * (NT + 1) + j];
-                            TOut* dst = dst0 + (size_t)m * plane;
+                        for (int m = ew; m < m_cnt; m += 8) store_rep<R>(dst0 + (size_t)m * plane, dcol[m * (NT + 1)]);
+                    }
+                } else {
 #pragma unroll
-                            for (int dr = 0; dr < R; ++dr)
-                                if (dr < nrows) store_rep<R>(dst + (size_t)dr * p.W, v);
-                        }
-                    } else {
-                        const int ext = col_cols[j], ncols = ext & 0xffff, nrows = ext >> 16;
+                    for (int t = 0; t < kColsPerLane; ++t) {
+                        const int j = lane + 32 * t;
+                        const long long off = col_off[j];
+                        if (off < 0) continue;
+                        const int ext = col_cols[j], ncl = ext & 0xffff, nrows = ext >> 16;
                         for (int m = ew; m < m_cnt; m += 8) {
                             const TOut o = from_f32<TOut>(D[m * (NT + 1) + j]);
-                            TOut* dst = base + info + (size_t)m * plane;
+                            TOut* dst = base + off + (size_t)m * plane;
                             for (int dr = 0; dr < nrows; ++dr)
-                                for (int dc = 0; dc < ncols; ++dc) dst[(size_t)dr * p.W + dc] = o;
+                                for (int dc = 0; dc < ncl; ++dc) dst[(size_t)dr * p.W + dc] = o;
                         }
                     }
                 }
@@ -630,14 +650,22 @@ gf_status launch_gx_tc(const __nv_bfloat16* gbar, const __nv_bfloat16* thetaT, v
     p.gX = gX; p.err_word = err_word;
     p.N = g.N; p.C_in = g.C_in; p.C_out = g.C_out; p.H = g.H; p.W = g.W; p.r = g.r; p.Hp = g.Hp; p.Wp = g.Wp; p.P = P;
     p.div_Wp = FastDiv((uint32_t)g.Wp);
+    p.div_Hp = FastDiv((uint32_t)g.Hp);
     p.n_ci_tiles = (g.C_in + 127) / 128;
     p.div_ci_tiles = FastDiv((uint32_t)p.n_ci_tiles);
-    const long long col_tiles = ((long long)g.N * P + NT - 1) / NT;
+    const int R = (g.W % g.r == 0 && g.Wp <= NT && (g.r == 2 || g.r == 4 || g.r == 8)) ? g.r : 0;
+    p.div_RWp = FastDiv((uint32_t)((R > 0 ? R : 1) * g.Wp));
+    p.tile_cols = R > 0 ? (NT / g.Wp) * g.Wp : NT;
+    {   // pieces must not straddle a tile start: the piece width divides tile_cols as well as P
+        int lv = p.gbar.logV;
+        while (lv > 0 && (p.tile_cols % (1 << lv)) != 0) --lv;
+        p.gbar.logV = lv;
+    }
+    const long long col_tiles = ((long long)g.N * P + p.tile_cols - 1) / p.tile_cols;
     const long long items = col_tiles * p.n_ci_tiles;
     const int n_chunks = (g.C_out + kTcBK - 1) / kTcBK;
     if (items * n_chunks > 0x7fffffffLL) return GF_ERR_UNSUPPORTED;
     p.items = (int)items;
-    const int R = (g.W % g.r == 0 && (g.r == 2 || g.r == 4 || g.r == 8)) ? g.r : 0;
     if (R == 2) return launch_gx_tc_v<__nv_bfloat16, NT, 2>(p, s);
     if (R == 4) return launch_gx_tc_v<__nv_bfloat16, NT, 4>(p, s);
     if (R == 8) return launch_gx_tc_v<__nv_bfloat16, NT, 8>(p, s);
