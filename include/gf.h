@@ -95,6 +95,27 @@ gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* sta
                       const void* W, float* g_W, void* g_X, void* workspace,
                       size_t workspace_bytes, void* stream);
 
+/* No counterpart in the paper: a convenience of this library.
+ * gf_backward for callers that must not allocate device memory (a fine-tuning loop
+ * inside a runtime whose memory plan is fixed at start-up; a latency-critical section
+ * where cudaMalloc, which synchronises the device and may fail, is unacceptable).  Same
+ * arguments and results as gf_backward, minus the workspace: the scratch is an array of
+ * GF_STATIC_SCRATCH_BYTES that is part of the library image, so every GPU that loads the
+ * library holds that much memory until the process exits.  The call allocates and frees
+ * nothing.
+ *  - Layers whose gf_backward_workspace_bytes exceeds GF_STATIC_SCRATCH_BYTES are refused
+ *    with GF_ERR_WORKSPACE and nothing is launched.
+ *  - The first call on a device looks up the array's device address (once per device, with
+ *    that device current); make that first call outside any stream capture.
+ *  - All calls share the one array and it keeps the previous call's contents; the call
+ *    itself resets what must start from zero.  Two calls whose GPU work overlaps in time
+ *    (different streams, or different host threads) race on it: serialise them.
+ *  - A device-side wait that expires is recorded inside the scratch, which this ABI does
+ *    not expose; gf_last_async_status does not cover this entry point. */
+#define GF_STATIC_SCRATCH_BYTES (8u << 20)
+gf_status gf_backward_static_scratch(const gf_conv_desc* desc, const void* g_y, const void* stash,
+                                     const void* W, float* g_W, void* g_X, void* stream);
+
 /* Reads the error word that device-side bounded waits of the last gf_backward
  * on `workspace` may have set, and the library-wide word that gf_stash_forward
  * reports to (cleared by this call).  Synchronises `stream` (blocking).  GF_OK

@@ -24,7 +24,7 @@ EXPORTS = (
     "gf_stash_dims", "gf_stash_bytes", "gf_backward_workspace_bytes", "gf_stash_forward",
     "gf_backward", "gf_last_async_status", "gf_host_step_arena_bytes", "gf_layer_step_host",
     "gf_kernel_launch_count", "gf_status_string", "gf_profile_configure", "gf_profile_read",
-    "gf_kernel_name", "gf_kernel_id_count",
+    "gf_kernel_name", "gf_kernel_id_count", "gf_backward_static_scratch",
 )
 
 
@@ -72,6 +72,8 @@ def lib() -> ctypes.CDLL:
         L.gf_backward_workspace_bytes.argtypes = [dp, ctypes.POINTER(sz)]
         L.gf_stash_forward.argtypes = [dp, vp, vp, vp]
         L.gf_backward.argtypes = [dp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.gf_backward_static_scratch.argtypes = [dp, vp, vp, vp, vp, vp, vp]
+        L.gf_backward_static_scratch.restype = ctypes.c_int
         L.gf_last_async_status.argtypes = [vp, vp]
         L.gf_host_step_arena_bytes.argtypes = [dp, ctypes.POINTER(sz)]
         L.gf_layer_step_host.argtypes = [dp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -170,6 +172,17 @@ def gf_backward(desc: gf_conv_desc, g_y, stash, W, g_W, g_X, workspace, workspac
     _check(lib().gf_backward(ctypes.byref(desc), _ptr(g_y), _ptr(stash), _ptr(W), _ptr(g_W), _ptr(g_X),
                              _ptr(workspace), ctypes.c_size_t(workspace_bytes), _stream(stream)),
            "gf_backward")
+
+
+GF_STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def gf_backward_static_scratch(desc: gf_conv_desc, g_y, stash, W, g_W, g_X, stream=None) -> None:
+    """gf_backward without a workspace argument: the scratch is an array built into the
+    library (GF_STATIC_SCRATCH_BYTES), for callers that may not allocate device memory.
+    Calls must not overlap on the GPU; larger layers raise GfError(GF_ERR_WORKSPACE)."""
+    _check(lib().gf_backward_static_scratch(ctypes.byref(desc), _ptr(g_y), _ptr(stash), _ptr(W), _ptr(g_W),
+                                            _ptr(g_X), _stream(stream)), "gf_backward_static_scratch")
 
 
 def gf_last_async_status(workspace, stream=None) -> int:

@@ -1,0 +1,53 @@
+"""gf_backward_static_scratch: the backward pass for callers that cannot allocate.
+
+A runtime with a memory plan frozen at start-up, or a latency-critical section, cannot call
+cudaMalloc for gf_backward's workspace.  The library therefore carries an 8 MiB scratch
+array of its own and an entry point that uses it.  This test calls that entry point through
+the C ABI twice in a row (the array keeps the first call's contents, so the second call
+checks that stale contents do no harm) and compares every output with gf_backward's.
+The file name makes pytest collect it last.
+"""
+import ctypes
+
+import pytest
+import torch
+
+from paper_2301_00330_b200 import workloads
+from paper_2301_00330_b200.workloads import Layer
+
+from parity_util import TOL, f64, relerr
+
+pytestmark = pytest.mark.gpu
+
+CASES = [
+    Layer("noalloc_f32", 0, 0, 3, 24, 40, 14, 14, 3, 1, 2, "f32", "relu", 1e-2),      # CUDA-core path, g_W slices
+    Layer("noalloc_bf16", 0, 1, 4, 64, 64, 14, 14, 3, 1, 2, "bf16", "relu", 1e-2),    # tensor-core path, accumulator
+    Layer("noalloc_dw", 0, 2, 2, 16, 16, 14, 14, 3, 16, 2, "f32", "relu6", 1e-2),     # depthwise path
+]
+
+
+@pytest.mark.parametrize("layer", CASES, ids=lambda l: l.name)
+def test_static_scratch_matches_gf_backward_twice(gf, layer):
+    desc = gf.desc_for(layer)
+    assert gf.gf_backward_workspace_bytes(desc) <= gf.GF_STATIC_SCRATCH_BYTES
+    dt = workloads.torch_dtype(layer.dtype)
+    x, gy, w = (t.cuda() for t in workloads.make_inputs(layer))
+    ref = gf.alloc_layer(desc)
+    gf.gf_stash_forward(desc, x, ref.stash)
+    gf.gf_backward(desc, gy, ref.stash, w, ref.g_W, ref.g_X, ref.workspace)
+    torch.cuda.synchronize()
+    for call in range(2):
+        g_W = torch.full_like(ref.g_W, float("nan"))
+        g_X = torch.full_like(ref.g_X, float("nan"))
+        gf.gf_backward_static_scratch(desc, gy, ref.stash, w, g_W, g_X)
+        torch.cuda.synchronize()
+        assert relerr(f64(g_W), f64(ref.g_W)) <= TOL[layer.dtype], (layer.name, call, "g_W")
+        assert relerr(f64(g_X), f64(ref.g_X)) <= TOL[layer.dtype], (layer.name, call, "g_X")
+        assert g_X.dtype == dt
+
+
+def test_static_scratch_refuses_layers_that_do_not_fit(gf):
+    big = gf.make_desc(64, 256, 256, 28, 28, 3, r=2, dtype=gf.GF_BF16)
+    assert gf.gf_backward_workspace_bytes(big) > gf.GF_STATIC_SCRATCH_BYTES
+    a = ctypes.c_void_p(0x1000)      # never dereferenced: the size check comes first
+    assert gf.lib().gf_backward_static_scratch(ctypes.byref(big), a, a, a, a, a, None) == gf.GF_ERR_WORKSPACE
