@@ -236,6 +236,23 @@ template <int R> __device__ __forceinline__ void store_rep(__nv_bfloat16* dst, f
     else *reinterpret_cast<uint4*>(dst) = make_uint4(w, w, w, w);
 }
 
+// UPC consecutive vectors of R copies each, as whole 16-byte stores (dst 16-byte aligned)
+template <int R, int UPC> __device__ __forceinline__ void store_chunk(float* dst, const float (&v)[UPC]) {
+    if constexpr (R == 2) *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[0], v[1], v[1]);
+    else store_rep<R>(dst, v[0]);
+}
+template <int R, int UPC> __device__ __forceinline__ void store_chunk(__nv_bfloat16* dst, const float (&v)[UPC]) {
+    uint32_t w[UPC];
+#pragma unroll
+    for (int i = 0; i < UPC; ++i) {
+        const __nv_bfloat162 b2 = __float2bfloat162_rn(v[i]);
+        w[i] = *reinterpret_cast<const uint32_t*>(&b2);
+    }
+    if constexpr (R == 2) *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+    else if constexpr (R == 4) *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[0], w[1], w[1]);
+    else *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[0], w[0], w[0]);
+}
+
 struct GxShared {
     uint64_t full[kGxStages], empty[kGxStages];
     uint64_t acc_full[2], acc_empty[2];
@@ -398,15 +415,42 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
                 const int m_cnt = min(128, p.C_in - ci0);
                 TOut* base = gx + (size_t)ci0 * plane;
                 if constexpr (R > 0) {
-                    // expansion in memory order: lane l writes the vectors l, l+32, ... of every plane
+                    // expansion in memory order, 16 bytes per store where possible: lane l owns the
+                    // chunks l, l+32, ... of UPC consecutive vectors each, for every plane
+                    constexpr int UPC = (16 / (R * (int)sizeof(TOut))) > 1 ? 16 / (R * (int)sizeof(TOut)) : 1;
                     const int n_units = ncols * R;
-                    for (int u = lane; u < n_units; u += 32) {
-                        const long long off = unit_off[u];
-                        if (off < 0) continue;
-                        const float* dcol = D + unit_src[u];
-                        TOut* dst0 = base + off;
+                    const bool plane_al = (plane * sizeof(TOut)) % 16 == 0 &&
+                                          (reinterpret_cast<uintptr_t>(gx) & 15) == 0;
+                    for (int u0 = lane * UPC; u0 < n_units; u0 += 32 * UPC) {
+                        long long off[UPC];
+                        int src[UPC];
+                        bool vec = plane_al && (u0 + UPC <= n_units);
+#pragma unroll
+                        for (int i = 0; i < UPC; ++i) {
+                            const bool in = u0 + i < n_units;
+                            off[i] = in ? unit_off[u0 + i] : -1;
+                            src[i] = in ? unit_src[u0 + i] : 0;
+                            vec = vec && off[i] >= 0 && off[i] == off[0] + (long long)i * R;
+                        }
+                        vec = vec && ((off[0] + (long long)ci0 * (long long)plane) * (long long)sizeof(TOut)) % 16 == 0;
+                        if (vec) {
+                            TOut* dst0 = base + off[0];
 #pragma unroll 4
-                        for (int m = ew; m < m_cnt; m += 8) store_rep<R>(dst0 + (size_t)m * plane, dcol[m * (NT + 1)]);
+                            for (int m = ew; m < m_cnt; m += 8) {
+                                float v[UPC];
+#pragma unroll
+                                for (int i = 0; i < UPC; ++i) v[i] = D[m * (NT + 1) + src[i]];
+                                store_chunk<R, UPC>(dst0 + (size_t)m * plane, v);
+                            }
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < UPC; ++i) {
+                                if (off[i] < 0) continue;
+                                TOut* dst0 = base + off[i];
+                                for (int m = ew; m < m_cnt; m += 8)
+                                    store_rep<R>(dst0 + (size_t)m * plane, D[m * (NT + 1) + src[i]]);
+                            }
+                        }
                     }
                 } else {
 #pragma unroll
