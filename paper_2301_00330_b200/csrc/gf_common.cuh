@@ -38,6 +38,29 @@ static inline gf_status after_launch() {
     return cudaPeekAtLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
 }
 
+// ---- programmatic dependent launch ---------------------------------------------------
+// Kernels launched through launch_pdl may be scheduled while the previous kernel of the
+// stream is still draining: their blocks run their set-up, then pdl_wait() blocks until
+// that previous kernel has completed and its writes are visible.  Every such kernel
+// calls pdl_launch_dependents() first (the next kernel may start being scheduled) and
+// pdl_wait() before it touches global memory, so stream order is preserved.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+static inline gf_status launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                   Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+    count_launch();
+    return e == cudaSuccess ? GF_OK : GF_ERR_CUDA;
+}
+
 static inline int64_t cdiv64(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
 // ---- division by a runtime constant ---------------------------------------

@@ -199,6 +199,8 @@ gf_status launch_gw_partial(const float* gbar, const void* stash, float* part, i
 // ---------------------------------------------------------------- gw_finish
 __global__ void gw_finish_kernel(const float* __restrict__ part, int S, size_t n_pairs, int taps,
                                  FastDiv div_taps, float* __restrict__ gW) {
+    pdl_launch_dependents();
+    pdl_wait();
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n_pairs * taps) return;
     const uint32_t pair = div_taps.div((uint32_t)i);
@@ -219,8 +221,8 @@ gf_status launch_gw_finish(const float* part, int splits, float* gW, const Geo& 
     const int taps = g.KH * g.KW;
     const size_t total = n_pairs * taps;
     if (total > 0x7fffffffULL) return GF_ERR_UNSUPPORTED;
-    gw_finish_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(part, splits, n_pairs, taps, FastDiv(taps), gW);
-    return after_launch();
+    return launch_pdl(gw_finish_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, s, part, splits, n_pairs,
+                      taps, FastDiv(taps), gW);
 }
 
 }  // namespace gf

@@ -197,11 +197,13 @@ __global__ void __launch_bounds__(kStreamThreads, 1) pool_stream_kernel(const Po
             bulk_g2s(buf(s), in + tile * p.S * strip_elems, bytes, &full[s]);
         }
     };
+    pdl_launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStreamStages; ++s) mbar_init(&full[s], 1);
         mbar_fence_init();
     }
     __syncthreads();
+    pdl_wait();                       // the input may come from the previous kernel of the stream
     if (threadIdx.x == 0)
         for (int it = 0; it < kStreamStages && it < n_my; ++it) issue(it);
 
@@ -362,8 +364,7 @@ static gf_status launch_stream_inst(const PoolParams& p, cudaStream_t s) {
         configured = true;
     }
     const long long grid = p.tiles < sm_count() ? p.tiles : sm_count();
-    pool_stream_kernel<TIn, TOut, R, G><<<(unsigned)grid, kStreamThreads, smem, s>>>(p);
-    return after_launch();
+    return launch_pdl(pool_stream_kernel<TIn, TOut, R, G>, dim3((unsigned)grid), dim3(kStreamThreads), smem, s, p);
 }
 
 template <typename TIn, typename TOut>

@@ -26,12 +26,12 @@ namespace gf {
 constexpr int kTcBK = 64;           // K elements per stage (one 128-byte swizzled row)
 constexpr int kGwLoaders = 256;     // gw_tc: 8 loader / epilogue warps + 1 MMA warp
 constexpr int kGwThreads = 288;
-constexpr int kGwStages = 3;
+constexpr int kGwStages = 6;
 constexpr int kGxLoaders = 256;     // gx_tc: 8 loader warps, 8 epilogue warps, 1 MMA warp
 constexpr int kGxEpi = 256;
 constexpr int kGxThreads = kGxLoaders + kGxEpi + 32;
 constexpr int kGxMmaWarp = (kGxLoaders + kGxEpi) / 32;
-constexpr int kGxStages = 4;
+constexpr int kGxStages = 7;
 
 // Source of an operand: a [n][C][P] bf16 array read along the flattened index
 // k = n*P + p (row c is a channel).  A plain [rows][pitch] matrix is the case P = pitch,
@@ -287,6 +287,7 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
     const int first = blockIdx.x, stride = gridDim.x;
     const int n_my = first < p.items ? (p.items - first + stride - 1) / stride : 0;
 
+    pdl_launch_dependents();
     if (tid == 0) {
         for (int s = 0; s < kGxStages; ++s) { mbar_init(&sh.full[s], kGxLoaders); mbar_init(&sh.empty[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&sh.acc_full[b], 1); mbar_init(&sh.acc_empty[b], 1); }
@@ -297,6 +298,7 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = sh.tmem_base;
+    pdl_wait();                       // operands come from the previous kernels of the stream
     bool ok = true;
     auto item_of = [&](int it, int& ci0, long long& col0, int& ncols) {
         uint32_t ct, cit;
@@ -515,6 +517,7 @@ __global__ void __launch_bounds__(kGwThreads) gw_tc_kernel(const GwTcParams p) {
     const int kc_end = (int)((long long)p.chunks_total * (split + 1) / p.S);
     const int n_chunks = kc_end - kc_begin;
 
+    pdl_launch_dependents();
     if (tid == 0) {
         for (int s = 0; s < kGwStages; ++s) { mbar_init(&sh.full[s], kGwLoaders); mbar_init(&sh.empty[s], 1); }
         mbar_init(&sh.accum, 1);
@@ -525,6 +528,7 @@ __global__ void __launch_bounds__(kGwThreads) gw_tc_kernel(const GwTcParams p) {
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = sh.tmem_base;
+    pdl_wait();                       // operands come from the previous kernels of the stream
     bool ok = true;
 
     if (warp < 8) {
@@ -596,6 +600,8 @@ __global__ void __launch_bounds__(1024) ksum_t_kernel(const T* __restrict__ W, _
                                                       float* __restrict__ gwu, int C_in, int C_out, int taps,
                                                       uint32_t* err_word) {
     __shared__ float tile[32][33];
+    pdl_launch_dependents();
+    pdl_wait();
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
     const int co0 = blockIdx.y * 32, ci0 = blockIdx.x * 32;
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0 && err_word) *err_word = 0u;
@@ -645,9 +651,11 @@ gf_status launch_ksum_t(const void* W, const Geo& g, __nv_bfloat16* thetaT, floa
     const int taps = g.KH * g.KW;
     dim3 grid((g.C_in + 31) / 32, (g.C_out + 31) / 32, 1);
     if (grid.y > 65535) return GF_ERR_UNSUPPORTED;
-    if (g.dtype == GF_F32) ksum_t_kernel<float><<<grid, 1024, 0, s>>>((const float*)W, thetaT, gwu, g.C_in, g.C_out, taps, err_word);
-    else ksum_t_kernel<__nv_bfloat16><<<grid, 1024, 0, s>>>((const __nv_bfloat16*)W, thetaT, gwu, g.C_in, g.C_out, taps, err_word);
-    return after_launch();
+    if (g.dtype == GF_F32)
+        return launch_pdl(ksum_t_kernel<float>, grid, dim3(1024), 0, s, (const float*)W, thetaT, gwu, g.C_in, g.C_out,
+                          taps, err_word);
+    return launch_pdl(ksum_t_kernel<__nv_bfloat16>, grid, dim3(1024), 0, s, (const __nv_bfloat16*)W, thetaT, gwu, g.C_in,
+                      g.C_out, taps, err_word);
 }
 
 static int sm_count_tc() {
@@ -669,8 +677,7 @@ static gf_status launch_gx_tc_inst(const GxTcParams& p, cudaStream_t s) {
         configured = true;
     }
     const int grid = p.items < sm_count_tc() ? p.items : sm_count_tc();
-    gx_tc_kernel<TOut, NT, R, LOGV><<<grid, kGxThreads, smem, s>>>(p);
-    return after_launch();
+    return launch_pdl(gx_tc_kernel<TOut, NT, R, LOGV>, dim3(grid), dim3(kGxThreads), smem, s, p);
 }
 
 template <typename TOut, int NT, int R>
@@ -724,8 +731,7 @@ static gf_status launch_gw_tc_inst(const GwTcParams& p, dim3 grid, cudaStream_t 
         GF_CUDA_TRY(cudaFuncSetAttribute(gw_tc_kernel<NT, LOGV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         configured = true;
     }
-    gw_tc_kernel<NT, LOGV><<<grid, kGwThreads, smem, s>>>(p);
-    return after_launch();
+    return launch_pdl(gw_tc_kernel<NT, LOGV>, grid, dim3(kGwThreads), smem, s, p);
 }
 
 gf_status launch_gw_tc(const __nv_bfloat16* gbar, const __nv_bfloat16* stash, float* gwu, int splits,
