@@ -192,14 +192,12 @@ __device__ __forceinline__ bool run_sync_loaders(uint64_t* full, uint64_t* empty
 // b_step = start-address advance of the B descriptor per step (32 bytes K-major, 2048
 // bytes MN-major); b_lbo = its leading byte offset.
 template <int STAGES>
-__device__ __forceinline__ bool mma_chunk(uint64_t* full, uint64_t* empty, unsigned char* dyn, int stage_bytes,
-                                          int a_bytes, int q, bool first, uint32_t d_tmem, uint32_t idesc,
-                                          uint32_t b_step, uint32_t b_lbo) {
+__device__ __forceinline__ bool mma_chunk(uint64_t* full, uint64_t* empty, int q, bool first, uint32_t a_addr,
+                                          uint32_t b_addr, uint32_t d_tmem, uint32_t idesc, uint32_t b_step,
+                                          uint32_t b_lbo) {
     const int s = q % STAGES;
     if (!mbar_wait_bounded(&full[s], (uint32_t)(q / STAGES) & 1u)) return false;
     tc_fence_after_sync();
-    const uint32_t a_addr = smem_u32(dyn + (size_t)s * stage_bytes);
-    const uint32_t b_addr = a_addr + a_bytes;
 #pragma unroll
     for (int ks = 0; ks < kTcBK / 16; ++ks) {
         const uint64_t adesc = umma_smem_desc(a_addr + ks * 32, 16, 1024);
@@ -264,11 +262,15 @@ struct GxShared {
 //        follow memory order: consecutive lanes write consecutive R-element vectors.
 // R == 0: any r; a tile is NT flattened patches, element-wise stores clipped at the edges.
 // LOGV: log2 of the piece width of gbar (0: 2-byte pieces through registers).
-template <typename TOut, int NT, int R, int LOGV>
+// ARES: the CTA keeps one c_i tile for all its items and holds that tile of thetaT (all of
+//       K) resident in shared memory; only the gbar tiles stream through the ring.
+template <typename TOut, int NT, int R, int LOGV, bool ARES>
 __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p) {
     constexpr int kABytes = 128 * kTcBK * 2;             // 16 KB
     constexpr int kBBytes = kTcBK * NT * 2;              // 64 k x NT columns
-    constexpr int kStageBytes = kABytes + kBBytes;
+    constexpr int kStageBytes = ARES ? kBBytes : kABytes + kBBytes;
+    constexpr int kBOff = ARES ? 0 : kABytes;
+    constexpr int kDBytes = (128 * (NT + 1) * 4 + 1023) / 1024 * 1024;
     constexpr int kColsPerLane = NT / 32;
     constexpr int kUnits = R > 0 ? NT * R : 1;           // R-element vectors of a tile's part of one plane
     constexpr int kColTab = R == 0 ? NT : 1;
@@ -281,11 +283,16 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
     __shared__ int col_cols[kColTab];             //         columns | rows << 16 of the patch inside the map
     unsigned char* dyn = align1024(dyn_raw);
     float* D = reinterpret_cast<float*>(dyn + (size_t)kGxStages * kStageBytes);   // [128][NT+1]
+    unsigned char* a_res = dyn + (size_t)kGxStages * kStageBytes + kDBytes;       // ARES: [n_chunks][128][64]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_chunks = (p.C_out + kTcBK - 1) / kTcBK;
-    const int first = blockIdx.x, stride = gridDim.x;
-    const int n_my = first < p.items ? (p.items - first + stride - 1) / stride : 0;
+    // items of this CTA: item = column tile * n_ci_tiles + c_i tile.  ARES: fixed c_i tile
+    // (blockIdx % n_ci_tiles; the grid is a multiple of n_ci_tiles), column tiles strided.
+    const int first = ARES ? (int)(blockIdx.x / p.n_ci_tiles) : (int)blockIdx.x;
+    const int stride = ARES ? (int)(gridDim.x / p.n_ci_tiles) : (int)gridDim.x;
+    const int total = ARES ? p.items / p.n_ci_tiles : p.items;
+    const int n_my = first < total ? (total - first + stride - 1) / stride : 0;
 
     pdl_launch_dependents();
     if (tid == 0) {
@@ -302,7 +309,8 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
     bool ok = true;
     auto item_of = [&](int it, int& ci0, long long& col0, int& ncols) {
         uint32_t ct, cit;
-        p.div_ci_tiles.divmod((uint32_t)(first + it * stride), ct, cit);
+        if constexpr (ARES) { ct = (uint32_t)(first + it * stride); cit = blockIdx.x % (uint32_t)p.n_ci_tiles; }
+        else p.div_ci_tiles.divmod((uint32_t)(first + it * stride), ct, cit);
         ci0 = (int)cit * 128;
         col0 = (long long)ct * p.tile_cols;
         ncols = (int)min((long long)p.tile_cols, p.gbar.k_total - col0);
@@ -331,8 +339,16 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
                     b_src = flat_ptr(p.gbar, pb.krow0, b_ok ? col0 + pb.j : 0);
                 }
                 const int k0 = kc * kTcBK;
-                pa.issue(tile, a_src + k0, (size_t)p.C_out, p.C_in - ci0 - pa.row0, k0 + pa.k < p.C_out, p.thetaT.base);
-                pb.issue(tile + kABytes, b_src + (size_t)k0 * p.P, (size_t)p.P, p.C_out - k0 - pb.krow0, b_ok,
+                if constexpr (ARES) {
+                    if (q == 0)      // the resident thetaT tile rides in the first copy group
+                        for (int c = 0; c < n_chunks; ++c)
+                            pa.issue(smem_u32(a_res) + c * kABytes, a_src + c * kTcBK, (size_t)p.C_out,
+                                     p.C_in - ci0 - pa.row0, c * kTcBK + pa.k < p.C_out, p.thetaT.base);
+                } else {
+                    pa.issue(tile, a_src + k0, (size_t)p.C_out, p.C_in - ci0 - pa.row0, k0 + pa.k < p.C_out,
+                             p.thetaT.base);
+                }
+                pb.issue(tile + kBOff, b_src + (size_t)k0 * p.P, (size_t)p.P, p.C_out - k0 - pb.krow0, b_ok,
                          p.gbar.base);
             });
         } else {
@@ -342,7 +358,7 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
                 int ci0, ncols; long long col0;
                 item_of(it, ci0, col0, ncols);
                 load_kmajor_scalar<128, kGxLoaders>(tile, p.thetaT, ci0, (long long)kc * kTcBK, tid);
-                load_mnmajor_scalar<NT, kGxLoaders>(tile + kABytes, p.gbar, kc * kTcBK, col0, ncols, tid);
+                load_mnmajor_scalar<NT, kGxLoaders>(tile + kBOff, p.gbar, kc * kTcBK, col0, ncols, tid);
             });
         }
     } else if (warp == kGxMmaWarp) {
@@ -351,9 +367,13 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
             for (int it = 0; it < n_my && ok; ++it) {
                 const int buf = it & 1;
                 if (it >= 2) ok = mbar_wait_bounded(&sh.acc_empty[buf], (uint32_t)((it >> 1) - 1) & 1u);
-                for (int kc = 0; kc < n_chunks && ok; ++kc)
-                    ok = mma_chunk<kGxStages>(sh.full, sh.empty, dyn, kStageBytes, kABytes, it * n_chunks + kc, kc == 0,
+                for (int kc = 0; kc < n_chunks && ok; ++kc) {
+                    const int q = it * n_chunks + kc;
+                    const uint32_t stage = smem_u32(dyn + (size_t)(q % kGxStages) * kStageBytes);
+                    const uint32_t a_addr = ARES ? smem_u32(a_res) + (uint32_t)(kc * kABytes) : stage;
+                    ok = mma_chunk<kGxStages>(sh.full, sh.empty, q, kc == 0, a_addr, stage + kBOff,
                                               tmem + (uint32_t)(buf * NT), kIdesc, 2048, 8192);
+                }
                 if (ok) umma_commit(&sh.acc_full[buf]);
             }
         }
@@ -581,7 +601,10 @@ __global__ void __launch_bounds__(kGwThreads) gw_tc_kernel(const GwTcParams p) {
         }
     } else if (lane == 0) {
         for (int it = 0; it < n_chunks && ok; ++it)
-            ok = mma_chunk<kGwStages>(sh.full, sh.empty, dyn, kStageBytes, kABytes, it, it == 0, tmem, kIdesc, 32, 16);
+        {
+            const uint32_t a_addr = smem_u32(dyn + (size_t)(it % kGwStages) * kStageBytes);
+            ok = mma_chunk<kGwStages>(sh.full, sh.empty, it, it == 0, a_addr, a_addr + kABytes, tmem, kIdesc, 32, 16);
+        }
         if (ok && n_chunks > 0) umma_commit(&sh.accum);
     }
     if (!ok) atomicOr(p.err_word, 4u);
@@ -668,16 +691,32 @@ static int sm_count_tc() {
     return n;
 }
 
-template <typename TOut, int NT, int R, int LOGV>
-static gf_status launch_gx_tc_inst(const GxTcParams& p, cudaStream_t s) {
-    constexpr size_t smem = (size_t)kGxStages * (128 * kTcBK * 2 + kTcBK * NT * 2) + (size_t)128 * (NT + 1) * 4 + 1024;
+constexpr size_t kGxAResMaxBytes = 128 * 1024;     // largest resident thetaT tile (C_out <= 512)
+
+template <typename TOut, int NT, int R, int LOGV, bool ARES>
+static gf_status launch_gx_tc_ares(const GxTcParams& p, int grid, cudaStream_t s) {
+    constexpr size_t d_bytes = ((size_t)128 * (NT + 1) * 4 + 1023) / 1024 * 1024;
+    constexpr size_t smem = ARES ? (size_t)kGxStages * (kTcBK * NT * 2) + d_bytes + kGxAResMaxBytes + 1024
+                                 : (size_t)kGxStages * (128 * kTcBK * 2 + kTcBK * NT * 2) + d_bytes + 1024;
     static bool configured = false;
     if (!configured) {
-        GF_CUDA_TRY(cudaFuncSetAttribute(gx_tc_kernel<TOut, NT, R, LOGV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        GF_CUDA_TRY(cudaFuncSetAttribute(gx_tc_kernel<TOut, NT, R, LOGV, ARES>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         configured = true;
     }
-    const int grid = p.items < sm_count_tc() ? p.items : sm_count_tc();
-    return launch_pdl(gx_tc_kernel<TOut, NT, R, LOGV>, dim3(grid), dim3(kGxThreads), smem, s, p);
+    return launch_pdl(gx_tc_kernel<TOut, NT, R, LOGV, ARES>, dim3(grid), dim3(kGxThreads), smem, s, p);
+}
+
+template <typename TOut, int NT, int R, int LOGV>
+static gf_status launch_gx_tc_inst(const GxTcParams& p, cudaStream_t s) {
+    int grid = p.items < sm_count_tc() ? p.items : sm_count_tc();
+    if constexpr (LOGV > 0) {
+        const size_t a_bytes = (size_t)((p.C_out + kTcBK - 1) / kTcBK) * 128 * kTcBK * 2;
+        const int g2 = grid / p.n_ci_tiles * p.n_ci_tiles;
+        if (a_bytes <= kGxAResMaxBytes && g2 >= p.n_ci_tiles)
+            return launch_gx_tc_ares<TOut, NT, R, LOGV, true>(p, g2, s);
+    }
+    return launch_gx_tc_ares<TOut, NT, R, LOGV, false>(p, grid, s);
 }
 
 template <typename TOut, int NT, int R>
