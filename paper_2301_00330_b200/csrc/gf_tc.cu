@@ -62,9 +62,7 @@ __device__ __forceinline__ void cp_async_piece(uint32_t dst, const void* src, bo
     else asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() {
-    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
 // A thread's share of a K-major tile [ROWS][64]: one piece position k along the row and
 // the rows row0, row0 + ROW_STEP, ...  The shared-memory offsets are the same for every
@@ -151,28 +149,23 @@ __device__ __forceinline__ unsigned char* align1024(unsigned char* p) {
 }
 
 // The loaders' side of a ring of STAGES stages over `total` chunks: issue(q, smem addr of the
-// stage) enqueues the asynchronous copies of chunk q; STAGES-1 chunks are in flight; a
-// chunk is published (proxy fence + arrive on full[stage]) once this thread's copies of
-// it have landed.
+// stage) enqueues the asynchronous copies of chunk q, then the thread hands its arrival on
+// full[stage] to the copy unit (cp.async.mbarrier.arrive.noinc: the arrival happens when
+// this thread's copies so far have landed).  Up to STAGES chunks are in flight and a chunk
+// is published the moment it is complete.  The consumer orders the landed data before its
+// tensor-core reads with a proxy fence.
 template <int STAGES, typename Issue>
 __device__ __forceinline__ bool run_async_loaders(uint64_t* full, uint64_t* empty, unsigned char* dyn, int stage_bytes,
                                                   int total, Issue issue) {
     bool ok = true;
-    for (int q = 0; q < total + STAGES - 1; ++q) {
-        if (q < total) {
-            const int s = q % STAGES;
-            if (q >= STAGES) ok = mbar_wait_bounded(&empty[s], (uint32_t)((q / STAGES) - 1) & 1u);
-            if (!ok) break;
-            issue(q, smem_u32(dyn + (size_t)s * stage_bytes));
-        }
-        cp_async_commit();
-        if (q >= STAGES - 1) {
-            cp_async_wait<STAGES - 1>();
-            fence_proxy_async_smem();
-            mbar_arrive(&full[(q - (STAGES - 1)) % STAGES]);
-        }
+    for (int q = 0; q < total; ++q) {
+        const int s = q % STAGES;
+        if (q >= STAGES) ok = mbar_wait_bounded(&empty[s], (uint32_t)((q / STAGES) - 1) & 1u);
+        if (!ok) break;
+        issue(q, smem_u32(dyn + (size_t)s * stage_bytes));
+        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&full[s])) : "memory");
     }
-    cp_async_wait<0>();
+    cp_async_wait_all();
     return ok;
 }
 template <int STAGES, typename Load>
@@ -197,6 +190,7 @@ __device__ __forceinline__ bool mma_chunk(uint64_t* full, uint64_t* empty, int q
                                           uint32_t b_lbo) {
     const int s = q % STAGES;
     if (!mbar_wait_bounded(&full[s], (uint32_t)(q / STAGES) & 1u)) return false;
+    fence_proxy_async_smem();      // copies landed through the generic proxy; the MMA reads through the async proxy
     tc_fence_after_sync();
 #pragma unroll
     for (int ks = 0; ks < kTcBK / 16; ++ks) {
