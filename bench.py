@@ -420,14 +420,93 @@ def run_ours(args) -> None:
         dist.destroy_process_group()
 
 
+def run_table(args) -> None:
+    """--table: every headline layer (and the paper's on-device shapes) timed once each way:
+    gf_stash_forward, gf_backward, and an exact backward through torch/cuDNN as context.
+    Prints one JSON line per layer and a markdown table; not the contract line."""
+    import torch
+    import paper_2301_00330_b200 as gf
+    from paper_2301_00330_b200 import workloads
+
+    torch.cuda.set_device(0)
+    gf.build_library()
+    peaks, which = measured_peaks()
+    layers = [l for l in workloads.all_headline_layers() if l.r > 1] + workloads.ondevice_table(2, "f32") \
+        + workloads.ondevice_table(4, "f32")
+    stream = torch.cuda.current_stream()
+    rows = []
+
+    def timed(fn, reps):
+        for _ in range(3):
+            fn(0)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda._sleep(int(3e-3 * 1.9e9))       # backlog: the calls below queue up behind it
+        e0.record(stream)
+        for i in range(reps):
+            fn(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / reps
+
+    for L in layers:
+        desc = gf.desc_for(L)
+        x0, gy0, w0 = workloads.make_inputs(L)
+        per_set = L.backward_bytes() + L.stash_bytes_moved()
+        n_sets = max(1, min(4, int(400e6 // per_set) + 1))
+        sets = [(torch.roll(x0, i, 0).cuda(), torch.roll(gy0, i, 0).cuda(), gf.alloc_layer(desc)) for i in range(n_sets)]
+        w = w0.cuda()
+        ws_bytes = gf.gf_backward_workspace_bytes(desc)
+        reps = 20 if per_set < 300e6 else 8
+
+        def stash(i):
+            x, _, b = sets[i % n_sets]
+            gf.gf_stash_forward(desc, x, b.stash, stream)
+
+        def bwd(i):
+            _, gy, b = sets[i % n_sets]
+            gf.gf_backward(desc, gy, b.stash, w, b.g_W, b.g_X, b.workspace, ws_bytes, stream)
+
+        def exact(i):
+            x, gy, _ = sets[i % n_sets]
+            torch.ops.aten.convolution_backward(gy, x, w, None, [1, 1], [L.pad, L.pad], [1, 1], False, [0, 0],
+                                                L.groups, [True, True, False])
+
+        t_stash, t_bwd = timed(stash, reps), timed(bwd, reps)
+        try:
+            t_exact = timed(exact, max(2, reps // 4))
+        except Exception:
+            t_exact = None
+        row = {"layer": L.name, "r": L.r, "dtype": L.dtype, "stash_us": t_stash, "backward_us": t_bwd,
+               "backward_alg_MB": L.backward_bytes() / 1e6,
+               "backward_gbs": L.backward_bytes() / t_bwd / 1e3,
+               "backward_frac_hbm": L.backward_bytes() / t_bwd / 1e3 / peaks["hbm_gbs"],
+               "stash_gbs": L.stash_bytes_moved() / t_stash / 1e3,
+               "stash_frac_hbm": L.stash_bytes_moved() / t_stash / 1e3 / peaks["hbm_gbs"],
+               "exact_cudnn_us": t_exact, "reduced_gflop": L.reduced_flops() / 1e9}
+        rows.append(row)
+        print(json.dumps(row), flush=True)
+        del sets
+        torch.cuda.empty_cache()
+    print(f"\n| layer | r | dtype | stash us | backward us | alg MB | GB/s | frac of {peaks['hbm_gbs']:.0f} GB/s ({which}) | exact cuDNN us |")
+    print("|---|---|---|---|---|---|---|---|---|")
+    for r in rows:
+        ex = f"{r['exact_cudnn_us']:.0f}" if r["exact_cudnn_us"] else "n/a"
+        print(f"| {r['layer']} | {r['r']} | {r['dtype']} | {r['stash_us']:.1f} | {r['backward_us']:.1f} | "
+              f"{r['backward_alg_MB']:.1f} | {r['backward_gbs']:.0f} | {r['backward_frac_hbm']:.2f} | {ex} |")
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--table", action="store_true", help="time every layer shape once (diagnostic table)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.table:
+        run_table(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
