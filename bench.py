@@ -136,13 +136,15 @@ def kernel_cost(name: str, L, splits: int) -> tuple[float, float]:
     """(algorithmic bytes, flops) of one launch of kernel `name` on layer L."""
     e = L.elem_bytes
     gbar = 4 * L.N * L.C_out * L.Hp * L.Wp          # fp32 patch means (CUDA-core path)
-    gbar16 = gbar // 2                              # bf16 patch means (tensor-core path)
+    # tensor-core path: bf16 patch means; fp32 layers carry (high, low) bf16 pairs, 4 bytes again
+    gbar16 = gbar // 2 if L.dtype == "bf16" else gbar
     pairs = L.C_out * L.C_ig
     M = L.N * L.Hp * L.Wp
     mix = 2.0 * M * L.C_out * L.C_ig
-    tc = L.dtype == "bf16" and L.groups == 1
+    tc = L.groups == 1 and L.C_out % 8 == 0
     table = {
-        "gx_tc": (gbar16 + 2 * pairs + e * L.numel_x(), mix),
+        "split_f32": (8 * L.numel_stash(), L.numel_stash()),
+        "gx_tc": (gbar16 + e * pairs + e * L.numel_x(), mix),
         "gw_tc": (gbar16 + e * L.numel_stash() + 4 * splits * pairs, mix),
         "stash_pool": (e * (L.numel_x() + L.numel_stash()), L.numel_x()),
         "gy_pool": (e * L.numel_gy() + (gbar16 if tc else gbar), L.numel_gy()),
@@ -385,7 +387,7 @@ def run_ours(args) -> None:
         return
 
     # split count of the reduced g_W contraction, needed for its byte count
-    if layer.dtype == "bf16" and layer.groups == 1:      # tensor-core path: 128 x 128 tiles, one wave of CTAs
+    if layer.groups == 1 and layer.C_out % 8 == 0 and layer.r >= 2:      # tensor-core path: 128 x 128 tiles, one wave of CTAs
         tiles = ((layer.C_out + 127) // 128) * ((layer.C_in + 127) // 128)
         chunks = -(-(layer.N * layer.Hp * layer.Wp) // 64)
         splits = max(1, min(chunks, -(-148 // tiles)))

@@ -21,7 +21,7 @@ int g_prof_created = 0;          // event pairs that exist
 int g_prof_used = 0;             // event pairs recorded since the last read
 int g_prof_slot_kid[kProfPairs];
 const char* const kKernelNames[K_COUNT] = {
-    "stash_pool", "ksum", "gy_pool", "gx_mix", "gw_partial", "gw_finish", "dw_fused", "exact_gx", "exact_gw", "gx_tc", "gw_tc"};
+    "stash_pool", "ksum", "gy_pool", "gx_mix", "gw_partial", "gw_finish", "dw_fused", "exact_gx", "exact_gw", "gx_tc", "gw_tc", "split_f32"};
 }  // namespace
 
 ProfScope::ProfScope(int kernel_id, cudaStream_t s) : slot(-1), stream(s) {
@@ -107,6 +107,7 @@ Workspace plan_workspace(const Geo& g) {
     Workspace w;
     w.off_err = 0;
     size_t off = 256;
+    w.off_split = 0;
     if (g.r == 1) { w.off_tsum = w.off_gbar = w.off_part = off; w.splits = 0; w.total = off; return w; }
     w.off_tsum = off; off += align_up((size_t)g.C_out * g.C_ig * 4, 256);
     w.off_gbar = off; off += align_up((size_t)g.N * g.C_out * g.Hp * g.Wp * 4, 256);
@@ -115,6 +116,10 @@ Workspace plan_workspace(const Geo& g) {
     if (is_depthwise(g)) { const int ds = depthwise_splits(g); if (ds > s) s = ds; }
     w.splits = s;
     w.off_part = off; off += align_up((size_t)s * g.C_out * g.C_ig * 4, 256);
+    if (tc_eligible(g) && g.dtype == GF_F32) {
+        // fp32 stash as (high, low) bf16 arrays for the tensor-core contraction
+        w.off_split = off; off += 2 * align_up((size_t)g.N * g.C_in * g.Hp * g.Wp * 2, 256);
+    }
     w.total = off;
     return w;
 }
@@ -165,7 +170,7 @@ gf_status gf_stash_forward(const gf_conv_desc* desc, const void* x, void* stash,
     if (g.r == 1) return launch_copy(x, stash, (size_t)planes * g.H * g.W * g.esize, s);
     uint32_t* err = global_err_word();
     if (!err) return GF_ERR_CUDA;
-    return launch_pool(K_STASH_POOL, x, g.dtype, stash, g.dtype, /*mean=*/false, planes, g.H, g.W, g.r, err, s);
+    return launch_pool(K_STASH_POOL, x, g.dtype, stash, nullptr, g.dtype, /*mean=*/false, planes, g.H, g.W, g.r, err, s);
 }
 
 gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* stash, const void* W,
@@ -204,21 +209,35 @@ gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* sta
 
     if (tc_eligible(g)) {
         // tensor-core path: theta sums (transposed, bf16; clears the error word), patch
-        // means of g_y as bf16, then the two contractions on tcgen05
+        // means of g_y as bf16, then the two contractions on tcgen05.  fp32 layers carry
+        // every operand as a (high, low) bf16 pair: v = hi + lo up to 2^-17 |v|.
+        const bool split = g.dtype == GF_F32;
+        const size_t P = (size_t)g.Hp * g.Wp;
+        // low parts sit 16-byte aligned behind the high parts, inside the fp32-sized regions
+        const long long theta_lo = split ? (long long)align_up((size_t)g.C_in * g.C_out, 8) : 0;
+        const long long gbar_lo = split ? (long long)align_up((size_t)g.N * g.C_out * P, 8) : 0;
+        const long long stash_lo = split ? (long long)(align_up((size_t)g.N * g.C_in * P * 2, 256) / 2) : 0;
         __nv_bfloat16* thetaT = reinterpret_cast<__nv_bfloat16*>(tsum);
         __nv_bfloat16* gbar16 = reinterpret_cast<__nv_bfloat16*>(gbar);
-        st = launch_ksum_t(W, g, thetaT, g_W ? part : nullptr, err, s);
+        st = launch_ksum_t(W, g, thetaT, split ? thetaT + theta_lo : nullptr, g_W ? part : nullptr, err, s);
         if (st != GF_OK) return st;
-        st = launch_pool(K_GY_POOL, g_y, g.dtype, gbar16, GF_BF16, /*mean=*/true, (int64_t)g.N * g.C_out, g.H, g.W,
-                         g.r, err, s);
+        st = launch_pool(K_GY_POOL, g_y, g.dtype, gbar16, split ? gbar16 + gbar_lo : nullptr, GF_BF16, /*mean=*/true,
+                         (int64_t)g.N * g.C_out, g.H, g.W, g.r, err, s);
         if (st != GF_OK) return st;
         if (g_X) {
-            st = launch_gx_tc(gbar16, thetaT, g_X, err, g, s);
+            st = launch_gx_tc(gbar16, gbar_lo, thetaT, theta_lo, g_X, err, g, s);
             if (st != GF_OK) return st;
         }
         if (g_W) {
+            const __nv_bfloat16* stash16 = static_cast<const __nv_bfloat16*>(stash);
+            if (split) {
+                __nv_bfloat16* sp = reinterpret_cast<__nv_bfloat16*>(base + ws.off_split);
+                st = launch_split_f32(static_cast<const float*>(stash), sp, sp + stash_lo, (size_t)g.N * g.C_in * P, s);
+                if (st != GF_OK) return st;
+                stash16 = sp;
+            }
             const int splits = tc_gw_splits(g);
-            st = launch_gw_tc(gbar16, static_cast<const __nv_bfloat16*>(stash), part, splits, err, g, s);
+            st = launch_gw_tc(gbar16, gbar_lo, stash16, stash_lo, part, splits, err, g, s);
             if (st != GF_OK) return st;
             st = launch_gw_finish(part, 1, g_W, g, s);
             if (st != GF_OK) return st;
@@ -230,7 +249,7 @@ gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* sta
     // patch means of g_y, read once
     st = launch_ksum(W, g, tsum, err, s);
     if (st != GF_OK) return st;
-    st = launch_pool(K_GY_POOL, g_y, g.dtype, gbar, GF_F32, /*mean=*/true, (int64_t)g.N * g.C_out, g.H, g.W, g.r, err, s);
+    st = launch_pool(K_GY_POOL, g_y, g.dtype, gbar, nullptr, GF_F32, /*mean=*/true, (int64_t)g.N * g.C_out, g.H, g.W, g.r, err, s);
     if (st != GF_OK) return st;
     if (g_X) {
         st = launch_gx_mix(gbar, tsum, g_X, g, s);

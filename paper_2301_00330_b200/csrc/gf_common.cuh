@@ -14,7 +14,7 @@ void count_launch(int n = 1);
 
 enum KernelId {
     K_STASH_POOL = 0, K_KSUM, K_GY_POOL, K_GX_MIX, K_GW_PARTIAL, K_GW_FINISH, K_DW_FUSED,
-    K_EXACT_GX, K_EXACT_GW, K_GX_TC, K_GW_TC, K_COUNT
+    K_EXACT_GX, K_EXACT_GW, K_GX_TC, K_GW_TC, K_SPLIT, K_COUNT
 };
 
 // Brackets the launches made during its lifetime with a pair of events when
@@ -147,16 +147,16 @@ Geo make_geo(const gf_conv_desc& d);
 
 // ---- workspace layout of gf_backward ---------------------------------------
 // [ error word (256 B) | theta sum fp32 [C_out,C_ig] | gbar fp32 [N,C_out,Hp,Wp] |
-//   split partials fp32 [S, C_out, C_ig] ]
+//   split partials fp32 [S, C_out, C_ig] | fp32 tensor-core layers: stash as bf16 (high, low) ]
 struct Workspace {
-    size_t off_err, off_tsum, off_gbar, off_part, total;
+    size_t off_err, off_tsum, off_gbar, off_part, off_split, total;
     int splits;           // S: number of partial g_W matrices
 };
 Workspace plan_workspace(const Geo& g);
 
 // ---- kernel entry points (host launchers) ----------------------------------
 // pool: out[plane, a, b] = sum (or mean) of in[plane] over patch (a,b)
-gf_status launch_pool(int kernel_id, const void* in, int in_dtype, void* out, int out_dtype, bool mean,
+gf_status launch_pool(int kernel_id, const void* in, int in_dtype, void* out, void* out_lo, int out_dtype, bool mean,
                       int64_t planes, int H, int W, int r, uint32_t* err_word, cudaStream_t s);
 gf_status launch_copy(const void* in, void* out, size_t bytes, cudaStream_t s);
 
@@ -172,12 +172,14 @@ int depthwise_splits(const Geo& g);
 // tensor-core path (bf16 operands, dense layers)
 bool tc_eligible(const Geo& g);
 int tc_gw_splits(const Geo& g);
-gf_status launch_ksum_t(const void* W, const Geo& g, __nv_bfloat16* thetaT, float* gwu, uint32_t* err_word,
-                        cudaStream_t s);
-gf_status launch_gx_tc(const __nv_bfloat16* gbar, const __nv_bfloat16* thetaT, void* gX, uint32_t* err_word,
-                       const Geo& g, cudaStream_t s);
-gf_status launch_gw_tc(const __nv_bfloat16* gbar, const __nv_bfloat16* stash, float* gwu, int splits,
-                       uint32_t* err_word, const Geo& g, cudaStream_t s);
+gf_status launch_ksum_t(const void* W, const Geo& g, __nv_bfloat16* thetaT, __nv_bfloat16* thetaT_lo, float* gwu,
+                        uint32_t* err_word, cudaStream_t s);
+gf_status launch_split_f32(const float* in, __nv_bfloat16* hi, __nv_bfloat16* lo, size_t n, cudaStream_t s);
+gf_status launch_gx_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const __nv_bfloat16* thetaT,
+                       long long theta_lo_off, void* gX, uint32_t* err_word, const Geo& g, cudaStream_t s);
+gf_status launch_gw_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const __nv_bfloat16* stash,
+                       long long stash_lo_off, float* gwu, int splits, uint32_t* err_word, const Geo& g,
+                       cudaStream_t s);
 gf_status launch_exact(const void* gy, const void* x, const void* W, float* gW, void* gX,
                        const Geo& g, cudaStream_t s);
 

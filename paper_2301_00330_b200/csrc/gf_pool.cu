@@ -27,6 +27,7 @@ constexpr int kStreamStages = 6;
 struct PoolParams {
     const void* in;
     void* out;
+    void* out_lo;      // bf16 output only: low parts, out = rn(v), out_lo = rn(v - out); NULL: plain output
     uint32_t* err_word;
     long long planes, total_elems, tiles;
     int H, W, r, Hp, Wp;
@@ -91,6 +92,17 @@ template <int G> __device__ __forceinline__ void store_vec(__nv_bfloat16* dst, c
         *dst = __float2bfloat16_rn(a[0]);
     }
 }
+
+// G outputs as (high, low) bf16 pairs into two arrays
+template <int G>
+__device__ __forceinline__ void store_split(__nv_bfloat16* hi, __nv_bfloat16* lo, const float (&a)[G]) {
+    float l[G];
+#pragma unroll
+    for (int k = 0; k < G; ++k) l[k] = a[k] - __bfloat162float(__float2bfloat16_rn(a[k]));
+    store_vec<G>(hi, a);
+    store_vec<G>(lo, l);
+}
+template <int G> __device__ __forceinline__ void store_split(float*, float*, const float (&)[G]) {}
 
 // ---- tile geometry (shared by the two tiled kernels) ------------------------------
 struct Tile { long long g0, out_base; int len, np, a0, na; };
@@ -171,7 +183,8 @@ __device__ __forceinline__ void reduce_item(const PoolParams& p, const TIn* buf,
 #pragma unroll
         for (int k = 0; k < G; ++k) acc[k] *= p.inv_full;
     }
-    store_vec<G>(dst + o, acc);
+    if (p.out_lo) store_split<G>(dst + o, static_cast<TOut*>(p.out_lo) + (dst - static_cast<TOut*>(p.out)) + o, acc);
+    else store_vec<G>(dst + o, acc);
 }
 
 template <typename TIn, typename TOut, int R, int G>
@@ -283,7 +296,12 @@ __global__ void __launch_bounds__(kPoolThreads) pool_tile_kernel(const PoolParam
             cnt = nr * nc;
         }
         if (p.mean) s *= (cnt == p.r * p.r) ? p.inv_full : 1.0f / (float)cnt;
-        out[g.out_base + o] = from_f32<TOut>(s);
+        if (p.out_lo) {
+            const float a[1] = {s};
+            store_split<1>(out + g.out_base + o, static_cast<TOut*>(p.out_lo) + g.out_base + o, a);
+        } else {
+            out[g.out_base + o] = from_f32<TOut>(s);
+        }
     }
 }
 
@@ -314,7 +332,12 @@ __global__ void __launch_bounds__(kPoolThreads) pool_bigpatch_kernel(const PoolP
         t = warp_sum(t);
         if (threadIdx.x == 0) {
             if (p.mean) t /= (float)(nr * nc);
-            out[o] = from_f32<TOut>(t);
+            if (p.out_lo) {
+                const float a[1] = {t};
+                store_split<1>(out + o, static_cast<TOut*>(p.out_lo) + o, a);
+            } else {
+                out[o] = from_f32<TOut>(t);
+            }
         }
     }
 }
@@ -408,11 +431,12 @@ static gf_status pool_dispatch(PoolParams& p, size_t e, cudaStream_t s) {
     return after_launch();
 }
 
-gf_status launch_pool(int kernel_id, const void* in, int in_dtype, void* out, int out_dtype, bool mean,
+gf_status launch_pool(int kernel_id, const void* in, int in_dtype, void* out, void* out_lo, int out_dtype, bool mean,
                       int64_t planes, int H, int W, int r, uint32_t* err_word, cudaStream_t s) {
     ProfScope prof(kernel_id, s);
     PoolParams p;
-    p.in = in; p.out = out; p.err_word = err_word; p.planes = planes; p.total_elems = planes * H * W;
+    if (out_lo && out_dtype != GF_BF16) return GF_ERR_UNSUPPORTED;
+    p.in = in; p.out = out; p.out_lo = out_lo; p.err_word = err_word; p.planes = planes; p.total_elems = planes * H * W;
     p.H = H; p.W = W; p.r = r; p.mean = mean ? 1 : 0;
     p.Hp = (H + r - 1) / r; p.Wp = (W + r - 1) / r;
     p.div_plane_out = FastDiv(p.Hp * p.Wp);
@@ -423,6 +447,7 @@ gf_status launch_pool(int kernel_id, const void* in, int in_dtype, void* out, in
     if (in_dtype == GF_F32 && out_dtype == GF_F32) return pool_dispatch<float, float>(p, e, s);
     if (in_dtype == GF_BF16 && out_dtype == GF_BF16) return pool_dispatch<__nv_bfloat16, __nv_bfloat16>(p, e, s);
     if (in_dtype == GF_BF16 && out_dtype == GF_F32) return pool_dispatch<__nv_bfloat16, float>(p, e, s);
+    if (in_dtype == GF_F32 && out_dtype == GF_BF16) return pool_dispatch<float, __nv_bfloat16>(p, e, s);
     return GF_ERR_UNSUPPORTED;
 }
 

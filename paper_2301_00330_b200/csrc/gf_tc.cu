@@ -26,12 +26,14 @@ namespace gf {
 constexpr int kTcBK = 64;           // K elements per stage (one 128-byte swizzled row)
 constexpr int kGwLoaders = 256;     // gw_tc: 8 loader / epilogue warps + 1 MMA warp
 constexpr int kGwThreads = 288;
-constexpr int kGwStages = 6;
+constexpr int kGwStagesMax = 6;
+__host__ __device__ constexpr int gw_stages(int split) { return split == 2 ? 3 : 6; }
 constexpr int kGxLoaders = 256;     // gx_tc: 8 loader warps, 8 epilogue warps, 1 MMA warp
 constexpr int kGxEpi = 256;
 constexpr int kGxThreads = kGxLoaders + kGxEpi + 32;
 constexpr int kGxMmaWarp = (kGxLoaders + kGxEpi) / 32;
-constexpr int kGxStages = 7;
+constexpr int kGxStagesMax = 7;
+__host__ __device__ constexpr int gx_stages(int split, bool ares) { return split == 2 ? (ares ? 4 : 3) : 7; }
 
 // Source of an operand: a [n][C][P] bf16 array read along the flattened index
 // k = n*P + p (row c is a channel).  A plain [rows][pitch] matrix is the case P = pitch,
@@ -44,6 +46,7 @@ struct FlatSrc {
     long long k_total;  // N*P
     FastDiv div_P;
     int logV;
+    long long lo_off;   // split operands: elements from the high-part array to the low-part array (0: none)
 };
 
 __device__ __forceinline__ const __nv_bfloat16* flat_ptr(const FlatSrc& s, int c, long long k) {
@@ -184,10 +187,12 @@ __device__ __forceinline__ bool run_sync_loaders(uint64_t* full, uint64_t* empty
 // One chunk of the MMA thread's work: wait for the stage, four K = 16 steps, release it.
 // b_step = start-address advance of the B descriptor per step (32 bytes K-major, 2048
 // bytes MN-major); b_lbo = its leading byte offset.
-template <int STAGES>
+// SPLIT == 2: every operand is a pair of bf16 tiles (high and low parts of an fp32 value);
+// the product is hi*hi + hi*lo + lo*hi (the lo*lo term, 2^-18 relative, is dropped).
+template <int STAGES, int SPLIT>
 __device__ __forceinline__ bool mma_chunk(uint64_t* full, uint64_t* empty, int q, bool first, uint32_t a_addr,
-                                          uint32_t b_addr, uint32_t d_tmem, uint32_t idesc, uint32_t b_step,
-                                          uint32_t b_lbo) {
+                                          uint32_t a_lo, uint32_t b_addr, uint32_t b_lo, uint32_t d_tmem,
+                                          uint32_t idesc, uint32_t b_step, uint32_t b_lbo) {
     const int s = q % STAGES;
     if (!mbar_wait_bounded(&full[s], (uint32_t)(q / STAGES) & 1u)) return false;
     fence_proxy_async_smem();      // copies landed through the generic proxy; the MMA reads through the async proxy
@@ -197,6 +202,10 @@ __device__ __forceinline__ bool mma_chunk(uint64_t* full, uint64_t* empty, int q
         const uint64_t adesc = umma_smem_desc(a_addr + ks * 32, 16, 1024);
         const uint64_t bdesc = umma_smem_desc(b_addr + ks * b_step, b_lbo, 1024);
         umma_bf16(d_tmem, adesc, bdesc, idesc, !(first && ks == 0));
+        if constexpr (SPLIT == 2) {
+            umma_bf16(d_tmem, adesc, umma_smem_desc(b_lo + ks * b_step, b_lbo, 1024), idesc, 1u);
+            umma_bf16(d_tmem, umma_smem_desc(a_lo + ks * 32, 16, 1024), bdesc, idesc, 1u);
+        }
     }
     umma_commit(&empty[s]);
     return true;
@@ -246,7 +255,7 @@ template <int R, int UPC> __device__ __forceinline__ void store_chunk(__nv_bfloa
 }
 
 struct GxShared {
-    uint64_t full[kGxStages], empty[kGxStages];
+    uint64_t full[kGxStagesMax], empty[kGxStagesMax];
     uint64_t acc_full[2], acc_empty[2];
     uint32_t tmem_base;
 };
@@ -258,12 +267,15 @@ struct GxShared {
 // LOGV: log2 of the piece width of gbar (0: 2-byte pieces through registers).
 // ARES: the CTA keeps one c_i tile for all its items and holds that tile of thetaT (all of
 //       K) resident in shared memory; only the gbar tiles stream through the ring.
-template <typename TOut, int NT, int R, int LOGV, bool ARES>
+// SPLIT: 1 = bf16 operands; 2 = fp32 data carried as (high, low) bf16 pairs.
+template <typename TOut, int NT, int R, int LOGV, bool ARES, int SPLIT>
 __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p) {
+    constexpr int kGxStages = gx_stages(SPLIT, ARES);
     constexpr int kABytes = 128 * kTcBK * 2;             // 16 KB
     constexpr int kBBytes = kTcBK * NT * 2;              // 64 k x NT columns
-    constexpr int kStageBytes = ARES ? kBBytes : kABytes + kBBytes;
-    constexpr int kBOff = ARES ? 0 : kABytes;
+    // stage: [A hi][A lo] (unless resident) [B hi][B lo]
+    constexpr int kStageBytes = SPLIT * (ARES ? kBBytes : kABytes + kBBytes);
+    constexpr int kBOff = ARES ? 0 : SPLIT * kABytes;
     constexpr int kDBytes = (128 * (NT + 1) * 4 + 1023) / 1024 * 1024;
     constexpr int kColsPerLane = NT / 32;
     constexpr int kUnits = R > 0 ? NT * R : 1;           // R-element vectors of a tile's part of one plane
@@ -335,15 +347,22 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
                 const int k0 = kc * kTcBK;
                 if constexpr (ARES) {
                     if (q == 0)      // the resident thetaT tile rides in the first copy group
-                        for (int c = 0; c < n_chunks; ++c)
-                            pa.issue(smem_u32(a_res) + c * kABytes, a_src + c * kTcBK, (size_t)p.C_out,
-                                     p.C_in - ci0 - pa.row0, c * kTcBK + pa.k < p.C_out, p.thetaT.base);
+                        for (int c = 0; c < SPLIT * n_chunks; ++c) {
+                            const int cc = c < n_chunks ? c : c - n_chunks;
+                            pa.issue(smem_u32(a_res) + c * kABytes,
+                                     a_src + (c < n_chunks ? 0 : p.thetaT.lo_off) + cc * kTcBK, (size_t)p.C_out,
+                                     p.C_in - ci0 - pa.row0, cc * kTcBK + pa.k < p.C_out, p.thetaT.base);
+                        }
                 } else {
-                    pa.issue(tile, a_src + k0, (size_t)p.C_out, p.C_in - ci0 - pa.row0, k0 + pa.k < p.C_out,
-                             p.thetaT.base);
+#pragma unroll
+                    for (int h = 0; h < SPLIT; ++h)
+                        pa.issue(tile + h * kABytes, a_src + h * p.thetaT.lo_off + k0, (size_t)p.C_out,
+                                 p.C_in - ci0 - pa.row0, k0 + pa.k < p.C_out, p.thetaT.base);
                 }
-                pb.issue(tile + kBOff, b_src + (size_t)k0 * p.P, (size_t)p.P, p.C_out - k0 - pb.krow0, b_ok,
-                         p.gbar.base);
+#pragma unroll
+                for (int h = 0; h < SPLIT; ++h)
+                    pb.issue(tile + kBOff + h * kBBytes, b_src + h * p.gbar.lo_off + (size_t)k0 * p.P, (size_t)p.P,
+                             p.C_out - k0 - pb.krow0, b_ok, p.gbar.base);
             });
         } else {
             ok = run_sync_loaders<kGxStages>(sh.full, sh.empty, dyn, kStageBytes, n_my * n_chunks,
@@ -351,8 +370,14 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
                 const int it = q / n_chunks, kc = q - it * n_chunks;
                 int ci0, ncols; long long col0;
                 item_of(it, ci0, col0, ncols);
-                load_kmajor_scalar<128, kGxLoaders>(tile, p.thetaT, ci0, (long long)kc * kTcBK, tid);
-                load_mnmajor_scalar<NT, kGxLoaders>(tile + kBOff, p.gbar, kc * kTcBK, col0, ncols, tid);
+#pragma unroll
+                for (int h = 0; h < SPLIT; ++h) {
+                    FlatSrc a = p.thetaT, b = p.gbar;
+                    a.base += h * a.lo_off;
+                    b.base += h * b.lo_off;
+                    load_kmajor_scalar<128, kGxLoaders>(tile + h * kABytes, a, ci0, (long long)kc * kTcBK, tid);
+                    load_mnmajor_scalar<NT, kGxLoaders>(tile + kBOff + h * kBBytes, b, kc * kTcBK, col0, ncols, tid);
+                }
             });
         }
     } else if (warp == kGxMmaWarp) {
@@ -365,8 +390,10 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
                     const int q = it * n_chunks + kc;
                     const uint32_t stage = smem_u32(dyn + (size_t)(q % kGxStages) * kStageBytes);
                     const uint32_t a_addr = ARES ? smem_u32(a_res) + (uint32_t)(kc * kABytes) : stage;
-                    ok = mma_chunk<kGxStages>(sh.full, sh.empty, q, kc == 0, a_addr, stage + kBOff,
-                                              tmem + (uint32_t)(buf * NT), kIdesc, 2048, 8192);
+                    const uint32_t a_lo = ARES ? a_addr + (uint32_t)(n_chunks * kABytes) : stage + kABytes;
+                    ok = mma_chunk<kGxStages, SPLIT>(sh.full, sh.empty, q, kc == 0, a_addr, a_lo, stage + kBOff,
+                                                     stage + kBOff + kBBytes, tmem + (uint32_t)(buf * NT), kIdesc,
+                                                     2048, 8192);
                 }
                 if (ok) umma_commit(&sh.acc_full[buf]);
             }
@@ -504,7 +531,7 @@ struct GwTcParams {
 };
 
 struct GwShared {
-    uint64_t full[kGwStages], empty[kGwStages];
+    uint64_t full[kGwStagesMax], empty[kGwStagesMax];
     uint64_t accum;
     uint32_t tmem_base;
 };
@@ -515,11 +542,13 @@ __device__ __forceinline__ void red_add_v4(float* dst, uint32_t a, uint32_t b, u
                  : "memory");
 }
 
-template <int NT, int LOGV>
+template <int NT, int LOGV, int SPLIT>
 __global__ void __launch_bounds__(kGwThreads) gw_tc_kernel(const GwTcParams p) {
+    constexpr int kGwStages = gw_stages(SPLIT);
     constexpr int kABytes = 128 * kTcBK * 2;
     constexpr int kBBytes = NT * kTcBK * 2;
-    constexpr int kStageBytes = kABytes + kBBytes;
+    constexpr int kBOff = SPLIT * kABytes;                  // stage: [A hi][A lo][B hi][B lo]
+    constexpr int kStageBytes = SPLIT * (kABytes + kBBytes);
     constexpr uint32_t kIdesc = umma_idesc_bf16(128, NT, 0, 0);
     extern __shared__ unsigned char dyn_raw[];
     __shared__ GwShared sh;
@@ -559,14 +588,25 @@ __global__ void __launch_bounds__(kGwThreads) gw_tc_kernel(const GwTcParams p) {
                 const uint32_t pp = (uint32_t)(k_ok ? kk : 0) - n * (uint32_t)p.gbar.P;
                 const __nv_bfloat16* a_src = p.gbar.base + ((size_t)n * p.C_out + co0 + pa.row0) * p.gbar.P + pp;
                 const __nv_bfloat16* b_src = p.stash.base + ((size_t)n * p.C_in + ci0 + pb.row0) * p.gbar.P + pp;
-                pa.issue(tile, a_src, (size_t)p.gbar.P, p.C_out - co0 - pa.row0, k_ok, p.gbar.base);
-                pb.issue(tile + kABytes, b_src, (size_t)p.gbar.P, p.C_in - ci0 - pb.row0, k_ok, p.stash.base);
+#pragma unroll
+                for (int h = 0; h < SPLIT; ++h) {
+                    pa.issue(tile + h * kABytes, a_src + h * p.gbar.lo_off, (size_t)p.gbar.P, p.C_out - co0 - pa.row0,
+                             k_ok, p.gbar.base);
+                    pb.issue(tile + kBOff + h * kBBytes, b_src + h * p.stash.lo_off, (size_t)p.gbar.P,
+                             p.C_in - ci0 - pb.row0, k_ok, p.stash.base);
+                }
             });
         } else {
             ok = run_sync_loaders<kGwStages>(sh.full, sh.empty, dyn, kStageBytes, n_chunks, [&](int it, unsigned char* tile) {
                 const long long k0 = (long long)(kc_begin + it) * kTcBK;
-                load_kmajor_scalar<128, kGwLoaders>(tile, p.gbar, co0, k0, tid);
-                load_kmajor_scalar<NT, kGwLoaders>(tile + kABytes, p.stash, ci0, k0, tid);
+#pragma unroll
+                for (int h = 0; h < SPLIT; ++h) {
+                    FlatSrc a = p.gbar, b = p.stash;
+                    a.base += h * a.lo_off;
+                    b.base += h * b.lo_off;
+                    load_kmajor_scalar<128, kGwLoaders>(tile + h * kABytes, a, co0, k0, tid);
+                    load_kmajor_scalar<NT, kGwLoaders>(tile + kBOff + h * kBBytes, b, ci0, k0, tid);
+                }
             });
         }
         if (ok && n_chunks > 0) ok = mbar_wait_bounded(&sh.accum, 0);
@@ -597,7 +637,8 @@ __global__ void __launch_bounds__(kGwThreads) gw_tc_kernel(const GwTcParams p) {
         for (int it = 0; it < n_chunks && ok; ++it)
         {
             const uint32_t a_addr = smem_u32(dyn + (size_t)(it % kGwStages) * kStageBytes);
-            ok = mma_chunk<kGwStages>(sh.full, sh.empty, it, it == 0, a_addr, a_addr + kABytes, tmem, kIdesc, 32, 16);
+            ok = mma_chunk<kGwStages, SPLIT>(sh.full, sh.empty, it, it == 0, a_addr, a_addr + kABytes, a_addr + kBOff,
+                                             a_addr + kBOff + kBBytes, tmem, kIdesc, 32, 16);
         }
         if (ok && n_chunks > 0) umma_commit(&sh.accum);
     }
@@ -614,8 +655,8 @@ __global__ void __launch_bounds__(kGwThreads) gw_tc_kernel(const GwTcParams p) {
 // contiguous.  Also clears the error word and g_W's unique-value accumulator.
 template <typename T>
 __global__ void __launch_bounds__(1024) ksum_t_kernel(const T* __restrict__ W, __nv_bfloat16* __restrict__ thetaT,
-                                                      float* __restrict__ gwu, int C_in, int C_out, int taps,
-                                                      uint32_t* err_word) {
+                                                      __nv_bfloat16* __restrict__ thetaT_lo, float* __restrict__ gwu,
+                                                      int C_in, int C_out, int taps, uint32_t* err_word) {
     __shared__ float tile[32][33];
     pdl_launch_dependents();
     pdl_wait();
@@ -634,20 +675,45 @@ __global__ void __launch_bounds__(1024) ksum_t_kernel(const T* __restrict__ W, _
     }
     __syncthreads();
     const int ci = ci0 + ty, co = co0 + tx;
-    if (ci < C_in && co < C_out) thetaT[(size_t)ci * C_out + co] = __float2bfloat16_rn(tile[tx][ty]);
+    if (ci < C_in && co < C_out) {
+        const float v = tile[tx][ty];
+        const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+        thetaT[(size_t)ci * C_out + co] = hi;
+        if (thetaT_lo) thetaT_lo[(size_t)ci * C_out + co] = __float2bfloat16_rn(v - __bfloat162float(hi));
+    }
+}
+
+// fp32 -> (high, low) bf16 pair: hi = rn(v), lo = rn(v - hi); v - hi - lo is below 2^-17 |v|.
+__global__ void __launch_bounds__(256) split_f32_kernel(const float* __restrict__ in, __nv_bfloat16* __restrict__ hi,
+                                                        __nv_bfloat16* __restrict__ lo, size_t n4) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n4) return;
+    const float4 v = __ldcs(reinterpret_cast<const float4*>(in) + i);
+    const float f[4] = {v.x, v.y, v.z, v.w};
+    __nv_bfloat16 h[4], l[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        h[k] = __float2bfloat16_rn(f[k]);
+        l[k] = __float2bfloat16_rn(f[k] - __bfloat162float(h[k]));
+    }
+    reinterpret_cast<uint2*>(hi)[i] = *reinterpret_cast<uint2*>(h);
+    reinterpret_cast<uint2*>(lo)[i] = *reinterpret_cast<uint2*>(l);
 }
 
 // ================================================================== host side
-static FlatSrc make_flat(const void* base, int C, int P, long long k_total) {
+static FlatSrc make_flat(const void* base, int C, int P, long long k_total, long long lo_off) {
     FlatSrc s;
     s.base = static_cast<const __nv_bfloat16*>(base);
     s.C = C; s.P = P; s.k_total = k_total; s.div_P = FastDiv((uint32_t)P);
-    s.logV = (P % 8 == 0) ? 3 : (P % 4 == 0) ? 2 : (P % 2 == 0) ? 1 : 0;
+    s.logV = (P % 8 == 0) ? 3 : (P % 4 == 0) ? 2 : 0;      // 16- or 8-byte pieces, else element-wise
+    s.lo_off = lo_off;
     return s;
 }
 
 bool tc_eligible(const Geo& g) {
-    return g.dtype == GF_BF16 && g.G == 1 && g.r >= 2 && g.C_out % 8 == 0 &&
+    return (g.dtype == GF_BF16 || g.dtype == GF_F32) && g.G == 1 && g.r >= 2 && g.C_out % 8 == 0 &&
            (long long)g.N * g.Hp * g.Wp < (1LL << 31);
 }
 
@@ -662,17 +728,24 @@ int tc_gw_splits(const Geo& g) {
     return s;
 }
 
-gf_status launch_ksum_t(const void* W, const Geo& g, __nv_bfloat16* thetaT, float* gwu, uint32_t* err_word,
-                        cudaStream_t s) {
+gf_status launch_ksum_t(const void* W, const Geo& g, __nv_bfloat16* thetaT, __nv_bfloat16* thetaT_lo, float* gwu,
+                        uint32_t* err_word, cudaStream_t s) {
     ProfScope prof(K_KSUM, s);
     const int taps = g.KH * g.KW;
     dim3 grid((g.C_in + 31) / 32, (g.C_out + 31) / 32, 1);
     if (grid.y > 65535) return GF_ERR_UNSUPPORTED;
     if (g.dtype == GF_F32)
-        return launch_pdl(ksum_t_kernel<float>, grid, dim3(1024), 0, s, (const float*)W, thetaT, gwu, g.C_in, g.C_out,
-                          taps, err_word);
-    return launch_pdl(ksum_t_kernel<__nv_bfloat16>, grid, dim3(1024), 0, s, (const __nv_bfloat16*)W, thetaT, gwu, g.C_in,
-                      g.C_out, taps, err_word);
+        return launch_pdl(ksum_t_kernel<float>, grid, dim3(1024), 0, s, (const float*)W, thetaT, thetaT_lo, gwu, g.C_in,
+                          g.C_out, taps, err_word);
+    return launch_pdl(ksum_t_kernel<__nv_bfloat16>, grid, dim3(1024), 0, s, (const __nv_bfloat16*)W, thetaT, thetaT_lo,
+                      gwu, g.C_in, g.C_out, taps, err_word);
+}
+
+gf_status launch_split_f32(const float* in, __nv_bfloat16* hi, __nv_bfloat16* lo, size_t n, cudaStream_t s) {
+    ProfScope prof(K_SPLIT, s);
+    if (n % 4 != 0 || n / 4 > 0x7fffffffULL * 256ULL) return GF_ERR_UNSUPPORTED;
+    const size_t n4 = n / 4;
+    return launch_pdl(split_f32_kernel, dim3((unsigned)((n4 + 255) / 256)), dim3(256), 0, s, in, hi, lo, n4);
 }
 
 static int sm_count_tc() {
@@ -685,52 +758,65 @@ static int sm_count_tc() {
     return n;
 }
 
-constexpr size_t kGxAResMaxBytes = 128 * 1024;     // largest resident thetaT tile (C_out <= 512)
+constexpr size_t kSmemLimit = 227 * 1024;
 
-template <typename TOut, int NT, int R, int LOGV, bool ARES>
-static gf_status launch_gx_tc_ares(const GxTcParams& p, int grid, cudaStream_t s) {
+template <typename TOut, int NT, int R, int LOGV, bool ARES, int SPLIT>
+static gf_status launch_gx_tc_ares(const GxTcParams& p, int grid, size_t a_res_bytes, cudaStream_t s) {
     constexpr size_t d_bytes = ((size_t)128 * (NT + 1) * 4 + 1023) / 1024 * 1024;
-    constexpr size_t smem = ARES ? (size_t)kGxStages * (kTcBK * NT * 2) + d_bytes + kGxAResMaxBytes + 1024
-                                 : (size_t)kGxStages * (128 * kTcBK * 2 + kTcBK * NT * 2) + d_bytes + 1024;
-    static bool configured = false;
-    if (!configured) {
-        GF_CUDA_TRY(cudaFuncSetAttribute(gx_tc_kernel<TOut, NT, R, LOGV, ARES>,
+    constexpr size_t ring = (size_t)gx_stages(SPLIT, ARES) * SPLIT * (kTcBK * NT * 2 + (ARES ? 0 : 128 * kTcBK * 2));
+    const size_t smem = ring + d_bytes + (ARES ? a_res_bytes : 0) + 1024;
+    static size_t configured = 0;
+    if (smem > configured) {
+        GF_CUDA_TRY(cudaFuncSetAttribute(gx_tc_kernel<TOut, NT, R, LOGV, ARES, SPLIT>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        configured = true;
+        configured = smem;
     }
-    return launch_pdl(gx_tc_kernel<TOut, NT, R, LOGV, ARES>, dim3(grid), dim3(kGxThreads), smem, s, p);
+    return launch_pdl(gx_tc_kernel<TOut, NT, R, LOGV, ARES, SPLIT>, dim3(grid), dim3(kGxThreads), smem, s, p);
 }
 
-template <typename TOut, int NT, int R, int LOGV>
+template <typename TOut, int NT, int R, int LOGV, int SPLIT>
 static gf_status launch_gx_tc_inst(const GxTcParams& p, cudaStream_t s) {
-    int grid = p.items < sm_count_tc() ? p.items : sm_count_tc();
+    const int grid = p.items < sm_count_tc() ? p.items : sm_count_tc();
     if constexpr (LOGV > 0) {
-        const size_t a_bytes = (size_t)((p.C_out + kTcBK - 1) / kTcBK) * 128 * kTcBK * 2;
+        constexpr size_t d_bytes = ((size_t)128 * (NT + 1) * 4 + 1023) / 1024 * 1024;
+        constexpr size_t ring = (size_t)gx_stages(SPLIT, true) * SPLIT * (kTcBK * NT * 2);
+        // the kernel's static shared memory (barriers, offset tables) counts against the same limit
+        constexpr size_t fixed = 512 + (R > 0 ? (size_t)NT * R * 10 : (size_t)NT * 12);
+        const size_t a_bytes = (size_t)SPLIT * ((p.C_out + kTcBK - 1) / kTcBK) * 128 * kTcBK * 2;
         const int g2 = grid / p.n_ci_tiles * p.n_ci_tiles;
-        if (a_bytes <= kGxAResMaxBytes && g2 >= p.n_ci_tiles)
-            return launch_gx_tc_ares<TOut, NT, R, LOGV, true>(p, g2, s);
+        if (ring + d_bytes + a_bytes + 1024 + fixed <= kSmemLimit && g2 >= p.n_ci_tiles)
+            return launch_gx_tc_ares<TOut, NT, R, LOGV, true, SPLIT>(p, g2, a_bytes, s);
     }
-    return launch_gx_tc_ares<TOut, NT, R, LOGV, false>(p, grid, s);
+    return launch_gx_tc_ares<TOut, NT, R, LOGV, false, SPLIT>(p, grid, 0, s);
 }
 
-template <typename TOut, int NT, int R>
+template <typename TOut, int NT, int R, int SPLIT>
 static gf_status launch_gx_tc_v(const GxTcParams& p, cudaStream_t s) {
     switch (p.gbar.logV) {
-        case 3: return launch_gx_tc_inst<TOut, NT, R, 3>(p, s);
-        case 2: return launch_gx_tc_inst<TOut, NT, R, 2>(p, s);
-        case 1: return launch_gx_tc_inst<TOut, NT, R, 1>(p, s);
-        default: return launch_gx_tc_inst<TOut, NT, R, 0>(p, s);
+        case 3: return launch_gx_tc_inst<TOut, NT, R, 3, SPLIT>(p, s);
+        case 2: return launch_gx_tc_inst<TOut, NT, R, 2, SPLIT>(p, s);
+        default: return launch_gx_tc_inst<TOut, NT, R, 0, SPLIT>(p, s);
     }
 }
 
-gf_status launch_gx_tc(const __nv_bfloat16* gbar, const __nv_bfloat16* thetaT, void* gX, uint32_t* err_word,
-                       const Geo& g, cudaStream_t s) {
+template <typename TOut, int NT, int SPLIT>
+static gf_status launch_gx_tc_r(const GxTcParams& p, int R, cudaStream_t s) {
+    if (R == 2) return launch_gx_tc_v<TOut, NT, 2, SPLIT>(p, s);
+    if (R == 4) return launch_gx_tc_v<TOut, NT, 4, SPLIT>(p, s);
+    if (R == 8) return launch_gx_tc_v<TOut, NT, 8, SPLIT>(p, s);
+    return launch_gx_tc_v<TOut, NT, 0, SPLIT>(p, s);
+}
+
+// gbar / thetaT: bf16 arrays; *_lo_off: elements from the high-part to the low-part array
+// (fp32 layers: operands carried as bf16 pairs), 0 for plain bf16 layers.
+gf_status launch_gx_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const __nv_bfloat16* thetaT,
+                       long long theta_lo_off, void* gX, uint32_t* err_word, const Geo& g, cudaStream_t s) {
     ProfScope prof(K_GX_TC, s);
     constexpr int NT = 64;
     GxTcParams p;
     const int P = g.Hp * g.Wp;
-    p.gbar = make_flat(gbar, g.C_out, P, (long long)g.N * P);
-    p.thetaT = make_flat(thetaT, g.C_in, g.C_out, g.C_out);
+    p.gbar = make_flat(gbar, g.C_out, P, (long long)g.N * P, gbar_lo_off);
+    p.thetaT = make_flat(thetaT, g.C_in, g.C_out, g.C_out, theta_lo_off);
     p.gX = gX; p.err_word = err_word;
     p.N = g.N; p.C_in = g.C_in; p.C_out = g.C_out; p.H = g.H; p.W = g.W; p.r = g.r; p.Hp = g.Hp; p.Wp = g.Wp; p.P = P;
     p.div_Wp = FastDiv((uint32_t)g.Wp);
@@ -743,49 +829,53 @@ gf_status launch_gx_tc(const __nv_bfloat16* gbar, const __nv_bfloat16* thetaT, v
     {   // pieces must not straddle a tile start: the piece width divides tile_cols as well as P
         int lv = p.gbar.logV;
         while (lv > 0 && (p.tile_cols % (1 << lv)) != 0) --lv;
-        p.gbar.logV = lv;
+        p.gbar.logV = lv == 1 ? 0 : lv;
     }
     const long long col_tiles = ((long long)g.N * P + p.tile_cols - 1) / p.tile_cols;
     const long long items = col_tiles * p.n_ci_tiles;
     const int n_chunks = (g.C_out + kTcBK - 1) / kTcBK;
     if (items * n_chunks > 0x7fffffffLL) return GF_ERR_UNSUPPORTED;
     p.items = (int)items;
-    if (R == 2) return launch_gx_tc_v<__nv_bfloat16, NT, 2>(p, s);
-    if (R == 4) return launch_gx_tc_v<__nv_bfloat16, NT, 4>(p, s);
-    if (R == 8) return launch_gx_tc_v<__nv_bfloat16, NT, 8>(p, s);
-    return launch_gx_tc_v<__nv_bfloat16, NT, 0>(p, s);
+    if (g.dtype == GF_F32) return launch_gx_tc_r<float, NT, 2>(p, R, s);
+    return launch_gx_tc_r<__nv_bfloat16, NT, 1>(p, R, s);
 }
 
-template <int NT, int LOGV>
+template <int NT, int LOGV, int SPLIT>
 static gf_status launch_gw_tc_inst(const GwTcParams& p, dim3 grid, cudaStream_t s) {
-    constexpr size_t smem = (size_t)kGwStages * (128 * kTcBK * 2 + NT * kTcBK * 2) + 1024;
+    constexpr size_t smem = (size_t)gw_stages(SPLIT) * SPLIT * (128 * kTcBK * 2 + NT * kTcBK * 2) + 1024;
     static bool configured = false;
     if (!configured) {
-        GF_CUDA_TRY(cudaFuncSetAttribute(gw_tc_kernel<NT, LOGV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        GF_CUDA_TRY(cudaFuncSetAttribute(gw_tc_kernel<NT, LOGV, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         configured = true;
     }
-    return launch_pdl(gw_tc_kernel<NT, LOGV>, grid, dim3(kGwThreads), smem, s, p);
+    return launch_pdl(gw_tc_kernel<NT, LOGV, SPLIT>, grid, dim3(kGwThreads), smem, s, p);
 }
 
-gf_status launch_gw_tc(const __nv_bfloat16* gbar, const __nv_bfloat16* stash, float* gwu, int splits,
-                       uint32_t* err_word, const Geo& g, cudaStream_t s) {
+template <int NT, int SPLIT>
+static gf_status launch_gw_tc_v(const GwTcParams& p, dim3 grid, cudaStream_t s) {
+    switch (p.gbar.logV) {
+        case 3: return launch_gw_tc_inst<NT, 3, SPLIT>(p, grid, s);
+        case 2: return launch_gw_tc_inst<NT, 2, SPLIT>(p, grid, s);
+        default: return launch_gw_tc_inst<NT, 0, SPLIT>(p, grid, s);
+    }
+}
+
+gf_status launch_gw_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const __nv_bfloat16* stash,
+                       long long stash_lo_off, float* gwu, int splits, uint32_t* err_word, const Geo& g,
+                       cudaStream_t s) {
     ProfScope prof(K_GW_TC, s);
     constexpr int NT = 128;
     GwTcParams p;
     const int P = g.Hp * g.Wp;
     const long long K = (long long)g.N * P;
-    p.gbar = make_flat(gbar, g.C_out, P, K);
-    p.stash = make_flat(stash, g.C_in, P, K);
+    p.gbar = make_flat(gbar, g.C_out, P, K, gbar_lo_off);
+    p.stash = make_flat(stash, g.C_in, P, K, stash_lo_off);
     p.gwu = gwu; p.err_word = err_word; p.C_in = g.C_in; p.C_out = g.C_out; p.S = splits;
     p.chunks_total = (int)((K + kTcBK - 1) / kTcBK);
     if ((g.C_out + 127) / 128 > 65535 || splits > 65535) return GF_ERR_UNSUPPORTED;
     dim3 grid((g.C_in + NT - 1) / NT, (g.C_out + 127) / 128, splits);
-    switch (p.gbar.logV) {
-        case 3: return launch_gw_tc_inst<NT, 3>(p, grid, s);
-        case 2: return launch_gw_tc_inst<NT, 2>(p, grid, s);
-        case 1: return launch_gw_tc_inst<NT, 1>(p, grid, s);
-        default: return launch_gw_tc_inst<NT, 0>(p, grid, s);
-    }
+    if (g.dtype == GF_F32) return launch_gw_tc_v<NT, 2>(p, grid, s);
+    return launch_gw_tc_v<NT, 1>(p, grid, s);
 }
 
 }  // namespace gf
