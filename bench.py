@@ -435,6 +435,8 @@ def run_table(args) -> None:
     peaks, which = measured_peaks()
     layers = [l for l in workloads.all_headline_layers() if l.r > 1] + workloads.ondevice_table(2, "f32") \
         + workloads.ondevice_table(4, "f32")
+    if args.only:
+        layers = [l for l in layers if any(k in f"{l.name}/r{l.r}/{l.dtype}" for k in args.only.split(","))]
     stream = torch.cuda.current_stream()
     rows = []
 
@@ -475,6 +477,14 @@ def run_table(args) -> None:
                                                 L.groups, [True, True, False])
 
         t_stash, t_bwd = timed(stash, reps), timed(bwd, reps)
+        # per-kernel event times of the backward call (each bracketed, so a few us high)
+        gf.gf_profile_configure(2)
+        torch.cuda._sleep(int(3e-3 * 1.9e9))
+        for i in range(4):
+            bwd(i)
+        torch.cuda.synchronize()
+        kern = {k: round(ms / n * 1e3, 1) for k, (n, ms) in gf.gf_profile_read().items()}
+        gf.gf_profile_configure(0)
         try:
             t_exact = timed(exact, max(2, reps // 4))
         except Exception:
@@ -485,7 +495,7 @@ def run_table(args) -> None:
                "backward_frac_hbm": L.backward_bytes() / t_bwd / 1e3 / peaks["hbm_gbs"],
                "stash_gbs": L.stash_bytes_moved() / t_stash / 1e3,
                "stash_frac_hbm": L.stash_bytes_moved() / t_stash / 1e3 / peaks["hbm_gbs"],
-               "exact_cudnn_us": t_exact, "reduced_gflop": L.reduced_flops() / 1e9}
+               "exact_cudnn_us": t_exact, "reduced_gflop": L.reduced_flops() / 1e9, "kernels_us": kern}
         rows.append(row)
         print(json.dumps(row), flush=True)
         del sets
@@ -505,6 +515,7 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--table", action="store_true", help="time every layer shape once (diagnostic table)")
+    ap.add_argument("--only", default="", help="--table: comma-separated substrings of name/rR/dtype to keep")
     args = ap.parse_args()
     if args.table:
         run_table(args)

@@ -110,15 +110,17 @@ Workspace plan_workspace(const Geo& g) {
     w.off_split = 0;
     if (g.r == 1) { w.off_tsum = w.off_gbar = w.off_part = off; w.splits = 0; w.total = off; return w; }
     w.off_tsum = off; off += align_up((size_t)g.C_out * g.C_ig * 4, 256);
-    w.off_gbar = off; off += align_up((size_t)g.N * g.C_out * g.Hp * g.Wp * 4, 256);
+    const size_t pitch = tc_eligible(g) ? (size_t)tc_pitch(g) : (size_t)g.Hp * g.Wp;
+    w.off_gbar = off; off += align_up((size_t)g.N * g.C_out * pitch * 4, 256);
     int s = dense_splits(g);
     if (tc_eligible(g)) { const int ts = tc_gw_splits(g); if (ts > s) s = ts; }
     if (is_depthwise(g)) { const int ds = depthwise_splits(g); if (ds > s) s = ds; }
     w.splits = s;
     w.off_part = off; off += align_up((size_t)s * g.C_out * g.C_ig * 4, 256);
-    if (tc_eligible(g) && g.dtype == GF_F32) {
-        // fp32 stash as (high, low) bf16 arrays for the tensor-core contraction
-        w.off_split = off; off += 2 * align_up((size_t)g.N * g.C_in * g.Hp * g.Wp * 2, 256);
+    if (tc_eligible(g) && (g.dtype == GF_F32 || pitch != (size_t)g.Hp * g.Wp)) {
+        // the stash as the tensor-core contraction reads it: bf16 in the operand pitch, fp32
+        // values as (high, low) pairs
+        w.off_split = off; off += 2 * align_up((size_t)g.N * g.C_in * pitch * 2, 256);
     }
     w.total = off;
     return w;
@@ -170,7 +172,7 @@ gf_status gf_stash_forward(const gf_conv_desc* desc, const void* x, void* stash,
     if (g.r == 1) return launch_copy(x, stash, (size_t)planes * g.H * g.W * g.esize, s);
     uint32_t* err = global_err_word();
     if (!err) return GF_ERR_CUDA;
-    return launch_pool(K_STASH_POOL, x, g.dtype, stash, nullptr, g.dtype, /*mean=*/false, planes, g.H, g.W, g.r, err, s);
+    return launch_pool(K_STASH_POOL, x, g.dtype, stash, nullptr, g.dtype, /*mean=*/false, planes, g.H, g.W, g.r, 0, err, s);
 }
 
 gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* stash, const void* W,
@@ -213,16 +215,17 @@ gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* sta
         // every operand as a (high, low) bf16 pair: v = hi + lo up to 2^-17 |v|.
         const bool split = g.dtype == GF_F32;
         const size_t P = (size_t)g.Hp * g.Wp;
+        const size_t pitch = (size_t)tc_pitch(g);     // > P: planes padded so that rows can be copied in aligned pieces
         // low parts sit 16-byte aligned behind the high parts, inside the fp32-sized regions
         const long long theta_lo = split ? (long long)align_up((size_t)g.C_in * g.C_out, 8) : 0;
-        const long long gbar_lo = split ? (long long)align_up((size_t)g.N * g.C_out * P, 8) : 0;
-        const long long stash_lo = split ? (long long)(align_up((size_t)g.N * g.C_in * P * 2, 256) / 2) : 0;
+        const long long gbar_lo = split ? (long long)align_up((size_t)g.N * g.C_out * pitch, 8) : 0;
+        const long long stash_lo = split ? (long long)(align_up((size_t)g.N * g.C_in * pitch * 2, 256) / 2) : 0;
         __nv_bfloat16* thetaT = reinterpret_cast<__nv_bfloat16*>(tsum);
         __nv_bfloat16* gbar16 = reinterpret_cast<__nv_bfloat16*>(gbar);
         st = launch_ksum_t(W, g, thetaT, split ? thetaT + theta_lo : nullptr, g_W ? part : nullptr, err, s);
         if (st != GF_OK) return st;
         st = launch_pool(K_GY_POOL, g_y, g.dtype, gbar16, split ? gbar16 + gbar_lo : nullptr, GF_BF16, /*mean=*/true,
-                         (int64_t)g.N * g.C_out, g.H, g.W, g.r, err, s);
+                         (int64_t)g.N * g.C_out, g.H, g.W, g.r, (int)pitch, err, s);
         if (st != GF_OK) return st;
         if (g_X) {
             st = launch_gx_tc(gbar16, gbar_lo, thetaT, theta_lo, g_X, err, g, s);
@@ -230,9 +233,13 @@ gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* sta
         }
         if (g_W) {
             const __nv_bfloat16* stash16 = static_cast<const __nv_bfloat16*>(stash);
-            if (split) {
+            if (split || pitch != P) {
                 __nv_bfloat16* sp = reinterpret_cast<__nv_bfloat16*>(base + ws.off_split);
-                st = launch_split_f32(static_cast<const float*>(stash), sp, sp + stash_lo, (size_t)g.N * g.C_in * P, s);
+                if (pitch == P)
+                    st = launch_split_f32(static_cast<const float*>(stash), sp, sp + stash_lo, (size_t)g.N * g.C_in * P, s);
+                else
+                    st = launch_repack(stash, g.dtype, sp, split ? sp + stash_lo : nullptr, (long long)g.N * g.C_in,
+                                       (int)P, (int)pitch, s);
                 if (st != GF_OK) return st;
                 stash16 = sp;
             }
@@ -249,7 +256,7 @@ gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* sta
     // patch means of g_y, read once
     st = launch_ksum(W, g, tsum, err, s);
     if (st != GF_OK) return st;
-    st = launch_pool(K_GY_POOL, g_y, g.dtype, gbar, nullptr, GF_F32, /*mean=*/true, (int64_t)g.N * g.C_out, g.H, g.W, g.r, err, s);
+    st = launch_pool(K_GY_POOL, g_y, g.dtype, gbar, nullptr, GF_F32, /*mean=*/true, (int64_t)g.N * g.C_out, g.H, g.W, g.r, 0, err, s);
     if (st != GF_OK) return st;
     if (g_X) {
         st = launch_gx_mix(gbar, tsum, g_X, g, s);

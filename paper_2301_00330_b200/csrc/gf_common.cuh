@@ -155,9 +155,10 @@ struct Workspace {
 Workspace plan_workspace(const Geo& g);
 
 // ---- kernel entry points (host launchers) ----------------------------------
-// pool: out[plane, a, b] = sum (or mean) of in[plane] over patch (a,b)
+// pool: out[plane, a, b] = sum (or mean) of in[plane] over patch (a,b).  out_lo: bf16 low
+// parts (NULL: none).  out_pitch: elements between output planes, 0 = dense; a gap is zeroed.
 gf_status launch_pool(int kernel_id, const void* in, int in_dtype, void* out, void* out_lo, int out_dtype, bool mean,
-                      int64_t planes, int H, int W, int r, uint32_t* err_word, cudaStream_t s);
+                      int64_t planes, int H, int W, int r, int out_pitch, uint32_t* err_word, cudaStream_t s);
 gf_status launch_copy(const void* in, void* out, size_t bytes, cudaStream_t s);
 
 gf_status launch_ksum(const void* W, const Geo& g, float* tsum, uint32_t* err_word, cudaStream_t s);
@@ -172,6 +173,11 @@ int depthwise_splits(const Geo& g);
 // tensor-core path (bf16 operands, dense layers)
 bool tc_eligible(const Geo& g);
 int tc_gw_splits(const Geo& g);
+// elements between the (image, channel) planes of the tensor-core operands: Hp*Wp, or
+// that rounded up to 8 when plain rows could not be copied in aligned pieces
+int tc_pitch(const Geo& g);
+gf_status launch_repack(const void* in, int in_dtype, __nv_bfloat16* hi, __nv_bfloat16* lo, long long rows, int P,
+                        int pitch, cudaStream_t s);
 gf_status launch_ksum_t(const void* W, const Geo& g, __nv_bfloat16* thetaT, __nv_bfloat16* thetaT_lo, float* gwu,
                         uint32_t* err_word, cudaStream_t s);
 gf_status launch_split_f32(const float* in, __nv_bfloat16* hi, __nv_bfloat16* lo, size_t n, cudaStream_t s);

@@ -35,6 +35,8 @@ struct PoolParams {
     int BR;      // patch rows per tile (== Hp when P > 1)
     int bands;   // tiles along the patch rows of one plane (1 when P > 1)
     int mean;    // 1: patch mean, 0: patch sum
+    int plane_out;   // Hp * Wp
+    int out_pitch;   // elements between output planes (>= plane_out; the gap is written as zeros)
     long long strips;   // streamed kernel: planes * H / r strips of r rows
     int S;              // streamed kernel: strips per tile
     FastDiv div_bands, div_plane_out /* Hp*Wp */, div_Wp;
@@ -104,6 +106,38 @@ __device__ __forceinline__ void store_split(__nv_bfloat16* hi, __nv_bfloat16* lo
 }
 template <int G> __device__ __forceinline__ void store_split(float*, float*, const float (&)[G]) {}
 
+// Destination index of output `og` (flattened over the planes), G outputs at a time
+// (G | Wp, so they stay inside a plane).  With a padded plane pitch the writer of a
+// plane's last outputs also clears the pad.
+template <typename TOut, int G>
+__device__ __forceinline__ long long out_index(const PoolParams& p, long long og) {
+    if (p.out_pitch == p.plane_out) return og;
+    uint32_t pl, rem;
+    p.div_plane_out.divmod((uint32_t)og, pl, rem);
+    const long long base = (long long)pl * p.out_pitch;
+    if ((int)rem + G == p.plane_out) {
+        TOut* hi = static_cast<TOut*>(p.out) + base;
+        TOut* lo = p.out_lo ? static_cast<TOut*>(p.out_lo) + base : nullptr;
+        for (int k = p.plane_out; k < p.out_pitch; ++k) {
+            hi[k] = from_f32<TOut>(0.f);
+            if (lo) lo[k] = from_f32<TOut>(0.f);
+        }
+    }
+    return base + rem;
+}
+
+// one output value (or its high/low pair)
+template <typename TOut>
+__device__ __forceinline__ void store_one(const PoolParams& p, long long idx, float v) {
+    TOut* out = static_cast<TOut*>(p.out);
+    if (p.out_lo) {
+        const float a[1] = {v};
+        store_split<1>(out + idx, static_cast<TOut*>(p.out_lo) + idx, a);
+    } else {
+        out[idx] = from_f32<TOut>(v);
+    }
+}
+
 // ---- tile geometry (shared by the two tiled kernels) ------------------------------
 struct Tile { long long g0, out_base; int len, np, a0, na; };
 __device__ __forceinline__ Tile tile_of(const PoolParams& p, long long t) {
@@ -159,7 +193,7 @@ __device__ __forceinline__ int stage_plain(const TIn* __restrict__ in, long long
 // R*W contiguous elements that produce the Wp contiguous outputs s*Wp .. s*Wp+Wp-1.
 // A tile is S consecutive strips (plane boundaries do not matter).
 template <typename TIn, typename TOut, int R, int G>
-__device__ __forceinline__ void reduce_item(const PoolParams& p, const TIn* buf, TOut* dst, uint32_t q) {
+__device__ __forceinline__ void reduce_item(const PoolParams& p, const TIn* buf, long long og0, uint32_t q) {
     const uint32_t o = q * G;
     uint32_t A, b;
     p.div_Wp.divmod(o, A, b);
@@ -183,8 +217,10 @@ __device__ __forceinline__ void reduce_item(const PoolParams& p, const TIn* buf,
 #pragma unroll
         for (int k = 0; k < G; ++k) acc[k] *= p.inv_full;
     }
-    if (p.out_lo) store_split<G>(dst + o, static_cast<TOut*>(p.out_lo) + (dst - static_cast<TOut*>(p.out)) + o, acc);
-    else store_vec<G>(dst + o, acc);
+    const long long idx = out_index<TOut, G>(p, og0 + o);
+    TOut* dst = static_cast<TOut*>(p.out) + idx;
+    if (p.out_lo) store_split<G>(dst, static_cast<TOut*>(p.out_lo) + idx, acc);
+    else store_vec<G>(dst, acc);
 }
 
 template <typename TIn, typename TOut, int R, int G>
@@ -192,7 +228,6 @@ __global__ void __launch_bounds__(kStreamThreads, 1) pool_stream_kernel(const Po
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     __shared__ uint64_t full[kStreamStages];
     const TIn* __restrict__ in = static_cast<const TIn*>(p.in);
-    TOut* __restrict__ out = static_cast<TOut*>(p.out);
     const long long first = blockIdx.x, stride = gridDim.x;
     const int n_my = first < p.tiles ? (int)((p.tiles - first + stride - 1) / stride) : 0;
     const int strip_elems = R * p.W;
@@ -237,7 +272,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) pool_stream_kernel(const Po
         }
         if (ok) {
             const uint32_t nitems = (uint32_t)(ns * p.Wp) / G;
-            TOut* dst = out + tile * p.S * p.Wp;
+            const long long dst = tile * p.S * p.Wp;      // first output of the tile, flattened over planes
             const TIn* b = buf(s);
             uint32_t q = threadIdx.x;
             for (; q + kStreamThreads < nitems; q += 2 * kStreamThreads) {   // two independent items in flight
@@ -267,7 +302,6 @@ template <typename TIn, typename TOut, int R>
 __global__ void __launch_bounds__(kPoolThreads) pool_tile_kernel(const PoolParams p) {
     __shared__ uint4 smem_v[kPoolTileBytes / 16 + 1];
     const TIn* __restrict__ in = static_cast<const TIn*>(p.in);
-    TOut* __restrict__ out = static_cast<TOut*>(p.out);
     const Tile g = tile_of(p, blockIdx.x);
     const int shift = stage_plain<TIn, kPoolThreads>(in, p.total_elems, g.g0, g.len, smem_v);
     const TIn* smem = reinterpret_cast<const TIn*>(smem_v);
@@ -296,12 +330,7 @@ __global__ void __launch_bounds__(kPoolThreads) pool_tile_kernel(const PoolParam
             cnt = nr * nc;
         }
         if (p.mean) s *= (cnt == p.r * p.r) ? p.inv_full : 1.0f / (float)cnt;
-        if (p.out_lo) {
-            const float a[1] = {s};
-            store_split<1>(out + g.out_base + o, static_cast<TOut*>(p.out_lo) + g.out_base + o, a);
-        } else {
-            out[g.out_base + o] = from_f32<TOut>(s);
-        }
+        store_one<TOut>(p, out_index<TOut, 1>(p, g.out_base + o), s);
     }
 }
 
@@ -311,7 +340,6 @@ template <typename TIn, typename TOut>
 __global__ void __launch_bounds__(kPoolThreads) pool_bigpatch_kernel(const PoolParams p) {
     __shared__ float warp_part[kPoolThreads / 32];
     const TIn* __restrict__ in = static_cast<const TIn*>(p.in);
-    TOut* __restrict__ out = static_cast<TOut*>(p.out);
     const long long o = blockIdx.x;
     const int plane_out = p.Hp * p.Wp;
     const long long pl = o / plane_out;
@@ -332,12 +360,7 @@ __global__ void __launch_bounds__(kPoolThreads) pool_bigpatch_kernel(const PoolP
         t = warp_sum(t);
         if (threadIdx.x == 0) {
             if (p.mean) t /= (float)(nr * nc);
-            if (p.out_lo) {
-                const float a[1] = {t};
-                store_split<1>(out + o, static_cast<TOut*>(p.out_lo) + o, a);
-            } else {
-                out[o] = from_f32<TOut>(t);
-            }
+            store_one<TOut>(p, out_index<TOut, 1>(p, o), t);
         }
     }
 }
@@ -432,13 +455,17 @@ static gf_status pool_dispatch(PoolParams& p, size_t e, cudaStream_t s) {
 }
 
 gf_status launch_pool(int kernel_id, const void* in, int in_dtype, void* out, void* out_lo, int out_dtype, bool mean,
-                      int64_t planes, int H, int W, int r, uint32_t* err_word, cudaStream_t s) {
+                      int64_t planes, int H, int W, int r, int out_pitch, uint32_t* err_word, cudaStream_t s) {
     ProfScope prof(kernel_id, s);
     PoolParams p;
     if (out_lo && out_dtype != GF_BF16) return GF_ERR_UNSUPPORTED;
     p.in = in; p.out = out; p.out_lo = out_lo; p.err_word = err_word; p.planes = planes; p.total_elems = planes * H * W;
     p.H = H; p.W = W; p.r = r; p.mean = mean ? 1 : 0;
     p.Hp = (H + r - 1) / r; p.Wp = (W + r - 1) / r;
+    p.plane_out = p.Hp * p.Wp;
+    p.out_pitch = out_pitch > 0 ? out_pitch : p.plane_out;
+    if (p.out_pitch < p.plane_out) return GF_ERR_BAD_DESC;
+    if (p.out_pitch != p.plane_out && planes * p.plane_out > 0x7fffffffLL) return GF_ERR_UNSUPPORTED;
     p.div_plane_out = FastDiv(p.Hp * p.Wp);
     p.div_Wp = FastDiv(p.Wp);
     p.inv_full = 1.0f / ((float)r * (float)r);

@@ -217,10 +217,25 @@ struct GxTcParams {
     FlatSrc thetaT;                     // [C_in][C_out] as a flat source with P = C_out
     void* gX;
     uint32_t* err_word;
-    int N, C_in, C_out, H, W, r, Hp, Wp, P;
+    int N, C_in, C_out, H, W, r, Hp, Wp;
+    int P;                              // elements between the planes of gbar (>= Hp*Wp; the gap holds zeros)
+    int P_live;                         // Hp*Wp
     int n_ci_tiles, items;
     int tile_cols;                      // flattened columns per tile: whole patch rows (R > 0) or NT
-    FastDiv div_Wp, div_Hp, div_RWp, div_ci_tiles;
+    // padded planes with R > 0: a tile is rows_per_tile patch rows of ONE image, loaded from
+    // the 8-element boundary below its first column (tiles_per_img tiles per image); 0 otherwise
+    int rows_per_tile, tiles_per_img;
+    FastDiv div_Wp, div_Hp, div_RWp, div_ci_tiles, div_tiles_per_img;
+};
+
+// One unit of work of gx_tc: a 128-row c_i tile times a column tile.
+struct GxItem {
+    int ci0;
+    long long col0;     // first column loaded (flattened over images with pitch P)
+    int ncols;          // columns loaded
+    uint32_t A0;        // R > 0: first patch row, counted over all images
+    int shift;          //        tile column of that row's first patch
+    int nlive;          //        patches of the tile
 };
 
 // R consecutive copies of v
@@ -313,13 +328,30 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
     const uint32_t tmem = sh.tmem_base;
     pdl_wait();                       // operands come from the previous kernels of the stream
     bool ok = true;
-    auto item_of = [&](int it, int& ci0, long long& col0, int& ncols) {
+    auto item_of = [&](int it) {
+        GxItem w;
         uint32_t ct, cit;
         if constexpr (ARES) { ct = (uint32_t)(first + it * stride); cit = blockIdx.x % (uint32_t)p.n_ci_tiles; }
         else p.div_ci_tiles.divmod((uint32_t)(first + it * stride), ct, cit);
-        ci0 = (int)cit * 128;
-        col0 = (long long)ct * p.tile_cols;
-        ncols = (int)min((long long)p.tile_cols, p.gbar.k_total - col0);
+        w.ci0 = (int)cit * 128;
+        if (R > 0 && p.rows_per_tile > 0) {
+            uint32_t n, t;
+            p.div_tiles_per_img.divmod(ct, n, t);
+            const int a0 = (int)t * p.rows_per_tile;
+            const int ps = a0 * p.Wp;
+            w.shift = ps & 7;
+            w.col0 = (long long)n * p.P + (ps - w.shift);
+            w.nlive = min(p.rows_per_tile, p.Hp - a0) * p.Wp;
+            w.ncols = w.shift + w.nlive;
+            w.A0 = n * (uint32_t)p.Hp + (uint32_t)a0;
+        } else {
+            w.col0 = (long long)ct * p.tile_cols;
+            w.ncols = (int)min((long long)p.tile_cols, p.gbar.k_total - w.col0);
+            w.shift = 0;
+            w.nlive = w.ncols;
+            w.A0 = R > 0 ? p.div_Wp.div((uint32_t)w.col0) : 0u;
+        }
+        return w;
     };
 
     if (warp < kGxLoaders / 32) {
@@ -336,13 +368,12 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
                                               [&](int q, uint32_t tile) {
                 const int it = q / n_chunks, kc = q - it * n_chunks;
                 if (it != cur_it) {                        // per item: this thread's first source elements
-                    long long col0;
-                    int ncols;
-                    item_of(it, ci0, col0, ncols);
+                    const GxItem w = item_of(it);
+                    ci0 = w.ci0;
                     cur_it = it;
                     a_src = p.thetaT.base + (size_t)(ci0 + pa.row0) * p.C_out + pa.k;
-                    b_ok = pb.j < ncols;
-                    b_src = flat_ptr(p.gbar, pb.krow0, b_ok ? col0 + pb.j : 0);
+                    b_ok = pb.j < w.ncols;
+                    b_src = flat_ptr(p.gbar, pb.krow0, b_ok ? w.col0 + pb.j : 0);
                 }
                 const int k0 = kc * kTcBK;
                 if constexpr (ARES) {
@@ -368,15 +399,14 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
             ok = run_sync_loaders<kGxStages>(sh.full, sh.empty, dyn, kStageBytes, n_my * n_chunks,
                                              [&](int q, unsigned char* tile) {
                 const int it = q / n_chunks, kc = q - it * n_chunks;
-                int ci0, ncols; long long col0;
-                item_of(it, ci0, col0, ncols);
+                const GxItem w = item_of(it);
 #pragma unroll
                 for (int h = 0; h < SPLIT; ++h) {
                     FlatSrc a = p.thetaT, b = p.gbar;
                     a.base += h * a.lo_off;
                     b.base += h * b.lo_off;
-                    load_kmajor_scalar<128, kGxLoaders>(tile + h * kABytes, a, ci0, (long long)kc * kTcBK, tid);
-                    load_mnmajor_scalar<NT, kGxLoaders>(tile + kBOff + h * kBBytes, b, kc * kTcBK, col0, ncols, tid);
+                    load_kmajor_scalar<128, kGxLoaders>(tile + h * kABytes, a, w.ci0, (long long)kc * kTcBK, tid);
+                    load_mnmajor_scalar<NT, kGxLoaders>(tile + kBOff + h * kBBytes, b, kc * kTcBK, w.col0, w.ncols, tid);
                 }
             });
         }
@@ -405,13 +435,14 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
         const size_t plane = (size_t)p.H * p.W;
         for (int it = 0; it < n_my; ++it) {
             const int buf = it & 1;
-            int ci0, ncols; long long col0;
-            item_of(it, ci0, col0, ncols);
+            const GxItem w = item_of(it);
+            const int ci0 = w.ci0, ncols = w.ncols;
+            const long long col0 = w.col0;
             if constexpr (R > 0) {
                 // vector u of the tile's part of a plane, in memory order: patch row ta of the tile,
                 // pixel row dr of that patch row, patch jb of the row
-                const uint32_t A0 = p.div_Wp.div((uint32_t)col0);          // first global patch row
-                for (int u = et; u < ncols * R; u += kGxEpi) {
+                const uint32_t A0 = w.A0;                                  // first patch row, over all images
+                for (int u = et; u < w.nlive * R; u += kGxEpi) {
                     uint32_t ta, rem, dr, jb, n, a;
                     p.div_RWp.divmod((uint32_t)u, ta, rem);
                     p.div_Wp.divmod(rem, dr, jb);
@@ -419,7 +450,7 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
                     const int row = (int)a * R + (int)dr;
                     unit_off[u] = row < p.H ? (long long)n * p.C_in * p.H * p.W + (long long)row * p.W + (long long)jb * R
                                             : -1;
-                    unit_src[u] = (unsigned short)(ta * p.Wp + jb);
+                    unit_src[u] = (unsigned short)(w.shift + ta * p.Wp + jb);
                 }
             } else {
                 for (int j = et; j < NT; j += kGxEpi) {      // patch offsets of this tile's columns
@@ -428,10 +459,12 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
                     if (j < ncols) {
                         const long long c = col0 + j;
                         const uint32_t n = p.gbar.div_P.div((uint32_t)c), pp = (uint32_t)c - n * (uint32_t)p.P;
-                        uint32_t a, b;
-                        p.div_Wp.divmod(pp, a, b);
-                        off = (long long)n * p.C_in * p.H * p.W + (long long)a * p.r * p.W + (long long)b * p.r;
-                        ext = min(p.r, p.W - (int)b * p.r) | (min(p.r, p.H - (int)a * p.r) << 16);
+                        if ((int)pp < p.P_live) {               // not a pad column
+                            uint32_t a, b;
+                            p.div_Wp.divmod(pp, a, b);
+                            off = (long long)n * p.C_in * p.H * p.W + (long long)a * p.r * p.W + (long long)b * p.r;
+                            ext = min(p.r, p.W - (int)b * p.r) | (min(p.r, p.H - (int)a * p.r) << 16);
+                        }
                     }
                     col_off[j] = off;
                     col_cols[j] = ext;
@@ -461,7 +494,7 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
                     // expansion in memory order, 16 bytes per store where possible: lane l owns the
                     // chunks l, l+32, ... of UPC consecutive vectors each, for every plane
                     constexpr int UPC = (16 / (R * (int)sizeof(TOut))) > 1 ? 16 / (R * (int)sizeof(TOut)) : 1;
-                    const int n_units = ncols * R;
+                    const int n_units = w.nlive * R;
                     const bool plane_al = (plane * sizeof(TOut)) % 16 == 0 &&
                                           (reinterpret_cast<uintptr_t>(gx) & 15) == 0;
                     for (int u0 = lane * UPC; u0 < n_units; u0 += 32 * UPC) {
@@ -702,6 +735,24 @@ __global__ void __launch_bounds__(256) split_f32_kernel(const float* __restrict_
     reinterpret_cast<uint2*>(lo)[i] = *reinterpret_cast<uint2*>(l);
 }
 
+// [rows][P] -> bf16 [rows][pitch] with a zeroed gap, fp32 inputs as (high, low) pairs:
+// the stash in the plane pitch the tensor-core loaders want.
+template <typename TIn>
+__global__ void __launch_bounds__(256) repack_kernel(const TIn* __restrict__ in, __nv_bfloat16* __restrict__ hi,
+                                                     __nv_bfloat16* __restrict__ lo, long long total, int P, int pitch,
+                                                     FastDiv div_pitch) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    uint32_t row, k;
+    div_pitch.divmod((uint32_t)i, row, k);
+    const float v = (int)k < P ? to_f32(in[(size_t)row * P + k]) : 0.f;
+    const __nv_bfloat16 h = __float2bfloat16_rn(v);
+    hi[i] = h;
+    if (lo) lo[i] = __float2bfloat16_rn(v - __bfloat162float(h));
+}
+
 // ================================================================== host side
 static FlatSrc make_flat(const void* base, int C, int P, long long k_total, long long lo_off) {
     FlatSrc s;
@@ -714,11 +765,34 @@ static FlatSrc make_flat(const void* base, int C, int P, long long k_total, long
 
 bool tc_eligible(const Geo& g) {
     return (g.dtype == GF_BF16 || g.dtype == GF_F32) && g.G == 1 && g.r >= 2 && g.C_out % 8 == 0 &&
-           (long long)g.N * g.Hp * g.Wp < (1LL << 31);
+           (long long)g.N * (((long long)g.Hp * g.Wp + 7) / 8 * 8) < (1LL << 31);
+}
+
+int tc_pitch(const Geo& g) {
+    const long long P = (long long)g.Hp * g.Wp;
+    if (P % 4 == 0) return (int)P;                  // 8- or 16-byte pieces of plain rows
+    const long long pitch = (P + 7) / 8 * 8;
+    const long long C = g.C_in > g.C_out ? g.C_in : g.C_out;
+    if ((long long)g.N * C * pitch > 0x7fffffffLL) return (int)P;     // 32-bit indexing of the padded copies
+    return (int)pitch;
+}
+
+gf_status launch_repack(const void* in, int in_dtype, __nv_bfloat16* hi, __nv_bfloat16* lo, long long rows, int P,
+                        int pitch, cudaStream_t s) {
+    ProfScope prof(K_SPLIT, s);
+    const long long total = rows * pitch;
+    if (total > 0x7fffffffLL) return GF_ERR_UNSUPPORTED;
+    if (total == 0) return GF_OK;
+    const dim3 grid((unsigned)((total + 255) / 256));
+    if (in_dtype == GF_F32)
+        return launch_pdl(repack_kernel<float>, grid, dim3(256), 0, s, (const float*)in, hi, lo, total, P, pitch,
+                          FastDiv((uint32_t)pitch));
+    return launch_pdl(repack_kernel<__nv_bfloat16>, grid, dim3(256), 0, s, (const __nv_bfloat16*)in, hi, lo, total, P,
+                      pitch, FastDiv((uint32_t)pitch));
 }
 
 int tc_gw_splits(const Geo& g) {
-    const long long K = (long long)g.N * g.Hp * g.Wp;
+    const long long K = (long long)g.N * tc_pitch(g);
     const int chunks = (int)((K + kTcBK - 1) / kTcBK);
     const int tiles = ((g.C_in + 127) / 128) * ((g.C_out + 127) / 128);
     int s = (148 + tiles - 1) / tiles;
@@ -814,7 +888,9 @@ gf_status launch_gx_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const _
     ProfScope prof(K_GX_TC, s);
     constexpr int NT = 64;
     GxTcParams p;
-    const int P = g.Hp * g.Wp;
+    const int P = tc_pitch(g);                      // gbar's plane pitch
+    const bool padded = P != g.Hp * g.Wp;
+    p.P_live = g.Hp * g.Wp;
     p.gbar = make_flat(gbar, g.C_out, P, (long long)g.N * P, gbar_lo_off);
     p.thetaT = make_flat(thetaT, g.C_in, g.C_out, g.C_out, theta_lo_off);
     p.gX = gX; p.err_word = err_word;
@@ -823,15 +899,27 @@ gf_status launch_gx_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const _
     p.div_Hp = FastDiv((uint32_t)g.Hp);
     p.n_ci_tiles = (g.C_in + 127) / 128;
     p.div_ci_tiles = FastDiv((uint32_t)p.n_ci_tiles);
-    const int R = (g.W % g.r == 0 && g.Wp <= NT && (g.r == 2 || g.r == 4 || g.r == 8)) ? g.r : 0;
+    int R = (g.W % g.r == 0 && g.Wp <= NT && (g.r == 2 || g.r == 4 || g.r == 8)) ? g.r : 0;
+    if (padded && g.Wp > NT - 7) R = 0;             // no room for the alignment slack of a row-aligned tile
     p.div_RWp = FastDiv((uint32_t)((R > 0 ? R : 1) * g.Wp));
     p.tile_cols = R > 0 ? (NT / g.Wp) * g.Wp : NT;
-    {   // pieces must not straddle a tile start: the piece width divides tile_cols as well as P
+    p.rows_per_tile = 0;
+    p.tiles_per_img = 1;
+    long long col_tiles;
+    if (padded && R > 0) {
+        // tiles of whole patch rows of one image, loaded from an 8-element boundary
+        p.rows_per_tile = (NT - 7) / g.Wp;
+        if (p.rows_per_tile > g.Hp) p.rows_per_tile = g.Hp;
+        p.tiles_per_img = (g.Hp + p.rows_per_tile - 1) / p.rows_per_tile;
+        col_tiles = (long long)g.N * p.tiles_per_img;
+    } else {
+        // pieces must not straddle a tile start: the piece width divides tile_cols as well as P
         int lv = p.gbar.logV;
         while (lv > 0 && (p.tile_cols % (1 << lv)) != 0) --lv;
         p.gbar.logV = lv == 1 ? 0 : lv;
+        col_tiles = ((long long)g.N * P + p.tile_cols - 1) / p.tile_cols;
     }
-    const long long col_tiles = ((long long)g.N * P + p.tile_cols - 1) / p.tile_cols;
+    p.div_tiles_per_img = FastDiv((uint32_t)p.tiles_per_img);
     const long long items = col_tiles * p.n_ci_tiles;
     const int n_chunks = (g.C_out + kTcBK - 1) / kTcBK;
     if (items * n_chunks > 0x7fffffffLL) return GF_ERR_UNSUPPORTED;
@@ -866,7 +954,7 @@ gf_status launch_gw_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const _
     ProfScope prof(K_GW_TC, s);
     constexpr int NT = 128;
     GwTcParams p;
-    const int P = g.Hp * g.Wp;
+    const int P = tc_pitch(g);                      // plane pitch of both operands; gaps hold zeros
     const long long K = (long long)g.N * P;
     p.gbar = make_flat(gbar, g.C_out, P, K, gbar_lo_off);
     p.stash = make_flat(stash, g.C_in, P, K, stash_lo_off);

@@ -45,6 +45,12 @@ SMALL = [
     L("many_small_planes", 5, 33, 47, 6, 6, 3, 1, 2),
     L("r8_16x16", 3, 20, 36, 16, 16, 3, 1, 8),
     L("r4_32x32", 2, 20, 12, 32, 32, 1, 1, 4),
+    # patch planes whose size is not a multiple of 4: the tensor-core operands get a padded pitch
+    L("pitch_rows_multi", 3, 24, 40, 30, 30, 3, 1, 2),      # 15x15 patches, several row tiles per image
+    L("pitch_generic", 2, 16, 16, 9, 11, 3, 1, 2),          # 5x6 patches, partial patches
+    L("pitch_r4_28x28", 2, 24, 16, 28, 28, 1, 1, 4),        # 7x7 patches
+    L("pitch_wide_rows", 1, 8, 8, 6, 118, 3, 1, 2),         # 3x59 patches: rows too wide for a row tile
+    L("pitch_many_images", 37, 136, 72, 14, 14, 1, 1, 2),   # 7x7 patches, two c_i tiles, many items per CTA
 ]
 
 
