@@ -62,6 +62,17 @@ static uint32_t* global_err_word() {
 
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = 148;
+    }
+    return n;
+}
+
 Geo make_geo(const gf_conv_desc& d) {
     Geo g;
     g.N = d.N; g.C_in = d.C_in; g.C_out = d.C_out; g.H = d.H; g.W = d.W;

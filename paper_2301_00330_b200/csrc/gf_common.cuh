@@ -63,6 +63,9 @@ static inline gf_status launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 blo
 
 static inline int64_t cdiv64(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
+// SMs of the current device (148 when the query fails)
+int sm_count();
+
 // ---- division by a runtime constant ---------------------------------------
 // q = n / d for any 32-bit n via one multiply-high, an add and two shifts.
 struct FastDiv {

@@ -63,6 +63,22 @@ __device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, u
                  : "memory");
 }
 
+// One contiguous shared -> global copy by the copy engine (same alignment rules), as part
+// of the issuing thread's current bulk group.  bulk_commit() closes the group;
+// bulk_wait_read<N>() returns once all but the N most recent groups of this thread have
+// finished READING shared memory (the source may be reused); bulk_wait_all() once every
+// group has completed.
+__device__ __forceinline__ void bulk_s2g(void* dst_gmem, const void* src_smem, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst_gmem), "r"(smem_u32(src_smem)),
+                 "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 // Orders generic-proxy writes to shared memory before later asynchronous-proxy
 // accesses (copy engine, tensor core) to the same locations.
 __device__ __forceinline__ void fence_proxy_async_smem() {

@@ -14,6 +14,7 @@
 //  pool_bigpatch_kernel patches too large for a tile: one CTA per output value.
 #include "gf_common.cuh"
 #include "gf_pipe.cuh"
+#include "gf_span.cuh"
 
 namespace gf {
 
@@ -42,39 +43,6 @@ struct PoolParams {
     FastDiv div_bands, div_plane_out /* Hp*Wp */, div_Wp;
     float inv_full;  // 1 / r^2
 };
-
-// ---- NE consecutive shared-memory elements as floats -----------------------------
-template <int NE> __device__ __forceinline__ void load_span(const float* p, float (&v)[NE]) {
-    if constexpr (NE >= 4) {
-#pragma unroll
-        for (int i = 0; i < NE / 4; ++i) {
-            const float4 t = reinterpret_cast<const float4*>(p)[i];
-            v[4 * i] = t.x; v[4 * i + 1] = t.y; v[4 * i + 2] = t.z; v[4 * i + 3] = t.w;
-        }
-    } else {
-        const float2 t = *reinterpret_cast<const float2*>(p);
-        v[0] = t.x; v[1] = t.y;
-    }
-}
-__device__ __forceinline__ void unpack_bf16x2(uint32_t u, float& lo, float& hi) {
-    lo = __uint_as_float(u << 16);
-    hi = __uint_as_float(u & 0xffff0000u);
-}
-template <int NE> __device__ __forceinline__ void load_span(const __nv_bfloat16* p, float (&v)[NE]) {
-    if constexpr (NE >= 8) {
-#pragma unroll
-        for (int i = 0; i < NE / 8; ++i) {
-            const uint4 t = reinterpret_cast<const uint4*>(p)[i];
-            unpack_bf16x2(t.x, v[8 * i], v[8 * i + 1]); unpack_bf16x2(t.y, v[8 * i + 2], v[8 * i + 3]);
-            unpack_bf16x2(t.z, v[8 * i + 4], v[8 * i + 5]); unpack_bf16x2(t.w, v[8 * i + 6], v[8 * i + 7]);
-        }
-    } else if constexpr (NE == 4) {
-        const uint2 t = *reinterpret_cast<const uint2*>(p);
-        unpack_bf16x2(t.x, v[0], v[1]); unpack_bf16x2(t.y, v[2], v[3]);
-    } else {
-        unpack_bf16x2(*reinterpret_cast<const uint32_t*>(p), v[0], v[1]);
-    }
-}
 
 // ---- G consecutive outputs ---------------------------------------------------------
 template <int G> __device__ __forceinline__ void store_vec(float* dst, const float (&a)[G]) {
@@ -371,7 +339,6 @@ static int gcd_int(int a, int b) { while (b) { int t = a % b; a = b; b = t; } re
 // Tiling for the streamed kernel: S strips per tile, a multiple of the count that
 // makes a tile a multiple of 16 bytes (so that every tile starts 16-byte aligned),
 // sized so that every CTA of the persistent grid gets the same number of tiles.
-static int sm_count();
 static bool plan_stream(PoolParams& p, size_t e) {
     if (!(p.r == 2 || p.r == 4 || p.r == 8) || p.W % p.r != 0 || p.H % p.r != 0) return false;
     const long long strip_bytes = (long long)p.r * p.W * (long long)e;
@@ -388,16 +355,6 @@ static bool plan_stream(PoolParams& p, size_t e) {
     p.S = (int)S;
     p.tiles = cdiv64(p.strips, p.S);
     return p.tiles <= 0x7fffffffLL;
-}
-
-static int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-            n = 148;
-    }
-    return n;
 }
 
 template <typename TIn, typename TOut, int R, int G>

@@ -822,16 +822,6 @@ gf_status launch_split_f32(const float* in, __nv_bfloat16* hi, __nv_bfloat16* lo
     return launch_pdl(split_f32_kernel, dim3((unsigned)((n4 + 255) / 256)), dim3(256), 0, s, in, hi, lo, n4);
 }
 
-static int sm_count_tc() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-            n = 148;
-    }
-    return n;
-}
-
 constexpr size_t kSmemLimit = 227 * 1024;
 
 template <typename TOut, int NT, int R, int LOGV, bool ARES, int SPLIT>
@@ -850,7 +840,7 @@ static gf_status launch_gx_tc_ares(const GxTcParams& p, int grid, size_t a_res_b
 
 template <typename TOut, int NT, int R, int LOGV, int SPLIT>
 static gf_status launch_gx_tc_inst(const GxTcParams& p, cudaStream_t s) {
-    const int grid = p.items < sm_count_tc() ? p.items : sm_count_tc();
+    const int grid = p.items < sm_count() ? p.items : sm_count();
     if constexpr (LOGV > 0) {
         constexpr size_t d_bytes = ((size_t)128 * (NT + 1) * 4 + 1023) / 1024 * 1024;
         constexpr size_t ring = (size_t)gx_stages(SPLIT, true) * SPLIT * (kTcBK * NT * 2);

@@ -45,6 +45,13 @@ SMALL = [
     L("many_small_planes", 5, 33, 47, 6, 6, 3, 1, 2),
     L("r8_16x16", 3, 20, 36, 16, 16, 3, 1, 8),
     L("r4_32x32", 2, 20, 12, 32, 32, 1, 1, 4),
+    # depthwise, streamed kernel: ring wrap-around (more tiles per CTA than ring slots), bands of
+    # large planes, r = 8, 7-wide patch rows
+    L("dw_ring_wrap", 16, 640, 640, 28, 28, 3, 640, 2),
+    L("dw_band_ring", 4, 64, 64, 160, 120, 3, 64, 2),
+    L("dw_r8", 2, 12, 12, 32, 32, 3, 12, 8),
+    L("dw_14x14", 3, 40, 40, 14, 14, 3, 40, 2),
+    L("dw_k5_r4", 2, 24, 24, 16, 48, 5, 24, 4),
     # patch planes whose size is not a multiple of 4: the tensor-core operands get a padded pitch
     L("pitch_rows_multi", 3, 24, 40, 30, 30, 3, 1, 2),      # 15x15 patches, several row tiles per image
     L("pitch_generic", 2, 16, 16, 9, 11, 3, 1, 2),          # 5x6 patches, partial patches
