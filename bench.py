@@ -232,6 +232,22 @@ def run_reference(args) -> None:
 
 
 # --------------------------------------------------------------------------- GPU arm
+def max_over_ranks(ms: float, dist, device) -> float:
+    """The slowest rank's time: the job is done when the last replica is."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value_us(ms_total: float, steps: int, world: int) -> float:
+    """us per layer step of the whole job: every rank ran `steps` layer steps of its own
+    replica in ms_total (max over ranks), so the job did steps * world of them."""
+    return ms_total * 1e3 / (steps * world)
+
+
 def run_ours(args) -> None:
     import torch
     import paper_2301_00330_b200 as gf
@@ -350,12 +366,9 @@ def run_ours(args) -> None:
         launches += replays * n_sets * launches_per_step     # kernels the replays ran
     ms_total = ev0.elapsed_time(ev1)
     assert gf.gf_last_async_status(sets[0][2].workspace) == gf.GF_OK
-    if dist is not None:
-        t = torch.tensor([ms_total], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, dist, "cuda")
     ms_per_step = ms_total / args.steps
-    value = ms_total * 1e3 / (args.steps * world)      # us per layer over all ranks' layers
+    value = job_value_us(ms_total, args.steps, world)
 
     # ---- end to end: host buffers in, host buffers out, through the C ABI ----
     hx, hgy, hw = x0.pin_memory(), gy0.pin_memory(), w0.pin_memory()
@@ -372,13 +385,10 @@ def run_ours(args) -> None:
     ev1.record(stream)
     torch.cuda.synchronize()
     e2e_ms = ev0.elapsed_time(ev1)
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, dist, "cuda")
     h2d = sum(t.numel() * t.element_size() for t in (hx, hgy, hw))
     d2h = sum(t.numel() * t.element_size() for t in (h_gW, h_gX))
-    e2e = {"value": e2e_ms * 1e3 / (e2e_steps * world), "unit": UNIT, "h2d_bytes_per_step": h2d,
+    e2e = {"value": job_value_us(e2e_ms, e2e_steps, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
            "d2h_bytes_per_step": d2h, "steps": e2e_steps, "api": "gf_layer_step_host (pinned host buffers)"}
 
     if rank != 0:

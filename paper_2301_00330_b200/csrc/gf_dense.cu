@@ -215,12 +215,45 @@ __global__ void gw_finish_kernel(const float* __restrict__ part, int S, size_t n
     gW[i] = ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
 }
 
+// Many partial matrices (S >= 16): 32 pairs per block, the partials dealt to the block's 8
+// warps, every load of a warp independent; the sum order is fixed.
+__global__ void __launch_bounds__(256) gw_finish_wide_kernel(const float* __restrict__ part, int S, size_t n_pairs,
+                                                             int taps, FastDiv div_taps, float* __restrict__ gW) {
+    __shared__ float red[8][33];
+    pdl_launch_dependents();
+    pdl_wait();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const size_t pair0 = (size_t)blockIdx.x * 32, pair = pair0 + lane;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    if (pair < n_pairs) {
+        int k = warp;
+        for (; k + 24 < S; k += 32) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) acc[u] += part[(size_t)(k + 8 * u) * n_pairs + pair];
+        }
+        for (; k < S; k += 8) acc[0] += part[(size_t)k * n_pairs + pair];
+    }
+    red[warp][lane] = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+    __syncthreads();
+    const int n_here = (int)min((size_t)32, n_pairs - pair0);
+    for (int o = threadIdx.x; o < n_here * taps; o += 256) {
+        const uint32_t pl = div_taps.div((uint32_t)o);
+        float v = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) v += red[w][pl];
+        gW[pair0 * taps + o] = v;
+    }
+}
+
 gf_status launch_gw_finish(const float* part, int splits, float* gW, const Geo& g, cudaStream_t s) {
     ProfScope prof(K_GW_FINISH, s);
     const size_t n_pairs = (size_t)g.C_out * g.C_ig;
     const int taps = g.KH * g.KW;
     const size_t total = n_pairs * taps;
     if (total > 0x7fffffffULL) return GF_ERR_UNSUPPORTED;
+    if (splits >= 16)
+        return launch_pdl(gw_finish_wide_kernel, dim3((unsigned)((n_pairs + 31) / 32)), dim3(256), 0, s, part, splits,
+                          n_pairs, taps, FastDiv(taps), gW);
     return launch_pdl(gw_finish_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, s, part, splits, n_pairs,
                       taps, FastDiv(taps), gW);
 }
