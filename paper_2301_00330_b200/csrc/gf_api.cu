@@ -139,6 +139,36 @@ Workspace plan_workspace(const Geo& g) {
 
 static bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
+// ---- side stream ----------------------------------------------------------------------------
+// The two contractions of the tensor-core path are independent of each other.  The g_W
+// chain (stash repack, contraction, broadcast to the taps) is put on a library-owned
+// second stream between a fork event and a join event, so that it shares the SMs with
+// the g_X contraction instead of queueing behind it.  One stream and event pair per
+// device, created on first use; the host-side sequence is serialised by a mutex.
+struct SideStream {
+    cudaStream_t stream = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr;
+    bool ok = false;
+};
+std::mutex g_side_mu;
+
+static SideStream* side_stream() {
+    static SideStream side[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    SideStream& sd = side[dev];
+    if (!sd.ok) {
+        if (cudaStreamCreateWithFlags(&sd.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&sd.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&sd.join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        sd.ok = true;
+    }
+    return &sd;
+}
+
+gf_status backward_impl(const gf_conv_desc* desc, const void* g_y, const void* stash, const void* W, float* g_W,
+                        void* g_X, void* workspace, size_t workspace_bytes, void* stream, bool may_fork);
+
 }  // namespace gf
 
 using namespace gf;
@@ -188,6 +218,14 @@ gf_status gf_stash_forward(const gf_conv_desc* desc, const void* x, void* stash,
 
 gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* stash, const void* W,
                       float* g_W, void* g_X, void* workspace, size_t workspace_bytes, void* stream) {
+    return backward_impl(desc, g_y, stash, W, g_W, g_X, workspace, workspace_bytes, stream, /*may_fork=*/true);
+}
+
+}  // extern "C"
+
+namespace gf {
+gf_status backward_impl(const gf_conv_desc* desc, const void* g_y, const void* stash, const void* W, float* g_W,
+                        void* g_X, void* workspace, size_t workspace_bytes, void* stream, bool may_fork) {
     if (!desc || !g_y || !W || !workspace) return GF_ERR_NULL;
     if (g_W && !stash) return GF_ERR_NULL;
     gf_status st = validate(desc);
@@ -238,11 +276,24 @@ gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* sta
         st = launch_pool(K_GY_POOL, g_y, g.dtype, gbar16, split ? gbar16 + gbar_lo : nullptr, GF_BF16, /*mean=*/true,
                          (int64_t)g.N * g.C_out, g.H, g.W, g.r, (int)pitch, err, s);
         if (st != GF_OK) return st;
+        // both outputs wanted: the g_W chain goes to the side stream, forked here
+        SideStream* side = (may_fork && g_X && g_W) ? side_stream() : nullptr;
+        std::unique_lock<std::mutex> side_lock;
+        cudaStream_t sw = s;                          // stream of the g_W chain
+        int gx_ctas = 0, gw_splits = tc_gw_splits(g);
+        if (side) {
+            tc_partition(g, &gx_ctas, &gw_splits);    // side by side: each kernel gets its share of the SMs
+            side_lock = std::unique_lock<std::mutex>(g_side_mu);
+            GF_CUDA_TRY(cudaEventRecord(side->fork, s));
+            GF_CUDA_TRY(cudaStreamWaitEvent(side->stream, side->fork, 0));
+            sw = side->stream;
+        }
         if (g_X) {
-            st = launch_gx_tc(gbar16, gbar_lo, thetaT, theta_lo, g_X, err, g, s);
+            st = launch_gx_tc(gbar16, gbar_lo, thetaT, theta_lo, g_X, gx_ctas, err, g, s);
             if (st != GF_OK) return st;
         }
         if (g_W) {
+            cudaStream_t s = sw;                      // shadows: everything below runs on the g_W chain's stream
             const __nv_bfloat16* stash16 = static_cast<const __nv_bfloat16*>(stash);
             if (split || pitch != P) {
                 __nv_bfloat16* sp = reinterpret_cast<__nv_bfloat16*>(base + ws.off_split);
@@ -254,11 +305,14 @@ gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* sta
                 if (st != GF_OK) return st;
                 stash16 = sp;
             }
-            const int splits = tc_gw_splits(g);
-            st = launch_gw_tc(gbar16, gbar_lo, stash16, stash_lo, part, splits, err, g, s);
+            st = launch_gw_tc(gbar16, gbar_lo, stash16, stash_lo, part, gw_splits, err, g, s);
             if (st != GF_OK) return st;
             st = launch_gw_finish(part, 1, g_W, g, s);
             if (st != GF_OK) return st;
+        }
+        if (side) {                                   // join: the caller's stream waits for the g_W chain
+            GF_CUDA_TRY(cudaEventRecord(side->join, side->stream));
+            GF_CUDA_TRY(cudaStreamWaitEvent(s, side->join, 0));
         }
         return GF_OK;
     }
@@ -281,6 +335,9 @@ gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* sta
     }
     return GF_OK;
 }
+}  // namespace gf
+
+extern "C" {
 
 gf_status gf_last_async_status(const void* workspace, void* stream) {
     if (!workspace) return GF_ERR_NULL;

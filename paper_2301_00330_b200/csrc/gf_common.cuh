@@ -157,6 +157,11 @@ struct Workspace {
 };
 Workspace plan_workspace(const Geo& g);
 
+// gf_backward's body.  may_fork: the tensor-core path may run its g_W chain on the
+// library's side stream (created on first use); false keeps everything on `stream`.
+gf_status backward_impl(const gf_conv_desc* desc, const void* g_y, const void* stash, const void* W, float* g_W,
+                        void* g_X, void* workspace, size_t workspace_bytes, void* stream, bool may_fork);
+
 // ---- kernel entry points (host launchers) ----------------------------------
 // pool: out[plane, a, b] = sum (or mean) of in[plane] over patch (a,b).  out_lo: bf16 low
 // parts (NULL: none).  out_pitch: elements between output planes, 0 = dense; a gap is zeroed.
@@ -184,8 +189,12 @@ gf_status launch_repack(const void* in, int in_dtype, __nv_bfloat16* hi, __nv_bf
 gf_status launch_ksum_t(const void* W, const Geo& g, __nv_bfloat16* thetaT, __nv_bfloat16* thetaT_lo, float* gwu,
                         uint32_t* err_word, cudaStream_t s);
 gf_status launch_split_f32(const float* in, __nv_bfloat16* hi, __nv_bfloat16* lo, size_t n, cudaStream_t s);
+// max_ctas: CTAs the kernel may use (0: one per SM)
 gf_status launch_gx_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const __nv_bfloat16* thetaT,
-                       long long theta_lo_off, void* gX, uint32_t* err_word, const Geo& g, cudaStream_t s);
+                       long long theta_lo_off, void* gX, int max_ctas, uint32_t* err_word, const Geo& g,
+                       cudaStream_t s);
+// shares of the SMs when the two contractions run side by side: CTAs of gx_tc, K-splits of gw_tc
+void tc_partition(const Geo& g, int* gx_ctas, int* gw_splits);
 gf_status launch_gw_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const __nv_bfloat16* stash,
                        long long stash_lo_off, float* gwu, int splits, uint32_t* err_word, const Geo& g,
                        cudaStream_t s);

@@ -39,5 +39,7 @@ extern "C" gf_status gf_backward_static_scratch(const gf_conv_desc* desc, const 
     if (!scratch) return GF_ERR_CUDA;
     // gf_backward itself resets what has to start from zero (the error word, the g_W
     // accumulator); everything else in the scratch is overwritten before it is read.
-    return gf_backward(desc, g_y, stash, W, g_W, g_X, scratch, (size_t)GF_STATIC_SCRATCH_BYTES, stream);
+    // Single stream: the side stream of gf_backward would be a resource created on first use.
+    return gf::backward_impl(desc, g_y, stash, W, g_W, g_X, scratch, (size_t)GF_STATIC_SCRATCH_BYTES, stream,
+                             /*may_fork=*/false);
 }

@@ -221,6 +221,7 @@ struct GxTcParams {
     int P;                              // elements between the planes of gbar (>= Hp*Wp; the gap holds zeros)
     int P_live;                         // Hp*Wp
     int n_ci_tiles, items;
+    int max_ctas;                       // CTAs the kernel may use (all SMs, or its share of them)
     int tile_cols;                      // flattened columns per tile: whole patch rows (R > 0) or NT
     // padded planes with R > 0: a tile is rows_per_tile patch rows of ONE image, loaded from
     // the 8-element boundary below its first column (tiles_per_img tiles per image); 0 otherwise
@@ -791,11 +792,45 @@ gf_status launch_repack(const void* in, int in_dtype, __nv_bfloat16* hi, __nv_bf
                       pitch, FastDiv((uint32_t)pitch));
 }
 
+// When the two contractions run side by side (g_W chain on the side stream), each gets a
+// share of the SMs: both kernels hold one CTA per SM, so their grids must add up to the
+// SM count to be resident together.  The g_X kernel is bound by the HBM write rate, which
+// it reaches with a fraction of the SMs; the g_W kernel by the rate at which its CTAs fill
+// shared memory.  The g_W share balances the two: measured on the 256 -> 256, 28 x 28,
+// r = 2 layer the step was shortest at about 50 of 148 SMs, where the bytes the g_W kernel
+// stages equal the bytes of g_X; the share scales with that ratio.
+void tc_partition(const Geo& g, int* gx_ctas, int* gw_splits) {
+    const int sms = sm_count();
+    const long long K = (long long)g.N * tc_pitch(g);
+    const long long chunks = (K + kTcBK - 1) / kTcBK;
+    const int tiles = ((g.C_in + 127) / 128) * ((g.C_out + 127) / 128);
+    const int split_ops = g.dtype == GF_F32 ? 2 : 1;
+    const double staged = (double)tiles * (double)chunks * (128 + 128) * kTcBK * 2.0 * split_ops;
+    const double gx_bytes = (double)g.N * g.C_in * g.H * g.W * (double)g.esize;
+    int n_gw = (int)(staged / gx_bytes * 0.35 * sms + 0.5);
+    if (n_gw < sms / 6) n_gw = sms / 6;
+    if (n_gw > sms / 2) n_gw = sms / 2;
+    int s = n_gw / tiles;
+    if (s < 1) s = 1;
+    if (s > chunks) s = (int)chunks;
+    if (s > 65535) s = 65535;
+    const int n_ci_tiles = (g.C_in + 127) / 128;
+    int gx = sms - s * tiles;
+    gx = gx / n_ci_tiles * n_ci_tiles;
+    if (gx < n_ci_tiles || gx < sms / 3) {          // no sensible split: both kernels take the whole GPU in turn
+        *gx_ctas = sms;
+        *gw_splits = tc_gw_splits(g);
+        return;
+    }
+    *gx_ctas = gx;
+    *gw_splits = s;
+}
+
 int tc_gw_splits(const Geo& g) {
     const long long K = (long long)g.N * tc_pitch(g);
     const int chunks = (int)((K + kTcBK - 1) / kTcBK);
     const int tiles = ((g.C_in + 127) / 128) * ((g.C_out + 127) / 128);
-    int s = (148 + tiles - 1) / tiles;
+    int s = (sm_count() + tiles - 1) / tiles;
     if (s > chunks) s = chunks;
     if (s < 1) s = 1;
     if (s > 65535) s = 65535;
@@ -840,7 +875,8 @@ static gf_status launch_gx_tc_ares(const GxTcParams& p, int grid, size_t a_res_b
 
 template <typename TOut, int NT, int R, int LOGV, int SPLIT>
 static gf_status launch_gx_tc_inst(const GxTcParams& p, cudaStream_t s) {
-    const int grid = p.items < sm_count() ? p.items : sm_count();
+    const int sms = p.max_ctas;
+    const int grid = p.items < sms ? p.items : sms;
     if constexpr (LOGV > 0) {
         constexpr size_t d_bytes = ((size_t)128 * (NT + 1) * 4 + 1023) / 1024 * 1024;
         constexpr size_t ring = (size_t)gx_stages(SPLIT, true) * SPLIT * (kTcBK * NT * 2);
@@ -874,7 +910,8 @@ static gf_status launch_gx_tc_r(const GxTcParams& p, int R, cudaStream_t s) {
 // gbar / thetaT: bf16 arrays; *_lo_off: elements from the high-part to the low-part array
 // (fp32 layers: operands carried as bf16 pairs), 0 for plain bf16 layers.
 gf_status launch_gx_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const __nv_bfloat16* thetaT,
-                       long long theta_lo_off, void* gX, uint32_t* err_word, const Geo& g, cudaStream_t s) {
+                       long long theta_lo_off, void* gX, int max_ctas, uint32_t* err_word, const Geo& g,
+                       cudaStream_t s) {
     ProfScope prof(K_GX_TC, s);
     constexpr int NT = 64;
     GxTcParams p;
@@ -884,6 +921,7 @@ gf_status launch_gx_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const _
     p.gbar = make_flat(gbar, g.C_out, P, (long long)g.N * P, gbar_lo_off);
     p.thetaT = make_flat(thetaT, g.C_in, g.C_out, g.C_out, theta_lo_off);
     p.gX = gX; p.err_word = err_word;
+    p.max_ctas = (max_ctas > 0 && max_ctas < sm_count()) ? max_ctas : sm_count();
     p.N = g.N; p.C_in = g.C_in; p.C_out = g.C_out; p.H = g.H; p.W = g.W; p.r = g.r; p.Hp = g.Hp; p.Wp = g.Wp; p.P = P;
     p.div_Wp = FastDiv((uint32_t)g.Wp);
     p.div_Hp = FastDiv((uint32_t)g.Hp);
