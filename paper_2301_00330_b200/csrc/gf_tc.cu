@@ -792,38 +792,97 @@ gf_status launch_repack(const void* in, int in_dtype, __nv_bfloat16* hi, __nv_bf
                       pitch, FastDiv((uint32_t)pitch));
 }
 
+// How gx_tc cuts a layer into column tiles (shared by its launcher and by the SM-share model).
+struct GxPlan {
+    int R;                 // expansion factor handled by the row-aligned path, 0: generic path
+    int tile_cols, rows_per_tile, tiles_per_img, logV;
+    long long col_tiles;
+    bool padded, ares;     // padded plane pitch; resident thetaT tile possible
+};
+constexpr int kGxNT = 64;
+constexpr size_t kSmemLimit = 227 * 1024;
+
+static GxPlan gx_plan(const Geo& g) {
+    constexpr int NT = kGxNT;
+    GxPlan d;
+    const int P = tc_pitch(g);
+    d.padded = P != g.Hp * g.Wp;
+    d.R = (g.W % g.r == 0 && g.Wp <= NT && (g.r == 2 || g.r == 4 || g.r == 8)) ? g.r : 0;
+    if (d.padded && g.Wp > NT - 7) d.R = 0;         // no room for the alignment slack of a row-aligned tile
+    d.tile_cols = d.R > 0 ? (NT / g.Wp) * g.Wp : NT;
+    d.rows_per_tile = 0;
+    d.tiles_per_img = 1;
+    d.logV = (P % 8 == 0) ? 3 : (P % 4 == 0) ? 2 : 0;
+    if (d.padded && d.R > 0) {
+        // tiles of whole patch rows of one image, loaded from an 8-element boundary
+        d.rows_per_tile = (NT - 7) / g.Wp;
+        if (d.rows_per_tile > g.Hp) d.rows_per_tile = g.Hp;
+        d.tiles_per_img = (g.Hp + d.rows_per_tile - 1) / d.rows_per_tile;
+        d.col_tiles = (long long)g.N * d.tiles_per_img;
+    } else {
+        // pieces must not straddle a tile start: the piece width divides tile_cols as well as P
+        int lv = d.logV;
+        while (lv > 0 && (d.tile_cols % (1 << lv)) != 0) --lv;
+        d.logV = lv == 1 ? 0 : lv;
+        d.col_tiles = ((long long)g.N * P + d.tile_cols - 1) / d.tile_cols;
+    }
+    // shared memory of the variant that keeps its thetaT tile resident
+    const int split = g.dtype == GF_F32 ? 2 : 1;
+    const size_t d_bytes = ((size_t)128 * (NT + 1) * 4 + 1023) / 1024 * 1024;
+    const size_t ring = (size_t)gx_stages(split, true) * split * (kTcBK * NT * 2);
+    const size_t fixed = 512 + (d.R > 0 ? (size_t)NT * d.R * 10 : (size_t)NT * 12);
+    const size_t a_bytes = (size_t)split * ((g.C_out + kTcBK - 1) / kTcBK) * 128 * kTcBK * 2;
+    d.ares = d.logV > 0 && ring + d_bytes + a_bytes + 1024 + fixed <= kSmemLimit;
+    return d;
+}
+
 // When the two contractions run side by side (g_W chain on the side stream), each gets a
 // share of the SMs: both kernels hold one CTA per SM, so their grids must add up to the
-// SM count to be resident together.  The g_X kernel is bound by the HBM write rate, which
-// it reaches with a fraction of the SMs; the g_W kernel by the rate at which its CTAs fill
-// shared memory.  The g_W share balances the two: measured on the 256 -> 256, 28 x 28,
-// r = 2 layer the step was shortest at about 50 of 148 SMs, where the bytes the g_W kernel
-// stages equal the bytes of g_X; the share scales with that ratio.
+// SM count to be resident together.  The shares follow a cost model in SM-microseconds,
+// its constants fitted to per-kernel timings over the layer table: the g_X kernel costs
+// 0.25 us per MB it writes or 0.15 us per MB it stages in shared memory, whichever is
+// larger; the g_W kernel 0.14 us per MB it stages (0.22 with fp32 operand pairs, three MMAs per step).  The g_X grid is then trimmed to the
+// smallest one with the same number of rounds of column tiles, which costs it nothing and
+// leaves more SMs to the other kernel.
 void tc_partition(const Geo& g, int* gx_ctas, int* gw_splits) {
     const int sms = sm_count();
-    const long long K = (long long)g.N * tc_pitch(g);
-    const long long chunks = (K + kTcBK - 1) / kTcBK;
-    const int tiles = ((g.C_in + 127) / 128) * ((g.C_out + 127) / 128);
-    const int split_ops = g.dtype == GF_F32 ? 2 : 1;
-    const double staged = (double)tiles * (double)chunks * (128 + 128) * kTcBK * 2.0 * split_ops;
-    const double gx_bytes = (double)g.N * g.C_in * g.H * g.W * (double)g.esize;
-    int n_gw = (int)(staged / gx_bytes * 0.35 * sms + 0.5);
-    if (n_gw < sms / 6) n_gw = sms / 6;
-    if (n_gw > sms / 2) n_gw = sms / 2;
-    int s = n_gw / tiles;
-    if (s < 1) s = 1;
-    if (s > chunks) s = (int)chunks;
-    if (s > 65535) s = 65535;
+    const GxPlan d = gx_plan(g);
+    const double split = g.dtype == GF_F32 ? 2.0 : 1.0;
     const int n_ci_tiles = (g.C_in + 127) / 128;
-    int gx = sms - s * tiles;
-    gx = gx / n_ci_tiles * n_ci_tiles;
-    if (gx < n_ci_tiles || gx < sms / 3) {          // no sensible split: both kernels take the whole GPU in turn
+    const long long chunks_x = (g.C_out + kTcBK - 1) / kTcBK;
+    const double staged_x = (double)d.col_tiles * n_ci_tiles * chunks_x * split * (kTcBK * kGxNT * 2 + (d.ares ? 0 : 128 * kTcBK * 2));
+    const double out_x = (double)g.N * g.C_in * g.H * g.W * (double)g.esize;
+    const double w_x = fmax(0.25e-6 * out_x, 0.15e-6 * staged_x);
+    const long long chunks_w = ((long long)g.N * tc_pitch(g) + kTcBK - 1) / kTcBK;
+    const int tiles_w = n_ci_tiles * ((g.C_out + 127) / 128);
+    const double staged_w = (double)tiles_w * chunks_w * split * (128 + 128) * kTcBK * 2;
+    const double w_w = (g.dtype == GF_F32 ? 0.22e-6 : 0.14e-6) * staged_w;
+    int n_gw = (int)(sms * w_w / (w_w + w_x) + 0.5);
+    if (n_gw < sms / 5) n_gw = sms / 5;
+    if (n_gw > sms * 3 / 5) n_gw = sms * 3 / 5;
+    // the g_X grid: smallest with as many rounds as the budget allows
+    int gx;
+    if (d.ares) {
+        int per_ci = (sms - n_gw) / n_ci_tiles;
+        if (per_ci < 1) per_ci = 1;
+        const long long rounds = (d.col_tiles + per_ci - 1) / per_ci;
+        gx = (int)((d.col_tiles + rounds - 1) / rounds) * n_ci_tiles;
+    } else {
+        const long long items = d.col_tiles * n_ci_tiles;
+        const int budget = sms - n_gw;
+        const long long rounds = (items + budget - 1) / budget;
+        gx = (int)((items + rounds - 1) / rounds);
+    }
+    long long s = (sms - gx) / tiles_w;
+    if (s > chunks_w) s = chunks_w;
+    if (s > 65535) s = 65535;
+    if (s < 1 || gx < 1 || gx > sms) {              // no sensible split: both kernels take the whole GPU in turn
         *gx_ctas = sms;
         *gw_splits = tc_gw_splits(g);
         return;
     }
     *gx_ctas = gx;
-    *gw_splits = s;
+    *gw_splits = (int)s;
 }
 
 int tc_gw_splits(const Geo& g) {
@@ -856,8 +915,6 @@ gf_status launch_split_f32(const float* in, __nv_bfloat16* hi, __nv_bfloat16* lo
     const size_t n4 = n / 4;
     return launch_pdl(split_f32_kernel, dim3((unsigned)((n4 + 255) / 256)), dim3(256), 0, s, in, hi, lo, n4);
 }
-
-constexpr size_t kSmemLimit = 227 * 1024;
 
 template <typename TOut, int NT, int R, int LOGV, bool ARES, int SPLIT>
 static gf_status launch_gx_tc_ares(const GxTcParams& p, int grid, size_t a_res_bytes, cudaStream_t s) {
@@ -913,10 +970,9 @@ gf_status launch_gx_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const _
                        long long theta_lo_off, void* gX, int max_ctas, uint32_t* err_word, const Geo& g,
                        cudaStream_t s) {
     ProfScope prof(K_GX_TC, s);
-    constexpr int NT = 64;
+    constexpr int NT = kGxNT;
     GxTcParams p;
     const int P = tc_pitch(g);                      // gbar's plane pitch
-    const bool padded = P != g.Hp * g.Wp;
     p.P_live = g.Hp * g.Wp;
     p.gbar = make_flat(gbar, g.C_out, P, (long long)g.N * P, gbar_lo_off);
     p.thetaT = make_flat(thetaT, g.C_in, g.C_out, g.C_out, theta_lo_off);
@@ -927,26 +983,14 @@ gf_status launch_gx_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const _
     p.div_Hp = FastDiv((uint32_t)g.Hp);
     p.n_ci_tiles = (g.C_in + 127) / 128;
     p.div_ci_tiles = FastDiv((uint32_t)p.n_ci_tiles);
-    int R = (g.W % g.r == 0 && g.Wp <= NT && (g.r == 2 || g.r == 4 || g.r == 8)) ? g.r : 0;
-    if (padded && g.Wp > NT - 7) R = 0;             // no room for the alignment slack of a row-aligned tile
+    const GxPlan d = gx_plan(g);
+    const int R = d.R;
     p.div_RWp = FastDiv((uint32_t)((R > 0 ? R : 1) * g.Wp));
-    p.tile_cols = R > 0 ? (NT / g.Wp) * g.Wp : NT;
-    p.rows_per_tile = 0;
-    p.tiles_per_img = 1;
-    long long col_tiles;
-    if (padded && R > 0) {
-        // tiles of whole patch rows of one image, loaded from an 8-element boundary
-        p.rows_per_tile = (NT - 7) / g.Wp;
-        if (p.rows_per_tile > g.Hp) p.rows_per_tile = g.Hp;
-        p.tiles_per_img = (g.Hp + p.rows_per_tile - 1) / p.rows_per_tile;
-        col_tiles = (long long)g.N * p.tiles_per_img;
-    } else {
-        // pieces must not straddle a tile start: the piece width divides tile_cols as well as P
-        int lv = p.gbar.logV;
-        while (lv > 0 && (p.tile_cols % (1 << lv)) != 0) --lv;
-        p.gbar.logV = lv == 1 ? 0 : lv;
-        col_tiles = ((long long)g.N * P + p.tile_cols - 1) / p.tile_cols;
-    }
+    p.tile_cols = d.tile_cols;
+    p.rows_per_tile = d.rows_per_tile;
+    p.tiles_per_img = d.tiles_per_img;
+    p.gbar.logV = d.logV;
+    const long long col_tiles = d.col_tiles;
     p.div_tiles_per_img = FastDiv((uint32_t)p.tiles_per_img);
     const long long items = col_tiles * p.n_ci_tiles;
     const int n_chunks = (g.C_out + kTcBK - 1) / kTcBK;
