@@ -160,7 +160,9 @@ __device__ __forceinline__ int stage_plain(const TIn* __restrict__ in, long long
 // "strips": strip s is the R image rows [s*R, s*R+R) of the [planes*H, W] matrix,
 // R*W contiguous elements that produce the Wp contiguous outputs s*Wp .. s*Wp+Wp-1.
 // A tile is S consecutive strips (plane boundaries do not matter).
-template <typename TIn, typename TOut, int R, int G>
+// EXT: the output has a low-part array and/or a padded plane pitch (tensor-core operands);
+// the plain case keeps to one vector store at og0 + o.
+template <typename TIn, typename TOut, int R, int G, bool EXT>
 __device__ __forceinline__ void reduce_item(const PoolParams& p, const TIn* buf, long long og0, uint32_t q) {
     const uint32_t o = q * G;
     uint32_t A, b;
@@ -185,13 +187,17 @@ __device__ __forceinline__ void reduce_item(const PoolParams& p, const TIn* buf,
 #pragma unroll
         for (int k = 0; k < G; ++k) acc[k] *= p.inv_full;
     }
-    const long long idx = out_index<TOut, G>(p, og0 + o);
-    TOut* dst = static_cast<TOut*>(p.out) + idx;
-    if (p.out_lo) store_split<G>(dst, static_cast<TOut*>(p.out_lo) + idx, acc);
-    else store_vec<G>(dst, acc);
+    if constexpr (EXT) {
+        const long long idx = out_index<TOut, G>(p, og0 + o);
+        TOut* dst = static_cast<TOut*>(p.out) + idx;
+        if (p.out_lo) store_split<G>(dst, static_cast<TOut*>(p.out_lo) + idx, acc);
+        else store_vec<G>(dst, acc);
+    } else {
+        store_vec<G>(static_cast<TOut*>(p.out) + og0 + o, acc);
+    }
 }
 
-template <typename TIn, typename TOut, int R, int G>
+template <typename TIn, typename TOut, int R, int G, bool EXT>
 __global__ void __launch_bounds__(kStreamThreads, 1) pool_stream_kernel(const PoolParams p) {
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     __shared__ uint64_t full[kStreamStages];
@@ -244,10 +250,10 @@ __global__ void __launch_bounds__(kStreamThreads, 1) pool_stream_kernel(const Po
             const TIn* b = buf(s);
             uint32_t q = threadIdx.x;
             for (; q + kStreamThreads < nitems; q += 2 * kStreamThreads) {   // two independent items in flight
-                reduce_item<TIn, TOut, R, G>(p, b, dst, q);
-                reduce_item<TIn, TOut, R, G>(p, b, dst, q + kStreamThreads);
+                reduce_item<TIn, TOut, R, G, EXT>(p, b, dst, q);
+                reduce_item<TIn, TOut, R, G, EXT>(p, b, dst, q + kStreamThreads);
             }
-            if (q < nitems) reduce_item<TIn, TOut, R, G>(p, b, dst, q);
+            if (q < nitems) reduce_item<TIn, TOut, R, G, EXT>(p, b, dst, q);
         }
         failed = __syncthreads_or(!ok);     // also: every thread is done reading slot s
         done = it + 1;
@@ -357,17 +363,23 @@ static bool plan_stream(PoolParams& p, size_t e) {
     return p.tiles <= 0x7fffffffLL;
 }
 
-template <typename TIn, typename TOut, int R, int G>
-static gf_status launch_stream_inst(const PoolParams& p, cudaStream_t s) {
+template <typename TIn, typename TOut, int R, int G, bool EXT>
+static gf_status launch_stream_ext(const PoolParams& p, cudaStream_t s) {
     constexpr size_t smem = (size_t)kStreamStages * kStreamTileBytes;
     static bool configured = false;
     if (!configured) {
-        GF_CUDA_TRY(cudaFuncSetAttribute(pool_stream_kernel<TIn, TOut, R, G>,
+        GF_CUDA_TRY(cudaFuncSetAttribute(pool_stream_kernel<TIn, TOut, R, G, EXT>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         configured = true;
     }
     const long long grid = p.tiles < sm_count() ? p.tiles : sm_count();
-    return launch_pdl(pool_stream_kernel<TIn, TOut, R, G>, dim3((unsigned)grid), dim3(kStreamThreads), smem, s, p);
+    return launch_pdl(pool_stream_kernel<TIn, TOut, R, G, EXT>, dim3((unsigned)grid), dim3(kStreamThreads), smem, s, p);
+}
+
+template <typename TIn, typename TOut, int R, int G>
+static gf_status launch_stream_inst(const PoolParams& p, cudaStream_t s) {
+    if (p.out_lo || p.out_pitch != p.plane_out) return launch_stream_ext<TIn, TOut, R, G, true>(p, s);
+    return launch_stream_ext<TIn, TOut, R, G, false>(p, s);
 }
 
 template <typename TIn, typename TOut>

@@ -841,7 +841,8 @@ static GxPlan gx_plan(const Geo& g) {
 // SM count to be resident together.  The shares follow a cost model in SM-microseconds,
 // its constants fitted to per-kernel timings over the layer table: the g_X kernel costs
 // 0.25 us per MB it writes or 0.15 us per MB it stages in shared memory, whichever is
-// larger; the g_W kernel 0.14 us per MB it stages (0.22 with fp32 operand pairs, three MMAs per step).  The g_X grid is then trimmed to the
+// larger; the g_W kernel 0.14 us per MB it stages (0.22 with fp32 operand pairs, three
+// MMAs per step).  The g_X grid is then trimmed to the
 // smallest one with the same number of rounds of column tiles, which costs it nothing and
 // leaves more SMs to the other kernel.
 void tc_partition(const Geo& g, int* gx_ctas, int* gw_splits) {
