@@ -35,10 +35,18 @@ FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # SMs x FMA lanes x 2 flop x 
 # DRAM bytes per launch of a kernel from one ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by kernel name, with the sha1 of the source file
 # at capture time; a changed source makes the entry stale (reported as null).
-NCU_TRAFFIC: dict[str, dict] = {}
+# Captured on the bench layer (profiles/step_resnet3x3_256_N64_28x28_r2_bf16.md).  Writes of a
+# single launch stay in the 126 MB L2 past the end of the kernel, so dram__bytes_write is 0
+# there and the figure is the read side.
+NCU_TRAFFIC: dict[str, dict] = {
+    "gx_tc": {"bytes": 6584832, "sha1": "0f52a7deddf63f0abcf2fbec0951bddaaef366b3"},
+    "gw_tc": {"bytes": 13128448, "sha1": "0f52a7deddf63f0abcf2fbec0951bddaaef366b3"},
+    "stash_pool": {"bytes": 25704192, "sha1": "af0ecc32d79557b642afe63bede04d88db66f208"},
+    "gy_pool": {"bytes": 25703936, "sha1": "af0ecc32d79557b642afe63bede04d88db66f208"},
+}
 
 KERNEL_SOURCE = {
-    "stash_pool": "gf_pool.cu", "gy_pool": "gf_pool.cu", "ksum": "gf_dense.cu", "gx_mix": "gf_dense.cu",
+    "stash_pool": "gf_pool.cu", "gy_pool": "gf_pool.cu", "ksum": "gf_tc.cu", "gx_mix": "gf_dense.cu",
     "gw_partial": "gf_dense.cu", "gw_finish": "gf_dense.cu", "dw_fused": "gf_depthwise.cu",
     "gx_tc": "gf_tc.cu", "gw_tc": "gf_tc.cu",
 }
