@@ -36,6 +36,7 @@ struct PoolParams {
     int BR;      // patch rows per tile (== Hp when P > 1)
     int bands;   // tiles along the patch rows of one plane (1 when P > 1)
     int mean;    // 1: patch mean, 0: patch sum
+    int lin_log_lpr; // linear mode of the streamed kernel: log2(16-byte vectors per image row)
     int plane_out;   // Hp * Wp
     int out_pitch;   // elements between output planes (>= plane_out; the gap is written as zeros)
     long long strips;   // streamed kernel: planes * H / r strips of r rows
@@ -197,6 +198,77 @@ __device__ __forceinline__ void reduce_item(const PoolParams& p, const TIn* buf,
     }
 }
 
+// Linear mode (narrow maps whose row is a power-of-two number of 16-byte vectors, a strip
+// no more than a warp wide): thread t takes vectors t, t + 512, ... of the tile, so a warp
+// reads 512 contiguous bytes without bank conflicts; the vector's share of its patches is
+// summed in registers, the R rows of a strip (and, for R wider than a vector, the vectors
+// of a patch row) are combined with shuffles, and the lanes of a strip's first row write.
+// A strip's vectors divide the block size, so a thread keeps its place inside the strip
+// from vector to vector: what it needs for that is worked out once per kernel.
+template <typename TIn, int R>
+struct LinearLane {
+    static constexpr int VE = 16 / (int)sizeof(TIn);
+    static constexpr int NP = VE >= R ? VE / R : 1;          // patch values a vector contributes to
+    static constexpr int VPP = R > VE ? R / VE : 1;          // vectors per patch row
+    static constexpr int LOG_R = R == 2 ? 1 : R == 4 ? 2 : 3;
+    int lpr;              // vectors per image row
+    bool writer;          // this lane writes its strip's outputs
+    uint32_t o0;          // output index (within the tile) of its first vector's first patch
+    uint32_t o_step;      // advance per round of 512 vectors
+    __device__ __forceinline__ void init(const PoolParams& p) {
+        lpr = 1 << p.lin_log_lpr;
+        const uint32_t lanes = (uint32_t)lpr << LOG_R;                 // vectors per strip
+        const uint32_t ls = threadIdx.x & (lanes - 1);
+        writer = ls < (uint32_t)lpr && (ls & (VPP - 1)) == 0;
+        o0 = (threadIdx.x >> (p.lin_log_lpr + LOG_R)) * (uint32_t)p.Wp + (VPP > 1 ? ls / VPP : ls * NP);
+        o_step = (uint32_t)(kStreamThreads >> (p.lin_log_lpr + LOG_R)) * (uint32_t)p.Wp;
+    }
+};
+
+// One vector per lane; every lane of a warp takes part (inactive ones add zeros).
+template <typename TIn, typename TOut, int R, bool EXT>
+__device__ __forceinline__ void reduce_linear(const PoolParams& p, const LinearLane<TIn, R>& ln, const TIn* buf,
+                                              long long og0, uint32_t v, uint32_t o, bool active) {
+    using LL = LinearLane<TIn, R>;
+    float val[LL::VE];
+    if (active) load_span<LL::VE>(buf + (size_t)v * LL::VE, val);
+    else {
+#pragma unroll
+        for (int k = 0; k < LL::VE; ++k) val[k] = 0.f;
+    }
+    float sum[LL::NP];
+#pragma unroll
+    for (int j = 0; j < LL::NP; ++j) {
+        constexpr int W_ = LL::VE >= R ? R : LL::VE;
+        float t = val[j * W_];
+#pragma unroll
+        for (int k = 1; k < W_; ++k) t += val[j * W_ + k];
+        sum[j] = t;
+    }
+#pragma unroll
+    for (int i = 0; i < LL::LOG_R; ++i) {
+#pragma unroll
+        for (int j = 0; j < LL::NP; ++j) sum[j] += __shfl_xor_sync(0xffffffffu, sum[j], ln.lpr << i);
+    }
+#pragma unroll
+    for (int d = 1; d < LL::VPP; d <<= 1) sum[0] += __shfl_xor_sync(0xffffffffu, sum[0], d);
+    if (active && ln.writer) {
+        if (p.mean) {
+#pragma unroll
+            for (int j = 0; j < LL::NP; ++j) sum[j] *= p.inv_full;
+        }
+        if constexpr (EXT) {
+            const long long idx = out_index<TOut, LL::NP>(p, og0 + o);
+            TOut* dst = static_cast<TOut*>(p.out) + idx;
+            if (p.out_lo) store_split<LL::NP>(dst, static_cast<TOut*>(p.out_lo) + idx, sum);
+            else store_vec<LL::NP>(dst, sum);
+        } else {
+            store_vec<LL::NP>(static_cast<TOut*>(p.out) + og0 + o, sum);
+        }
+    }
+}
+
+// G == 0 selects the linear mode.
 template <typename TIn, typename TOut, int R, int G, bool EXT>
 __global__ void __launch_bounds__(kStreamThreads, 1) pool_stream_kernel(const PoolParams p) {
     extern __shared__ __align__(128) unsigned char dyn_smem[];
@@ -219,6 +291,8 @@ __global__ void __launch_bounds__(kStreamThreads, 1) pool_stream_kernel(const Po
             bulk_g2s(buf(s), in + tile * p.S * strip_elems, bytes, &full[s]);
         }
     };
+    LinearLane<TIn, R> lane_ctx;
+    if constexpr (G == 0) lane_ctx.init(p);
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStreamStages; ++s) mbar_init(&full[s], 1);
@@ -245,15 +319,23 @@ __global__ void __launch_bounds__(kStreamThreads, 1) pool_stream_kernel(const Po
             __syncthreads();
         }
         if (ok) {
-            const uint32_t nitems = (uint32_t)(ns * p.Wp) / G;
             const long long dst = tile * p.S * p.Wp;      // first output of the tile, flattened over planes
             const TIn* b = buf(s);
-            uint32_t q = threadIdx.x;
-            for (; q + kStreamThreads < nitems; q += 2 * kStreamThreads) {   // two independent items in flight
-                reduce_item<TIn, TOut, R, G, EXT>(p, b, dst, q);
-                reduce_item<TIn, TOut, R, G, EXT>(p, b, dst, q + kStreamThreads);
+            if constexpr (G == 0) {
+                const uint32_t nvec = bytes >> 4, nvec_up = (nvec + 31u) & ~31u;   // whole warps take part
+                uint32_t o = lane_ctx.o0;
+#pragma unroll 2
+                for (uint32_t v = threadIdx.x; v < nvec_up; v += kStreamThreads, o += lane_ctx.o_step)
+                    reduce_linear<TIn, TOut, R, EXT>(p, lane_ctx, b, dst, v, o, v < nvec);
+            } else {
+                const uint32_t nitems = (uint32_t)(ns * p.Wp) / (G > 0 ? G : 1);
+                uint32_t q = threadIdx.x;
+                for (; q + kStreamThreads < nitems; q += 2 * kStreamThreads) {   // two independent items in flight
+                    reduce_item<TIn, TOut, R, (G > 0 ? G : 1), EXT>(p, b, dst, q);
+                    reduce_item<TIn, TOut, R, (G > 0 ? G : 1), EXT>(p, b, dst, q + kStreamThreads);
+                }
+                if (q < nitems) reduce_item<TIn, TOut, R, (G > 0 ? G : 1), EXT>(p, b, dst, q);
             }
-            if (q < nitems) reduce_item<TIn, TOut, R, G, EXT>(p, b, dst, q);
         }
         failed = __syncthreads_or(!ok);     // also: every thread is done reading slot s
         done = it + 1;
@@ -353,6 +435,19 @@ static bool plan_stream(PoolParams& p, size_t e) {
     const int s_max = (int)(kStreamTileBytes / strip_bytes) / q * q;
     if (s_max < 1) return false;
     p.strips = p.planes * (p.H / p.r);
+    {   // linear mode: a row is a power-of-two number of 16-byte vectors and a strip fits a warp
+        const long long row_bytes = (long long)p.W * (long long)e;
+        p.lin_log_lpr = -1;
+        if (row_bytes % 16 == 0) {
+            const long long lpr = row_bytes / 16;
+            // (r = 2 stays with the item mode: measured faster there, four outputs per index computation)
+            if ((lpr & (lpr - 1)) == 0 && lpr * p.r <= 32 && p.r >= 4) {
+                int l = 0;
+                while ((1LL << l) < lpr) ++l;
+                p.lin_log_lpr = l;
+            }
+        }
+    }
     const long long ctas = sm_count();
     const long long per_cta = cdiv64(p.strips, ctas);                 // strips per CTA
     const long long tiles_per_cta = cdiv64(per_cta, s_max);
@@ -384,9 +479,11 @@ static gf_status launch_stream_inst(const PoolParams& p, cudaStream_t s) {
 
 template <typename TIn, typename TOut>
 static gf_status launch_stream(const PoolParams& p, cudaStream_t s) {
-    const int G = p.Wp % 4 == 0 ? 4 : (p.Wp % 2 == 0 ? 2 : 1);
+    int G = p.Wp % 4 == 0 ? 4 : (p.Wp % 2 == 0 ? 2 : 1);
+    if (p.lin_log_lpr >= 0) G = 0;
 #define GF_STREAM_CASE(RR, GG) \
     if (p.r == RR && G == GG) return launch_stream_inst<TIn, TOut, RR, GG>(p, s);
+    GF_STREAM_CASE(2, 0) GF_STREAM_CASE(4, 0) GF_STREAM_CASE(8, 0)
     GF_STREAM_CASE(2, 4) GF_STREAM_CASE(2, 2) GF_STREAM_CASE(2, 1)
     GF_STREAM_CASE(4, 4) GF_STREAM_CASE(4, 2) GF_STREAM_CASE(4, 1)
     GF_STREAM_CASE(8, 4) GF_STREAM_CASE(8, 2) GF_STREAM_CASE(8, 1)
@@ -430,6 +527,7 @@ gf_status launch_pool(int kernel_id, const void* in, int in_dtype, void* out, vo
     if (out_lo && out_dtype != GF_BF16) return GF_ERR_UNSUPPORTED;
     p.in = in; p.out = out; p.out_lo = out_lo; p.err_word = err_word; p.planes = planes; p.total_elems = planes * H * W;
     p.H = H; p.W = W; p.r = r; p.mean = mean ? 1 : 0;
+    p.lin_log_lpr = -1;
     p.Hp = (H + r - 1) / r; p.Wp = (W + r - 1) / r;
     p.plane_out = p.Hp * p.Wp;
     p.out_pitch = out_pitch > 0 ? out_pitch : p.plane_out;

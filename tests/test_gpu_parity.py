@@ -45,6 +45,12 @@ SMALL = [
     L("many_small_planes", 5, 33, 47, 6, 6, 3, 1, 2),
     L("r8_16x16", 3, 20, 36, 16, 16, 3, 1, 8),
     L("r4_32x32", 2, 20, 12, 32, 32, 1, 1, 4),
+    # narrow power-of-two maps: the pooling kernel's shuffle mode at its extremes
+    L("lin_8x8_r8", 3, 16, 24, 8, 8, 3, 1, 8),
+    L("lin_8x8_r2", 3, 16, 24, 8, 8, 1, 1, 2),
+    L("lin_32x32_r8", 2, 8, 16, 32, 32, 3, 1, 8),
+    L("lin_16x64_r2", 2, 8, 8, 16, 64, 3, 1, 2),
+    L("lin_many_tiles", 8, 256, 128, 16, 16, 1, 1, 4),
     # depthwise, streamed kernel: ring wrap-around (more tiles per CTA than ring slots), bands of
     # large planes, r = 8, 7-wide patch rows
     L("dw_ring_wrap", 16, 640, 640, 28, 28, 3, 640, 2),
