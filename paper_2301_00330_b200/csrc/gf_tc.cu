@@ -20,6 +20,7 @@
 // and returns.
 #include "gf_common.cuh"
 #include "gf_tc.cuh"
+#include "gf_tma.cuh"
 
 namespace gf {
 
@@ -227,6 +228,11 @@ struct GxTcParams {
     // the 8-element boundary below its first column (tiles_per_img tiles per image); 0 otherwise
     int rows_per_tile, tiles_per_img;
     FastDiv div_Wp, div_Hp, div_RWp, div_ci_tiles, div_tiles_per_img;
+    // thetaT as a tensor map [part][C_in][C_out] (part: high / low halves of fp32 values), box
+    // 64 x 128: its tiles are fetched by the copy engine when tma_a is 1, by the loader
+    // threads otherwise
+    int tma_a;
+    CUtensorMap tm_theta;
 };
 
 // One unit of work of gx_tc: a 128-row c_i tile times a column tile.
@@ -285,7 +291,7 @@ struct GxShared {
 //       K) resident in shared memory; only the gbar tiles stream through the ring.
 // SPLIT: 1 = bf16 operands; 2 = fp32 data carried as (high, low) bf16 pairs.
 template <typename TOut, int NT, int R, int LOGV, bool ARES, int SPLIT>
-__global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p) {
+__global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const __grid_constant__ GxTcParams p) {
     constexpr int kGxStages = gx_stages(SPLIT, ARES);
     constexpr int kABytes = 128 * kTcBK * 2;             // 16 KB
     constexpr int kBBytes = kTcBK * NT * 2;              // 64 k x NT columns
@@ -318,7 +324,10 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
 
     pdl_launch_dependents();
     if (tid == 0) {
-        for (int s = 0; s < kGxStages; ++s) { mbar_init(&sh.full[s], kGxLoaders); mbar_init(&sh.empty[s], 1); }
+        // a stage is full when every loader thread's copies have landed, plus (tensor-map mode)
+        // thread 0's arrival that carries the bytes the copy engine delivers
+        const int tma_a = (LOGV > 0 && p.tma_a) ? 1 : 0;
+        for (int s = 0; s < kGxStages; ++s) { mbar_init(&sh.full[s], kGxLoaders + tma_a); mbar_init(&sh.empty[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&sh.acc_full[b], 1); mbar_init(&sh.acc_empty[b], 1); }
         mbar_fence_init();
     }
@@ -377,7 +386,30 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
                     b_src = flat_ptr(p.gbar, pb.krow0, b_ok ? w.col0 + pb.j : 0);
                 }
                 const int k0 = kc * kTcBK;
-                if constexpr (ARES) {
+                uint64_t* full_s = &sh.full[q % kGxStages];
+                if (p.tma_a) {
+                    // thetaT tiles by the copy engine: 64 x 128 boxes at (k, c_i, part)
+                    if (tid == 0) {
+                        if constexpr (ARES) {
+                            if (q == 0) {     // the resident tile rides with the first stage
+                                mbar_expect_tx(full_s, (uint32_t)(SPLIT * n_chunks * kABytes));
+                                for (int c = 0; c < SPLIT * n_chunks; ++c) {
+                                    const int cc = c < n_chunks ? c : c - n_chunks;
+                                    tma_load_3d(a_res + (size_t)c * kABytes, &p.tm_theta, cc * kTcBK, ci0, c < n_chunks ? 0 : 1,
+                                                full_s);
+                                }
+                            } else {
+                                mbar_arrive(full_s);
+                            }
+                        } else {
+                            mbar_expect_tx(full_s, (uint32_t)(SPLIT * kABytes));
+#pragma unroll
+                            for (int h = 0; h < SPLIT; ++h)
+                                tma_load_3d(dyn + (size_t)(q % kGxStages) * kStageBytes + h * kABytes, &p.tm_theta, k0, ci0, h,
+                                            full_s);
+                        }
+                    }
+                } else if constexpr (ARES) {
                     if (q == 0)      // the resident thetaT tile rides in the first copy group
                         for (int c = 0; c < SPLIT * n_chunks; ++c) {
                             const int cc = c < n_chunks ? c : c - n_chunks;
@@ -548,7 +580,12 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const GxTcParams p
             asm volatile("bar.sync 1, 256;" ::: "memory");   // D and the offsets are free again
         }
     }
-    if (!ok) atomicOr(p.err_word, 2u);
+    if (!ok) {
+        atomicOr(p.err_word, 2u);
+        // copies of the copy engine may still be on their way to this CTA's shared memory:
+        // a bounded pause (about a millisecond) before the CTA gives it up
+        if (p.tma_a) { const long long t0 = clock64(); while (clock64() - t0 < 2000000LL) {} }
+    }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -992,6 +1029,14 @@ gf_status launch_gx_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const _
     p.tiles_per_img = d.tiles_per_img;
     p.gbar.logV = d.logV;
     const long long col_tiles = d.col_tiles;
+    p.tma_a = 0;
+    if (d.logV > 0) {
+        const int parts = g.dtype == GF_F32 ? 2 : 1;
+        const uint64_t part_stride = parts == 2 ? (uint64_t)theta_lo_off : (uint64_t)g.C_in * g.C_out;
+        if (make_tmap_bf16(&p.tm_theta, thetaT, 3, (uint64_t)g.C_out, (uint64_t)g.C_in, (uint64_t)parts, (uint64_t)g.C_out,
+                           part_stride, 128))
+            p.tma_a = 1;
+    }
     p.div_tiles_per_img = FastDiv((uint32_t)p.tiles_per_img);
     const long long items = col_tiles * p.n_ci_tiles;
     const int n_chunks = (g.C_out + kTcBK - 1) / kTcBK;
