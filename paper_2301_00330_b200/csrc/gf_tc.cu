@@ -228,6 +228,7 @@ struct GxTcParams {
     // the 8-element boundary below its first column (tiles_per_img tiles per image); 0 otherwise
     int rows_per_tile, tiles_per_img;
     FastDiv div_Wp, div_Hp, div_RWp, div_ci_tiles, div_tiles_per_img;
+    FastDiv div_rW, div_W, div_r;       // r*W, W, r: pixel walk of the R == 1 epilogue
     // thetaT as a tensor map [part][C_in][C_out] (part: high / low halves of fp32 values), box
     // 64 x 128: its tiles are fetched by the copy engine when tma_a is 1, by the loader
     // threads otherwise
@@ -285,6 +286,9 @@ struct GxShared {
 // R > 0: r == R, r | W and Wp <= NT.  A tile is a run of whole patch rows (of consecutive
 //        images), so its part of a g_X plane is made of whole pixel rows and the stores
 //        follow memory order: consecutive lanes write consecutive R-element vectors.
+// R == 1: any r with Wp <= NT (partial patches at the right and bottom edges allowed): tiles
+//        of whole patch rows as above; the epilogue walks the tile's pixels in memory order,
+//        consecutive lanes on consecutive pixels of a row, one element per store.
 // R == 0: any r; a tile is NT flattened patches, element-wise stores clipped at the edges.
 // LOGV: log2 of the piece width of gbar (0: 2-byte pieces through registers).
 // ARES: the CTA keeps one c_i tile for all its items and holds that tile of thetaT (all of
@@ -300,7 +304,7 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const __grid_const
     constexpr int kBOff = ARES ? 0 : SPLIT * kABytes;
     constexpr int kDBytes = (128 * (NT + 1) * 4 + 1023) / 1024 * 1024;
     constexpr int kColsPerLane = NT / 32;
-    constexpr int kUnits = R > 0 ? NT * R : 1;           // R-element vectors of a tile's part of one plane
+    constexpr int kUnits = R >= 2 ? NT * R : 1;          // R-element vectors of a tile's part of one plane
     constexpr int kColTab = R == 0 ? NT : 1;
     constexpr uint32_t kIdesc = umma_idesc_bf16(128, NT, /*A K-major*/ 0, /*B MN-major*/ 1);
     extern __shared__ unsigned char dyn_raw[];
@@ -471,7 +475,7 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const __grid_const
             const GxItem w = item_of(it);
             const int ci0 = w.ci0, ncols = w.ncols;
             const long long col0 = w.col0;
-            if constexpr (R > 0) {
+            if constexpr (R >= 2) {
                 // vector u of the tile's part of a plane, in memory order: patch row ta of the tile,
                 // pixel row dr of that patch row, patch jb of the row
                 const uint32_t A0 = w.A0;                                  // first patch row, over all images
@@ -485,7 +489,7 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const __grid_const
                                             : -1;
                     unit_src[u] = (unsigned short)(w.shift + ta * p.Wp + jb);
                 }
-            } else {
+            } else if constexpr (R == 0) {
                 for (int j = et; j < NT; j += kGxEpi) {      // patch offsets of this tile's columns
                     long long off = -1;
                     int ext = 0;
@@ -523,7 +527,25 @@ __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const __grid_const
             if (ok) {
                 const int m_cnt = min(128, p.C_in - ci0);
                 TOut* base = gx + (size_t)ci0 * plane;
-                if constexpr (R > 0) {
+                if constexpr (R == 1) {
+                    // pixels of the tile's part of a plane in memory order: patch row ta of the tile,
+                    // pixel row dr of it (rows below the map are skipped), column x; the same
+                    // pixel of every plane m comes from D[m][patch of the pixel]
+                    const uint32_t rW = (uint32_t)(p.r * p.W);
+                    const uint32_t n_pix = (uint32_t)(w.nlive / p.Wp) * rW;
+                    for (uint32_t e = lane; e < n_pix; e += 32) {
+                        uint32_t ta, rem, dr, x, n, a;
+                        p.div_rW.divmod(e, ta, rem);
+                        p.div_W.divmod(rem, dr, x);
+                        p.div_Hp.divmod(w.A0 + ta, n, a);
+                        const int row = (int)a * p.r + (int)dr;
+                        if (row >= p.H) continue;
+                        const int src = w.shift + (int)ta * p.Wp + (int)p.div_r.div(x);
+                        TOut* dst0 = base + (long long)n * p.C_in * p.H * p.W + (long long)row * p.W + x;
+                        for (int m = ew; m < m_cnt; m += 8)
+                            dst0[(size_t)m * plane] = from_f32<TOut>(D[m * (NT + 1) + src]);
+                    }
+                } else if constexpr (R >= 2) {
                     // expansion in memory order, 16 bytes per store where possible: lane l owns the
                     // chunks l, l+32, ... of UPC consecutive vectors each, for every plane
                     constexpr int UPC = (16 / (R * (int)sizeof(TOut))) > 1 ? 16 / (R * (int)sizeof(TOut)) : 1;
@@ -844,9 +866,26 @@ static GxPlan gx_plan(const Geo& g) {
     GxPlan d;
     const int P = tc_pitch(g);
     d.padded = P != g.Hp * g.Wp;
-    d.R = (g.W % g.r == 0 && g.Wp <= NT && (g.r == 2 || g.r == 4 || g.r == 8)) ? g.r : 0;
-    if (d.padded && g.Wp > NT - 7) d.R = 0;         // no room for the alignment slack of a row-aligned tile
+    const bool fits = g.Wp <= (d.padded ? NT - 7 : NT);   // padded: room for the alignment slack of a row tile
+    d.R = !fits ? 0 : (g.W % g.r == 0 && (g.r == 2 || g.r == 4 || g.r == 8)) ? g.r : 1;
     d.tile_cols = d.R > 0 ? (NT / g.Wp) * g.Wp : NT;
+    const int n_ci_tiles = (g.C_in + 127) / 128;
+    if (d.R > 0 && !d.padded) {
+        // Few, large tiles leave SMs idle (every patch of a tile expands to r x r pixels of
+        // 128 planes, all written by one CTA): shorten the tiles until there is one per SM.
+        // Only lengths that keep the tile starts on the copy-piece boundary P allows.
+        const long long total_rows = (long long)g.N * g.Hp;
+        const int piece = (P % 8 == 0) ? 8 : (P % 4 == 0) ? 4 : 1;
+        const int rows_max = NT / g.Wp;
+        if (d.tile_cols % piece == 0) {
+            int rows = rows_max;
+            for (int cand = rows_max - 1; cand >= 1; --cand) {
+                if (((total_rows + rows - 1) / rows) * n_ci_tiles >= sm_count()) break;
+                if ((cand * g.Wp) % piece == 0) rows = cand;
+            }
+            d.tile_cols = rows * g.Wp;
+        }
+    }
     d.rows_per_tile = 0;
     d.tiles_per_img = 1;
     d.logV = (P % 8 == 0) ? 3 : (P % 4 == 0) ? 2 : 0;
@@ -854,6 +893,13 @@ static GxPlan gx_plan(const Geo& g) {
         // tiles of whole patch rows of one image, loaded from an 8-element boundary
         d.rows_per_tile = (NT - 7) / g.Wp;
         if (d.rows_per_tile > g.Hp) d.rows_per_tile = g.Hp;
+        while (d.rows_per_tile > 1 &&
+               (long long)g.N * ((g.Hp + d.rows_per_tile - 1) / d.rows_per_tile) * n_ci_tiles < sm_count())
+            --d.rows_per_tile;                      // as above: at least one tile per SM
+        {   // even tiles: 7 rows in two tiles are 4 + 3, not 6 + 1
+            const int t = (g.Hp + d.rows_per_tile - 1) / d.rows_per_tile;
+            d.rows_per_tile = (g.Hp + t - 1) / t;
+        }
         d.tiles_per_img = (g.Hp + d.rows_per_tile - 1) / d.rows_per_tile;
         d.col_tiles = (long long)g.N * d.tiles_per_img;
     } else {
@@ -999,6 +1045,7 @@ static gf_status launch_gx_tc_r(const GxTcParams& p, int R, cudaStream_t s) {
     if (R == 2) return launch_gx_tc_v<TOut, NT, 2, SPLIT>(p, s);
     if (R == 4) return launch_gx_tc_v<TOut, NT, 4, SPLIT>(p, s);
     if (R == 8) return launch_gx_tc_v<TOut, NT, 8, SPLIT>(p, s);
+    if (R == 1) return launch_gx_tc_v<TOut, NT, 1, SPLIT>(p, s);
     return launch_gx_tc_v<TOut, NT, 0, SPLIT>(p, s);
 }
 
@@ -1024,6 +1071,9 @@ gf_status launch_gx_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const _
     const GxPlan d = gx_plan(g);
     const int R = d.R;
     p.div_RWp = FastDiv((uint32_t)((R > 0 ? R : 1) * g.Wp));
+    p.div_rW = FastDiv((uint32_t)(g.r * g.W));
+    p.div_W = FastDiv((uint32_t)g.W);
+    p.div_r = FastDiv((uint32_t)g.r);
     p.tile_cols = d.tile_cols;
     p.rows_per_tile = d.rows_per_tile;
     p.tiles_per_img = d.tiles_per_img;
