@@ -39,10 +39,10 @@ FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # SMs x FMA lanes x 2 flop x 
 # single launch stay in the 126 MB L2 past the end of the kernel, so dram__bytes_write is 0
 # there and the figure is the read side.
 NCU_TRAFFIC: dict[str, dict] = {
-    "gx_tc": {"bytes": 6584832, "sha1": "0f52a7deddf63f0abcf2fbec0951bddaaef366b3"},
-    "gw_tc": {"bytes": 13128448, "sha1": "0f52a7deddf63f0abcf2fbec0951bddaaef366b3"},
-    "stash_pool": {"bytes": 25704192, "sha1": "af0ecc32d79557b642afe63bede04d88db66f208"},
-    "gy_pool": {"bytes": 25703936, "sha1": "af0ecc32d79557b642afe63bede04d88db66f208"},
+    "gx_tc": {"bytes": 6591744, "sha1": "5d0d5d5b046b08b6758a596ff64c9eb89a4b82ec"},
+    "gw_tc": {"bytes": 13128192, "sha1": "5d0d5d5b046b08b6758a596ff64c9eb89a4b82ec"},
+    "stash_pool": {"bytes": 25704192, "sha1": "32489a8cbb4cb6666eb457a8564921407388dd58"},
+    "gy_pool": {"bytes": 25703936, "sha1": "32489a8cbb4cb6666eb457a8564921407388dd58"},
 }
 
 KERNEL_SOURCE = {
