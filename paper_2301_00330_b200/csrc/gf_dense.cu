@@ -215,6 +215,24 @@ __global__ void gw_finish_kernel(const float* __restrict__ part, int S, size_t n
     gW[i] = ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
 }
 
+// One partial matrix (the tensor-core path accumulates in place): a pure broadcast of
+// every unique value to its taps, four consecutive outputs (one 16-byte store) per thread.
+__global__ void __launch_bounds__(256) gw_broadcast_kernel(const float* __restrict__ part, size_t total, FastDiv div_taps,
+                                                           float* __restrict__ gW) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+    if (i >= total) return;
+    float v[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) v[k] = i + k < total ? part[div_taps.div((uint32_t)(i + k))] : 0.f;
+    if (i + 4 <= total) {
+        *reinterpret_cast<float4*>(gW + i) = make_float4(v[0], v[1], v[2], v[3]);
+    } else {
+        for (int k = 0; i + k < total; ++k) gW[i + k] = v[k];
+    }
+}
+
 // Many partial matrices (S >= 16): 32 pairs per block, the partials dealt to the block's 8
 // warps, every load of a warp independent; the sum order is fixed.
 __global__ void __launch_bounds__(256) gw_finish_wide_kernel(const float* __restrict__ part, int S, size_t n_pairs,
@@ -251,6 +269,9 @@ gf_status launch_gw_finish(const float* part, int splits, float* gW, const Geo& 
     const int taps = g.KH * g.KW;
     const size_t total = n_pairs * taps;
     if (total > 0x7fffffffULL) return GF_ERR_UNSUPPORTED;
+    if (splits == 1)
+        return launch_pdl(gw_broadcast_kernel, dim3((unsigned)((total / 4 + 256) / 256)), dim3(256), 0, s, part, total,
+                          FastDiv(taps), gW);
     if (splits >= 16)
         return launch_pdl(gw_finish_wide_kernel, dim3((unsigned)((n_pairs + 31) / 32)), dim3(256), 0, s, part, splits,
                           n_pairs, taps, FastDiv(taps), gW);
