@@ -271,10 +271,13 @@ gf_status backward_impl(const gf_conv_desc* desc, const void* g_y, const void* s
         const long long stash_lo = split ? (long long)(align_up((size_t)g.N * g.C_in * pitch * 2, 256) / 2) : 0;
         __nv_bfloat16* thetaT = reinterpret_cast<__nv_bfloat16*>(tsum);
         __nv_bfloat16* gbar16 = reinterpret_cast<__nv_bfloat16*>(gbar);
-        st = launch_ksum_t(W, g, thetaT, split ? thetaT + theta_lo : nullptr, g_W ? part : nullptr, err, s);
-        if (st != GF_OK) return st;
+        // the gradient filter first; the theta sums (which also clear the error word and the g_W
+        // accumulator) are launched behind it and work next to it
         st = launch_pool(K_GY_POOL, g_y, g.dtype, gbar16, split ? gbar16 + gbar_lo : nullptr, GF_BF16, /*mean=*/true,
                          (int64_t)g.N * g.C_out, g.H, g.W, g.r, (int)pitch, err, s);
+        if (st != GF_OK) return st;
+        st = launch_ksum_t(W, g, thetaT, split ? thetaT + theta_lo : nullptr, g_W ? part : nullptr, err,
+                           /*beside_pool=*/true, s);
         if (st != GF_OK) return st;
         // both outputs wanted: the g_W chain goes to the side stream, forked here
         SideStream* side = (may_fork && g_X && g_W) ? side_stream() : nullptr;

@@ -186,8 +186,9 @@ int tc_gw_splits(const Geo& g);
 int tc_pitch(const Geo& g);
 gf_status launch_repack(const void* in, int in_dtype, __nv_bfloat16* hi, __nv_bfloat16* lo, long long rows, int P,
                         int pitch, cudaStream_t s);
+// beside_pool: launched right behind the gradient-filter pooling kernel, works next to it
 gf_status launch_ksum_t(const void* W, const Geo& g, __nv_bfloat16* thetaT, __nv_bfloat16* thetaT_lo, float* gwu,
-                        uint32_t* err_word, cudaStream_t s);
+                        uint32_t* err_word, bool beside_pool, cudaStream_t s);
 gf_status launch_split_f32(const float* in, __nv_bfloat16* hi, __nv_bfloat16* lo, size_t n, cudaStream_t s);
 // max_ctas: CTAs the kernel may use (0: one per SM)
 gf_status launch_gx_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const __nv_bfloat16* thetaT,

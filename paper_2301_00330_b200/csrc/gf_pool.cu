@@ -293,13 +293,15 @@ __global__ void __launch_bounds__(kStreamThreads, 1) pool_stream_kernel(const Po
     };
     LinearLane<TIn, R> lane_ctx;
     if constexpr (G == 0) lane_ctx.init(p);
-    pdl_launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStreamStages; ++s) mbar_init(&full[s], 1);
         mbar_fence_init();
     }
     __syncthreads();
     pdl_wait();                       // the input may come from the previous kernel of the stream
+    // The next kernel of the stream may start only now: it then knows that every kernel
+    // before this one has completed (the theta-sum kernel works next to this one on that basis).
+    pdl_launch_dependents();
     if (threadIdx.x == 0)
         for (int it = 0; it < kStreamStages && it < n_my; ++it) issue(it);
 

@@ -749,10 +749,16 @@ __global__ void __launch_bounds__(kGwThreads) gw_tc_kernel(const GwTcParams p) {
 template <typename T>
 __global__ void __launch_bounds__(1024) ksum_t_kernel(const T* __restrict__ W, __nv_bfloat16* __restrict__ thetaT,
                                                       __nv_bfloat16* __restrict__ thetaT_lo, float* __restrict__ gwu,
-                                                      int C_in, int C_out, int taps, uint32_t* err_word) {
+                                                      int C_in, int C_out, int taps, uint32_t* err_word,
+                                                      int late_wait) {
     __shared__ float tile[32][33];
     pdl_launch_dependents();
-    pdl_wait();
+    // late_wait: the kernel before this one in the stream is the gradient-filter pooling
+    // kernel, which releases its dependents only after everything before IT has completed and
+    // neither produces this kernel's inputs nor touches its outputs.  So this kernel works
+    // next to it right away and waits for it at its END, which keeps the stream's order for
+    // whatever comes after (the contractions need both).
+    if (!late_wait) pdl_wait();
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
     const int co0 = blockIdx.y * 32, ci0 = blockIdx.x * 32;
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0 && err_word) *err_word = 0u;
@@ -774,6 +780,7 @@ __global__ void __launch_bounds__(1024) ksum_t_kernel(const T* __restrict__ W, _
         thetaT[(size_t)ci * C_out + co] = hi;
         if (thetaT_lo) thetaT_lo[(size_t)ci * C_out + co] = __float2bfloat16_rn(v - __bfloat162float(hi));
     }
+    if (late_wait) pdl_wait();
 }
 
 // fp32 -> (high, low) bf16 pair: hi = rn(v), lo = rn(v - hi); v - hi - lo is below 2^-17 |v|.
@@ -981,16 +988,16 @@ int tc_gw_splits(const Geo& g) {
 }
 
 gf_status launch_ksum_t(const void* W, const Geo& g, __nv_bfloat16* thetaT, __nv_bfloat16* thetaT_lo, float* gwu,
-                        uint32_t* err_word, cudaStream_t s) {
+                        uint32_t* err_word, bool beside_pool, cudaStream_t s) {
     ProfScope prof(K_KSUM, s);
     const int taps = g.KH * g.KW;
     dim3 grid((g.C_in + 31) / 32, (g.C_out + 31) / 32, 1);
     if (grid.y > 65535) return GF_ERR_UNSUPPORTED;
     if (g.dtype == GF_F32)
         return launch_pdl(ksum_t_kernel<float>, grid, dim3(1024), 0, s, (const float*)W, thetaT, thetaT_lo, gwu, g.C_in,
-                          g.C_out, taps, err_word);
+                          g.C_out, taps, err_word, beside_pool ? 1 : 0);
     return launch_pdl(ksum_t_kernel<__nv_bfloat16>, grid, dim3(1024), 0, s, (const __nv_bfloat16*)W, thetaT, thetaT_lo,
-                      gwu, g.C_in, g.C_out, taps, err_word);
+                      gwu, g.C_in, g.C_out, taps, err_word, beside_pool ? 1 : 0);
 }
 
 gf_status launch_split_f32(const float* in, __nv_bfloat16* hi, __nv_bfloat16* lo, size_t n, cudaStream_t s) {
