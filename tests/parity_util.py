@@ -35,7 +35,9 @@ class Guarded:
 
     def __init__(self, shape, dtype, device="cuda"):
         n = int(np.prod(shape))
-        self.sentinel = 90 if dtype == torch.uint8 else SENTINEL
+        # byte buffers (the workspace) start as all-ones: NaN as bf16 or fp32, so that scratch which
+        # the library reads without having written it shows up in the results
+        self.sentinel = 255 if dtype == torch.uint8 else SENTINEL
         self.raw = torch.full((n + 2 * GUARD,), self.sentinel, dtype=dtype, device=device)
         self.t = self.raw[GUARD:GUARD + n].view(shape)
         assert self.t.data_ptr() % 16 == 0
