@@ -6,3 +6,4 @@ library is the only implementation: nothing here computes on the CPU.
 from . import workloads  # noqa: F401
 from .binding import *  # noqa: F401,F403
 from .binding import build_library, lib, library_path  # noqa: F401
+from .autograd import FilteredConv2d, filtered_conv2d  # noqa: F401
