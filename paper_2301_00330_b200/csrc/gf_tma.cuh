@@ -9,7 +9,7 @@
 //
 // Rules kept by every caller: the innermost coordinate times 2 bytes is a multiple of 16;
 // global strides are multiples of 16 bytes; the shared-memory destination is 1024-byte
-// aligned; no multicast.
+// aligned; every copy goes to the issuing CTA alone.
 #pragma once
 
 #include <cuda.h>
