@@ -28,7 +28,7 @@ constexpr int kTcBK = 64;           // K elements per stage (one 128-byte swizzl
 constexpr int kGwLoaders = 256;     // gw_tc: 8 loader / epilogue warps + 1 MMA warp
 constexpr int kGwThreads = 288;
 constexpr int kGwStagesMax = 6;
-__host__ __device__ constexpr int gw_stages(int split) { return split == 2 ? 3 : 6; }
+__host__ __device__ constexpr int gw_stages(int split, int nt) { return split == 2 ? 3 : nt == 256 ? 4 : 6; }
 constexpr int kGxLoaders = 256;     // gx_tc: 8 loader warps, 8 epilogue warps, 1 MMA warp
 constexpr int kGxEpi = 256;
 constexpr int kGxThreads = kGxLoaders + kGxEpi + 32;
@@ -637,7 +637,7 @@ __device__ __forceinline__ void red_add_v4(float* dst, uint32_t a, uint32_t b, u
 
 template <int NT, int LOGV, int SPLIT>
 __global__ void __launch_bounds__(kGwThreads) gw_tc_kernel(const GwTcParams p) {
-    constexpr int kGwStages = gw_stages(SPLIT);
+    constexpr int kGwStages = gw_stages(SPLIT, NT);
     constexpr int kABytes = 128 * kTcBK * 2;
     constexpr int kBBytes = NT * kTcBK * 2;
     constexpr int kBOff = SPLIT * kABytes;                  // stage: [A hi][A lo][B hi][B lo]
@@ -858,6 +858,20 @@ gf_status launch_repack(const void* in, int in_dtype, __nv_bfloat16* hi, __nv_bf
                       pitch, FastDiv((uint32_t)pitch));
 }
 
+// Output tiles of gw_tc are 128 (c_o) x 128 or 256 (c_i).  The wide tile fetches the gbar
+// operand once for twice the outputs and issues N = 256 MMAs, which run at the full
+// tensor-core rate.  It pays on long contractions over many c_i (measured: -11 % and -18 % of
+// the backward call on the 512 -> 512 and 512 -> 2048 layers at 16 x 16, r = 2; within noise
+// on shorter ones), so it is taken for bf16 layers (two operand parts would not leave room
+// for a ring) with C_in >= 512, at least 200 K chunks, and little extra padding of C_in.
+static int gw_tile_n(const Geo& g) {
+    if (g.dtype != GF_BF16 || g.C_in < 512) return 128;
+    const long long chunks = ((long long)g.N * tc_pitch(g) + kTcBK - 1) / kTcBK;
+    if (chunks < 200) return 128;
+    const int pad128 = (g.C_in + 127) / 128 * 128, pad256 = (g.C_in + 255) / 256 * 256;
+    return pad256 * 100 <= pad128 * 115 ? 256 : 128;
+}
+
 // How gx_tc cuts a layer into column tiles (shared by its launcher and by the SM-share model).
 struct GxPlan {
     int R;                 // expansion factor handled by the row-aligned path, 0: generic path
@@ -945,8 +959,9 @@ void tc_partition(const Geo& g, int* gx_ctas, int* gw_splits) {
     const double out_x = (double)g.N * g.C_in * g.H * g.W * (double)g.esize;
     const double w_x = fmax(0.25e-6 * out_x, 0.15e-6 * staged_x);
     const long long chunks_w = ((long long)g.N * tc_pitch(g) + kTcBK - 1) / kTcBK;
-    const int tiles_w = n_ci_tiles * ((g.C_out + 127) / 128);
-    const double staged_w = (double)tiles_w * chunks_w * split * (128 + 128) * kTcBK * 2;
+    const int nt_w = gw_tile_n(g);
+    const int tiles_w = ((g.C_in + nt_w - 1) / nt_w) * ((g.C_out + 127) / 128);
+    const double staged_w = (double)tiles_w * chunks_w * split * (128 + nt_w) * kTcBK * 2;
     const double w_w = (g.dtype == GF_F32 ? 0.22e-6 : 0.14e-6) * staged_w;
     int n_gw = (int)(sms * w_w / (w_w + w_x) + 0.5);
     if (n_gw < sms / 5) n_gw = sms / 5;
@@ -979,7 +994,8 @@ void tc_partition(const Geo& g, int* gx_ctas, int* gw_splits) {
 int tc_gw_splits(const Geo& g) {
     const long long K = (long long)g.N * tc_pitch(g);
     const int chunks = (int)((K + kTcBK - 1) / kTcBK);
-    const int tiles = ((g.C_in + 127) / 128) * ((g.C_out + 127) / 128);
+    const int nt = gw_tile_n(g);
+    const int tiles = ((g.C_in + nt - 1) / nt) * ((g.C_out + 127) / 128);
     int s = (sm_count() + tiles - 1) / tiles;
     if (s > chunks) s = chunks;
     if (s < 1) s = 1;
@@ -1105,7 +1121,7 @@ gf_status launch_gx_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const _
 
 template <int NT, int LOGV, int SPLIT>
 static gf_status launch_gw_tc_inst(const GwTcParams& p, dim3 grid, cudaStream_t s) {
-    constexpr size_t smem = (size_t)gw_stages(SPLIT) * SPLIT * (128 * kTcBK * 2 + NT * kTcBK * 2) + 1024;
+    constexpr size_t smem = (size_t)gw_stages(SPLIT, NT) * SPLIT * (128 * kTcBK * 2 + NT * kTcBK * 2) + 1024;
     static bool configured = false;
     if (!configured) {
         GF_CUDA_TRY(cudaFuncSetAttribute(gw_tc_kernel<NT, LOGV, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -1127,7 +1143,7 @@ gf_status launch_gw_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const _
                        long long stash_lo_off, float* gwu, int splits, uint32_t* err_word, const Geo& g,
                        cudaStream_t s) {
     ProfScope prof(K_GW_TC, s);
-    constexpr int NT = 128;
+    const int NT = gw_tile_n(g);
     GwTcParams p;
     const int P = tc_pitch(g);                      // plane pitch of both operands; gaps hold zeros
     const long long K = (long long)g.N * P;
@@ -1137,8 +1153,9 @@ gf_status launch_gw_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const _
     p.chunks_total = (int)((K + kTcBK - 1) / kTcBK);
     if ((g.C_out + 127) / 128 > 65535 || splits > 65535) return GF_ERR_UNSUPPORTED;
     dim3 grid((g.C_in + NT - 1) / NT, (g.C_out + 127) / 128, splits);
-    if (g.dtype == GF_F32) return launch_gw_tc_v<NT, 2>(p, grid, s);
-    return launch_gw_tc_v<NT, 1>(p, grid, s);
+    if (g.dtype == GF_F32) return launch_gw_tc_v<128, 2>(p, grid, s);
+    if (NT == 256) return launch_gw_tc_v<256, 1>(p, grid, s);
+    return launch_gw_tc_v<128, 1>(p, grid, s);
 }
 
 }  // namespace gf

@@ -51,6 +51,9 @@ SMALL = [
     L("lin_32x32_r8", 2, 8, 16, 32, 32, 3, 1, 8),
     L("lin_16x64_r2", 2, 8, 8, 16, 64, 3, 1, 2),
     L("lin_many_tiles", 8, 256, 128, 16, 16, 1, 1, 4),
+    # long contraction over many input channels: the 128 x 256 output tiles of the g_W kernel (bf16),
+    # with a ragged last tile
+    L("gw_wide_tile", 200, 700, 72, 16, 16, 1, 1, 2),
     # depthwise, streamed kernel: ring wrap-around (more tiles per CTA than ring slots), bands of
     # large planes, r = 8, 7-wide patch rows
     L("dw_ring_wrap", 16, 640, 640, 28, 28, 3, 640, 2),
