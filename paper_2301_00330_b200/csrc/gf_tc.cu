@@ -34,7 +34,9 @@ constexpr int kGxEpi = 256;
 constexpr int kGxThreads = kGxLoaders + kGxEpi + 32;
 constexpr int kGxMmaWarp = (kGxLoaders + kGxEpi) / 32;
 constexpr int kGxStagesMax = 7;
-__host__ __device__ constexpr int gx_stages(int split, bool ares) { return split == 2 ? (ares ? 4 : 3) : 7; }
+__host__ __device__ constexpr int gx_stages(int split, bool ares, int nt = 64) {
+    return split == 2 ? (ares ? 4 : 3) : nt == 128 ? (ares ? 4 : 4) : 7;
+}
 
 // Source of an operand: a [n][C][P] bf16 array read along the flattened index
 // k = n*P + p (row c is a channel).  A plain [rows][pitch] matrix is the case P = pitch,
@@ -296,7 +298,7 @@ struct GxShared {
 // SPLIT: 1 = bf16 operands; 2 = fp32 data carried as (high, low) bf16 pairs.
 template <typename TOut, int NT, int R, int LOGV, bool ARES, int SPLIT>
 __global__ void __launch_bounds__(kGxThreads, 1) gx_tc_kernel(const __grid_constant__ GxTcParams p) {
-    constexpr int kGxStages = gx_stages(SPLIT, ARES);
+    constexpr int kGxStages = gx_stages(SPLIT, ARES, NT);
     constexpr int kABytes = 128 * kTcBK * 2;             // 16 KB
     constexpr int kBBytes = kTcBK * NT * 2;              // 64 k x NT columns
     // stage: [A hi][A lo] (unless resident) [B hi][B lo]
@@ -879,11 +881,15 @@ struct GxPlan {
     long long col_tiles;
     bool padded, ares;     // padded plane pitch; resident thetaT tile possible
 };
-constexpr int kGxNT = 64;
 constexpr size_t kSmemLimit = 227 * 1024;
 
+// Column tiles of gx_tc are 64 or 128 wide.  The wide tile halves the traffic of the thetaT
+// operand when that has to be streamed (C_out too large for a resident tile) and the number
+// of MMA rounds; it needs a 66 KB staging tile, so it is kept to bf16 layers with C_out >= 1024.
+static int gx_tile_n(const Geo& g) { return (g.dtype == GF_BF16 && g.C_out >= 1024) ? 128 : 64; }
+
 static GxPlan gx_plan(const Geo& g) {
-    constexpr int NT = kGxNT;
+    const int NT = gx_tile_n(g);
     GxPlan d;
     const int P = tc_pitch(g);
     d.padded = P != g.Hp * g.Wp;
@@ -933,7 +939,7 @@ static GxPlan gx_plan(const Geo& g) {
     // shared memory of the variant that keeps its thetaT tile resident
     const int split = g.dtype == GF_F32 ? 2 : 1;
     const size_t d_bytes = ((size_t)128 * (NT + 1) * 4 + 1023) / 1024 * 1024;
-    const size_t ring = (size_t)gx_stages(split, true) * split * (kTcBK * NT * 2);
+    const size_t ring = (size_t)gx_stages(split, true, NT) * split * (kTcBK * NT * 2);
     const size_t fixed = 512 + (d.R > 0 ? (size_t)NT * d.R * 10 : (size_t)NT * 12);
     const size_t a_bytes = (size_t)split * ((g.C_out + kTcBK - 1) / kTcBK) * 128 * kTcBK * 2;
     d.ares = d.logV > 0 && ring + d_bytes + a_bytes + 1024 + fixed <= kSmemLimit;
@@ -955,7 +961,7 @@ void tc_partition(const Geo& g, int* gx_ctas, int* gw_splits) {
     const double split = g.dtype == GF_F32 ? 2.0 : 1.0;
     const int n_ci_tiles = (g.C_in + 127) / 128;
     const long long chunks_x = (g.C_out + kTcBK - 1) / kTcBK;
-    const double staged_x = (double)d.col_tiles * n_ci_tiles * chunks_x * split * (kTcBK * kGxNT * 2 + (d.ares ? 0 : 128 * kTcBK * 2));
+    const double staged_x = (double)d.col_tiles * n_ci_tiles * chunks_x * split * (kTcBK * gx_tile_n(g) * 2 + (d.ares ? 0 : 128 * kTcBK * 2));
     const double out_x = (double)g.N * g.C_in * g.H * g.W * (double)g.esize;
     const double w_x = fmax(0.25e-6 * out_x, 0.15e-6 * staged_x);
     const long long chunks_w = ((long long)g.N * tc_pitch(g) + kTcBK - 1) / kTcBK;
@@ -1026,7 +1032,7 @@ gf_status launch_split_f32(const float* in, __nv_bfloat16* hi, __nv_bfloat16* lo
 template <typename TOut, int NT, int R, int LOGV, bool ARES, int SPLIT>
 static gf_status launch_gx_tc_ares(const GxTcParams& p, int grid, size_t a_res_bytes, cudaStream_t s) {
     constexpr size_t d_bytes = ((size_t)128 * (NT + 1) * 4 + 1023) / 1024 * 1024;
-    constexpr size_t ring = (size_t)gx_stages(SPLIT, ARES) * SPLIT * (kTcBK * NT * 2 + (ARES ? 0 : 128 * kTcBK * 2));
+    constexpr size_t ring = (size_t)gx_stages(SPLIT, ARES, NT) * SPLIT * (kTcBK * NT * 2 + (ARES ? 0 : 128 * kTcBK * 2));
     const size_t smem = ring + d_bytes + (ARES ? a_res_bytes : 0) + 1024;
     static size_t configured = 0;
     if (smem > configured) {
@@ -1043,7 +1049,7 @@ static gf_status launch_gx_tc_inst(const GxTcParams& p, cudaStream_t s) {
     const int grid = p.items < sms ? p.items : sms;
     if constexpr (LOGV > 0) {
         constexpr size_t d_bytes = ((size_t)128 * (NT + 1) * 4 + 1023) / 1024 * 1024;
-        constexpr size_t ring = (size_t)gx_stages(SPLIT, true) * SPLIT * (kTcBK * NT * 2);
+        constexpr size_t ring = (size_t)gx_stages(SPLIT, true, NT) * SPLIT * (kTcBK * NT * 2);
         // the kernel's static shared memory (barriers, offset tables) counts against the same limit
         constexpr size_t fixed = 512 + (R > 0 ? (size_t)NT * R * 10 : (size_t)NT * 12);
         const size_t a_bytes = (size_t)SPLIT * ((p.C_out + kTcBK - 1) / kTcBK) * 128 * kTcBK * 2;
@@ -1078,7 +1084,6 @@ gf_status launch_gx_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const _
                        long long theta_lo_off, void* gX, int max_ctas, uint32_t* err_word, const Geo& g,
                        cudaStream_t s) {
     ProfScope prof(K_GX_TC, s);
-    constexpr int NT = kGxNT;
     GxTcParams p;
     const int P = tc_pitch(g);                      // gbar's plane pitch
     p.P_live = g.Hp * g.Wp;
@@ -1115,8 +1120,9 @@ gf_status launch_gx_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const _
     const int n_chunks = (g.C_out + kTcBK - 1) / kTcBK;
     if (items * n_chunks > 0x7fffffffLL) return GF_ERR_UNSUPPORTED;
     p.items = (int)items;
-    if (g.dtype == GF_F32) return launch_gx_tc_r<float, NT, 2>(p, R, s);
-    return launch_gx_tc_r<__nv_bfloat16, NT, 1>(p, R, s);
+    if (g.dtype == GF_F32) return launch_gx_tc_r<float, 64, 2>(p, R, s);
+    if (gx_tile_n(g) == 128) return launch_gx_tc_r<__nv_bfloat16, 128, 1>(p, R, s);
+    return launch_gx_tc_r<__nv_bfloat16, 64, 1>(p, R, s);
 }
 
 template <int NT, int LOGV, int SPLIT>

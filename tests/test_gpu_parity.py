@@ -54,6 +54,10 @@ SMALL = [
     # long contraction over many input channels: the 128 x 256 output tiles of the g_W kernel (bf16),
     # with a ragged last tile
     L("gw_wide_tile", 200, 700, 72, 16, 16, 1, 1, 2),
+    # many output channels: the 128-wide column tiles of the g_X kernel (bf16), ragged in every direction
+    L("gx_wide_tile", 3, 40, 1032, 16, 16, 1, 1, 2),
+    L("gx_wide_tile_partial", 2, 24, 1024, 14, 14, 1, 1, 4),
+    L("gx_wide_tile_7x7", 5, 136, 1024, 14, 14, 1, 1, 2),
     # depthwise, streamed kernel: ring wrap-around (more tiles per CTA than ring slots), bands of
     # large planes, r = 8, 7-wide patch rows
     L("dw_ring_wrap", 16, 640, 640, 28, 28, 3, 640, 2),
