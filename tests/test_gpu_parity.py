@@ -149,3 +149,36 @@ def test_oracle_disagrees_when_a_mistake_is_planted(gf):
     wrong_mean = gsum / 4.0
     gx_wrong = oracle.reduced_gx(wrong_mean, oracle.kernel_sum(f64(w)), 1, 7, 7, 2)
     assert relerr(f64(gX), gx_wrong) > 100 * TOL["f32"]
+
+
+def test_back_to_back_steps_in_a_cuda_graph(gf):
+    """Steps replayed from a CUDA graph on ONE set of buffers (every kernel of a step starts as
+    early as the dependency rules of the library allow) give what a single eager call gives."""
+    layer = L("graph_steps", 8, 256, 256, 28, 28, 3, 1, 2, "bf16")
+    x, gy, w = workloads.make_inputs(layer)
+    desc = gf.desc_for(layer)
+    xd, gyd, wd = x.cuda(), gy.cuda(), w.cuda()
+    buf = gf.alloc_layer(desc)
+    ws_bytes = gf.gf_backward_workspace_bytes(desc)
+    stream = torch.cuda.Stream()
+
+    def step():
+        gf.gf_stash_forward(desc, xd, buf.stash, stream)
+        gf.gf_backward(desc, gyd, buf.stash, wd, buf.g_W, buf.g_X, buf.workspace, ws_bytes, stream)
+
+    with torch.cuda.stream(stream):
+        step()
+    torch.cuda.synchronize()
+    gW_ref, gX_ref = buf.g_W.clone(), buf.g_X.clone()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        for _ in range(4):
+            step()
+    for _ in range(5):
+        buf.g_W.zero_()
+        buf.g_X.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert gf.gf_last_async_status(buf.workspace) == gf.GF_OK
+        assert torch.equal(buf.g_X, gX_ref)
+        assert relerr(f64(buf.g_W), f64(gW_ref)) <= 1e-5
