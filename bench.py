@@ -40,9 +40,9 @@ FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # SMs x FMA lanes x 2 flop x 
 # there and the figure is the read side.
 NCU_TRAFFIC: dict[str, dict] = {
     "gx_tc": {"bytes": 6591488, "sha1": "89d154e96ff4d360afd232422b68bd39714d857e"},
-    "gw_tc": {"bytes": 13127936, "sha1": "89d154e96ff4d360afd232422b68bd39714d857e"},
-    "stash_pool": {"bytes": 25704192, "sha1": "d3a2deb333a72205f7254934fa713c3053f7326c"},
-    "gy_pool": {"bytes": 25703936, "sha1": "d3a2deb333a72205f7254934fa713c3053f7326c"},
+    "gw_tc": {"bytes": 13128192, "sha1": "89d154e96ff4d360afd232422b68bd39714d857e"},
+    "stash_pool": {"bytes": 25703936, "sha1": "c38ad61ccbdf77bc96e7bf40af6f901fbfce0590"},
+    "gy_pool": {"bytes": 25703936, "sha1": "c38ad61ccbdf77bc96e7bf40af6f901fbfce0590"},
 }
 
 KERNEL_SOURCE = {
