@@ -90,7 +90,15 @@ gf_status gf_stash_forward(const gf_conv_desc* desc, const void* x, void* stash,
  * output may be NULL and is then skipped (a first trained layer needs no g_X).
  * `workspace` is device scratch of at least gf_backward_workspace_bytes; its
  * contents are undefined afterwards, and two calls that overlap in time must
- * not share it. */
+ * not share it.
+ * Streams: everything is ordered after what `stream` held before the call, and
+ * whatever is put on `stream` after the call is ordered after all of the call's
+ * work.  When both outputs are wanted on the tensor-core path, part of the work
+ * (the g_W contraction) runs on a second stream owned by the library, forked
+ * from and joined back into `stream` with events; that stream and its two
+ * events are created by the first such call on a device (host-side resources,
+ * no device memory).  Host threads calling concurrently are serialised while
+ * they enqueue. */
 gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* stash,
                       const void* W, float* g_W, void* g_X, void* workspace,
                       size_t workspace_bytes, void* stream);
