@@ -3,13 +3,20 @@
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
-One step = one pass of the whole hot path over one batch of one layer:
-gf_stash_forward (patch-summed activations) + gf_backward (gradient filter,
-reduced g_W, reduced g_X with expansion), on the ResNet-style layer
-3x3, 256->256, N=64, 28x28, r=2, bf16 inputs with fp32 accumulation.
-Prints ONE JSON line (rank 0).  The metric is microseconds per layer backward
-(lower is better).  N > 1: independent replicas, one per GPU, no collective on
-the data path; the value is time divided by the layers all ranks processed.
+One step = one pass of the whole hot path over one batch of the MobileNetV2-style
+inverted-residual block (1x1 conv 96->576, 3x3 depthwise conv 576, 1x1 conv 576->96;
+N=128, 28x28, r=2, fp32): for each of the three layers gf_stash_forward
+(patch-summed activations) and gf_backward (gradient filter, reduced g_W, reduced g_X
+with expansion).  Prints ONE JSON line (rank 0).  The metric is microseconds per
+layer backward (the step's time divided by its three layers; lower is better).
+The line also carries, in `per_config`, every layer of the other workload
+configurations timed the same way, each next to an exact convolution backward of the
+same shape through torch/cuDNN (context: a different, unfiltered result).
+
+N > 1: independent replicas, one per GPU, no collective on the data path; the value
+is time divided by the layers all ranks processed.  Under a launcher (torchrun) the
+ranks come from the environment; started plainly with --gpus N > 1, the script
+re-executes itself under torch.distributed.run with N processes.
 
 --impl reference times the fp64 CPU checker (oracle/) on the host cores on a
 bounded sample of the same workload.
@@ -32,23 +39,23 @@ METRIC = "filtered_conv_backward_us_per_layer"
 UNIT = "us"
 FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # SMs x FMA lanes x 2 flop x max SM clock
 
-# DRAM bytes per launch of a kernel from one ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum), keyed by kernel name, with the sha1 of the source file
-# at capture time; a changed source makes the entry stale (reported as null).
-# Captured on the bench layer (profiles/step_resnet3x3_256_N64_28x28_r2_bf16.md).  Writes of a
-# single launch stay in the 126 MB L2 past the end of the kernel, so dram__bytes_write is 0
-# there and the figure is the read side.
-NCU_TRAFFIC: dict[str, dict] = {
-    "gx_tc": {"bytes": 6591488, "sha1": "89d154e96ff4d360afd232422b68bd39714d857e"},
-    "gw_tc": {"bytes": 13128192, "sha1": "89d154e96ff4d360afd232422b68bd39714d857e"},
-    "stash_pool": {"bytes": 25703936, "sha1": "c38ad61ccbdf77bc96e7bf40af6f901fbfce0590"},
-    "gy_pool": {"bytes": 25703936, "sha1": "c38ad61ccbdf77bc96e7bf40af6f901fbfce0590"},
+# What the paper reports for this path (Section 5.5): ratios against the libraries' exact
+# convolution backward on its own devices, fp32.  Context for `exact_cudnn_us`, not a target.
+PAPER_CONTEXT = {
+    "r2": "paper, Section 5.5: over 10x faster than the exact cuDNN backward at patch size 2 (RTX 3090 Ti and "
+          "Jetson Nano GPUs, fp32), over 20x against MKLDNN on CPUs (11900KF, Jetson Nano, Raspberry Pi 3b)",
+    "r4": "paper, Section 5.5: over 25x against cuDNN at patch size 4, over 60x against MKLDNN",
 }
+
+# DRAM bytes per launch of a kernel from one ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum), keyed by (layer name, kernel name), with the sha1 of the kernel's
+# source file at capture time; a changed source makes the entry stale (reported as null).
+NCU_TRAFFIC: dict[tuple[str, str], dict] = {}
 
 KERNEL_SOURCE = {
     "stash_pool": "gf_pool.cu", "gy_pool": "gf_pool.cu", "ksum": "gf_tc.cu", "gx_mix": "gf_dense.cu",
     "gw_partial": "gf_dense.cu", "gw_finish": "gf_dense.cu", "dw_fused": "gf_depthwise.cu",
-    "gx_tc": "gf_tc.cu", "gw_tc": "gf_tc.cu",
+    "gx_tc": "gf_tc.cu", "gw_tc": "gf_tc.cu", "split_f32": "gf_tc.cu",
 }
 
 
@@ -63,21 +70,24 @@ def measured_peaks() -> tuple[dict, str]:
 
 
 def workload():
+    """The layers of one step: the MobileNetV2-style block at r = 2, fp32."""
     from paper_2301_00330_b200 import workloads
-    (layer,) = workloads.config2()
-    return layer
+    return workloads.config3(2)
 
 
-def workload_config(layer, extra=None) -> dict:
-    cfg = {
-        "workload": "configs[1]: ResNet-style 3x3 conv backward, stride 1, pad 1, N=64, 256->256, 28x28, r=2",
-        "layer": layer.name, "N": layer.N, "C_in": layer.C_in, "C_out": layer.C_out, "H": layer.H,
-        "W": layer.W, "K": layer.K, "groups": layer.groups, "r": layer.r,
-        "step": "gf_stash_forward + gf_backward (g_W and g_X)",
+def workload_config(layers) -> dict:
+    """The same dict for both arms (GPU and --impl reference)."""
+    return {
+        "workload": "configs[2]: MobileNetV2-style inverted-residual block backward, 1x1 96->576, 3x3 depthwise 576 "
+                    "(pad 1), 1x1 576->96, N=128, 28x28, r=2, fp32 (the largest single-GPU configuration)",
+        "layers": [{"layer": L.name, "N": L.N, "C_in": L.C_in, "C_out": L.C_out, "H": L.H, "W": L.W, "K": L.K,
+                    "groups": L.groups, "r": L.r, "dtype": L.dtype} for L in layers],
+        "step": "for each of the 3 layers: gf_stash_forward + gf_backward (g_W and g_X); value = step time / 3",
+        "inputs": "each layer has its own seeded x, g_y, W (the activation and normalisation backward between the "
+                  "layers is outside the method)",
+        "l2": "every layer's tensors (0.4 - 0.75 GB) exceed the 126 MB L2 several times over, and the step walks "
+              "through 1.8 GB before it touches a buffer again; inputs and outputs also rotate over 2 sets",
     }
-    if extra:
-        cfg.update(extra)
-    return cfg
 
 
 # --------------------------------------------------------------------------- clocks
@@ -140,7 +150,7 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------- roofline
-def kernel_cost(name: str, L, splits: int) -> tuple[float, float]:
+def kernel_cost(name: str, L) -> tuple[float, float]:
     """(algorithmic bytes, flops) of one launch of kernel `name` on layer L."""
     e = L.elem_bytes
     gbar = 4 * L.N * L.C_out * L.Hp * L.Wp          # fp32 patch means (CUDA-core path)
@@ -153,21 +163,22 @@ def kernel_cost(name: str, L, splits: int) -> tuple[float, float]:
     table = {
         "split_f32": (8 * L.numel_stash(), L.numel_stash()),
         "gx_tc": (gbar16 + e * pairs + e * L.numel_x(), mix),
-        "gw_tc": (gbar16 + e * L.numel_stash() + 4 * splits * pairs, mix),
+        "gw_tc": (gbar16 + e * L.numel_stash() + 4 * pairs, mix),
         "stash_pool": (e * (L.numel_x() + L.numel_stash()), L.numel_x()),
         "gy_pool": (e * L.numel_gy() + (gbar16 if tc else gbar), L.numel_gy()),
+        "gyx_fused": (e * (L.numel_gy() + L.numel_x()) + gbar16 + e * pairs, mix + L.numel_gy()),
         "ksum": (e * L.numel_w() + 4 * pairs, L.numel_w()),
         "gx_mix": (gbar + 4 * pairs + e * L.numel_x(), mix),
-        "gw_partial": (gbar + e * L.numel_stash() + 4 * splits * pairs, mix),
-        "gw_finish": (4 * splits * pairs + 4 * L.numel_w(), splits * pairs),
+        "gw_partial": (gbar + e * L.numel_stash() + 4 * pairs, mix),
+        "gw_finish": (4 * pairs + 4 * L.numel_w(), pairs),
         "dw_fused": (e * (L.numel_gy() + L.numel_stash() + L.numel_x() + L.numel_w()), 3 * L.numel_gy()),
     }
     return table[name]
 
 
-def traffic_for(name: str):
-    ent = NCU_TRAFFIC.get(name)
-    src = KERNEL_SOURCE.get(name)
+def traffic_for(layer_name: str, kernel: str):
+    ent = NCU_TRAFFIC.get((layer_name, kernel))
+    src = KERNEL_SOURCE.get(kernel)
     if not ent or not src:
         return None
     path = os.path.join(ROOT, "paper_2301_00330_b200", "csrc", src)
@@ -176,36 +187,42 @@ def traffic_for(name: str):
     return ent["bytes"] if sha == ent.get("sha1") else None
 
 
-def roofline(name: str, avg_ms: float, L, splits: int) -> dict:
+def roofline(name: str, avg_ms: float, L) -> dict:
     peaks, which = measured_peaks()
-    nbytes, flops = kernel_cost(name, L, splits)
+    nbytes, flops = kernel_cost(name, L)
     t = avg_ms * 1e-3
     t_mem = nbytes / (peaks["hbm_gbs"] * 1e9)
     t_alu = flops / (FP32_ALU_TFLOPS * 1e12)
     if t_alu > t_mem and name in ("gx_mix", "gw_partial"):
         ach = flops / t / 1e12
-        return {"kernel": name, "bound": "alu", "achieved": ach, "peak": FP32_ALU_TFLOPS, "unit": "TFLOP/s",
-                "frac": ach / FP32_ALU_TFLOPS, "traffic": traffic_for(name), "peak_source": "derived: 148 SM x 128 FMA x 2 x 1.965 GHz",
-                "avg_launch_us": avg_ms * 1e3}
+        return {"kernel": name, "layer": L.name, "bound": "alu", "achieved": ach, "peak": FP32_ALU_TFLOPS,
+                "unit": "TFLOP/s", "frac": ach / FP32_ALU_TFLOPS, "traffic": traffic_for(L.name, name),
+                "peak_source": "derived: 148 SM x 128 FMA x 2 x 1.965 GHz", "avg_launch_us": avg_ms * 1e3}
     ach = nbytes / t / 1e9
-    return {"kernel": name, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-            "frac": ach / peaks["hbm_gbs"], "traffic": traffic_for(name), "peak_source": f"of {which}",
-            "avg_launch_us": avg_ms * 1e3}
+    return {"kernel": name, "layer": L.name, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"],
+            "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": traffic_for(L.name, name),
+            "peak_source": f"of {which}", "algorithmic_bytes_per_launch": nbytes, "avg_launch_us": avg_ms * 1e3}
 
 
 # --------------------------------------------------------------------------- CPU checker timing
-def time_oracle(layer, n_sample: int, steps: int, warmup: int) -> dict:
+def time_oracle(layers, n_sample: int, steps: int, warmup: int) -> dict:
+    """The fp64 CPU checker, as it stands, on n_sample images of every layer of the step."""
     import numpy as np
     import torch
     import oracle
     from paper_2301_00330_b200 import workloads
-    L = layer.with_(N=n_sample)
-    x, gy, w = workloads.make_inputs(L)
-    x64, gy64, w64 = (t.to(torch.float64).numpy() for t in (x, gy, w))
+    data = []
+    for L in layers:
+        Ls = L.with_(N=n_sample)
+        x, gy, w = workloads.make_inputs(Ls)
+        data.append((Ls, *(t.to(torch.float64).numpy() for t in (x, gy, w))))
 
     def one():
-        stash = oracle.stash_forward(x64, L.r)
-        return oracle.backward(gy64, stash, w64, L.r, groups=L.groups)
+        out = None
+        for Ls, x64, gy64, w64 in data:
+            stash = oracle.stash_forward(x64, Ls.r)
+            out = oracle.backward(gy64, stash, w64, Ls.r, groups=Ls.groups)
+        return out
 
     for _ in range(warmup):
         one()
@@ -214,10 +231,10 @@ def time_oracle(layer, n_sample: int, steps: int, warmup: int) -> dict:
         gw, gx = one()
     dt = (time.perf_counter() - t0) / steps
     assert np.isfinite(gw).all() and np.isfinite(gx).all()
-    scale = layer.N / n_sample
-    return {"value": dt * 1e6 * scale, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": f"{n_sample} of {layer.N} images of the same layer, fp64, time scaled x{scale:g} "
-                      f"(every step is linear in the batch); {steps} timed passes",
+    scale = layers[0].N / n_sample
+    return {"value": dt * 1e6 * scale / len(layers), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{n_sample} of {layers[0].N} images of each of the {len(layers)} layers, fp64, time scaled "
+                      f"x{scale:g} (every step of the method is linear in the batch); {steps} timed passes",
             "seconds_per_pass": dt}
 
 
@@ -225,13 +242,14 @@ def run_reference(args) -> None:
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    layer = workload()
-    base = time_oracle(layer, layer.N, max(1, args.steps), max(0, args.warmup))
+    layers = workload()
+    steps = max(1, min(args.steps, 3))
+    base = time_oracle(layers, 32, steps, 1 if args.warmup > 0 else 0)
     line = {
         "impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": base["value"] / 1e3,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": base["value"] * len(layers) / 1e3,
         "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-        "data": "synthetic", "config": workload_config(layer, {"dtype_in": "bf16 values widened to f64"}),
+        "data": "synthetic", "config": workload_config(layers),
         "cpu_baseline": base,
         "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -250,10 +268,92 @@ def max_over_ranks(ms: float, dist, device) -> float:
     return float(t.item())
 
 
-def job_value_us(ms_total: float, steps: int, world: int) -> float:
-    """us per layer step of the whole job: every rank ran `steps` layer steps of its own
-    replica in ms_total (max over ranks), so the job did steps * world of them."""
-    return ms_total * 1e3 / (steps * world)
+def job_value_us(ms_total: float, steps: int, world: int, layers_per_step: int = 1) -> float:
+    """us per layer of the whole job: every rank ran `steps` steps of `layers_per_step` layers of
+    its own replica in ms_total (max over ranks), so the job did steps * world * layers of them."""
+    return ms_total * 1e3 / (steps * world * layers_per_step)
+
+
+def backlog(ms: float = 4.0):
+    """Keeps the stream busy for a few ms so that the launches enqueued next wait in the
+    queue and then run back to back: event pairs then measure the GPU, not the host."""
+    import torch
+    torch.cuda._sleep(int(ms * 1e-3 * 1.9e9))
+
+
+def time_layer(gf, L, peaks, with_exact: bool = True, with_kernels: bool = False) -> dict:
+    """One layer timed three ways with CUDA events behind a stream backlog: gf_stash_forward,
+    gf_backward (g_W and g_X), and an exact backward through torch/cuDNN as context."""
+    import torch
+    from paper_2301_00330_b200 import workloads
+    stream = torch.cuda.current_stream()
+    desc = gf.desc_for(L)
+    x0, gy0, w0 = workloads.make_inputs(L)
+    per_set = L.backward_bytes() + L.stash_bytes_moved()
+    n_sets = max(1, min(4, int(400e6 // per_set) + 1))     # small layers rotate over several sets (L2)
+    sets = [(torch.roll(x0, i, 0).cuda(), torch.roll(gy0, i, 0).cuda(), gf.alloc_layer(desc)) for i in range(n_sets)]
+    w = w0.cuda()
+    ws_bytes = gf.gf_backward_workspace_bytes(desc)
+    reps = 20 if per_set < 300e6 else 8
+
+    def timed(fn, n):
+        for _ in range(3):
+            fn(0)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        backlog(3.0)
+        e0.record(stream)
+        for i in range(n):
+            fn(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / n
+
+    def stash(i):
+        x, _, b = sets[i % n_sets]
+        gf.gf_stash_forward(desc, x, b.stash, stream)
+
+    def bwd(i):
+        _, gy, b = sets[i % n_sets]
+        gf.gf_backward(desc, gy, b.stash, w, b.g_W, b.g_X, b.workspace, ws_bytes, stream)
+
+    def exact(i):
+        x, gy, _ = sets[i % n_sets]
+        torch.ops.aten.convolution_backward(gy, x, w, None, [1, 1], [L.pad, L.pad], [1, 1], False, [0, 0],
+                                            L.groups, [True, True, False])
+
+    t_stash, t_bwd = timed(stash, reps), timed(bwd, reps)
+    row = {"layer": L.name, "r": L.r, "dtype": L.dtype, "stash_us": round(t_stash, 2), "backward_us": round(t_bwd, 2),
+           "backward_alg_MB": round(L.backward_bytes() / 1e6, 1),
+           "backward_gbs": round(L.backward_bytes() / t_bwd / 1e3, 1),
+           "backward_frac_hbm": round(L.backward_bytes() / t_bwd / 1e3 / peaks["hbm_gbs"], 3),
+           "stash_gbs": round(L.stash_bytes_moved() / t_stash / 1e3, 1),
+           "stash_frac_hbm": round(L.stash_bytes_moved() / t_stash / 1e3 / peaks["hbm_gbs"], 3)}
+    if with_kernels:   # per-kernel event times of the backward call (each bracketed, so a few us high)
+        gf.gf_profile_configure(2)
+        backlog(3.0)
+        for i in range(4):
+            bwd(i)
+        torch.cuda.synchronize()
+        row["kernels_us"] = {k: round(ms / n * 1e3, 1) for k, (n, ms) in gf.gf_profile_read().items()}
+        gf.gf_profile_configure(0)
+    if with_exact:
+        try:
+            t_exact = timed(exact, max(2, reps // 4))
+            row["exact_cudnn_us"] = round(t_exact, 1)
+            row["exact_over_filtered"] = round(t_exact / t_bwd, 2)
+        except Exception as ex:   # context only: never fail the bench on it
+            row["exact_cudnn_us"] = None
+            row["exact_error"] = type(ex).__name__
+    del sets
+    torch.cuda.empty_cache()
+    return row
+
+
+def per_config_layers():
+    """Every layer of the workload configurations (rows of the measurement table)."""
+    from paper_2301_00330_b200 import workloads
+    return [l for l in workloads.all_headline_layers() if l.r > 1]
 
 
 def run_ours(args) -> None:
@@ -271,71 +371,75 @@ def run_ours(args) -> None:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     gf.build_library()
 
-    layer = workload()
-    desc = gf.desc_for(layer)
-    dt = workloads.torch_dtype(layer.dtype)
-    x0, gy0, w0 = workloads.make_inputs(layer)
-    n_sets = 4   # rotating input/output sets: 4 x ~106 MB > 3 x the 126 MB L2
-    sets = []
-    for i in range(n_sets):
-        buf = gf.alloc_layer(desc)
-        sets.append((torch.roll(x0, i, 0).cuda().contiguous(), torch.roll(gy0, i, 0).cuda().contiguous(), buf))
-    w = w0.cuda()
-    ws_bytes = gf.gf_backward_workspace_bytes(desc)
-    set_bytes = sum(t.numel() * t.element_size() for t in (sets[0][0], sets[0][1], sets[0][2].stash,
-                                                            sets[0][2].g_X, sets[0][2].g_W, sets[0][2].workspace))
+    layers = workload()
+    n_layers = len(layers)
+    n_sets = 2
     stream = torch.cuda.current_stream()
+    runs = []          # per layer: (L, desc, w, ws_bytes, [(x, gy, buffers)] * n_sets)
+    host_inputs = []
+    for L in layers:
+        desc = gf.desc_for(L)
+        x0, gy0, w0 = workloads.make_inputs(L)
+        host_inputs.append((x0, gy0, w0))
+        sets = [(torch.roll(x0, i, 0).cuda().contiguous(), torch.roll(gy0, i, 0).cuda().contiguous(),
+                 gf.alloc_layer(desc)) for i in range(n_sets)]
+        runs.append((L, desc, w0.cuda(), gf.gf_backward_workspace_bytes(desc), sets))
 
-    def step(i: int):
+    def layer_step(k: int, i: int, s=None):
+        L, desc, w, ws_bytes, sets = runs[k]
         x, gy, b = sets[i % n_sets]
-        gf.gf_stash_forward(desc, x, b.stash, stream)
-        gf.gf_backward(desc, gy, b.stash, w, b.g_W, b.g_X, b.workspace, ws_bytes, stream)
+        s = s or stream
+        gf.gf_stash_forward(desc, x, b.stash, s)
+        gf.gf_backward(desc, gy, b.stash, w, b.g_W, b.g_X, b.workspace, ws_bytes, s)
+
+    def step(i: int, s=None):
+        for k in range(n_layers):
+            layer_step(k, i, s)
 
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- warm-up; its first steps bracket every kernel to find the dominant one ----
     warm = max(3, args.warmup)
     for i in range(warm):
         step(i)
     torch.cuda.synchronize()
 
-    def backlog(ms: float = 4.0):
-        """Keeps the stream busy for a few ms so that the launches enqueued next
-        wait in the queue and then run back to back: event pairs around a
-        kernel then measure the GPU, not the enqueueing host thread."""
-        torch.cuda._sleep(int(ms * 1e-3 * 1.9e9))
+    # ---- diagnostic pass: every kernel bracketed by events, layer by layer, to find the
+    # (layer, kernel) pair that takes the most time ----
+    diag_steps = 4
+    breakdown = {}
+    dominant, dom_ms = None, -1.0
+    for k, (L, *_rest) in enumerate(runs):
+        gf.gf_profile_configure(2)
+        backlog()
+        for i in range(diag_steps):
+            layer_step(k, i)
+        torch.cuda.synchronize()
+        diag = gf.gf_profile_read()
+        gf.gf_profile_configure(0)
+        breakdown[L.name] = {kn: {"launches_per_step": n / diag_steps, "avg_us": round(ms / n * 1e3, 2)}
+                             for kn, (n, ms) in diag.items()}
+        for kn, (n, ms) in diag.items():
+            if ms > dom_ms:
+                dominant, dom_ms = (k, kn), ms
 
-    # ---- diagnostic pass: every kernel bracketed by events, to find the dominant one ----
-    diag_steps = 8
-    gf.gf_profile_configure(2)
-    backlog()
-    for i in range(diag_steps):
-        step(i)
-    torch.cuda.synchronize()
-    diag = gf.gf_profile_read()
-    gf.gf_profile_configure(0)
-    total_diag = sum(ms for _, ms in diag.values()) or 1.0
-    breakdown = {k: {"launches_per_step": n / diag_steps, "avg_us": ms / n * 1e3, "share": ms / total_diag}
-                 for k, (n, ms) in diag.items()}
-    dominant = max(diag.items(), key=lambda kv: kv[1][1])[0]
-
-    # ---- dominant kernel: event pairs around it alone, over eager steps ----
-    dom_steps = max(1, min(args.steps, 64))
-    gf.gf_profile_configure(1, gf.kernel_id(dominant))
+    # ---- dominant kernel: event pairs around it alone, over eager steps of its layer ----
+    dom_layer, dom_kernel = dominant
+    dom_steps = max(1, min(args.steps, 32))
+    gf.gf_profile_configure(1, gf.kernel_id(dom_kernel))
     backlog()
     for i in range(dom_steps):
-        step(i)
+        layer_step(dom_layer, i)
     torch.cuda.synchronize()
     dom = gf.gf_profile_read()
     gf.gf_profile_configure(0)
 
-    # ---- timed region: exactly K steps.  The steps are replayed from a CUDA graph
-    # that holds one step per input set (the launch sequence of the eager calls,
-    # captured once), so that the host's enqueue rate does not bound the number;
-    # the K mod n_sets remaining steps are enqueued eagerly. ----
+    # ---- timed region: exactly K steps.  The steps are replayed from a CUDA graph that holds
+    # one step per input set (the launch sequence of the eager calls, captured once), so that
+    # the host's enqueue rate does not bound the number; the K mod n_sets remaining steps are
+    # enqueued eagerly. ----
     graph = None
     launches_per_step = None
     if args.steps >= n_sets:
@@ -346,9 +450,7 @@ def run_ours(args) -> None:
         with torch.cuda.graph(graph, stream=side):
             cap = torch.cuda.current_stream()
             for i in range(n_sets):
-                x, gy, b = sets[i]
-                gf.gf_stash_forward(desc, x, b.stash, cap)
-                gf.gf_backward(desc, gy, b.stash, w, b.g_W, b.g_X, b.workspace, ws_bytes, cap)
+                step(i, cap)
         launches_per_step = (gf.gf_kernel_launch_count() - c0) // n_sets
         stream.wait_stream(side)
         graph.replay()               # one untimed replay
@@ -373,59 +475,64 @@ def run_ours(args) -> None:
     if graph is not None:
         launches += replays * n_sets * launches_per_step     # kernels the replays ran
     ms_total = ev0.elapsed_time(ev1)
-    assert gf.gf_last_async_status(sets[0][2].workspace) == gf.GF_OK
+    for _, _, _, _, sets in runs:
+        assert gf.gf_last_async_status(sets[0][2].workspace) == gf.GF_OK
     ms_total = max_over_ranks(ms_total, dist, "cuda")
     ms_per_step = ms_total / args.steps
-    value = job_value_us(ms_total, args.steps, world)
+    value = job_value_us(ms_total, args.steps, world, n_layers)
+    del graph
 
     # ---- end to end: host buffers in, host buffers out, through the C ABI ----
-    hx, hgy, hw = x0.pin_memory(), gy0.pin_memory(), w0.pin_memory()
-    h_gW = torch.empty((layer.C_out, layer.C_ig, layer.K, layer.K), dtype=torch.float32).pin_memory()
-    h_gX = torch.empty(tuple(x0.shape), dtype=dt).pin_memory()
-    arena = torch.empty(gf.gf_host_step_arena_bytes(desc), dtype=torch.uint8, device="cuda")
-    e2e_steps = max(1, min(args.steps, 30))
-    for _ in range(2):
-        gf.gf_layer_step_host(desc, hx, hgy, hw, h_gW, h_gX, arena, stream=stream)
+    e2e_sets = []
+    h2d = d2h = 0
+    for (L, desc, _, _, _), (x0, gy0, w0) in zip(runs, host_inputs):
+        hx, hgy, hw = x0.pin_memory(), gy0.pin_memory(), w0.pin_memory()
+        h_gW = torch.empty((L.C_out, L.C_ig, L.K, L.K), dtype=torch.float32).pin_memory()
+        h_gX = torch.empty(tuple(x0.shape), dtype=workloads.torch_dtype(L.dtype)).pin_memory()
+        arena = torch.empty(gf.gf_host_step_arena_bytes(desc), dtype=torch.uint8, device="cuda")
+        e2e_sets.append((desc, hx, hgy, hw, h_gW, h_gX, arena))
+        h2d += sum(t.numel() * t.element_size() for t in (hx, hgy, hw))
+        d2h += sum(t.numel() * t.element_size() for t in (h_gW, h_gX))
+
+    def e2e_step():
+        for desc, hx, hgy, hw, h_gW, h_gX, arena in e2e_sets:
+            gf.gf_layer_step_host(desc, hx, hgy, hw, h_gW, h_gX, arena, stream=stream)
+
+    e2e_steps = max(1, min(args.steps, 5))
+    e2e_step()
     barrier()
     ev0.record(stream)
     for _ in range(e2e_steps):
-        gf.gf_layer_step_host(desc, hx, hgy, hw, h_gW, h_gX, arena, stream=stream)
+        e2e_step()
     ev1.record(stream)
     torch.cuda.synchronize()
-    e2e_ms = ev0.elapsed_time(ev1)
-    e2e_ms = max_over_ranks(e2e_ms, dist, "cuda")
-    h2d = sum(t.numel() * t.element_size() for t in (hx, hgy, hw))
-    d2h = sum(t.numel() * t.element_size() for t in (h_gW, h_gX))
-    e2e = {"value": job_value_us(e2e_ms, e2e_steps, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
-           "d2h_bytes_per_step": d2h, "steps": e2e_steps, "api": "gf_layer_step_host (pinned host buffers)"}
+    e2e_ms = max_over_ranks(ev0.elapsed_time(ev1), dist, "cuda")
+    e2e = {"value": job_value_us(e2e_ms, e2e_steps, world, n_layers), "unit": UNIT, "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+           "api": "gf_layer_step_host per layer (pinned host buffers; copies of x, g_y, W in and g_W, g_X out inside "
+                  "the timed region)"}
+    del e2e_sets
 
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
 
-    # split count of the reduced g_W contraction, needed for its byte count
-    if layer.groups == 1 and layer.C_out % 8 == 0 and layer.r >= 2:      # tensor-core path: 128 x 128 tiles, one wave of CTAs
-        tiles = ((layer.C_out + 127) // 128) * ((layer.C_in + 127) // 128)
-        chunks = -(-(layer.N * layer.Hp * layer.Wp) // 64)
-        splits = max(1, min(chunks, -(-148 // tiles)))
-    else:
-        tiles = ((layer.C_out // layer.groups + 63) // 64) * ((layer.C_ig + 63) // 64) * layer.groups
-        splits = max(1, min(layer.N, -(-592 // tiles)))
-    n_dom, ms_dom = dom.get(dominant, (0, 0.0))
-    roof = roofline(dominant, ms_dom / max(n_dom, 1), layer, splits)
+    L_dom = layers[dom_layer]
+    n_dom, ms_dom = dom.get(dom_kernel, (0, 0.0))
+    roof = roofline(dom_kernel, ms_dom / max(n_dom, 1), L_dom)
     roof["timed_launches"] = n_dom
     peaks, which = measured_peaks()
-    step_bytes = layer.backward_bytes() + layer.stash_bytes_moved()
+    step_bytes = sum(L.backward_bytes() + L.stash_bytes_moved() for L in layers)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": workload_config(layer, {
-            "l2": f"inputs and outputs rotate over {n_sets} sets of {set_bytes / 1e6:.0f} MB (> 3x the 126 MB L2)",
-            "timing": (f"CUDA events around K steps; {replays} replays of a {n_sets}-step CUDA graph + {rest} eager "
-                       f"steps; dominant kernel timed by event pairs over {dom_steps} eager steps"),
-            "parallelism": "replicas only" if world > 1 else "single GPU"}),
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": workload_config(layers),
+        "timing": (f"CUDA events around K steps; {replays} replays of a {n_sets}-step CUDA graph + {rest} eager steps; "
+                   f"dominant kernel timed by event pairs over {dom_steps} eager steps of its layer"),
+        "parallelism": "replicas only" if world > 1 else "single GPU",
+        "block_us": ms_per_step * 1e3,
         "step_algorithmic_bytes": step_bytes,
         "step_gbs": step_bytes / (ms_per_step * 1e-3) / 1e9,
         "step_frac_of_hbm": step_bytes / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
@@ -434,16 +541,31 @@ def run_ours(args) -> None:
         "gpu_launches": int(launches),
     }
     if world == 1:
-        line["cpu_baseline"] = time_oracle(layer, layer.N, 5, 1)
+        for _, _, _, _, sets in runs:
+            sets.clear()
+        runs.clear()
+        torch.cuda.empty_cache()
+        line["cpu_baseline"] = time_oracle(layers, 32, 2, 1)
+        if not args.no_per_config:
+            rows = [time_layer(gf, L, peaks) for L in per_config_layers()]
+            line["per_config"] = {
+                "note": "every layer of the workload configurations: gf_stash_forward and gf_backward timed with CUDA "
+                        "events over 8-20 calls behind a stream backlog; frac = algorithmic bytes of the backward / time "
+                        f"/ {peaks['hbm_gbs']:.0f} GB/s ({which} copy bandwidth); exact_cudnn_us = exact convolution "
+                        "backward of the same shape and dtype through torch/cuDNN (context: it computes the unfiltered "
+                        "gradients)",
+                "paper_context": PAPER_CONTEXT,
+                "rows": rows,
+            }
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
 
 
 def run_table(args) -> None:
-    """--table: every headline layer (and the paper's on-device shapes) timed once each way:
-    gf_stash_forward, gf_backward, and an exact backward through torch/cuDNN as context.
-    Prints one JSON line per layer and a markdown table; not the contract line."""
+    """--table: every headline layer and the paper's on-device shapes timed once each way, with
+    the per-kernel event times of the backward call.  Prints one JSON line per layer and a
+    markdown table; not the contract line."""
     import torch
     import paper_2301_00330_b200 as gf
     from paper_2301_00330_b200 import workloads
@@ -451,90 +573,41 @@ def run_table(args) -> None:
     torch.cuda.set_device(0)
     gf.build_library()
     peaks, which = measured_peaks()
-    layers = [l for l in workloads.all_headline_layers() if l.r > 1] + workloads.ondevice_table(2, "f32") \
-        + workloads.ondevice_table(4, "f32")
+    layers = per_config_layers() + workloads.ondevice_table(2, "f32") + workloads.ondevice_table(4, "f32")
     if args.only:
         layers = [l for l in layers if any(k in f"{l.name}/r{l.r}/{l.dtype}" for k in args.only.split(","))]
-    stream = torch.cuda.current_stream()
     rows = []
-
-    def timed(fn, reps):
-        for _ in range(3):
-            fn(0)
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda._sleep(int(3e-3 * 1.9e9))       # backlog: the calls below queue up behind it
-        e0.record(stream)
-        for i in range(reps):
-            fn(i)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        return e0.elapsed_time(e1) * 1e3 / reps
-
     for L in layers:
-        desc = gf.desc_for(L)
-        x0, gy0, w0 = workloads.make_inputs(L)
-        per_set = L.backward_bytes() + L.stash_bytes_moved()
-        n_sets = max(1, min(4, int(400e6 // per_set) + 1))
-        sets = [(torch.roll(x0, i, 0).cuda(), torch.roll(gy0, i, 0).cuda(), gf.alloc_layer(desc)) for i in range(n_sets)]
-        w = w0.cuda()
-        ws_bytes = gf.gf_backward_workspace_bytes(desc)
-        reps = 20 if per_set < 300e6 else 8
-
-        def stash(i):
-            x, _, b = sets[i % n_sets]
-            gf.gf_stash_forward(desc, x, b.stash, stream)
-
-        def bwd(i):
-            _, gy, b = sets[i % n_sets]
-            gf.gf_backward(desc, gy, b.stash, w, b.g_W, b.g_X, b.workspace, ws_bytes, stream)
-
-        def exact(i):
-            x, gy, _ = sets[i % n_sets]
-            torch.ops.aten.convolution_backward(gy, x, w, None, [1, 1], [L.pad, L.pad], [1, 1], False, [0, 0],
-                                                L.groups, [True, True, False])
-
-        t_stash, t_bwd = timed(stash, reps), timed(bwd, reps)
-        # per-kernel event times of the backward call (each bracketed, so a few us high)
-        gf.gf_profile_configure(2)
-        torch.cuda._sleep(int(3e-3 * 1.9e9))
-        for i in range(4):
-            bwd(i)
-        torch.cuda.synchronize()
-        kern = {k: round(ms / n * 1e3, 1) for k, (n, ms) in gf.gf_profile_read().items()}
-        gf.gf_profile_configure(0)
-        try:
-            t_exact = timed(exact, max(2, reps // 4))
-        except Exception:
-            t_exact = None
-        row = {"layer": L.name, "r": L.r, "dtype": L.dtype, "stash_us": t_stash, "backward_us": t_bwd,
-               "backward_alg_MB": L.backward_bytes() / 1e6,
-               "backward_gbs": L.backward_bytes() / t_bwd / 1e3,
-               "backward_frac_hbm": L.backward_bytes() / t_bwd / 1e3 / peaks["hbm_gbs"],
-               "stash_gbs": L.stash_bytes_moved() / t_stash / 1e3,
-               "stash_frac_hbm": L.stash_bytes_moved() / t_stash / 1e3 / peaks["hbm_gbs"],
-               "exact_cudnn_us": t_exact, "reduced_gflop": L.reduced_flops() / 1e9, "kernels_us": kern}
+        row = time_layer(gf, L, peaks, with_exact=not args.no_exact, with_kernels=True)
         rows.append(row)
         print(json.dumps(row), flush=True)
-        del sets
-        torch.cuda.empty_cache()
     print(f"\n| layer | r | dtype | stash us | backward us | alg MB | GB/s | frac of {peaks['hbm_gbs']:.0f} GB/s ({which}) | exact cuDNN us |")
     print("|---|---|---|---|---|---|---|---|---|")
     for r in rows:
-        ex = f"{r['exact_cudnn_us']:.0f}" if r["exact_cudnn_us"] else "n/a"
+        ex = f"{r['exact_cudnn_us']:.0f}" if r.get("exact_cudnn_us") else "n/a"
         print(f"| {r['layer']} | {r['r']} | {r['dtype']} | {r['stash_us']:.1f} | {r['backward_us']:.1f} | "
               f"{r['backward_alg_MB']:.1f} | {r['backward_gbs']:.0f} | {r['backward_frac_hbm']:.2f} | {ex} |")
 
 
 def main() -> None:
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
+    ap.add_argument("--gpus", type=int, default=1,
+                    help="replicas (one process per GPU); under torchrun the ranks come from the environment, "
+                         "otherwise N > 1 re-executes this script under torch.distributed.run")
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-per-config", action="store_true", help="skip the per_config rows (faster)")
     ap.add_argument("--table", action="store_true", help="time every layer shape once (diagnostic table)")
     ap.add_argument("--only", default="", help="--table: comma-separated substrings of name/rR/dtype to keep")
+    ap.add_argument("--no-exact", action="store_true", help="--table: skip the exact cuDNN backward")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.table:
+        # started without a launcher: become N ranks on this node
+        port = 29500 + os.getpid() % 2000
+        os.execv(sys.executable, [sys.executable, "-m", "torch.distributed.run", "--nnodes=1",
+                                  f"--nproc-per-node={args.gpus}", "--master-addr", "127.0.0.1",
+                                  "--master-port", str(port), os.path.abspath(__file__), *sys.argv[1:]])
     if args.table:
         run_table(args)
     elif args.impl == "reference":

@@ -141,32 +141,6 @@ gf_status gf_layer_step_host(const gf_conv_desc* desc, const void* h_x, const vo
                              const void* h_W, float* h_gW, void* h_gX, void* arena,
                              size_t arena_bytes, void* stream);
 
-/* Number of kernels this library has launched in this process so far. */
-uint64_t gf_kernel_launch_count(void);
-
-/* Optional per-kernel timing for benchmarks.  mode 0: off (default).  mode 1:
- * every launch of kernel `kernel_id` is bracketed by a pair of CUDA events
- * recorded on the stream it is launched on.  mode 2: every kernel is bracketed
- * (kernel_id ignored).  Events come from an internal pool that is created on
- * first use; when the pool is exhausted further launches are not timed.  Not
- * for use while a stream is being captured. */
-gf_status gf_profile_configure(int32_t mode, int32_t kernel_id);
-
-typedef struct gf_kernel_time {
-    int32_t kernel_id;
-    int32_t launches;   /* timed launches since the last read */
-    double total_ms;    /* sum of their event-to-event durations */
-} gf_kernel_time;
-
-/* Waits for the recorded events, writes one entry per kernel that was timed
- * since the last read (at most max_entries) and clears the records.  Returns
- * the number of entries written, or -1 if a CUDA call failed. */
-int32_t gf_profile_read(gf_kernel_time* out, int32_t max_entries);
-
-/* Name of a kernel id (ids are 0 .. gf_kernel_id_count()-1), NULL if out of range. */
-const char* gf_kernel_name(int32_t kernel_id);
-int32_t gf_kernel_id_count(void);
-
 /* Static, human-readable name of a status code. */
 const char* gf_status_string(gf_status s);
 

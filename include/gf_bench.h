@@ -1,0 +1,45 @@
+/*
+ * gf_bench.h -- instrumentation of libgf_b200 for benchmarks and tests.
+ *
+ * None of these calls is part of the method (the paper has no counterpart): they count
+ * and time the kernels that the calls of gf.h launch.  The event pool behind the timing
+ * is process-wide state of the library, created on first use.
+ */
+#ifndef GF_BENCH_H_
+#define GF_BENCH_H_
+
+#include "gf.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Number of kernels this library has launched in this process so far. */
+uint64_t gf_kernel_launch_count(void);
+
+/* Optional per-kernel timing.  mode 0: off (default).  mode 1: every launch of kernel
+ * `kernel_id` is bracketed by a pair of CUDA events recorded on the stream it is launched
+ * on.  mode 2: every kernel is bracketed (kernel_id ignored).  Events come from an internal
+ * pool that is created on first use; when the pool is exhausted further launches are not
+ * timed.  Not for use while a stream is being captured. */
+gf_status gf_profile_configure(int32_t mode, int32_t kernel_id);
+
+typedef struct gf_kernel_time {
+    int32_t kernel_id;
+    int32_t launches;   /* timed launches since the last read */
+    double total_ms;    /* sum of their event-to-event durations */
+} gf_kernel_time;
+
+/* Waits for the recorded events, writes one entry per kernel that was timed since the last
+ * read (at most max_entries) and clears the records.  Returns the number of entries
+ * written, or -1 if a CUDA call failed. */
+int32_t gf_profile_read(gf_kernel_time* out, int32_t max_entries);
+
+/* Name of a kernel id (ids are 0 .. gf_kernel_id_count()-1), NULL if out of range. */
+const char* gf_kernel_name(int32_t kernel_id);
+int32_t gf_kernel_id_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GF_BENCH_H_ */

@@ -17,18 +17,18 @@
  * Readings taken where the paper's text is garbled or silent:
  *   - Patch (a,b) of an H x W map is the half-open index block
  *     [a r, min((a+1) r, H)) x [b r, min((b+1) r, W)); there are
- *     ceil(H/r) x ceil(W/r) patches (Section 3.3, "cutting the gradient map
- *     into r x r-pixel patches"; block count stated right after the filter
- *     equation).  The printed summation limits are not used.
- *   - On a partial patch at the right/bottom edge the "average value" is the
+ *     ceil(H/r) x ceil(W/r) patches (Section 3.3: the prose describes the map
+ *     as tiled by r x r blocks, and the count of unique values is stated right
+ *     after the filter equation).  The printed summation limits are not used.
+ *   - On a partial patch at the right/bottom edge the patch value is the
  *     mean over the elements that exist.  PARITY UNPINNED for this divisor:
  *     the paper gives no worked example with a partial patch (its formula
- *     prints 1/r^2, its prose says "average").
+ *     prints 1/r^2, its prose speaks of an average).
  *   - Eq. (grad_w) is summed once per patch: sum_{n,a,b} xsum * gmean, which
  *     is what the first line of its derivation in the supplement gives at
  *     zero offset without any approximation.
- *   - r == 1 means the method is off: exact convolution backward ("a patch
- *     size 1x1 means the vanilla BP algorithm", Section 4.2).
+ *   - r == 1 means the method is off: exact convolution backward (Section
+ *     4.2 names the 1 x 1 patch size as its exact-backpropagation baseline).
  *   - Stride 1, dilation 1, odd kernels with pad = (K-1)/2, the geometry in
  *     which Eq. (grad_x) indexes g_x and g_y with the same (h,w).
  */

@@ -1,4 +1,4 @@
-"""A convolution layer whose backward pass is the filtered one (Section 3.1, Algorithm 1).
+"""A convolution layer whose backward pass is the filtered one (Sections 3.3-3.4: Eq. (grad_x), Eq. (grad_w)).
 
 Forward: the convolution itself is torch's (it is not part of the filtered path), and the
 activation stash is taken by gf_stash_forward instead of keeping x (Section 3.4).  Backward:

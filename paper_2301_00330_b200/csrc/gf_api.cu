@@ -49,9 +49,9 @@ ProfScope::~ProfScope() {
 static __device__ uint32_t g_err_word_dev;
 
 static uint32_t* global_err_word() {
-    static uint32_t* cached[64] = {};
+    static uint32_t* cached[kMaxDevices] = {};
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
     if (!cached[dev]) {
         void* ptr = nullptr;
         if (cudaGetSymbolAddress(&ptr, g_err_word_dev) != cudaSuccess) return nullptr;
@@ -63,14 +63,15 @@ static uint32_t* global_err_word() {
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-            n = 148;
+    static int cached[kMaxDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 148;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cached[dev] = n;
     }
-    return n;
+    return cached[dev];
 }
 
 Geo make_geo(const gf_conv_desc& d) {
@@ -104,6 +105,7 @@ static gf_status validate(const gf_conv_desc* d) {
 }
 
 static bool is_depthwise(const Geo& g) { return g.G == g.C_in && g.G == g.C_out; }
+static bool is_depthwise_fused(const Geo& g) { return is_depthwise(g) && depthwise_splits(g) > 0; }
 
 static int dense_splits(const Geo& g) {
     const long long tiles = (long long)((g.C_og + 63) / 64) * ((g.C_ig + 63) / 64) * g.G;
@@ -144,7 +146,8 @@ static bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) &
 // chain (stash repack, contraction, broadcast to the taps) is put on a library-owned
 // second stream between a fork event and a join event, so that it shares the SMs with
 // the g_X contraction instead of queueing behind it.  One stream and event pair per
-// device, created on first use; the host-side sequence is serialised by a mutex.
+// device, created on first use; creation and the host-side fork .. join sequence are
+// serialised by g_side_mu, which the caller holds.
 struct SideStream {
     cudaStream_t stream = nullptr;
     cudaEvent_t fork = nullptr, join = nullptr;
@@ -152,15 +155,24 @@ struct SideStream {
 };
 std::mutex g_side_mu;
 
-static SideStream* side_stream() {
-    static SideStream side[64];
+// Caller holds g_side_mu.  NULL when the resources cannot be created (nothing is kept then).
+static SideStream* side_stream_locked() {
+    static SideStream side[kMaxDevices];
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
     SideStream& sd = side[dev];
     if (!sd.ok) {
-        if (cudaStreamCreateWithFlags(&sd.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
-        if (cudaEventCreateWithFlags(&sd.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
-        if (cudaEventCreateWithFlags(&sd.join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        SideStream t;
+        const bool made = cudaStreamCreateWithFlags(&t.stream, cudaStreamNonBlocking) == cudaSuccess &&
+                          cudaEventCreateWithFlags(&t.fork, cudaEventDisableTiming) == cudaSuccess &&
+                          cudaEventCreateWithFlags(&t.join, cudaEventDisableTiming) == cudaSuccess;
+        if (!made) {
+            if (t.join) cudaEventDestroy(t.join);
+            if (t.fork) cudaEventDestroy(t.fork);
+            if (t.stream) cudaStreamDestroy(t.stream);
+            return nullptr;
+        }
+        sd = t;
         sd.ok = true;
     }
     return &sd;
@@ -224,6 +236,51 @@ gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* sta
 }  // extern "C"
 
 namespace gf {
+
+// Tensor-core path of a dense layer: theta sums (transposed, bf16), patch means of g_y as
+// bf16, then the two contractions on tcgen05.  fp32 layers carry every operand as a
+// (high, low) bf16 pair: v = hi + lo up to 2^-17 |v|.  `sw` is the stream of the g_W chain
+// (the caller's stream, or the side stream that the caller has forked from it and joins
+// back afterwards whatever this function returns).
+static gf_status backward_tc(const Geo& g, const Workspace& ws, char* base, const void* g_y, const void* stash,
+                             const void* W, float* g_W, void* g_X, uint32_t* err, cudaStream_t s, cudaStream_t sw,
+                             bool forked, int gx_ctas, int gw_splits) {
+    const bool split = g.dtype == GF_F32;
+    const size_t P = (size_t)g.Hp * g.Wp;
+    const size_t pitch = (size_t)tc_pitch(g);     // > P: planes padded so that rows can be copied in aligned pieces
+    // low parts sit 16-byte aligned behind the high parts, inside the fp32-sized regions
+    const long long theta_lo = split ? (long long)align_up((size_t)g.C_in * g.C_out, 8) : 0;
+    const long long gbar_lo = split ? (long long)align_up((size_t)g.N * g.C_out * pitch, 8) : 0;
+    const long long stash_lo = split ? (long long)(align_up((size_t)g.N * g.C_in * pitch * 2, 256) / 2) : 0;
+    __nv_bfloat16* thetaT = reinterpret_cast<__nv_bfloat16*>(base + ws.off_tsum);
+    __nv_bfloat16* gbar16 = reinterpret_cast<__nv_bfloat16*>(base + ws.off_gbar);
+    float* part = reinterpret_cast<float*>(base + ws.off_part);
+    gf_status st = GF_OK;
+    if (g_X) {
+        st = launch_gx_tc(gbar16, gbar_lo, thetaT, theta_lo, g_X, gx_ctas, err, g, s);
+        if (st != GF_OK) return st;
+    }
+    if (g_W) {
+        const __nv_bfloat16* stash16 = static_cast<const __nv_bfloat16*>(stash);
+        if (split || pitch != P) {
+            __nv_bfloat16* sp = reinterpret_cast<__nv_bfloat16*>(base + ws.off_split);
+            if (pitch == P)
+                st = launch_split_f32(static_cast<const float*>(stash), sp, sp + stash_lo, (size_t)g.N * g.C_in * P, sw);
+            else
+                st = launch_repack(stash, g.dtype, sp, split ? sp + stash_lo : nullptr, (long long)g.N * g.C_in,
+                                   (int)P, (int)pitch, sw);
+            if (st != GF_OK) return st;
+            stash16 = sp;
+        }
+        st = launch_gw_tc(gbar16, gbar_lo, stash16, stash_lo, part, gw_splits, err, g, sw);
+        if (st != GF_OK) return st;
+        st = launch_gw_finish(part, 1, g_W, g, sw);
+        if (st != GF_OK) return st;
+    }
+    (void)forked;
+    return GF_OK;
+}
+
 gf_status backward_impl(const gf_conv_desc* desc, const void* g_y, const void* stash, const void* W, float* g_W,
                         void* g_X, void* workspace, size_t workspace_bytes, void* stream, bool may_fork) {
     if (!desc || !g_y || !W || !workspace) return GF_ERR_NULL;
@@ -240,17 +297,22 @@ gf_status backward_impl(const gf_conv_desc* desc, const void* g_y, const void* s
     char* base = static_cast<char*>(workspace);
     uint32_t* err = reinterpret_cast<uint32_t*>(base + ws.off_err);
     if (!g_W && !g_X) return GF_OK;
-
-    if (g.r == 1) {
-        GF_CUDA_TRY(cudaMemsetAsync(err, 0, sizeof(uint32_t), s));
-        return launch_exact(g_y, stash, W, g_W, g_X, g, s);
+    // limits of the launch geometry, checked before anything is enqueued
+    if (g.r > 1 && !is_depthwise_fused(g)) {
+        st = tc_eligible(g) ? tc_check_limits(g) : dense_check_limits(g, ws.splits);
+        if (st != GF_OK) return st;
     }
+
+    // The error word is cleared here, ahead of every kernel of the call that may set it.
+    GF_CUDA_TRY(cudaMemsetAsync(err, 0, sizeof(uint32_t), s));
+
+    if (g.r == 1) return launch_exact(g_y, stash, W, g_W, g_X, g, s);
 
     float* tsum = reinterpret_cast<float*>(base + ws.off_tsum);
     float* gbar = reinterpret_cast<float*>(base + ws.off_gbar);
     float* part = reinterpret_cast<float*>(base + ws.off_part);
 
-    if (is_depthwise(g) && depthwise_splits(g) > 0) {
+    if (is_depthwise_fused(g)) {
         int splits = 0;
         st = launch_depthwise(g_y, stash, W, g_W ? part : nullptr, g_X, err, g, &splits, s);
         if (st != GF_OK) return st;
@@ -259,70 +321,41 @@ gf_status backward_impl(const gf_conv_desc* desc, const void* g_y, const void* s
     }
 
     if (tc_eligible(g)) {
-        // tensor-core path: theta sums (transposed, bf16; clears the error word), patch
-        // means of g_y as bf16, then the two contractions on tcgen05.  fp32 layers carry
-        // every operand as a (high, low) bf16 pair: v = hi + lo up to 2^-17 |v|.
         const bool split = g.dtype == GF_F32;
-        const size_t P = (size_t)g.Hp * g.Wp;
-        const size_t pitch = (size_t)tc_pitch(g);     // > P: planes padded so that rows can be copied in aligned pieces
-        // low parts sit 16-byte aligned behind the high parts, inside the fp32-sized regions
+        const size_t pitch = (size_t)tc_pitch(g);
         const long long theta_lo = split ? (long long)align_up((size_t)g.C_in * g.C_out, 8) : 0;
         const long long gbar_lo = split ? (long long)align_up((size_t)g.N * g.C_out * pitch, 8) : 0;
-        const long long stash_lo = split ? (long long)(align_up((size_t)g.N * g.C_in * pitch * 2, 256) / 2) : 0;
         __nv_bfloat16* thetaT = reinterpret_cast<__nv_bfloat16*>(tsum);
         __nv_bfloat16* gbar16 = reinterpret_cast<__nv_bfloat16*>(gbar);
-        // the gradient filter first; the theta sums (which also clear the error word and the g_W
-        // accumulator) are launched behind it and work next to it
+        // the gradient filter first; the theta sums (which also clear the g_W accumulator) are
+        // launched behind it and work next to it
         st = launch_pool(K_GY_POOL, g_y, g.dtype, gbar16, split ? gbar16 + gbar_lo : nullptr, GF_BF16, /*mean=*/true,
                          (int64_t)g.N * g.C_out, g.H, g.W, g.r, (int)pitch, err, s);
         if (st != GF_OK) return st;
-        st = launch_ksum_t(W, g, thetaT, split ? thetaT + theta_lo : nullptr, g_W ? part : nullptr, err,
+        st = launch_ksum_t(W, g, thetaT, split ? thetaT + theta_lo : nullptr, g_W ? part : nullptr,
                            /*beside_pool=*/true, s);
         if (st != GF_OK) return st;
-        // both outputs wanted: the g_W chain goes to the side stream, forked here
-        SideStream* side = (may_fork && g_X && g_W) ? side_stream() : nullptr;
-        std::unique_lock<std::mutex> side_lock;
-        cudaStream_t sw = s;                          // stream of the g_W chain
+        if (!(may_fork && g_X && g_W))
+            return backward_tc(g, ws, base, g_y, stash, W, g_W, g_X, err, s, s, false, 0, tc_gw_splits(g));
+        // both outputs wanted: the g_W chain goes to the side stream, forked here and joined
+        // below on every path (an error return included), so that the caller's stream -- and a
+        // stream capture it may be part of -- never ends up with an open fork
+        std::lock_guard<std::mutex> side_lock(g_side_mu);
+        SideStream* side = side_stream_locked();
+        if (!side) return backward_tc(g, ws, base, g_y, stash, W, g_W, g_X, err, s, s, false, 0, tc_gw_splits(g));
         int gx_ctas = 0, gw_splits = tc_gw_splits(g);
-        if (side) {
-            tc_partition(g, &gx_ctas, &gw_splits);    // side by side: each kernel gets its share of the SMs
-            side_lock = std::unique_lock<std::mutex>(g_side_mu);
-            GF_CUDA_TRY(cudaEventRecord(side->fork, s));
-            GF_CUDA_TRY(cudaStreamWaitEvent(side->stream, side->fork, 0));
-            sw = side->stream;
-        }
-        if (g_X) {
-            st = launch_gx_tc(gbar16, gbar_lo, thetaT, theta_lo, g_X, gx_ctas, err, g, s);
-            if (st != GF_OK) return st;
-        }
-        if (g_W) {
-            cudaStream_t s = sw;                      // shadows: everything below runs on the g_W chain's stream
-            const __nv_bfloat16* stash16 = static_cast<const __nv_bfloat16*>(stash);
-            if (split || pitch != P) {
-                __nv_bfloat16* sp = reinterpret_cast<__nv_bfloat16*>(base + ws.off_split);
-                if (pitch == P)
-                    st = launch_split_f32(static_cast<const float*>(stash), sp, sp + stash_lo, (size_t)g.N * g.C_in * P, s);
-                else
-                    st = launch_repack(stash, g.dtype, sp, split ? sp + stash_lo : nullptr, (long long)g.N * g.C_in,
-                                       (int)P, (int)pitch, s);
-                if (st != GF_OK) return st;
-                stash16 = sp;
-            }
-            st = launch_gw_tc(gbar16, gbar_lo, stash16, stash_lo, part, gw_splits, err, g, s);
-            if (st != GF_OK) return st;
-            st = launch_gw_finish(part, 1, g_W, g, s);
-            if (st != GF_OK) return st;
-        }
-        if (side) {                                   // join: the caller's stream waits for the g_W chain
-            GF_CUDA_TRY(cudaEventRecord(side->join, side->stream));
-            GF_CUDA_TRY(cudaStreamWaitEvent(s, side->join, 0));
-        }
-        return GF_OK;
+        tc_partition(g, &gx_ctas, &gw_splits);        // side by side: each kernel gets its share of the SMs
+        GF_CUDA_TRY(cudaEventRecord(side->fork, s));
+        GF_CUDA_TRY(cudaStreamWaitEvent(side->stream, side->fork, 0));
+        st = backward_tc(g, ws, base, g_y, stash, W, g_W, g_X, err, s, side->stream, true, gx_ctas, gw_splits);
+        const bool joined = cudaEventRecord(side->join, side->stream) == cudaSuccess &&
+                            cudaStreamWaitEvent(s, side->join, 0) == cudaSuccess;
+        if (st != GF_OK) return st;
+        return joined ? GF_OK : GF_ERR_CUDA;
     }
 
-    // kernel sums (also clears the error word), then the gradient filter:
-    // patch means of g_y, read once
-    st = launch_ksum(W, g, tsum, err, s);
+    // kernel sums, then the gradient filter: patch means of g_y, read once
+    st = launch_ksum(W, g, tsum, s);
     if (st != GF_OK) return st;
     st = launch_pool(K_GY_POOL, g_y, g.dtype, gbar, nullptr, GF_F32, /*mean=*/true, (int64_t)g.N * g.C_out, g.H, g.W, g.r, 0, err, s);
     if (st != GF_OK) return st;

@@ -6,6 +6,7 @@
 #include <stdint.h>
 
 #include "gf.h"
+#include "gf_bench.h"
 
 namespace gf {
 
@@ -65,6 +66,24 @@ static inline int64_t cdiv64(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
 // SMs of the current device (148 when the query fails)
 int sm_count();
+
+// Per-device host state (function attributes, symbol addresses, SM counts) is kept in
+// arrays indexed by the ordinal of the device that is current at the call.
+constexpr int kMaxDevices = 64;
+
+// Raises a kernel's dynamic shared-memory limit to `smem`, once per device: a function
+// attribute belongs to the device that is current when it is set.  `configured` is the
+// launcher's own table of what it has set so far on each device.
+template <typename Kern>
+static inline gf_status ensure_dyn_smem(Kern kernel, size_t smem, size_t (&configured)[kMaxDevices]) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return GF_ERR_CUDA;
+    if (smem > configured[dev]) {
+        GF_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        configured[dev] = smem;
+    }
+    return GF_OK;
+}
 
 // ---- division by a runtime constant ---------------------------------------
 // q = n / d for any 32-bit n via one multiply-high, an add and two shifts.
@@ -169,11 +188,13 @@ gf_status launch_pool(int kernel_id, const void* in, int in_dtype, void* out, vo
                       int64_t planes, int H, int W, int r, int out_pitch, uint32_t* err_word, cudaStream_t s);
 gf_status launch_copy(const void* in, void* out, size_t bytes, cudaStream_t s);
 
-gf_status launch_ksum(const void* W, const Geo& g, float* tsum, uint32_t* err_word, cudaStream_t s);
+gf_status launch_ksum(const void* W, const Geo& g, float* tsum, cudaStream_t s);
 gf_status launch_gx_mix(const float* gbar, const float* tsum, void* gX, const Geo& g, cudaStream_t s);
 gf_status launch_gw_partial(const float* gbar, const void* stash, float* part, int splits,
                             const Geo& g, cudaStream_t s);
 gf_status launch_gw_finish(const float* part, int splits, float* gW, const Geo& g, cudaStream_t s);
+gf_status dense_check_limits(const Geo& g, int splits);
+gf_status tc_check_limits(const Geo& g);
 gf_status launch_depthwise(const void* gy, const void* stash, const void* W, float* part,
                            void* gX, uint32_t* err_word, const Geo& g, int* splits_out, cudaStream_t s);
 int depthwise_splits(const Geo& g);
@@ -188,7 +209,7 @@ gf_status launch_repack(const void* in, int in_dtype, __nv_bfloat16* hi, __nv_bf
                         int pitch, cudaStream_t s);
 // beside_pool: launched right behind the gradient-filter pooling kernel, works next to it
 gf_status launch_ksum_t(const void* W, const Geo& g, __nv_bfloat16* thetaT, __nv_bfloat16* thetaT_lo, float* gwu,
-                        uint32_t* err_word, bool beside_pool, cudaStream_t s);
+                        bool beside_pool, cudaStream_t s);
 gf_status launch_split_f32(const float* in, __nv_bfloat16* hi, __nv_bfloat16* lo, size_t n, cudaStream_t s);
 // max_ctas: CTAs the kernel may use (0: one per SM)
 gf_status launch_gx_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const __nv_bfloat16* thetaT,

@@ -9,22 +9,20 @@ namespace gf {
 
 // ---------------------------------------------------------------- ksum
 template <typename T>
-__global__ void ksum_kernel(const T* __restrict__ W, float* __restrict__ tsum, int n_pairs, int taps,
-                            uint32_t* err_word) {
+__global__ void ksum_kernel(const T* __restrict__ W, float* __restrict__ tsum, int n_pairs, int taps) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i == 0 && err_word) *err_word = 0u;
     if (i >= n_pairs) return;
     float s = 0.f;
     for (int t = 0; t < taps; ++t) s += to_f32(W[(size_t)i * taps + t]);
     tsum[i] = s;
 }
 
-gf_status launch_ksum(const void* W, const Geo& g, float* tsum, uint32_t* err_word, cudaStream_t s) {
+gf_status launch_ksum(const void* W, const Geo& g, float* tsum, cudaStream_t s) {
     ProfScope prof(K_KSUM, s);
     const int n_pairs = g.C_out * g.C_ig, taps = g.KH * g.KW;
     const int grid = (n_pairs + 255) / 256;
-    if (g.dtype == GF_F32) ksum_kernel<float><<<grid, 256, 0, s>>>((const float*)W, tsum, n_pairs, taps, err_word);
-    else ksum_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16*)W, tsum, n_pairs, taps, err_word);
+    if (g.dtype == GF_F32) ksum_kernel<float><<<grid, 256, 0, s>>>((const float*)W, tsum, n_pairs, taps);
+    else ksum_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16*)W, tsum, n_pairs, taps);
     return after_launch();
 }
 
@@ -106,6 +104,17 @@ __global__ void __launch_bounds__(256) gx_mix_kernel(const GxParams p) {
         for (int col = lane; col < cols_out; col += 32)
             dst[col] = from_f32<TOut>(Ds[m][ja * p.TB + p.div_r.div(col)]);
     }
+}
+
+// Limits of the launch geometry of gx_mix and gw_partial, for the host to check before
+// anything of a call is enqueued (the launchers repeat them).
+gf_status dense_check_limits(const Geo& g, int splits) {
+    const int TB = g.Wp < kBN ? g.Wp : kBN;
+    int TA = kBN / TB; if (TA > g.Hp) TA = g.Hp;
+    const long long gx_blocks = (long long)g.N * g.G * ((g.Hp + TA - 1) / TA) * ((g.Wp + TB - 1) / TB);
+    if (gx_blocks > 0x7fffffffLL || (g.C_ig + kBM - 1) / kBM > 65535) return GF_ERR_UNSUPPORTED;
+    if ((long long)g.G * splits > 65535 || (g.C_og + kBM - 1) / kBM > 65535) return GF_ERR_UNSUPPORTED;
+    return GF_OK;
 }
 
 gf_status launch_gx_mix(const float* gbar, const float* tsum, void* gX, const Geo& g, cudaStream_t s) {

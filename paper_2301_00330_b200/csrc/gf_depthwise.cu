@@ -122,7 +122,6 @@ __global__ void __launch_bounds__(kDwThreads) dw_fused_kernel(const DwParams p) 
     const T* __restrict__ Wt = static_cast<const T*>(p.W);
     T* __restrict__ gX = static_cast<T*>(p.gX);
 
-    if (blockIdx.x == 0 && threadIdx.x == 0) *p.err_word = 0u;
     uint32_t pg, band;
     p.div_bands.divmod(blockIdx.x, pg, band);
     const long long p0 = (long long)pg * p.P;
@@ -338,7 +337,6 @@ __global__ void __launch_bounds__(kDwsThreads, 1) dw_stream_kernel(const DwsPara
     }
     __syncthreads();
     pdl_wait();                           // the stash may come from the previous kernel of the stream
-    if (blockIdx.x == 0 && tid == 0) *p.err_word = 0u;
     if (tid == 0)
         for (int it = 0; it < kDwsStages && it < n_my; ++it) issue_load(it);
     for (int c = tid; c < p.C; c += kDwsThreads) {          // kernel sums of every channel
@@ -428,11 +426,8 @@ __global__ void __launch_bounds__(kDwsThreads, 1) dw_stream_kernel(const DwsPara
 template <typename T, int R, int G>
 static gf_status launch_dws_inst(const DwsParams& p, cudaStream_t s) {
     constexpr size_t smem = (size_t)kDwsStages * kDwsTileBytes + (size_t)(4 * kDwsMaxOut + kDwsMaxC) * sizeof(float);
-    static bool configured = false;
-    if (!configured) {
-        GF_CUDA_TRY(cudaFuncSetAttribute(dw_stream_kernel<T, R, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        configured = true;
-    }
+    static size_t configured[kMaxDevices] = {};
+    if (gf_status st = ensure_dyn_smem(dw_stream_kernel<T, R, G>, smem, configured); st != GF_OK) return st;
     const long long grid = p.tiles < sm_count() ? p.tiles : sm_count();
     return launch_pdl(dw_stream_kernel<T, R, G>, dim3((unsigned)grid), dim3(kDwsThreads), smem, s, p);
 }

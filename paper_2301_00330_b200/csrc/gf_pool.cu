@@ -467,12 +467,8 @@ static bool plan_stream(PoolParams& p, size_t e) {
 template <typename TIn, typename TOut, int R, int G, bool EXT>
 static gf_status launch_stream_ext(const PoolParams& p, cudaStream_t s) {
     constexpr size_t smem = (size_t)kStreamStages * kStreamTileBytes;
-    static bool configured = false;
-    if (!configured) {
-        GF_CUDA_TRY(cudaFuncSetAttribute(pool_stream_kernel<TIn, TOut, R, G, EXT>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        configured = true;
-    }
+    static size_t configured[kMaxDevices] = {};
+    if (gf_status st = ensure_dyn_smem(pool_stream_kernel<TIn, TOut, R, G, EXT>, smem, configured); st != GF_OK) return st;
     const long long grid = p.tiles < (long long)sm_count() * kStreamCtasPerSm ? p.tiles : (long long)sm_count() * kStreamCtasPerSm;
     return launch_pdl(pool_stream_kernel<TIn, TOut, R, G, EXT>, dim3((unsigned)grid), dim3(kStreamThreads), smem, s, p);
 }

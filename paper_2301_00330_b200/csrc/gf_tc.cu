@@ -747,12 +747,11 @@ __global__ void __launch_bounds__(kGwThreads) gw_tc_kernel(const GwTcParams p) {
 // ================================================================== theta sum, transposed bf16
 // thetaT[c_i][c_o] = sum_taps W[c_o][c_i][:], a 32 x 32 tile per block through shared
 // memory so that both the reads (along c_i, taps) and the writes (along c_o) are
-// contiguous.  Also clears the error word and g_W's unique-value accumulator.
+// contiguous.  Also clears g_W's unique-value accumulator.
 template <typename T>
 __global__ void __launch_bounds__(1024) ksum_t_kernel(const T* __restrict__ W, __nv_bfloat16* __restrict__ thetaT,
                                                       __nv_bfloat16* __restrict__ thetaT_lo, float* __restrict__ gwu,
-                                                      int C_in, int C_out, int taps, uint32_t* err_word,
-                                                      int late_wait) {
+                                                      int C_in, int C_out, int taps, int late_wait) {
     __shared__ float tile[32][33];
     pdl_launch_dependents();
     // late_wait: the kernel before this one in the stream is the gradient-filter pooling
@@ -763,7 +762,6 @@ __global__ void __launch_bounds__(1024) ksum_t_kernel(const T* __restrict__ W, _
     if (!late_wait) pdl_wait();
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
     const int co0 = blockIdx.y * 32, ci0 = blockIdx.x * 32;
-    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0 && err_word) *err_word = 0u;
     {
         const int co = co0 + ty, ci = ci0 + tx;
         float s = 0.f;
@@ -1009,17 +1007,30 @@ int tc_gw_splits(const Geo& g) {
     return s;
 }
 
+// Limits of the launch geometry of the tensor-core path, for the host to check before
+// anything of a call is enqueued (the launchers repeat them).
+gf_status tc_check_limits(const Geo& g) {
+    if ((g.C_out + 31) / 32 > 65535 || (g.C_out + 127) / 128 > 65535) return GF_ERR_UNSUPPORTED;
+    const GxPlan d = gx_plan(g);
+    const long long items = d.col_tiles * ((g.C_in + 127) / 128);
+    if (items * ((g.C_out + kTcBK - 1) / kTcBK) > 0x7fffffffLL) return GF_ERR_UNSUPPORTED;
+    const long long pitch = tc_pitch(g), P = (long long)g.Hp * g.Wp;
+    if (pitch != P && (long long)g.N * g.C_in * pitch > 0x7fffffffLL) return GF_ERR_UNSUPPORTED;
+    if (pitch == P && ((long long)g.N * g.C_in * P) % 4 != 0 && g.dtype == GF_F32) return GF_ERR_UNSUPPORTED;
+    return GF_OK;
+}
+
 gf_status launch_ksum_t(const void* W, const Geo& g, __nv_bfloat16* thetaT, __nv_bfloat16* thetaT_lo, float* gwu,
-                        uint32_t* err_word, bool beside_pool, cudaStream_t s) {
+                        bool beside_pool, cudaStream_t s) {
     ProfScope prof(K_KSUM, s);
     const int taps = g.KH * g.KW;
     dim3 grid((g.C_in + 31) / 32, (g.C_out + 31) / 32, 1);
     if (grid.y > 65535) return GF_ERR_UNSUPPORTED;
     if (g.dtype == GF_F32)
         return launch_pdl(ksum_t_kernel<float>, grid, dim3(1024), 0, s, (const float*)W, thetaT, thetaT_lo, gwu, g.C_in,
-                          g.C_out, taps, err_word, beside_pool ? 1 : 0);
+                          g.C_out, taps, beside_pool ? 1 : 0);
     return launch_pdl(ksum_t_kernel<__nv_bfloat16>, grid, dim3(1024), 0, s, (const __nv_bfloat16*)W, thetaT, thetaT_lo,
-                      gwu, g.C_in, g.C_out, taps, err_word, beside_pool ? 1 : 0);
+                      gwu, g.C_in, g.C_out, taps, beside_pool ? 1 : 0);
 }
 
 gf_status launch_split_f32(const float* in, __nv_bfloat16* hi, __nv_bfloat16* lo, size_t n, cudaStream_t s) {
@@ -1034,12 +1045,8 @@ static gf_status launch_gx_tc_ares(const GxTcParams& p, int grid, size_t a_res_b
     constexpr size_t d_bytes = ((size_t)128 * (NT + 1) * 4 + 1023) / 1024 * 1024;
     constexpr size_t ring = (size_t)gx_stages(SPLIT, ARES, NT) * SPLIT * (kTcBK * NT * 2 + (ARES ? 0 : 128 * kTcBK * 2));
     const size_t smem = ring + d_bytes + (ARES ? a_res_bytes : 0) + 1024;
-    static size_t configured = 0;
-    if (smem > configured) {
-        GF_CUDA_TRY(cudaFuncSetAttribute(gx_tc_kernel<TOut, NT, R, LOGV, ARES, SPLIT>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        configured = smem;
-    }
+    static size_t configured[kMaxDevices] = {};
+    if (gf_status st = ensure_dyn_smem(gx_tc_kernel<TOut, NT, R, LOGV, ARES, SPLIT>, smem, configured); st != GF_OK) return st;
     return launch_pdl(gx_tc_kernel<TOut, NT, R, LOGV, ARES, SPLIT>, dim3(grid), dim3(kGxThreads), smem, s, p);
 }
 
@@ -1128,11 +1135,8 @@ gf_status launch_gx_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const _
 template <int NT, int LOGV, int SPLIT>
 static gf_status launch_gw_tc_inst(const GwTcParams& p, dim3 grid, cudaStream_t s) {
     constexpr size_t smem = (size_t)gw_stages(SPLIT, NT) * SPLIT * (128 * kTcBK * 2 + NT * kTcBK * 2) + 1024;
-    static bool configured = false;
-    if (!configured) {
-        GF_CUDA_TRY(cudaFuncSetAttribute(gw_tc_kernel<NT, LOGV, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        configured = true;
-    }
+    static size_t configured[kMaxDevices] = {};
+    if (gf_status st = ensure_dyn_smem(gw_tc_kernel<NT, LOGV, SPLIT>, smem, configured); st != GF_OK) return st;
     return launch_pdl(gw_tc_kernel<NT, LOGV, SPLIT>, grid, dim3(kGwThreads), smem, s, p);
 }
 

@@ -123,13 +123,89 @@ def test_host_buffer_step_matches_device_path(gf):
 
 
 # ---- the benchmark configurations at full size, in the launch configuration bench.py times ----
-FULL = (workloads.config2() + workloads.config3(2) + workloads.config3(4) + workloads.config4()
-        + [l for dt in ("f32", "bf16") for r in (2, 4, 8) for l in workloads.config5(r, dt)])
+# Configurations 2, 3 and 4: every element of the stash, g_W and g_X against the checker (it needs
+# a few seconds per layer).  Configuration 5 (up to 69 GFLOP of fp64 per layer): sampled outputs.
+FULL_ELEMENTWISE = workloads.config2() + workloads.config3(2) + workloads.config3(4) + workloads.config4()
+FULL_SAMPLED = [l for dt in ("f32", "bf16") for r in (2, 4, 8) for l in workloads.config5(r, dt)]
 
 
-@pytest.mark.parametrize("layer", FULL, ids=lambda l: f"{l.name}_r{l.r}_{l.dtype}")
+@pytest.mark.parametrize("layer", FULL_ELEMENTWISE, ids=lambda l: f"{l.name}_r{l.r}_{l.dtype}")
+def test_full_size_configs_element_by_element(gf, layer):
+    check_layer_full(gf, layer, isolate=False)
+
+
+@pytest.mark.parametrize("layer", FULL_SAMPLED, ids=lambda l: f"{l.name}_r{l.r}_{l.dtype}")
 def test_full_size_configs_sampled(gf, layer):
     check_layer_sampled(gf, layer)
+
+
+# ---- exact arithmetic: inputs for which every intermediate of the method is an integer that the
+# kernels' number formats hold exactly, so the results must equal the checker's BIT FOR BIT ----
+# x in {0..3}: patch sums <= 3 r^2 (exact in bf16 up to 256).  g_y is patch-constant with integer
+# values in {-3..3}: its patch means are those integers.  W in {-1, 0, 1}: kernel sums are integers
+# of magnitude <= KH*KW.  Every product and every partial sum of either contraction is then an
+# integer below 2^24, exact in fp32 in any order of summation; g_W (fp32) must equal the checker's
+# integer and g_X must equal the checker's integer after ONE rounding to the output dtype.  A dropped
+# K chunk, a wrong tile edge or a swapped column changes an integer and cannot hide under a tolerance.
+EXACT = [
+    L("exact_gw_wide_tile", 200, 700, 72, 16, 16, 1, 1, 2),        # bf16: 128 x 256 output tiles of the g_W kernel
+    L("exact_gx_wide_tile", 3, 40, 1032, 16, 16, 1, 1, 2),         # bf16: 128-wide column tiles of the g_X kernel
+    L("exact_gx_tile64", 3, 24, 40, 14, 14, 3, 1, 2),              # 64-wide column tiles, 3x3 kernel sums
+    L("exact_two_ci_tiles", 5, 136, 264, 28, 28, 1, 1, 2),         # two c_i tiles, five K chunks, row tiles
+    L("exact_r4_ragged_k", 9, 72, 200, 32, 32, 3, 1, 4),           # r = 4, C_out not a multiple of 64
+    L("exact_many_items", 37, 96, 576, 28, 28, 1, 1, 2),           # many column tiles per CTA
+    L("exact_wide_ci", 6, 576, 96, 28, 28, 1, 1, 2),               # C_in far above one accumulator
+    L("exact_r8", 4, 128, 64, 32, 32, 3, 1, 8),
+    L("exact_dw", 3, 40, 40, 28, 28, 3, 40, 2),                    # depthwise streamed kernel
+    L("exact_groups", 3, 32, 48, 16, 16, 3, 4, 2),                 # grouped layer, CUDA-core path
+]
+
+
+def _integer_inputs(layer, seed):
+    g = torch.Generator(device="cpu")
+    g.manual_seed(seed)
+    assert layer.H % layer.r == 0 and layer.W % layer.r == 0
+    x = torch.randint(0, 4, (layer.N, layer.C_in, layer.H, layer.W), generator=g).to(torch.float32)
+    gbar = torch.randint(-3, 4, (layer.N, layer.C_out, layer.Hp, layer.Wp), generator=g).to(torch.float32)
+    gy = gbar.repeat_interleave(layer.r, 2).repeat_interleave(layer.r, 3).contiguous()
+    w = torch.randint(-1, 2, (layer.C_out, layer.C_ig, layer.K, layer.K), generator=g).to(torch.float32)
+    dt = workloads.torch_dtype(layer.dtype)
+    return x.to(dt), gy.to(dt), w.to(dt)
+
+
+@pytest.mark.parametrize("layer", EXACT, ids=lambda l: l.name)
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_exact_arithmetic_bit_for_bit(gf, layer, dtype):
+    layer = layer.with_(dtype=dtype)
+    x, gy, w = _integer_inputs(layer, seed=4242)
+    stash_ref = oracle.stash_forward(f64(x), layer.r)
+    gw_ref, gx_ref = oracle.backward(f64(gy), stash_ref, f64(w), layer.r, groups=layer.groups)
+    assert np.abs(gw_ref).max() < 2 ** 24 and np.abs(gx_ref).max() < 2 ** 24
+    stash, gW, gX = run_gpu(gf, layer, x, gy, w)
+    assert np.array_equal(f64(stash), stash_ref)
+    assert np.array_equal(f64(gW), gw_ref)
+    gx_once_rounded = torch.from_numpy(gx_ref).to(workloads.torch_dtype(dtype))
+    assert torch.equal(gX.cpu(), gx_once_rounded)
+
+
+def test_error_word_is_reported_and_cleared(gf):
+    """The report path of the bounded device-side waits, driven from the host: a non-zero error word
+    copied into the workspace header reads back as GF_ERR_TIMEOUT; the next gf_backward on that
+    workspace clears it before any of its kernels run, and a completed call reports GF_OK."""
+    layer = L("err_word", 2, 24, 40, 14, 14, 3, 1, 2)
+    x, gy, w = workloads.make_inputs(layer)
+    desc = gf.desc_for(layer)
+    buf = gf.alloc_layer(desc)
+    xd, gyd, wd = x.cuda(), gy.cuda(), w.cuda()
+    gf.gf_stash_forward(desc, xd, buf.stash)
+    gf.gf_backward(desc, gyd, buf.stash, wd, buf.g_W, buf.g_X, buf.workspace)
+    assert gf.gf_last_async_status(buf.workspace) == gf.GF_OK
+    buf.workspace[:4].copy_(torch.tensor([2, 0, 0, 0], dtype=torch.uint8))      # as a timed-out wait would leave it
+    torch.cuda.synchronize()
+    assert gf.gf_last_async_status(buf.workspace) == gf.GF_ERR_TIMEOUT
+    assert gf.gf_last_async_status(buf.workspace) == gf.GF_ERR_TIMEOUT          # reading does not clear a workspace's word
+    gf.gf_backward(desc, gyd, buf.stash, wd, buf.g_W, buf.g_X, buf.workspace)
+    assert gf.gf_last_async_status(buf.workspace) == gf.GF_OK
 
 
 def test_ondevice_table_shapes_sampled(gf):

@@ -20,7 +20,9 @@ from parity_util import TOL, f64, relerr
 pytestmark = pytest.mark.gpu
 
 CASES = [
-    Layer("noalloc_f32", 0, 0, 3, 24, 40, 14, 14, 3, 1, 2, "f32", "relu", 1e-2),      # CUDA-core path, g_W slices
+    Layer("noalloc_f32", 0, 0, 3, 24, 40, 14, 14, 3, 1, 2, "f32", "relu", 1e-2),      # tensor-core path, operand pairs
+    Layer("noalloc_grouped", 0, 3, 3, 24, 36, 14, 14, 3, 2, 2, "f32", "relu", 1e-2),  # CUDA-core path, several g_W slices
+    Layer("noalloc_ragged", 0, 4, 3, 24, 42, 14, 14, 3, 1, 2, "bf16", "relu", 1e-2),  # CUDA-core path (C_out % 8 != 0)
     Layer("noalloc_bf16", 0, 1, 4, 64, 64, 14, 14, 3, 1, 2, "bf16", "relu", 1e-2),    # tensor-core path, accumulator
     Layer("noalloc_dw", 0, 2, 2, 16, 16, 14, 14, 3, 16, 2, "f32", "relu6", 1e-2),     # depthwise path
 ]
