@@ -55,7 +55,8 @@ NCU_TRAFFIC: dict[tuple[str, str], dict] = {}
 KERNEL_SOURCE = {
     "stash_pool": "gf_pool.cu", "gy_pool": "gf_pool.cu", "ksum": "gf_tc.cu", "gx_mix": "gf_dense.cu",
     "gw_partial": "gf_dense.cu", "gw_finish": "gf_dense.cu", "dw_fused": "gf_depthwise.cu",
-    "gx_tc": "gf_tc.cu", "gw_tc": "gf_tc.cu", "split_f32": "gf_tc.cu",
+    "gx_tc": "gf_tc.cu", "gw_tc": "gf_tc.cu", "split_f32": "gf_tc.cu", "gyx_fused": "gf_fused.cu",
+    "gw_tiled": "gf_fused.cu",
 }
 
 
@@ -167,6 +168,7 @@ def kernel_cost(name: str, L) -> tuple[float, float]:
         "stash_pool": (e * (L.numel_x() + L.numel_stash()), L.numel_x()),
         "gy_pool": (e * L.numel_gy() + (gbar16 if tc else gbar), L.numel_gy()),
         "gyx_fused": (e * (L.numel_gy() + L.numel_x()) + gbar16 + e * pairs, mix + L.numel_gy()),
+        "gw_tiled": (gbar16 + e * L.numel_stash() + 4 * pairs, mix),
         "ksum": (e * L.numel_w() + 4 * pairs, L.numel_w()),
         "gx_mix": (gbar + 4 * pairs + e * L.numel_x(), mix),
         "gw_partial": (gbar + e * L.numel_stash() + 4 * pairs, mix),

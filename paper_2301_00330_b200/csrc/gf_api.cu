@@ -21,7 +21,7 @@ int g_prof_created = 0;          // event pairs that exist
 int g_prof_used = 0;             // event pairs recorded since the last read
 int g_prof_slot_kid[kProfPairs];
 const char* const kKernelNames[K_COUNT] = {
-    "stash_pool", "ksum", "gy_pool", "gx_mix", "gw_partial", "gw_finish", "dw_fused", "exact_gx", "exact_gw", "gx_tc", "gw_tc", "split_f32"};
+    "stash_pool", "ksum", "gy_pool", "gx_mix", "gw_partial", "gw_finish", "dw_fused", "exact_gx", "exact_gw", "gx_tc", "gw_tc", "split_f32", "gyx_fused", "gw_tiled"};
 }  // namespace
 
 ProfScope::ProfScope(int kernel_id, cudaStream_t s) : slot(-1), stream(s) {
@@ -123,6 +123,14 @@ Workspace plan_workspace(const Geo& g) {
     w.off_split = 0;
     if (g.r == 1) { w.off_tsum = w.off_gbar = w.off_part = off; w.splits = 0; w.total = off; return w; }
     w.off_tsum = off; off += align_up((size_t)g.C_out * g.C_ig * 4, 256);
+    if (fused_path_ok(g)) {
+        // fused path: kernel sums (bf16, transposed) | tiled patch means | g_W unique-value matrix
+        w.off_gbar = off; off += align_up(fused_gbar_bytes(g), 256);
+        w.splits = 1;
+        w.off_part = off; off += align_up((size_t)g.C_out * g.C_ig * 4, 256);
+        w.total = off;
+        return w;
+    }
     const size_t pitch = tc_eligible(g) ? (size_t)tc_pitch(g) : (size_t)g.Hp * g.Wp;
     w.off_gbar = off; off += align_up((size_t)g.N * g.C_out * pitch * 4, 256);
     int s = dense_splits(g);
@@ -298,7 +306,7 @@ gf_status backward_impl(const gf_conv_desc* desc, const void* g_y, const void* s
     uint32_t* err = reinterpret_cast<uint32_t*>(base + ws.off_err);
     if (!g_W && !g_X) return GF_OK;
     // limits of the launch geometry, checked before anything is enqueued
-    if (g.r > 1 && !is_depthwise_fused(g)) {
+    if (g.r > 1 && !is_depthwise_fused(g) && !fused_path_ok(g)) {
         st = tc_eligible(g) ? tc_check_limits(g) : dense_check_limits(g, ws.splits);
         if (st != GF_OK) return st;
     }
@@ -317,6 +325,27 @@ gf_status backward_impl(const gf_conv_desc* desc, const void* g_y, const void* s
         st = launch_depthwise(g_y, stash, W, g_W ? part : nullptr, g_X, err, g, &splits, s);
         if (st != GF_OK) return st;
         if (g_W) return launch_gw_finish(part, splits, g_W, g, s);
+        return GF_OK;
+    }
+
+    if (fused_path_ok(g)) {
+        // theta sums (transposed bf16; fp32 layers: (high, low) pairs), then ONE kernel that reads
+        // g_y once, forms the patch means, contracts them with the theta sums on the tensor cores
+        // and writes the expanded g_X; the patch means it leaves behind feed the g_W contraction
+        const bool split = g.dtype == GF_F32;
+        const long long theta_lo = split ? (long long)align_up((size_t)g.C_in * g.C_out, 8) : 0;
+        __nv_bfloat16* thetaT = reinterpret_cast<__nv_bfloat16*>(tsum);
+        unsigned char* gbar_t = reinterpret_cast<unsigned char*>(gbar);
+        st = launch_ksum_t(W, g, thetaT, split ? thetaT + theta_lo : nullptr, g_W ? part : nullptr, /*beside_pool=*/false, s);
+        if (st != GF_OK) return st;
+        st = launch_gyx_fused(g_y, thetaT, theta_lo, g_X, g_W ? gbar_t : nullptr, err, g, s);
+        if (st != GF_OK) return st;
+        if (g_W) {
+            st = launch_gw_tiled(gbar_t, stash, part, err, g, s);
+            if (st != GF_OK) return st;
+            st = launch_gw_finish(part, 1, g_W, g, s);
+            if (st != GF_OK) return st;
+        }
         return GF_OK;
     }
 

@@ -15,7 +15,7 @@ void count_launch(int n = 1);
 
 enum KernelId {
     K_STASH_POOL = 0, K_KSUM, K_GY_POOL, K_GX_MIX, K_GW_PARTIAL, K_GW_FINISH, K_DW_FUSED,
-    K_EXACT_GX, K_EXACT_GW, K_GX_TC, K_GW_TC, K_SPLIT, K_COUNT
+    K_EXACT_GX, K_EXACT_GW, K_GX_TC, K_GW_TC, K_SPLIT, K_GYX_FUSED, K_GW_TILED, K_COUNT
 };
 
 // Brackets the launches made during its lifetime with a pair of events when
@@ -220,6 +220,14 @@ void tc_partition(const Geo& g, int* gx_ctas, int* gw_splits);
 gf_status launch_gw_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const __nv_bfloat16* stash,
                        long long stash_lo_off, float* gwu, int splits, uint32_t* err_word, const Geo& g,
                        cudaStream_t s);
+// fused gradient filter + reduced g_X (gyx_fused) and the g_W contraction on its tiled patch
+// means (gw_tiled); fused_path_ok: both kernels can take the layer
+bool fused_path_ok(const Geo& g);
+size_t fused_gbar_bytes(const Geo& g);
+gf_status launch_gyx_fused(const void* gy, const __nv_bfloat16* thetaT, long long theta_lo_off, void* gX,
+                           unsigned char* gbar_t, uint32_t* err_word, const Geo& g, cudaStream_t s);
+gf_status launch_gw_tiled(const unsigned char* gbar_t, const void* stash, float* gwu, uint32_t* err_word, const Geo& g,
+                          cudaStream_t s);
 gf_status launch_exact(const void* gy, const void* x, const void* W, float* gW, void* gX,
                        const Geo& g, cudaStream_t s);
 

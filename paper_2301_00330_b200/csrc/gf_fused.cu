@@ -1,0 +1,789 @@
+// Dense layers, r in {2,4,8} dividing H and W: the gradient filter (Section 3.3) fused with
+// the reduced input gradient (Eq. (grad_x)) and its expansion, and the reduced weight
+// gradient (Eq. (grad_w)) on the patch means that the fused kernel leaves behind.
+//
+//   gyx_fused   One persistent CTA per SM walks over tiles of up to 128 patches (whole patch
+//               rows of one image, or several whole images when an image has at most 64
+//               patches).  Per tile and per chunk of 64 output channels c_o:
+//                 copy engine   g_y pixels of the tile's patches -> shared memory (tiled
+//                               tensor-map copies, a ring of raw slabs of a few channels each);
+//                 pooling warps r x r patch means -> bf16 (fp32 layers: a (high, low) pair of
+//                               bf16), written straight into the 128-byte-swizzled operand tile
+//                               A[c_o][patch] the tensor core reads;
+//                 one thread    tcgen05.mma  D[patch, c_i] += A^T[patch, c_o] thetaT[c_i, c_o]
+//                               (thetaT tiles by the copy engine), accumulators in tensor memory;
+//                 epilogue      tcgen05.ld -> every value stored to its r x r pixels of g_X.
+//               g_y is read from HBM once and g_X written once.  The operand tile is also
+//               copied out (bulk shared -> global) as-is: the patch means in exactly the
+//               layout the g_W contraction wants for its own operand, 8 KB blocks of
+//               [64 c_o][64 patches].
+//   gw_tiled    D[c_o, c_i] = sum_k gbar[c_o, k] stash[c_i, k], k running over (tile, patch of
+//               the tile): the patch-mean blocks come in by bulk copies, the stash rows by
+//               asynchronous copies from the dense stash (fp32: split into (high, low) bf16 in
+//               shared memory); split over k, partial tiles added with vector reductions.
+//
+// Every wait is bounded: on expiry the CTA sets the error word, frees its tensor memory
+// and returns.  Every tensor map covers memory of this GPU only and every copy goes to the
+// issuing CTA alone.
+#include "gf_common.cuh"
+#include "gf_span.cuh"
+#include "gf_tc.cuh"
+#include "gf_tma.cuh"
+
+namespace gf {
+
+constexpr int kFuPool = 256;                 // warps 0-7: pooling
+constexpr int kFuEpi = 256;                  // warps 8-15: epilogue
+constexpr int kFuRawWarp = 16, kFuBWarp = 17, kFuMmaWarp = 18;
+constexpr int kFuThreads = 19 * 32;
+constexpr int kFuRawMax = 4, kFuAMax = 4;
+constexpr int kFuRawBudget = 32768;          // bytes of g_y per raw slab
+
+// How a layer is cut up; computed on the host (fused_plan) and shared by both kernels.
+struct FusedPlan {
+    bool ok = false;
+    int parts = 1;          // 1: bf16 operands; 2: fp32 values as (high, low) bf16 pairs
+    int IT = 1;             // images per tile (> 1 only when an image has <= 64 patches)
+    int RT = 0;             // patch rows per tile
+    int tiles_per_img = 1;  // IT == 1
+    long long tiles = 0;
+    int pr = 0;             // pixel rows per copy piece
+    int PW = 0;             // elements per piece and channel: pr * W
+    int pieces = 0;         // copy pieces per tile
+    int kc_raw = 0;         // channels per raw slab
+    int n_sub = 0;          // raw slabs per chunk of 64 channels
+    int MB = 1;             // 64-patch blocks per tile
+    int PT = 0;             // patch slots per tile: IT * RT * Wp
+    int G = 1;              // adjacent patches pooled by one thread
+    int NG = 0, n_groups = 0;   // c_i per accumulator, number of such groups
+    int n_chunks = 0;       // ceil(C_out / 64)
+    int a_stages = 0, raw_stages = 0;
+    bool reuse = false;     // the operand tiles of a whole tile stay in the ring: pooled once for all c_i groups
+    size_t raw_stage_bytes = 0, smem = 0, gbar_bytes = 0;
+};
+
+struct FusedParams {
+    CUtensorMap tm_gy;      // g_y as [N][C_out][H*W], box {PW, kc_raw, IT}
+    CUtensorMap tm_theta;   // thetaT as [part][C_in][C_out] bf16, box {64, NG, 1}, 128-byte swizzle
+    void* gX;
+    unsigned char* gbar_t;  // tiled patch means, NULL: not wanted
+    uint32_t* err_word;
+    int N, C_in, C_out, H, W, Hp, Wp, r;
+    int IT, RT, tiles_per_img, pr, PW, pieces, kc_raw, n_sub, MB, PT, PTG, NG, NGs, n_groups, n_chunks, reuse;
+    int a_stages, raw_stages, raw_stage_bytes, raw_tx_bytes, piece_bytes;
+    long long tiles;
+    FastDiv div_PTG, div_tiles_per_img, div_RTWp, div_Wp, div_ppr;
+    float inv_area;
+};
+
+struct FuShared {
+    uint64_t raw_full[kFuRawMax], raw_empty[kFuRawMax];
+    uint64_t a_full[kFuAMax], a_empty[kFuAMax];
+    uint64_t b_full[2], b_empty[2];
+    uint64_t acc_full[2], acc_empty[2];
+    uint32_t tmem_base;
+    int tab[128];           // per pooling item of a channel: element offset of its patches inside a raw slab
+};
+
+// Named barrier `id` over `nthreads` threads that also tells every one of them whether ANY
+// of them passed a true predicate: a failed (timed-out) wait of one thread ends the loop of all,
+// so that no thread is left alone at a later barrier.
+__device__ __forceinline__ bool bar_any(int id, int nthreads, bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, %2, %3, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "r"((uint32_t)pred), "r"(id), "r"(nthreads)
+        : "memory");
+    return r != 0;
+}
+
+__device__ __forceinline__ void fu_tile(const FusedParams& p, long long t, int& n0, int& a0) {
+    if (p.IT > 1) { n0 = (int)(t * p.IT); a0 = 0; return; }
+    uint32_t n, ti;
+    p.div_tiles_per_img.divmod((uint32_t)t, n, ti);
+    n0 = (int)n;
+    a0 = (int)ti * p.RT;
+}
+
+// R copies of v, streaming stores (g_X is written once and not read again by this call)
+template <int R> __device__ __forceinline__ void fu_store_rep(float* dst, float v) {
+    if constexpr (R == 2) __stcs(reinterpret_cast<float2*>(dst), make_float2(v, v));
+    else if constexpr (R == 4) __stcs(reinterpret_cast<float4*>(dst), make_float4(v, v, v, v));
+    else { __stcs(reinterpret_cast<float4*>(dst), make_float4(v, v, v, v)); __stcs(reinterpret_cast<float4*>(dst) + 1, make_float4(v, v, v, v)); }
+}
+template <int R> __device__ __forceinline__ void fu_store_rep(__nv_bfloat16* dst, float v) {
+    const uint32_t w = pack_bf16x2(v, v);
+    if constexpr (R == 2) __stcs(reinterpret_cast<unsigned int*>(dst), w);
+    else if constexpr (R == 4) __stcs(reinterpret_cast<uint2*>(dst), make_uint2(w, w));
+    else __stcs(reinterpret_cast<uint4*>(dst), make_uint4(w, w, w, w));
+}
+
+// One pooling item: G adjacent patches of one channel of a raw slab -> their means as bf16
+// (high part, and low part when SPLIT == 2) at [kk][m .. m+G) of the operand tile.
+template <typename T, int R, int G, int SPLIT>
+__device__ __forceinline__ void fu_pool_item(const FusedParams& p, const T* raw, const int* tab, unsigned char* a_stage,
+                                             int kk0, uint32_t q) {
+    uint32_t k, mg;
+    p.div_PTG.divmod(q, k, mg);
+    const T* src = raw + tab[mg] + (int)k * p.PW;
+    float acc[G];
+#pragma unroll
+    for (int j = 0; j < G; ++j) acc[j] = 0.f;
+#pragma unroll
+    for (int i = 0; i < R; ++i) {
+        float v[G * R];
+        load_span<G * R>(src + i * p.W, v);
+#pragma unroll
+        for (int j = 0; j < G; ++j) {
+            float s = v[j * R];
+#pragma unroll
+            for (int t = 1; t < R; ++t) s += v[j * R + t];
+            acc[j] += s;
+        }
+    }
+    const uint32_t off = mnmajor_off((uint32_t)kk0 + k, mg * G);
+    __nv_bfloat16 hi[G];
+#pragma unroll
+    for (int j = 0; j < G; ++j) { acc[j] *= p.inv_area; hi[j] = __float2bfloat16_rn(acc[j]); }
+    if constexpr (G == 2) *reinterpret_cast<__nv_bfloat162*>(a_stage + off) = __halves2bfloat162(hi[0], hi[1]);
+    else *reinterpret_cast<__nv_bfloat16*>(a_stage + off) = hi[0];
+    if constexpr (SPLIT == 2) {
+        __nv_bfloat16 lo[G];
+#pragma unroll
+        for (int j = 0; j < G; ++j) lo[j] = __float2bfloat16_rn(acc[j] - __bfloat162float(hi[j]));
+        if constexpr (G == 2) *reinterpret_cast<__nv_bfloat162*>(a_stage + 16384 + off) = __halves2bfloat162(lo[0], lo[1]);
+        else *reinterpret_cast<__nv_bfloat16*>(a_stage + 16384 + off) = lo[0];
+    }
+}
+
+template <typename T, int R, int G>
+__global__ void __launch_bounds__(kFuThreads, 1) gyx_fused_kernel(const __grid_constant__ FusedParams p) {
+    constexpr int SPLIT = sizeof(T) == 4 ? 2 : 1;
+    constexpr int kAStage = SPLIT * 16384;
+    extern __shared__ unsigned char dyn_raw[];
+    __shared__ FuShared sh;
+    unsigned char* dyn = align1024(dyn_raw);
+    const int b_stage_bytes = SPLIT * p.NG * 128;
+    unsigned char* a_ring = dyn;
+    unsigned char* b_ring = a_ring + (size_t)p.a_stages * kAStage;
+    unsigned char* raw_ring = b_ring + 2 * (size_t)b_stage_bytes;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const long long first = blockIdx.x, stride = gridDim.x;
+    const int n_my = first < p.tiles ? (int)((p.tiles - first + stride - 1) / stride) : 0;
+    const int AS = p.a_stages, RS = p.raw_stages;
+
+    if (tid == 0) {
+        for (int s = 0; s < kFuRawMax; ++s) { mbar_init(&sh.raw_full[s], 1); mbar_init(&sh.raw_empty[s], kFuPool); }
+        for (int s = 0; s < kFuAMax; ++s) { mbar_init(&sh.a_full[s], 1); mbar_init(&sh.a_empty[s], 1); }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&sh.b_full[s], 1); mbar_init(&sh.b_empty[s], 1);
+            mbar_init(&sh.acc_full[s], 1); mbar_init(&sh.acc_empty[s], 1);
+        }
+        mbar_fence_init();
+    }
+    if (warp == kFuMmaWarp) { tmem_alloc(&sh.tmem_base, (uint32_t)(2 * p.NGs)); tmem_relinquish(); }
+    if (tid < kFuPool) {
+        // where the patches of pooling item mg sit inside a raw slab (channel 0); the same for every tile
+        const int ppr = p.pr / p.r;
+        for (int mg = tid; mg < p.PTG; mg += kFuPool) {
+            uint32_t img_l, rem, a_l, b, pc, a_in;
+            p.div_RTWp.divmod((uint32_t)(mg * G), img_l, rem);
+            p.div_Wp.divmod(rem, a_l, b);
+            p.div_ppr.divmod(a_l, pc, a_in);
+            (void)ppr;
+            sh.tab[mg] = (int)((pc * (uint32_t)p.IT + img_l) * (uint32_t)(p.kc_raw * p.PW) + a_in * (uint32_t)(p.r * p.W) + b * (uint32_t)p.r);
+        }
+        // patch slots that no tile ever fills must read as zeros (they take part in the g_W contraction)
+        for (int i = tid; i < AS * kAStage / 16; i += kFuPool) reinterpret_cast<uint4*>(a_ring)[i] = make_uint4(0, 0, 0, 0);
+        fence_proxy_async_smem();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = sh.tmem_base;
+    pdl_launch_dependents();
+    pdl_wait();                       // thetaT comes from the previous kernel of the stream
+    bool ok = true;
+    const bool has_mma = p.gX != nullptr;                   // false: only the patch means are wanted
+    // c_i groups for which a tile is pooled
+    const int n_pool_groups = (p.reuse || !has_mma) ? 1 : p.n_groups;
+
+    if (warp < kFuPool / 32) {
+        // ================= pooling warps =================
+        int aq = 0, rq = 0;
+        const uint32_t items = (uint32_t)(p.kc_raw * p.PTG);
+        for (int it = 0; it < n_my && ok; ++it) {
+            const long long tile = first + (long long)it * stride;
+            for (int g = 0; g < n_pool_groups && ok; ++g) {
+                for (int c = 0; c < p.n_chunks && ok; ++c, ++aq) {
+                    const int s = aq % AS, u = aq / AS;
+                    unsigned char* a_stage = a_ring + (size_t)s * kAStage;
+                    // the copy-out of this stage's previous contents must have finished reading it
+                    if (tid == 0) bulk_wait_read<1>();
+                    if (u >= 1 && has_mma) ok = mbar_wait_bounded(&sh.a_empty[s], (uint32_t)(u - 1) & 1u);
+                    if (bar_any(1, kFuPool, !ok)) { ok = false; break; }
+                    for (int sub = 0; sub < p.n_sub && ok; ++sub, ++rq) {
+                        const int rs = rq % RS;
+                        ok = mbar_wait_bounded(&sh.raw_full[rs], (uint32_t)(rq / RS) & 1u);
+                        if (!ok) break;
+                        const T* raw = reinterpret_cast<const T*>(raw_ring + (size_t)rs * p.raw_stage_bytes);
+                        const int kk0 = sub * p.kc_raw;
+                        uint32_t q = tid;
+                        for (; q + kFuPool < items; q += 2 * kFuPool) {       // two independent items in flight
+                            fu_pool_item<T, R, G, SPLIT>(p, raw, sh.tab, a_stage, kk0, q);
+                            fu_pool_item<T, R, G, SPLIT>(p, raw, sh.tab, a_stage, kk0, q + kFuPool);
+                        }
+                        if (q < items) fu_pool_item<T, R, G, SPLIT>(p, raw, sh.tab, a_stage, kk0, q);
+                        mbar_arrive(&sh.raw_empty[rs]);
+                    }
+                    fence_proxy_async_smem();     // the tile is read by the tensor core and the copy engine
+                    if (bar_any(1, kFuPool, !ok)) { ok = false; break; }
+                    if (tid == 0) {
+                        if (p.gbar_t && g == 0) {
+                            for (int part = 0; part < SPLIT; ++part)
+                                for (int mb = 0; mb < p.MB; ++mb) {
+                                    unsigned char* dst = p.gbar_t + ((((size_t)tile * p.MB + mb) * SPLIT + part) * p.n_chunks + c) * 8192;
+                                    bulk_s2g(dst, a_stage + part * 16384 + mb * 8192, 8192);
+                                }
+                            bulk_commit();
+                        }
+                        mbar_arrive(&sh.a_full[s]);
+                    }
+                }
+            }
+        }
+        if (tid == 0) bulk_wait_all();
+    } else if (warp < (kFuPool + kFuEpi) / 32) {
+        // ================= epilogue warps: lane quarter warp & 3, interleaved 32-column chunks =================
+        const int et = tid - kFuPool, ew = et >> 5;
+        const int quarter = warp & 3, half = ew >> 2;
+        T* gx = static_cast<T*>(p.gX);
+        const size_t plane = (size_t)p.H * p.W;
+        const uint32_t m = (uint32_t)(quarter * 32 + lane);
+        uint32_t img_l, rem, a_l, b;
+        p.div_RTWp.divmod(m, img_l, rem);
+        p.div_Wp.divmod(rem, a_l, b);
+        int iq = 0;
+        for (int it = 0; it < n_my && ok && has_mma; ++it) {
+            const long long tile = first + (long long)it * stride;
+            int n0, a0;
+            fu_tile(p, tile, n0, a0);
+            const bool valid = (int)m < p.PT && n0 + (int)img_l < p.N && a0 + (int)a_l < p.Hp;
+            T* base_m = gx + ((size_t)(n0 + (int)img_l) * p.C_in) * plane + (size_t)((a0 + (int)a_l) * R) * p.W + (size_t)b * R;
+            for (int g = 0; g < p.n_groups && ok; ++g, ++iq) {
+                const int buf = iq & 1;
+                const int ci0 = g * p.NG;
+                const int ng = min(p.NG, p.C_in - ci0);
+                ok = mbar_wait_bounded(&sh.acc_full[buf], (uint32_t)(iq >> 1) & 1u);
+                tc_fence_after_sync();
+                if (ok) {
+                    for (int c = half * 32; c < ng; c += 64) {
+                        uint32_t v[32];
+                        tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * p.NGs + c), v);
+                        tmem_ld_wait();
+                        if (valid) {
+                            T* dst = base_m + (size_t)(ci0 + c) * plane;
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) {
+                                if (c + i < ng) {
+                                    const float val = __uint_as_float(v[i]);
+#pragma unroll
+                                    for (int dr = 0; dr < R; ++dr) fu_store_rep<R>(dst + (size_t)i * plane + (size_t)dr * p.W, val);
+                                }
+                            }
+                        }
+                    }
+                }
+                tc_fence_before_sync();
+                if (bar_any(2, kFuEpi, !ok)) { ok = false; break; }
+                if (et == 0) mbar_arrive(&sh.acc_empty[buf]);
+            }
+        }
+    } else if (warp == kFuRawWarp) {
+        // ================= copy engine: g_y slabs =================
+        if (lane == 0) {
+            int rq = 0;
+            for (int it = 0; it < n_my && ok; ++it) {
+                const long long tile = first + (long long)it * stride;
+                int n0, a0;
+                fu_tile(p, tile, n0, a0);
+                const int x0 = a0 * p.r * p.W;
+                for (int g = 0; g < n_pool_groups && ok; ++g)
+                    for (int c = 0; c < p.n_chunks && ok; ++c)
+                        for (int sub = 0; sub < p.n_sub && ok; ++sub, ++rq) {
+                            const int rs = rq % RS;
+                            if (rq >= RS) ok = mbar_wait_bounded(&sh.raw_empty[rs], (uint32_t)(rq / RS - 1) & 1u);
+                            if (!ok) break;
+                            unsigned char* dst = raw_ring + (size_t)rs * p.raw_stage_bytes;
+                            mbar_expect_tx(&sh.raw_full[rs], (uint32_t)p.raw_tx_bytes);
+                            for (int pc = 0; pc < p.pieces; ++pc)
+                                tma_load_3d(dst + (size_t)pc * p.piece_bytes, &p.tm_gy, x0 + pc * p.PW, c * kTcBK + sub * p.kc_raw, n0,
+                                            &sh.raw_full[rs]);
+                        }
+            }
+        }
+    } else if (warp == kFuBWarp) {
+        // ================= copy engine: thetaT tiles =================
+        if (lane == 0) {
+            int bq = 0;
+            for (int it = 0; it < n_my && ok && has_mma; ++it)
+                for (int g = 0; g < p.n_groups && ok; ++g)
+                    for (int c = 0; c < p.n_chunks && ok; ++c, ++bq) {
+                        const int bs = bq & 1;
+                        if (bq >= 2) ok = mbar_wait_bounded(&sh.b_empty[bs], (uint32_t)((bq >> 1) - 1) & 1u);
+                        if (!ok) break;
+                        unsigned char* dst = b_ring + (size_t)bs * b_stage_bytes;
+                        mbar_expect_tx(&sh.b_full[bs], (uint32_t)b_stage_bytes);
+                        for (int part = 0; part < SPLIT; ++part)
+                            tma_load_3d(dst + (size_t)part * p.NG * 128, &p.tm_theta, c * kTcBK, g * p.NG, part, &sh.b_full[bs]);
+                    }
+        }
+    } else {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            int aq = 0, bq = 0, iq = 0;
+            for (int it = 0; it < n_my && ok && has_mma; ++it) {
+                const int a_base = aq;
+                for (int g = 0; g < p.n_groups && ok; ++g, ++iq) {
+                    const int buf = iq & 1;
+                    const int ng16 = (min(p.NG, p.C_in - g * p.NG) + 15) & ~15;
+                    const uint32_t idesc = umma_idesc_bf16(128, ng16, /*A MN-major*/ 1, /*B K-major*/ 0);
+                    const uint32_t d_tmem = tmem + (uint32_t)(buf * p.NGs);
+                    if (iq >= 2) ok = mbar_wait_bounded(&sh.acc_empty[buf], (uint32_t)((iq >> 1) - 1) & 1u);
+                    const bool pooled = (g == 0) || !p.reuse;
+                    const bool release = (g == p.n_groups - 1) || !p.reuse;
+                    for (int c = 0; c < p.n_chunks && ok; ++c, ++bq) {
+                        int a_idx;
+                        if (pooled) {
+                            a_idx = aq++;
+                            ok = mbar_wait_bounded(&sh.a_full[a_idx % AS], (uint32_t)(a_idx / AS) & 1u);
+                        } else {
+                            a_idx = a_base + c;
+                        }
+                        const int s = a_idx % AS, bs = bq & 1;
+                        if (ok) ok = mbar_wait_bounded(&sh.b_full[bs], (uint32_t)(bq >> 1) & 1u);
+                        if (!ok) break;
+                        fence_proxy_async_smem();
+                        tc_fence_after_sync();
+                        const uint32_t a_addr = smem_u32(a_ring + (size_t)s * kAStage);
+                        const uint32_t b_addr = smem_u32(b_ring + (size_t)bs * b_stage_bytes);
+                        const uint32_t b_lo = b_addr + (uint32_t)(p.NG * 128);
+#pragma unroll
+                        for (int ks = 0; ks < kTcBK / 16; ++ks) {
+                            const uint64_t adesc = umma_smem_desc(a_addr + ks * 2048, 8192, 1024);
+                            const uint64_t bdesc = umma_smem_desc(b_addr + ks * 32, 16, 1024);
+                            umma_bf16(d_tmem, adesc, bdesc, idesc, !(c == 0 && ks == 0));
+                            if constexpr (SPLIT == 2) {
+                                umma_bf16(d_tmem, adesc, umma_smem_desc(b_lo + ks * 32, 16, 1024), idesc, 1u);
+                                umma_bf16(d_tmem, umma_smem_desc(a_addr + 16384 + ks * 2048, 8192, 1024), bdesc, idesc, 1u);
+                            }
+                        }
+                        umma_commit(&sh.b_empty[bs]);
+                        if (release) umma_commit(&sh.a_empty[s]);
+                    }
+                    if (ok) umma_commit(&sh.acc_full[buf]);
+                }
+            }
+        }
+    }
+    if (!ok) {
+        atomicOr(p.err_word, 16u);
+        // copies of the copy engine may still be on their way to this CTA's shared memory:
+        // a bounded pause (about a millisecond) before the CTA gives it up
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) {}
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    if (warp == kFuMmaWarp) tmem_dealloc(tmem, (uint32_t)(2 * p.NGs));
+}
+
+// ================================================================== gw_tiled
+constexpr int kGtLoaders = 256;     // 8 loader / epilogue warps + 1 MMA warp
+constexpr int kGtThreads = 288;
+constexpr int kGtStagesMax = 6;
+__host__ __device__ constexpr int gt_stages(int split) { return split == 2 ? 3 : 6; }
+
+struct GwTiledParams {
+    const unsigned char* gbar_t;    // [tile][mb][part][c_o chunk][8 KB]
+    const void* stash;              // dense [N][C_in][P] in the layer's dtype
+    float* gwu;                     // [C_out][C_in] fp32, zeroed beforehand; every CTA adds its slice
+    uint32_t* err_word;
+    int N, C_in, C_out, Hp, Wp, P;
+    int IT, RT, tiles_per_img, MB, n_chunks, S;
+    int logv;                       // log2 of the stash elements per asynchronous copy piece (pieces of 4, 8 or 16 bytes)
+    long long kchunks;              // tiles * MB
+    FastDiv div_tiles_per_img, div_P, div_MB;
+};
+
+struct GtShared {
+    uint64_t full[kGtStagesMax], empty[kGtStagesMax], landed[kGtStagesMax];
+    uint64_t accum;
+    uint32_t tmem_base;
+};
+
+__device__ __forceinline__ void cp_async_bytes(uint32_t dst, const void* src, int piece_bytes, uint32_t src_bytes) {
+    if (piece_bytes == 16) asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+    else if (piece_bytes == 8) asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+    else asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+
+// T: dtype of the stash.  fp32: the rows land as fp32 [128][64] in the stage's B region and are
+// split in place into the (high, low) bf16 tiles; bf16: the pieces land at their swizzled places.
+template <typename T>
+__global__ void __launch_bounds__(kGtThreads) gw_tiled_kernel(const GwTiledParams p) {
+    constexpr int SPLIT = sizeof(T) == 4 ? 2 : 1;
+    constexpr int ST = gt_stages(SPLIT);
+    constexpr int kABytes = 128 * kTcBK * 2;                 // 16 KB per part
+    constexpr int kBOff = SPLIT * kABytes;                   // stage: [A hi][A lo][B hi][B lo]
+    constexpr int kStageBytes = 2 * SPLIT * kABytes;
+    constexpr uint32_t kIdesc = umma_idesc_bf16(128, 128, 0, 0);
+    extern __shared__ unsigned char dyn_raw[];
+    __shared__ GtShared sh;
+    unsigned char* dyn = align1024(dyn_raw);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int ci0 = blockIdx.x * 128, co_blk = blockIdx.y * 2, split = blockIdx.z;
+    const long long kc_begin = p.kchunks * split / p.S, kc_end = p.kchunks * (split + 1) / p.S;
+    const int n_chunks = (int)(kc_end - kc_begin);
+    const int a_blocks = min(2, p.n_chunks - co_blk);       // 8 KB blocks of 64 c_o that exist for this tile
+
+    pdl_launch_dependents();
+    if (tid == 0) {
+        for (int s = 0; s < ST; ++s) {
+            mbar_init(&sh.full[s], kGtLoaders + 1); mbar_init(&sh.empty[s], 1); mbar_init(&sh.landed[s], kGtLoaders);
+        }
+        mbar_init(&sh.accum, 1);
+        mbar_fence_init();
+    }
+    if (warp == 8) { tmem_alloc(&sh.tmem_base, 128); tmem_relinquish(); }
+    if (a_blocks < 2)     // rows 64..127 of the A tiles are never loaded: keep them finite
+        for (int i = tid; i < ST * SPLIT * 512; i += kGtThreads) {
+            const int s = i / (SPLIT * 512), rest = i % (SPLIT * 512);
+            reinterpret_cast<uint4*>(dyn + (size_t)s * kStageBytes + (rest / 512) * kABytes + 8192)[rest % 512] = make_uint4(0, 0, 0, 0);
+        }
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = sh.tmem_base;
+    pdl_wait();                       // operands come from the previous kernels of the stream
+    bool ok = true;
+
+    if (warp < 8) {
+        const int V = 1 << p.logv;                          // elements per piece
+        const int piece_bytes = V * (int)sizeof(T);
+        const int ppr = kTcBK / V;                          // pieces per row
+        const int row_step = kGtLoaders / ppr;
+        const int k_me = (tid % ppr) * V, row0 = tid / ppr;
+        const T* st = static_cast<const T*>(p.stash);
+        // enqueue the copies of chunk q into its stage
+        auto issue = [&](int q) {
+            const int s = q % ST;
+            unsigned char* stage = dyn + (size_t)s * kStageBytes;
+            uint32_t tile, mb;
+            p.div_MB.divmod((uint32_t)(kc_begin + q), tile, mb);
+            if (tid == 0) {                                 // the patch-mean blocks: one bulk copy per part
+                mbar_expect_tx(&sh.full[s], (uint32_t)(SPLIT * a_blocks * 8192));
+                for (int part = 0; part < SPLIT; ++part)
+                    bulk_g2s(stage + part * kABytes,
+                             p.gbar_t + ((((size_t)tile * p.MB + mb) * SPLIT + part) * p.n_chunks + co_blk) * 8192,
+                             (uint32_t)(a_blocks * 8192), &sh.full[s]);
+            }
+            // this thread's piece: patches m .. m+V-1 of the tile
+            const int m = (int)mb * 64 + k_me;
+            int n_img, p0, nvalid;
+            if (p.IT > 1) {
+                uint32_t il, pp;
+                p.div_P.divmod((uint32_t)m, il, pp);
+                n_img = (int)tile * p.IT + (int)il;
+                p0 = (int)pp;
+                nvalid = ((int)il < p.IT && n_img < p.N) ? V : 0;
+            } else {
+                uint32_t n, ti;
+                p.div_tiles_per_img.divmod(tile, n, ti);
+                const int a0 = (int)ti * p.RT;
+                const int lim = min(p.RT, p.Hp - a0) * p.Wp - m;
+                n_img = (int)n;
+                p0 = a0 * p.Wp + m;
+                nvalid = lim < 0 ? 0 : (lim < V ? lim : V);
+            }
+            const T* src0 = st + ((size_t)n_img * p.C_in + ci0 + row0) * p.P + p0;
+            const size_t step = (size_t)row_step * p.P;
+            const uint32_t bdst = smem_u32(stage + kBOff);
+            for (int i = 0, row = row0; row < 128; ++i, row += row_step) {
+                const bool rv = nvalid > 0 && ci0 + row < p.C_in;
+                const uint32_t dst = SPLIT == 2 ? bdst + (uint32_t)(row * 256 + k_me * 4) : bdst + kmajor_off((uint32_t)row, (uint32_t)k_me);
+                cp_async_bytes(dst, rv ? (const void*)(src0 + i * step) : (const void*)st, piece_bytes,
+                               rv ? (uint32_t)(nvalid * (int)sizeof(T)) : 0u);
+            }
+            if constexpr (SPLIT == 2)
+                asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&sh.landed[s])) : "memory");
+            else
+                asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&sh.full[s])) : "memory");
+        };
+        const int ahead = ST - 1;
+        for (int q = 0; q < ahead && q < n_chunks; ++q) issue(q);
+        for (int q = 0; q < n_chunks && ok; ++q) {
+            const int qa = q + ahead;
+            if (qa < n_chunks) {
+                if (qa >= ST) ok = mbar_wait_bounded(&sh.empty[qa % ST], (uint32_t)(qa / ST - 1) & 1u);
+                if (ok) issue(qa);
+            }
+            if constexpr (SPLIT == 2) {
+                // fp32 rows -> (high, low) bf16 tiles, in place: thread = (row, half of the row)
+                const int s = q % ST;
+                ok = mbar_wait_bounded(&sh.landed[s], (uint32_t)(q / ST) & 1u);
+                unsigned char* bt = dyn + (size_t)s * kStageBytes + kBOff;
+                const int row = tid >> 1, hf = tid & 1;
+                float v[32];
+                if (ok) load_span<32>(reinterpret_cast<const float*>(bt + row * 256 + hf * 128), v);
+                // every row is in registers before any is overwritten
+                if (bar_any(1, kGtLoaders, !ok)) { ok = false; break; }
+                uint32_t hi[16], lo[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const __nv_bfloat16 h0 = __float2bfloat16_rn(v[2 * j]), h1 = __float2bfloat16_rn(v[2 * j + 1]);
+                    const __nv_bfloat162 h2 = __halves2bfloat162(h0, h1);
+                    hi[j] = *reinterpret_cast<const uint32_t*>(&h2);
+                    lo[j] = pack_bf16x2(v[2 * j] - __bfloat162float(h0), v[2 * j + 1] - __bfloat162float(h1));
+                }
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const uint32_t off = kmajor_off((uint32_t)row, (uint32_t)(hf * 32 + c * 8));
+                    *reinterpret_cast<uint4*>(bt + off) = make_uint4(hi[4 * c], hi[4 * c + 1], hi[4 * c + 2], hi[4 * c + 3]);
+                    *reinterpret_cast<uint4*>(bt + kABytes + off) = make_uint4(lo[4 * c], lo[4 * c + 1], lo[4 * c + 2], lo[4 * c + 3]);
+                }
+                fence_proxy_async_smem();
+                mbar_arrive(&sh.full[s]);
+            }
+        }
+        cp_async_wait_all();
+        if (ok && n_chunks > 0) ok = mbar_wait_bounded(&sh.accum, 0);
+        tc_fence_after_sync();
+        if (ok && n_chunks > 0) {
+            const int co = blockIdx.y * 128 + (warp & 3) * 32 + lane;
+            const int c_base = (warp >> 2) * 64;
+            float* out = p.gwu + (size_t)co * p.C_in + ci0;
+            const bool vec_ok = (p.C_in % 4 == 0);
+#pragma unroll 1
+            for (int c = c_base; c < c_base + 64; c += 32) {
+                uint32_t v[32];
+                tmem_ld32(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)c, v);
+                tmem_ld_wait();
+                if (co < p.C_out) {
+                    if (vec_ok && ci0 + c + 32 <= p.C_in) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4) red_add_v4(out + c + i, v[i], v[i + 1], v[i + 2], v[i + 3]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (ci0 + c + i < p.C_in) atomicAdd(out + c + i, __uint_as_float(v[i]));
+                    }
+                }
+            }
+        }
+    } else if (lane == 0) {
+        for (int q = 0; q < n_chunks && ok; ++q) {
+            const uint32_t a_addr = smem_u32(dyn + (size_t)(q % ST) * kStageBytes);
+            ok = mma_chunk<ST, SPLIT>(sh.full, sh.empty, q, q == 0, a_addr, a_addr + kABytes, a_addr + kBOff,
+                                      a_addr + kBOff + kABytes, tmem, kIdesc, 32, 16);
+        }
+        if (ok && n_chunks > 0) umma_commit(&sh.accum);
+    }
+    if (!ok) {
+        atomicOr(p.err_word, 32u);
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) {}
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    if (warp == 8) tmem_dealloc(tmem, 128);
+}
+
+// ================================================================== host side
+static int round_up_int(int v, int a) { return (v + a - 1) / a * a; }
+
+static FusedPlan fused_plan(const Geo& g) {
+    FusedPlan f;
+    if (!tc_eligible(g)) return f;
+    const int r = g.r, e = (int)g.esize;
+    if (!(r == 2 || r == 4 || r == 8) || g.H % r != 0 || g.W % r != 0) return f;
+    if (g.Wp > 128 || g.W > 256) return f;
+    if (((long long)g.H * g.W * e) % 16 != 0) return f;                 // plane stride of the g_y tensor map
+    f.parts = g.dtype == GF_F32 ? 2 : 1;
+    const int P = g.Hp * g.Wp;
+    if (P <= 64) {
+        f.IT = 128 / P;
+        if (f.IT > g.N) f.IT = g.N;
+        f.RT = g.Hp;
+        f.tiles_per_img = 1;
+        f.tiles = ((long long)g.N + f.IT - 1) / f.IT;
+    } else {
+        const int rt0 = g.Hp < 128 / g.Wp ? g.Hp : 128 / g.Wp;
+        f.tiles_per_img = (g.Hp + rt0 - 1) / rt0;
+        f.RT = (g.Hp + f.tiles_per_img - 1) / f.tiles_per_img;          // even tiles
+        f.tiles_per_img = (g.Hp + f.RT - 1) / f.RT;
+        f.IT = 1;
+        f.tiles = (long long)g.N * f.tiles_per_img;
+        if (((long long)f.RT * r * g.W * e) % 16 != 0) return f;         // every tile starts on a 16-byte boundary
+    }
+    // copy pieces: pr pixel rows (whole patch rows), at most 256 elements, a multiple of 16 bytes;
+    // the least overshoot past the tile's rows first, then the largest piece
+    const int band = f.RT * r;
+    int best_over = 1 << 30;
+    for (int pr = r; pr <= band && pr * g.W <= 256; pr += r) {
+        if ((pr * g.W * e) % 16 != 0) continue;
+        const int pieces = (band + pr - 1) / pr, over = pieces * pr - band;
+        if (over < best_over || (over == best_over && pr > f.pr)) { best_over = over; f.pr = pr; f.pieces = pieces; }
+    }
+    if (f.pr == 0) return f;
+    f.PW = f.pr * g.W;
+    f.PT = f.IT * f.RT * g.Wp;
+    f.MB = f.PT > 64 ? 2 : 1;
+    f.G = g.Wp % 2 == 0 ? 2 : 1;
+    const long long per_ch = (long long)f.pieces * f.IT * f.PW * e;      // bytes of one channel of a raw slab
+    if (per_ch > kFuRawBudget) return f;
+    f.kc_raw = 64;
+    while ((long long)f.kc_raw * per_ch > kFuRawBudget) f.kc_raw >>= 1;
+    f.raw_stage_bytes = (size_t)round_up_int((int)(f.kc_raw * per_ch), 1024);
+    f.n_sub = 64 / f.kc_raw;
+    f.n_chunks = (g.C_out + 63) / 64;
+    const int ng_max = 256 / f.parts;
+    f.NG = g.C_in > ng_max ? ng_max : round_up_int(g.C_in, 16);
+    f.n_groups = (g.C_in + f.NG - 1) / f.NG;
+    f.a_stages = f.parts == 2 ? 2 : 4;
+    f.reuse = f.n_groups > 1 && f.n_chunks <= f.a_stages;
+    const size_t fixed = (size_t)f.a_stages * f.parts * 16384 + 2 * (size_t)f.parts * f.NG * 128;
+    const size_t budget = 227 * 1024 - 1024 - 2048;       // alignment slack, static shared memory
+    if (fixed + 2 * f.raw_stage_bytes > budget) return f;
+    f.raw_stages = (int)((budget - fixed) / f.raw_stage_bytes);
+    if (f.raw_stages > kFuRawMax) f.raw_stages = kFuRawMax;
+    f.smem = fixed + (size_t)f.raw_stages * f.raw_stage_bytes + 1024;
+    if (f.tiles > (1LL << 30) || f.tiles * f.MB > (1LL << 30)) return f;
+    f.gbar_bytes = (size_t)f.tiles * f.MB * f.parts * f.n_chunks * 8192;
+    f.ok = true;
+    return f;
+}
+
+size_t fused_gbar_bytes(const Geo& g) { return fused_plan(g).gbar_bytes; }
+
+template <typename T, int R, int G>
+static gf_status launch_fused_inst(const FusedParams& p, size_t smem, cudaStream_t s) {
+    static size_t configured[kMaxDevices] = {};
+    if (gf_status st = ensure_dyn_smem(gyx_fused_kernel<T, R, G>, smem, configured); st != GF_OK) return st;
+    const long long grid = p.tiles < sm_count() ? p.tiles : sm_count();
+    return launch_pdl(gyx_fused_kernel<T, R, G>, dim3((unsigned)grid), dim3(kFuThreads), smem, s, p);
+}
+
+template <typename T>
+static gf_status launch_fused_t(const FusedParams& p, int G, size_t smem, cudaStream_t s) {
+#define GF_FU_CASE(RR, GG) if (p.r == RR && G == GG) return launch_fused_inst<T, RR, GG>(p, smem, s);
+    GF_FU_CASE(2, 2) GF_FU_CASE(2, 1) GF_FU_CASE(4, 2) GF_FU_CASE(4, 1) GF_FU_CASE(8, 2) GF_FU_CASE(8, 1)
+#undef GF_FU_CASE
+    return GF_ERR_UNSUPPORTED;
+}
+
+// thetaT: bf16 [C_in][C_out] (fp32 layers: the low parts theta_lo_off elements behind the high
+// parts); gbar_t: where the tiled patch means go (NULL: not wanted).
+gf_status launch_gyx_fused(const void* gy, const __nv_bfloat16* thetaT, long long theta_lo_off, void* gX,
+                           unsigned char* gbar_t, uint32_t* err_word, const Geo& g, cudaStream_t s) {
+    ProfScope prof(K_GYX_FUSED, s);
+    const FusedPlan f = fused_plan(g);
+    if (!f.ok) return GF_ERR_UNSUPPORTED;
+    FusedParams p;
+    if (!make_tmap_plain(&p.tm_gy, gy, (int)g.esize, (uint64_t)g.H * g.W, (uint64_t)g.C_out, (uint64_t)g.N,
+                         (uint64_t)g.H * g.W, (uint64_t)g.C_out * g.H * g.W, (uint32_t)f.PW, (uint32_t)f.kc_raw, (uint32_t)f.IT))
+        return GF_ERR_CUDA;
+    const uint64_t part_stride = f.parts == 2 ? (uint64_t)theta_lo_off : (uint64_t)g.C_in * g.C_out;
+    if (!make_tmap_bf16(&p.tm_theta, thetaT, 3, (uint64_t)g.C_out, (uint64_t)g.C_in, (uint64_t)f.parts, (uint64_t)g.C_out,
+                        part_stride, (uint32_t)f.NG))
+        return GF_ERR_CUDA;
+    p.gX = gX; p.gbar_t = gbar_t; p.err_word = err_word;
+    p.N = g.N; p.C_in = g.C_in; p.C_out = g.C_out; p.H = g.H; p.W = g.W; p.Hp = g.Hp; p.Wp = g.Wp; p.r = g.r;
+    p.IT = f.IT; p.RT = f.RT; p.tiles_per_img = f.tiles_per_img; p.pr = f.pr; p.PW = f.PW; p.pieces = f.pieces;
+    p.kc_raw = f.kc_raw; p.n_sub = f.n_sub; p.MB = f.MB; p.PT = f.PT; p.PTG = f.PT / f.G; p.NG = f.NG;
+    int ngs = 32;
+    while (ngs < f.NG) ngs <<= 1;
+    p.NGs = ngs;
+    p.n_groups = f.n_groups; p.n_chunks = f.n_chunks; p.reuse = f.reuse ? 1 : 0;
+    p.a_stages = f.a_stages; p.raw_stages = f.raw_stages; p.raw_stage_bytes = (int)f.raw_stage_bytes;
+    p.piece_bytes = f.IT * f.kc_raw * f.PW * (int)g.esize;
+    p.raw_tx_bytes = f.pieces * p.piece_bytes;
+    p.tiles = f.tiles;
+    p.div_PTG = FastDiv((uint32_t)p.PTG);
+    p.div_tiles_per_img = FastDiv((uint32_t)f.tiles_per_img);
+    p.div_RTWp = FastDiv((uint32_t)(f.RT * g.Wp));
+    p.div_Wp = FastDiv((uint32_t)g.Wp);
+    p.div_ppr = FastDiv((uint32_t)(f.pr / g.r));
+    p.inv_area = 1.0f / ((float)g.r * (float)g.r);
+    if (g.dtype == GF_F32) return launch_fused_t<float>(p, f.G, f.smem, s);
+    return launch_fused_t<__nv_bfloat16>(p, f.G, f.smem, s);
+}
+
+template <typename T>
+static gf_status launch_gw_tiled_inst(const GwTiledParams& p, dim3 grid, cudaStream_t s) {
+    constexpr int SPLIT = sizeof(T) == 4 ? 2 : 1;
+    constexpr size_t smem = (size_t)gt_stages(SPLIT) * 2 * SPLIT * 16384 + 1024;
+    static size_t configured[kMaxDevices] = {};
+    if (gf_status st = ensure_dyn_smem(gw_tiled_kernel<T>, smem, configured); st != GF_OK) return st;
+    return launch_pdl(gw_tiled_kernel<T>, grid, dim3(kGtThreads), smem, s, p);
+}
+
+// Widest asynchronous-copy piece (log2 of its elements) with which the stash rows of every
+// (tile, 64-patch block) can be copied: 16, 8 or 4 bytes; -1 when not even 4-byte pieces fit.
+static int gw_tiled_logv(const Geo& g, const FusedPlan& f) {
+    const int e = (int)g.esize;
+    const int P = g.Hp * g.Wp;
+    // element offsets a piece may start at are multiples of gcd(P, tile stride in patches, V)
+    int unit = P;
+    auto gcd = [](int a, int b) { while (b) { const int t = a % b; a = b; b = t; } return a; };
+    if (f.IT == 1) unit = gcd(unit, f.RT * g.Wp);
+    for (int lv = e == 4 ? 2 : 3; lv >= 0; --lv) {
+        const int V = 1 << lv;
+        if (V * e < 4) break;
+        if (unit % V == 0 && 64 % V == 0) return lv;
+    }
+    return -1;
+}
+
+bool fused_path_ok(const Geo& g) {
+    const FusedPlan f = fused_plan(g);
+    return f.ok && gw_tiled_logv(g, f) >= 0 && (g.C_out + 127) / 128 <= 65535 && (g.C_out + 31) / 32 <= 65535;
+}
+
+gf_status launch_gw_tiled(const unsigned char* gbar_t, const void* stash, float* gwu, uint32_t* err_word, const Geo& g,
+                          cudaStream_t s) {
+    ProfScope prof(K_GW_TILED, s);
+    const FusedPlan f = fused_plan(g);
+    if (!f.ok) return GF_ERR_UNSUPPORTED;
+    GwTiledParams p;
+    p.gbar_t = gbar_t; p.stash = stash; p.gwu = gwu; p.err_word = err_word;
+    p.N = g.N; p.C_in = g.C_in; p.C_out = g.C_out; p.Hp = g.Hp; p.Wp = g.Wp; p.P = g.Hp * g.Wp;
+    p.IT = f.IT; p.RT = f.RT; p.tiles_per_img = f.tiles_per_img; p.MB = f.MB; p.n_chunks = f.n_chunks;
+    p.logv = gw_tiled_logv(g, f);
+    if (p.logv < 0) return GF_ERR_UNSUPPORTED;
+    p.kchunks = f.tiles * f.MB;
+    p.div_tiles_per_img = FastDiv((uint32_t)f.tiles_per_img);
+    p.div_P = FastDiv((uint32_t)p.P);
+    p.div_MB = FastDiv((uint32_t)f.MB);
+    const int tiles_out = ((g.C_in + 127) / 128) * ((g.C_out + 127) / 128);
+    long long S = (sm_count() + tiles_out - 1) / tiles_out;
+    if (S > p.kchunks) S = p.kchunks;
+    if (S < 1) S = 1;
+    if (S > 65535) S = 65535;
+    p.S = (int)S;
+    if ((g.C_out + 127) / 128 > 65535) return GF_ERR_UNSUPPORTED;
+    dim3 grid((g.C_in + 127) / 128, (g.C_out + 127) / 128, (unsigned)S);
+    if (g.dtype == GF_F32) return launch_gw_tiled_inst<float>(p, grid, s);
+    return launch_gw_tiled_inst<__nv_bfloat16>(p, grid, s);
+}
+
+}  // namespace gf

@@ -108,4 +108,56 @@ __device__ __forceinline__ uint32_t mnmajor_off(uint32_t k, uint32_t j) {
            ((j & 7u) << 1);
 }
 
+
+constexpr int kTcBK = 64;           // K elements per stage (one 128-byte swizzled row)
+
+// ---- asynchronous copies ----------------------------------------------------------------------
+template <int LOGV>
+__device__ __forceinline__ void cp_async_piece(uint32_t dst, const void* src, bool valid) {
+    static_assert(LOGV >= 1 && LOGV <= 3, "pieces of 4, 8 or 16 bytes");
+    const uint32_t n = valid ? (uint32_t)(2 << LOGV) : 0u;     // source bytes; 0 = fill with zeros
+    if constexpr (LOGV == 3) asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
+    else if constexpr (LOGV == 2) asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
+    else asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+__device__ __forceinline__ unsigned char* align1024(unsigned char* p) {
+    return reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(p) + 1023) & ~uintptr_t(1023));
+}
+
+// One chunk of the MMA thread's work: wait for the stage, four K = 16 steps, release it.
+// b_step = start-address advance of the B descriptor per step (32 bytes K-major, 2048
+// bytes MN-major); b_lbo = its leading byte offset.
+// SPLIT == 2: every operand is a pair of bf16 tiles (high and low parts of an fp32 value);
+// the product is hi*hi + hi*lo + lo*hi (the lo*lo term, 2^-18 relative, is dropped).
+template <int STAGES, int SPLIT>
+__device__ __forceinline__ bool mma_chunk(uint64_t* full, uint64_t* empty, int q, bool first, uint32_t a_addr,
+                                          uint32_t a_lo, uint32_t b_addr, uint32_t b_lo, uint32_t d_tmem,
+                                          uint32_t idesc, uint32_t b_step, uint32_t b_lbo) {
+    const int s = q % STAGES;
+    if (!mbar_wait_bounded(&full[s], (uint32_t)(q / STAGES) & 1u)) return false;
+    fence_proxy_async_smem();      // copies landed through the generic proxy; the MMA reads through the async proxy
+    tc_fence_after_sync();
+#pragma unroll
+    for (int ks = 0; ks < kTcBK / 16; ++ks) {
+        const uint64_t adesc = umma_smem_desc(a_addr + ks * 32, 16, 1024);
+        const uint64_t bdesc = umma_smem_desc(b_addr + ks * b_step, b_lbo, 1024);
+        umma_bf16(d_tmem, adesc, bdesc, idesc, !(first && ks == 0));
+        if constexpr (SPLIT == 2) {
+            umma_bf16(d_tmem, adesc, umma_smem_desc(b_lo + ks * b_step, b_lbo, 1024), idesc, 1u);
+            umma_bf16(d_tmem, umma_smem_desc(a_lo + ks * 32, 16, 1024), bdesc, idesc, 1u);
+        }
+    }
+    umma_commit(&empty[s]);
+    return true;
+}
+
+__device__ __forceinline__ void red_add_v4(float* dst, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(__uint_as_float(a)),
+                 "f"(__uint_as_float(b)), "f"(__uint_as_float(c)), "f"(__uint_as_float(d))
+                 : "memory");
+}
+
 }  // namespace gf

@@ -44,4 +44,22 @@ bool make_tmap_bf16(CUtensorMap* out, const void* base, int rank, uint64_t d0, u
     return r == CUDA_SUCCESS;
 }
 
+bool make_tmap_plain(CUtensorMap* out, const void* base, int elem_bytes, uint64_t d0, uint64_t d1, uint64_t d2,
+                     uint64_t stride1, uint64_t stride2, uint32_t box0, uint32_t box1, uint32_t box2) {
+    PFN_cuTensorMapEncodeTiled enc = encoder();
+    if (!enc || (elem_bytes != 2 && elem_bytes != 4)) return false;
+    const uint64_t e = (uint64_t)elem_bytes;
+    if ((reinterpret_cast<uintptr_t>(base) & 15u) != 0 || (stride1 * e) % 16 != 0 || (stride2 * e) % 16 != 0) return false;
+    if (box0 < 1 || box0 > 256 || (box0 * e) % 16 != 0 || box1 < 1 || box1 > 256 || box2 < 1 || box2 > 256) return false;
+    cuuint64_t dims[3] = {d0, d1, d2};
+    cuuint64_t strides[2] = {stride1 * e, stride2 * e};
+    cuuint32_t box[3] = {box0, box1, box2};
+    cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = enc(out, elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+                           const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 }  // namespace gf

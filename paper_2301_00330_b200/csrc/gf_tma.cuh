@@ -27,6 +27,13 @@ namespace gf {
 bool make_tmap_bf16(CUtensorMap* out, const void* base, int rank, uint64_t d0, uint64_t d1, uint64_t d2,
                     uint64_t stride1, uint64_t stride2, uint32_t box1);
 
+// Plain (unswizzled) map of a dense tensor [d2][d1][d0] of 2-byte (bf16) or 4-byte (fp32)
+// elements, d0 contiguous, strides in ELEMENTS, box = {box0, box1, box2}: the box lands in
+// shared memory as a dense [box2][box1][box0] array.  box0 * elem_bytes is a multiple of 16
+// and box0 <= 256.  false as above.
+bool make_tmap_plain(CUtensorMap* out, const void* base, int elem_bytes, uint64_t d0, uint64_t d1, uint64_t d2,
+                     uint64_t stride1, uint64_t stride2, uint32_t box0, uint32_t box1, uint32_t box2);
+
 #ifdef __CUDACC__
 __device__ __forceinline__ void tma_load_3d(void* dst_smem, const CUtensorMap* m, int x, int y, int z, uint64_t* bar) {
     asm volatile(
