@@ -141,6 +141,18 @@ gf_status gf_layer_step_host(const gf_conv_desc* desc, const void* h_x, const vo
                              const void* h_W, float* h_gW, void* h_gX, void* arena,
                              size_t arena_bytes, void* stream);
 
+/* Dense layers with r in {2,4,8} dividing H and W can be computed two ways: the gradient
+ * filter (Section 3.3) as a pooling pass of its own followed by the two reduced contractions
+ * side by side, or one kernel that reads g_y once, forms the patch means and computes g_X
+ * (Eq. (grad_x)) in the same pass, followed by the g_W contraction (Eq. (grad_w)).  The
+ * library picks per layer (the fused kernel where it measured faster: many tiles of 128
+ * patches and either far more input than output channels or few channels).  This call
+ * overrides that choice for the whole process, for tuning and for tests; it does not change
+ * gf_backward_workspace_bytes, which always covers both.  Not to be called while another
+ * thread is inside gf_backward. */
+typedef enum gf_dense_path { GF_PATH_AUTO = 0, GF_PATH_FUSED = 1, GF_PATH_SPLIT = 2 } gf_dense_path;
+gf_status gf_set_dense_path(int32_t path);
+
 /* Static, human-readable name of a status code. */
 const char* gf_status_string(gf_status s);
 

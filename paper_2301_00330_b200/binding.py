@@ -19,12 +19,13 @@ GF_OK, GF_ERR_NULL, GF_ERR_BAD_DESC, GF_ERR_UNSUPPORTED = 0, 1, 2, 3
 GF_ERR_WORKSPACE, GF_ERR_ALIGN, GF_ERR_CUDA, GF_ERR_TIMEOUT = 4, 5, 6, 7
 GF_F32, GF_BF16 = 0, 1
 GF_NCHW, GF_NHWC = 0, 1
+GF_PATH_AUTO, GF_PATH_FUSED, GF_PATH_SPLIT = 0, 1, 2
 
 EXPORTS = (
     "gf_stash_dims", "gf_stash_bytes", "gf_backward_workspace_bytes", "gf_stash_forward",
     "gf_backward", "gf_last_async_status", "gf_host_step_arena_bytes", "gf_layer_step_host",
     "gf_kernel_launch_count", "gf_status_string", "gf_profile_configure", "gf_profile_read",
-    "gf_kernel_name", "gf_kernel_id_count", "gf_backward_static_scratch",
+    "gf_kernel_name", "gf_kernel_id_count", "gf_backward_static_scratch", "gf_set_dense_path",
 )
 
 
@@ -87,6 +88,8 @@ def lib() -> ctypes.CDLL:
         L.gf_kernel_name.restype = ctypes.c_char_p
         L.gf_kernel_id_count.argtypes = []
         L.gf_kernel_id_count.restype = ctypes.c_int32
+        L.gf_set_dense_path.argtypes = [ctypes.c_int32]
+        L.gf_set_dense_path.restype = ctypes.c_int
         L.gf_status_string.argtypes = [ctypes.c_int]
         L.gf_status_string.restype = ctypes.c_char_p
         for name in ("gf_stash_dims", "gf_stash_bytes", "gf_backward_workspace_bytes", "gf_stash_forward",
@@ -202,6 +205,11 @@ def gf_layer_step_host(desc: gf_conv_desc, h_x, h_gy, h_W, h_gW, h_gX, arena, ar
     _check(lib().gf_layer_step_host(ctypes.byref(desc), _ptr(h_x), _ptr(h_gy), _ptr(h_W), _ptr(h_gW),
                                     _ptr(h_gX), _ptr(arena), ctypes.c_size_t(arena_bytes), _stream(stream)),
            "gf_layer_step_host")
+
+
+def gf_set_dense_path(path: int) -> None:
+    """GF_PATH_AUTO (the library's choice per layer), GF_PATH_FUSED or GF_PATH_SPLIT, process-wide."""
+    _check(lib().gf_set_dense_path(int(path)), "gf_set_dense_path")
 
 
 def gf_kernel_launch_count() -> int:

@@ -104,6 +104,14 @@ static gf_status validate(const gf_conv_desc* d) {
     return GF_OK;
 }
 
+// gf_set_dense_path: 0 = the library's choice, 1 = fused pair wherever it can run, 2 = never
+static std::atomic<int> g_dense_path{0};
+static bool use_fused(const Geo& g) {
+    const int policy = g_dense_path.load(std::memory_order_relaxed);
+    if (policy == 2 || !fused_path_ok(g)) return false;
+    return policy == 1 || fused_path_preferred(g);
+}
+
 static bool is_depthwise(const Geo& g) { return g.G == g.C_in && g.G == g.C_out; }
 static bool is_depthwise_fused(const Geo& g) { return is_depthwise(g) && depthwise_splits(g) > 0; }
 
@@ -116,21 +124,27 @@ static int dense_splits(const Geo& g) {
     return (int)s;
 }
 
-Workspace plan_workspace(const Geo& g) {
+// Layout of one path; plan_workspace sizes the workspace for whichever is larger, so that the
+// size a caller was told stays valid whatever path a later call takes.
+static Workspace plan_fused(const Geo& g) {
+    // kernel sums (bf16, transposed) | tiled patch means | g_W unique-value matrix
+    Workspace w;
+    w.off_err = 0; w.off_split = 0; w.splits = 1;
+    size_t off = 256;
+    w.off_tsum = off; off += align_up((size_t)g.C_out * g.C_ig * 4, 256);
+    w.off_gbar = off; off += align_up(fused_gbar_bytes(g), 256);
+    w.off_part = off; off += align_up((size_t)g.C_out * g.C_ig * 4, 256);
+    w.total = off;
+    return w;
+}
+
+static Workspace plan_split(const Geo& g) {
     Workspace w;
     w.off_err = 0;
     size_t off = 256;
     w.off_split = 0;
     if (g.r == 1) { w.off_tsum = w.off_gbar = w.off_part = off; w.splits = 0; w.total = off; return w; }
     w.off_tsum = off; off += align_up((size_t)g.C_out * g.C_ig * 4, 256);
-    if (fused_path_ok(g)) {
-        // fused path: kernel sums (bf16, transposed) | tiled patch means | g_W unique-value matrix
-        w.off_gbar = off; off += align_up(fused_gbar_bytes(g), 256);
-        w.splits = 1;
-        w.off_part = off; off += align_up((size_t)g.C_out * g.C_ig * 4, 256);
-        w.total = off;
-        return w;
-    }
     const size_t pitch = tc_eligible(g) ? (size_t)tc_pitch(g) : (size_t)g.Hp * g.Wp;
     w.off_gbar = off; off += align_up((size_t)g.N * g.C_out * pitch * 4, 256);
     int s = dense_splits(g);
@@ -144,6 +158,15 @@ Workspace plan_workspace(const Geo& g) {
         w.off_split = off; off += 2 * align_up((size_t)g.N * g.C_in * pitch * 2, 256);
     }
     w.total = off;
+    return w;
+}
+
+Workspace plan_workspace(const Geo& g) {
+    const Workspace split = plan_split(g);
+    if (g.r == 1 || !fused_path_ok(g)) return split;
+    Workspace w = use_fused(g) ? plan_fused(g) : split;
+    const size_t other = use_fused(g) ? split.total : plan_fused(g).total;
+    if (other > w.total) w.total = other;
     return w;
 }
 
@@ -306,7 +329,8 @@ gf_status backward_impl(const gf_conv_desc* desc, const void* g_y, const void* s
     uint32_t* err = reinterpret_cast<uint32_t*>(base + ws.off_err);
     if (!g_W && !g_X) return GF_OK;
     // limits of the launch geometry, checked before anything is enqueued
-    if (g.r > 1 && !is_depthwise_fused(g) && !fused_path_ok(g)) {
+    const bool fused = g.r > 1 && !is_depthwise_fused(g) && use_fused(g);
+    if (g.r > 1 && !is_depthwise_fused(g) && !fused) {
         st = tc_eligible(g) ? tc_check_limits(g) : dense_check_limits(g, ws.splits);
         if (st != GF_OK) return st;
     }
@@ -328,7 +352,7 @@ gf_status backward_impl(const gf_conv_desc* desc, const void* g_y, const void* s
         return GF_OK;
     }
 
-    if (fused_path_ok(g)) {
+    if (fused) {
         // theta sums (transposed bf16; fp32 layers: (high, low) pairs), then ONE kernel that reads
         // g_y once, forms the patch means, contracts them with the theta sums on the tensor cores
         // and writes the expanded g_X; the patch means it leaves behind feed the g_W contraction
@@ -478,6 +502,12 @@ gf_status gf_layer_step_host(const gf_conv_desc* desc, const void* h_x, const vo
     if (st != GF_OK) return st;
     if (h_gW) GF_CUDA_TRY(cudaMemcpyAsync(h_gW, base + a.gw, w_elems * 4, cudaMemcpyDeviceToHost, s));
     if (h_gX) GF_CUDA_TRY(cudaMemcpyAsync(h_gX, base + a.gx, x_bytes, cudaMemcpyDeviceToHost, s));
+    return GF_OK;
+}
+
+gf_status gf_set_dense_path(int32_t path) {
+    if (path < 0 || path > 2) return GF_ERR_BAD_DESC;
+    g_dense_path.store(path, std::memory_order_relaxed);
     return GF_OK;
 }
 

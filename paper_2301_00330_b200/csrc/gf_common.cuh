@@ -221,8 +221,10 @@ gf_status launch_gw_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const _
                        long long stash_lo_off, float* gwu, int splits, uint32_t* err_word, const Geo& g,
                        cudaStream_t s);
 // fused gradient filter + reduced g_X (gyx_fused) and the g_W contraction on its tiled patch
-// means (gw_tiled); fused_path_ok: both kernels can take the layer
+// means (gw_tiled); fused_path_ok: both kernels can take the layer; fused_path_preferred:
+// the layer is of a kind on which they measured faster than the separate kernels
 bool fused_path_ok(const Geo& g);
+bool fused_path_preferred(const Geo& g);
 size_t fused_gbar_bytes(const Geo& g);
 gf_status launch_gyx_fused(const void* gy, const __nv_bfloat16* thetaT, long long theta_lo_off, void* gX,
                            unsigned char* gbar_t, uint32_t* err_word, const Geo& g, cudaStream_t s);

@@ -32,24 +32,26 @@
 
 namespace gf {
 
-constexpr int kFuPool = 256;                 // warps 0-7: pooling
-constexpr int kFuEpi = 256;                  // warps 8-15: epilogue
+constexpr int kFuWork = 512;                 // warps 0-15: workers (pool a tile, then write its part of g_X)
 constexpr int kFuRawWarp = 16, kFuBWarp = 17, kFuMmaWarp = 18;
 constexpr int kFuThreads = 19 * 32;
-constexpr int kFuRawMax = 4, kFuAMax = 4;
+constexpr int kFuRawMax = 4, kFuAMax = 4, kFuAccMax = 8;
 constexpr int kFuRawBudget = 32768;          // bytes of g_y per raw slab
 
 // How a layer is cut up; computed on the host (fused_plan) and shared by both kernels.
+// A tile is up to 128 patch slots: RT whole patch rows of one image (IT == 1; tile t is
+// rows [ti RT, ti RT + RT) of image n with ti = t / N, n = t % N, so that the short last
+// tiles of the images come last), or IT whole images when an image has at most 64 patches
+// (tile t = images [t IT, t IT + IT)).
 struct FusedPlan {
     bool ok = false;
     int parts = 1;          // 1: bf16 operands; 2: fp32 values as (high, low) bf16 pairs
-    int IT = 1;             // images per tile (> 1 only when an image has <= 64 patches)
+    int IT = 1;             // images per tile
     int RT = 0;             // patch rows per tile
     int tiles_per_img = 1;  // IT == 1
     long long tiles = 0;
-    int pr = 0;             // pixel rows per copy piece
-    int PW = 0;             // elements per piece and channel: pr * W
-    int pieces = 0;         // copy pieces per tile
+    int run = 0;            // elements of one channel of one image in a (full) tile: RT r W, contiguous in g_y
+    int PW = 0, pieces = 0; // the run is fetched as `pieces` boxes of PW elements (PW <= 256, the last may overshoot)
     int kc_raw = 0;         // channels per raw slab
     int n_sub = 0;          // raw slabs per chunk of 64 channels
     int MB = 1;             // 64-patch blocks per tile
@@ -59,6 +61,7 @@ struct FusedPlan {
     int n_chunks = 0;       // ceil(C_out / 64)
     int a_stages = 0, raw_stages = 0;
     bool reuse = false;     // the operand tiles of a whole tile stay in the ring: pooled once for all c_i groups
+    bool stash_tma = false; // every 64-patch block of the stash starts on a 16-byte boundary: tensor-map copies can fetch it
     size_t raw_stage_bytes = 0, smem = 0, gbar_bytes = 0;
 };
 
@@ -69,10 +72,12 @@ struct FusedParams {
     unsigned char* gbar_t;  // tiled patch means, NULL: not wanted
     uint32_t* err_word;
     int N, C_in, C_out, H, W, Hp, Wp, r;
-    int IT, RT, tiles_per_img, pr, PW, pieces, kc_raw, n_sub, MB, PT, PTG, NG, NGs, n_groups, n_chunks, reuse;
-    int a_stages, raw_stages, raw_stage_bytes, raw_tx_bytes, piece_bytes;
+    int IT, RT, PW, pieces, piece_bytes, kc_raw, n_sub, MB, PT, PTG, NG, NGs, n_groups, n_chunks, reuse;
+    int a_stages, raw_stages, raw_stage_bytes;
+    int kpar;               // channels of a raw slab pooled side by side: kFuWork / PTG
+    int n_acc;              // accumulators in tensor memory (a ring): 512 / NGs, at most kFuAccMax
     long long tiles;
-    FastDiv div_PTG, div_tiles_per_img, div_RTWp, div_Wp, div_ppr;
+    FastDiv div_PTG, div_N, div_RTWp, div_Wp, div_PW;
     float inv_area;
 };
 
@@ -80,9 +85,8 @@ struct FuShared {
     uint64_t raw_full[kFuRawMax], raw_empty[kFuRawMax];
     uint64_t a_full[kFuAMax], a_empty[kFuAMax];
     uint64_t b_full[2], b_empty[2];
-    uint64_t acc_full[2], acc_empty[2];
+    uint64_t acc_full[kFuAccMax], acc_empty[kFuAccMax];
     uint32_t tmem_base;
-    int tab[128];           // per pooling item of a channel: element offset of its patches inside a raw slab
 };
 
 // Named barrier `id` over `nthreads` threads that also tells every one of them whether ANY
@@ -101,12 +105,13 @@ __device__ __forceinline__ bool bar_any(int id, int nthreads, bool pred) {
     return r != 0;
 }
 
-__device__ __forceinline__ void fu_tile(const FusedParams& p, long long t, int& n0, int& a0) {
-    if (p.IT > 1) { n0 = (int)(t * p.IT); a0 = 0; return; }
-    uint32_t n, ti;
-    p.div_tiles_per_img.divmod((uint32_t)t, n, ti);
+// first image and first patch row of tile t
+__device__ __forceinline__ void fu_tile(int IT, int RT, const FastDiv& div_N, long long t, int& n0, int& a0) {
+    if (IT > 1) { n0 = (int)(t * IT); a0 = 0; return; }
+    uint32_t ti, n;
+    div_N.divmod((uint32_t)t, ti, n);
     n0 = (int)n;
-    a0 = (int)ti * p.RT;
+    a0 = (int)ti * RT;
 }
 
 // R copies of v, streaming stores (g_X is written once and not read again by this call)
@@ -122,42 +127,72 @@ template <int R> __device__ __forceinline__ void fu_store_rep(__nv_bfloat16* dst
     else __stcs(reinterpret_cast<uint4*>(dst), make_uint4(w, w, w, w));
 }
 
-// One pooling item: G adjacent patches of one channel of a raw slab -> their means as bf16
-// (high part, and low part when SPLIT == 2) at [kk][m .. m+G) of the operand tile.
-template <typename T, int R, int G, int SPLIT>
-__device__ __forceinline__ void fu_pool_item(const FusedParams& p, const T* raw, const int* tab, unsigned char* a_stage,
-                                             int kk0, uint32_t q) {
-    uint32_t k, mg;
-    p.div_PTG.divmod(q, k, mg);
-    const T* src = raw + tab[mg] + (int)k * p.PW;
-    float acc[G];
+// The G adjacent patches of a thread's pooling position, for NB channels of a raw slab at
+// once (their loads are independent, so they are all in flight together): the means as bf16
+// (high part, and low part when SPLIT == 2) go to [k][m .. m+G) of the operand tile.
+// src: the first channel's row of the raw slab; roff: where each of the R pixel rows of the
+// patches starts relative to that; kstep: elements between the channels taken; dst: the operand tile plus the part of the offset that depends on m alone;
+// jc: 16-byte chunk of m within its 128-byte row; k: first channel (within the 64 of the
+// tile); channels from k_lim on do not exist (their rows of the tile are written as zeros,
+// and so is everything when the position holds no patch of this tile: live == false).
+template <typename T, int R, int G, int SPLIT, int NB>
+__device__ __forceinline__ void fu_pool_n(const FusedParams& p, const T* src, const int (&roff)[R], int kstep, unsigned char* dst,
+                                          uint32_t jc, int k, int kpar, int k_lim, bool live) {
+    float acc[NB][G];
 #pragma unroll
-    for (int j = 0; j < G; ++j) acc[j] = 0.f;
+    for (int n = 0; n < NB; ++n)
+#pragma unroll
+        for (int j = 0; j < G; ++j) acc[n][j] = 0.f;
 #pragma unroll
     for (int i = 0; i < R; ++i) {
-        float v[G * R];
-        load_span<G * R>(src + i * p.W, v);
+        float v[NB][G * R];
 #pragma unroll
-        for (int j = 0; j < G; ++j) {
-            float s = v[j * R];
+        for (int n = 0; n < NB; ++n) load_span<G * R>(src + n * kstep + roff[i], v[n]);
 #pragma unroll
-            for (int t = 1; t < R; ++t) s += v[j * R + t];
-            acc[j] += s;
+        for (int n = 0; n < NB; ++n)
+#pragma unroll
+            for (int j = 0; j < G; ++j) {
+                float s = v[n][j * R];
+#pragma unroll
+                for (int t = 1; t < R; ++t) s += v[n][j * R + t];
+                acc[n][j] += s;
+            }
+    }
+#pragma unroll
+    for (int n = 0; n < NB; ++n) {
+        const uint32_t kk = (uint32_t)(k + n * kpar);
+        const bool keep = live && (int)kk < k_lim;
+        unsigned char* d = dst + (kk >> 3) * 1024u + (kk & 7u) * 128u + (((jc ^ kk) & 7u) << 4);
+        __nv_bfloat16 hi[G];
+#pragma unroll
+        for (int j = 0; j < G; ++j) { acc[n][j] = keep ? acc[n][j] * p.inv_area : 0.f; hi[j] = __float2bfloat16_rn(acc[n][j]); }
+        if constexpr (G == 2) *reinterpret_cast<__nv_bfloat162*>(d) = __halves2bfloat162(hi[0], hi[1]);
+        else *reinterpret_cast<__nv_bfloat16*>(d) = hi[0];
+        if constexpr (SPLIT == 2) {
+            __nv_bfloat16 lo[G];
+#pragma unroll
+            for (int j = 0; j < G; ++j) lo[j] = __float2bfloat16_rn(acc[n][j] - __bfloat162float(hi[j]));
+            if constexpr (G == 2) *reinterpret_cast<__nv_bfloat162*>(d + 16384) = __halves2bfloat162(lo[0], lo[1]);
+            else *reinterpret_cast<__nv_bfloat16*>(d + 16384) = lo[0];
         }
     }
-    const uint32_t off = mnmajor_off((uint32_t)kk0 + k, mg * G);
-    __nv_bfloat16 hi[G];
-#pragma unroll
-    for (int j = 0; j < G; ++j) { acc[j] *= p.inv_area; hi[j] = __float2bfloat16_rn(acc[j]); }
-    if constexpr (G == 2) *reinterpret_cast<__nv_bfloat162*>(a_stage + off) = __halves2bfloat162(hi[0], hi[1]);
-    else *reinterpret_cast<__nv_bfloat16*>(a_stage + off) = hi[0];
-    if constexpr (SPLIT == 2) {
-        __nv_bfloat16 lo[G];
-#pragma unroll
-        for (int j = 0; j < G; ++j) lo[j] = __float2bfloat16_rn(acc[j] - __bfloat162float(hi[j]));
-        if constexpr (G == 2) *reinterpret_cast<__nv_bfloat162*>(a_stage + 16384 + off) = __halves2bfloat162(lo[0], lo[1]);
-        else *reinterpret_cast<__nv_bfloat16*>(a_stage + 16384 + off) = lo[0];
-    }
+}
+
+// One raw slab: thread (kl, mg) pools position mg of the channels kl, kl + kpar, ... of the
+// slab, in batches whose loads overlap.  kk0: first channel of the slab within its chunk.
+template <typename T, int R, int G, int SPLIT>
+__device__ __forceinline__ void fu_pool_slab(const FusedParams& p, const T* src, const int (&roff)[R], unsigned char* dst,
+                                             uint32_t jc, int kk0, int kl, int k_lim, bool live) {
+    constexpr int NB = R == 2 ? 4 : R == 4 ? 2 : 1;      // R = 8: one item already is 8 rows of loads
+    const int kpar = p.kpar, kstep = kpar * p.PW;
+    int k = kl;
+    if constexpr (NB >= 4)
+        for (; k + 3 * kpar < p.kc_raw; k += 4 * kpar)
+            fu_pool_n<T, R, G, SPLIT, 4>(p, src + k * p.PW, roff, kstep, dst, jc, kk0 + k, kpar, k_lim, live);
+    if constexpr (NB >= 2)
+        for (; k + kpar < p.kc_raw; k += 2 * kpar)
+            fu_pool_n<T, R, G, SPLIT, 2>(p, src + k * p.PW, roff, kstep, dst, jc, kk0 + k, kpar, k_lim, live);
+    for (; k < p.kc_raw; k += kpar) fu_pool_n<T, R, G, SPLIT, 1>(p, src + k * p.PW, roff, kstep, dst, jc, kk0 + k, kpar, k_lim, live);
 }
 
 template <typename T, int R, int G>
@@ -178,28 +213,17 @@ __global__ void __launch_bounds__(kFuThreads, 1) gyx_fused_kernel(const __grid_c
     const int AS = p.a_stages, RS = p.raw_stages;
 
     if (tid == 0) {
-        for (int s = 0; s < kFuRawMax; ++s) { mbar_init(&sh.raw_full[s], 1); mbar_init(&sh.raw_empty[s], kFuPool); }
+        for (int s = 0; s < kFuRawMax; ++s) { mbar_init(&sh.raw_full[s], 1); mbar_init(&sh.raw_empty[s], kFuWork / 32); }
         for (int s = 0; s < kFuAMax; ++s) { mbar_init(&sh.a_full[s], 1); mbar_init(&sh.a_empty[s], 1); }
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(&sh.b_full[s], 1); mbar_init(&sh.b_empty[s], 1);
-            mbar_init(&sh.acc_full[s], 1); mbar_init(&sh.acc_empty[s], 1);
-        }
+        for (int s = 0; s < 2; ++s) { mbar_init(&sh.b_full[s], 1); mbar_init(&sh.b_empty[s], 1); }
+        for (int s = 0; s < kFuAccMax; ++s) { mbar_init(&sh.acc_full[s], 1); mbar_init(&sh.acc_empty[s], 1); }
         mbar_fence_init();
     }
-    if (warp == kFuMmaWarp) { tmem_alloc(&sh.tmem_base, (uint32_t)(2 * p.NGs)); tmem_relinquish(); }
-    if (tid < kFuPool) {
-        // where the patches of pooling item mg sit inside a raw slab (channel 0); the same for every tile
-        const int ppr = p.pr / p.r;
-        for (int mg = tid; mg < p.PTG; mg += kFuPool) {
-            uint32_t img_l, rem, a_l, b, pc, a_in;
-            p.div_RTWp.divmod((uint32_t)(mg * G), img_l, rem);
-            p.div_Wp.divmod(rem, a_l, b);
-            p.div_ppr.divmod(a_l, pc, a_in);
-            (void)ppr;
-            sh.tab[mg] = (int)((pc * (uint32_t)p.IT + img_l) * (uint32_t)(p.kc_raw * p.PW) + a_in * (uint32_t)(p.r * p.W) + b * (uint32_t)p.r);
-        }
+    const int n_acc = p.n_acc;
+    if (warp == kFuMmaWarp) { tmem_alloc(&sh.tmem_base, (uint32_t)(n_acc * p.NGs)); tmem_relinquish(); }
+    if (tid < kFuWork) {
         // patch slots that no tile ever fills must read as zeros (they take part in the g_W contraction)
-        for (int i = tid; i < AS * kAStage / 16; i += kFuPool) reinterpret_cast<uint4*>(a_ring)[i] = make_uint4(0, 0, 0, 0);
+        for (int i = tid; i < AS * kAStage / 16; i += kFuWork) reinterpret_cast<uint4*>(a_ring)[i] = make_uint4(0, 0, 0, 0);
         fence_proxy_async_smem();
     }
     tc_fence_before_sync();
@@ -210,41 +234,72 @@ __global__ void __launch_bounds__(kFuThreads, 1) gyx_fused_kernel(const __grid_c
     pdl_wait();                       // thetaT comes from the previous kernel of the stream
     bool ok = true;
     const bool has_mma = p.gX != nullptr;                   // false: only the patch means are wanted
-    // c_i groups for which a tile is pooled
-    const int n_pool_groups = (p.reuse || !has_mma) ? 1 : p.n_groups;
+    // passes over a tile's g_y: one when its operand tiles stay in the ring for every c_i
+    // group (or no g_X is wanted), else one per c_i group
+    const int n_pass = (p.reuse || !has_mma) ? 1 : p.n_groups;
 
-    if (warp < kFuPool / 32) {
-        // ================= pooling warps =================
-        int aq = 0, rq = 0;
-        const uint32_t items = (uint32_t)(p.kc_raw * p.PTG);
+    if (warp < kFuWork / 32) {
+        // ================= workers: pool the tile, then expand its accumulators into g_X =================
+        // Pooling: thread (kl, mg) takes position mg (G adjacent patch slots) of the channels kl,
+        // kl + kpar, ... of every raw slab; where those patches sit inside a slab and inside the
+        // operand tile is the same for every tile.
+        uint32_t kl, mg;
+        p.div_PTG.divmod((uint32_t)tid, kl, mg);
+        const bool pool_active = (int)kl < p.kpar;
+        uint32_t pimg, prem, pa, pb;
+        p.div_RTWp.divmod(mg * G, pimg, prem);
+        p.div_Wp.divmod(prem, pa, pb);
+        // a raw slab is [piece][image of the tile][channel][PW]: where the R pixel rows of the position start
+        int roff[R];
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+            uint32_t pc, within;
+            p.div_PW.divmod((pa * (uint32_t)R + (uint32_t)i) * (uint32_t)p.W + pb * (uint32_t)R, pc, within);
+            roff[i] = (int)((pc * (uint32_t)p.IT + pimg) * (uint32_t)(p.kc_raw * p.PW) + within);
+        }
+        const uint32_t pj = mg * G;
+        const uint32_t pool_dst = (pj >> 6) * 8192u + ((pj & 7u) << 1), pool_jc = (pj & 63u) >> 3;
+        // Expansion: lane quarter warp & 3 of tensor memory = patch slots 32 (warp & 3) + lane;
+        // the four warps of a quarter take interleaved 32-column chunks.
+        const int quarter = warp & 3, cset = warp >> 2;
+        T* gx = static_cast<T*>(p.gX);
+        const size_t plane = (size_t)p.H * p.W;
+        const uint32_t m = (uint32_t)(quarter * 32 + lane);
+        uint32_t eimg, erem, ea, eb;
+        p.div_RTWp.divmod(m, eimg, erem);
+        p.div_Wp.divmod(erem, ea, eb);
+        int aq = 0, rq = 0, iq = 0;
         for (int it = 0; it < n_my && ok; ++it) {
             const long long tile = first + (long long)it * stride;
-            for (int g = 0; g < n_pool_groups && ok; ++g) {
+            int n0, a0;
+            fu_tile(p.IT, p.RT, p.div_N, tile, n0, a0);
+            const bool pool_live = n0 + (int)pimg < p.N && a0 + (int)pa < p.Hp;
+            const bool e_valid = (int)m < p.PT && n0 + (int)eimg < p.N && a0 + (int)ea < p.Hp;
+            T* base_m = gx + ((size_t)(n0 + (int)eimg) * p.C_in) * plane + (size_t)((a0 + (int)ea) * R) * p.W + (size_t)eb * R;
+            for (int pass = 0; pass < n_pass && ok; ++pass) {
                 for (int c = 0; c < p.n_chunks && ok; ++c, ++aq) {
                     const int s = aq % AS, u = aq / AS;
                     unsigned char* a_stage = a_ring + (size_t)s * kAStage;
                     // the copy-out of this stage's previous contents must have finished reading it
                     if (tid == 0) bulk_wait_read<1>();
                     if (u >= 1 && has_mma) ok = mbar_wait_bounded(&sh.a_empty[s], (uint32_t)(u - 1) & 1u);
-                    if (bar_any(1, kFuPool, !ok)) { ok = false; break; }
+                    if (bar_any(1, kFuWork, !ok)) { ok = false; break; }
+                    const int k_lim = p.C_out - c * kTcBK;
                     for (int sub = 0; sub < p.n_sub && ok; ++sub, ++rq) {
                         const int rs = rq % RS;
                         ok = mbar_wait_bounded(&sh.raw_full[rs], (uint32_t)(rq / RS) & 1u);
                         if (!ok) break;
-                        const T* raw = reinterpret_cast<const T*>(raw_ring + (size_t)rs * p.raw_stage_bytes);
-                        const int kk0 = sub * p.kc_raw;
-                        uint32_t q = tid;
-                        for (; q + kFuPool < items; q += 2 * kFuPool) {       // two independent items in flight
-                            fu_pool_item<T, R, G, SPLIT>(p, raw, sh.tab, a_stage, kk0, q);
-                            fu_pool_item<T, R, G, SPLIT>(p, raw, sh.tab, a_stage, kk0, q + kFuPool);
-                        }
-                        if (q < items) fu_pool_item<T, R, G, SPLIT>(p, raw, sh.tab, a_stage, kk0, q);
-                        mbar_arrive(&sh.raw_empty[rs]);
+                        if (pool_active)
+                            fu_pool_slab<T, R, G, SPLIT>(p, reinterpret_cast<const T*>(raw_ring + (size_t)rs * p.raw_stage_bytes), roff,
+                                                         a_stage + pool_dst, pool_jc, sub * p.kc_raw, (int)kl, k_lim, pool_live);
+                        // one arrival per warp (hundreds of arrivals on one barrier would queue up behind each other)
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&sh.raw_empty[rs]);
                     }
                     fence_proxy_async_smem();     // the tile is read by the tensor core and the copy engine
-                    if (bar_any(1, kFuPool, !ok)) { ok = false; break; }
+                    if (bar_any(1, kFuWork, !ok)) { ok = false; break; }
                     if (tid == 0) {
-                        if (p.gbar_t && g == 0) {
+                        if (p.gbar_t && pass == 0) {
                             for (int part = 0; part < SPLIT; ++part)
                                 for (int mb = 0; mb < p.MB; ++mb) {
                                     unsigned char* dst = p.gbar_t + ((((size_t)tile * p.MB + mb) * SPLIT + part) * p.n_chunks + c) * 8192;
@@ -255,72 +310,60 @@ __global__ void __launch_bounds__(kFuThreads, 1) gyx_fused_kernel(const __grid_c
                         mbar_arrive(&sh.a_full[s]);
                     }
                 }
-            }
-        }
-        if (tid == 0) bulk_wait_all();
-    } else if (warp < (kFuPool + kFuEpi) / 32) {
-        // ================= epilogue warps: lane quarter warp & 3, interleaved 32-column chunks =================
-        const int et = tid - kFuPool, ew = et >> 5;
-        const int quarter = warp & 3, half = ew >> 2;
-        T* gx = static_cast<T*>(p.gX);
-        const size_t plane = (size_t)p.H * p.W;
-        const uint32_t m = (uint32_t)(quarter * 32 + lane);
-        uint32_t img_l, rem, a_l, b;
-        p.div_RTWp.divmod(m, img_l, rem);
-        p.div_Wp.divmod(rem, a_l, b);
-        int iq = 0;
-        for (int it = 0; it < n_my && ok && has_mma; ++it) {
-            const long long tile = first + (long long)it * stride;
-            int n0, a0;
-            fu_tile(p, tile, n0, a0);
-            const bool valid = (int)m < p.PT && n0 + (int)img_l < p.N && a0 + (int)a_l < p.Hp;
-            T* base_m = gx + ((size_t)(n0 + (int)img_l) * p.C_in) * plane + (size_t)((a0 + (int)a_l) * R) * p.W + (size_t)b * R;
-            for (int g = 0; g < p.n_groups && ok; ++g, ++iq) {
-                const int buf = iq & 1;
-                const int ci0 = g * p.NG;
-                const int ng = min(p.NG, p.C_in - ci0);
-                ok = mbar_wait_bounded(&sh.acc_full[buf], (uint32_t)(iq >> 1) & 1u);
-                tc_fence_after_sync();
-                if (ok) {
-                    for (int c = half * 32; c < ng; c += 64) {
-                        uint32_t v[32];
-                        tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * p.NGs + c), v);
-                        tmem_ld_wait();
-                        if (valid) {
-                            T* dst = base_m + (size_t)(ci0 + c) * plane;
+                if (!has_mma || !ok) continue;
+                // the c_i groups this pass has fed
+                const int g_lo = p.reuse ? 0 : pass, g_hi = p.reuse ? p.n_groups : pass + 1;
+                for (int g = g_lo; g < g_hi && ok; ++g, ++iq) {
+                    const int buf = iq % n_acc;
+                    const int ci0 = g * p.NG;
+                    const int ng = min(p.NG, p.C_in - ci0);
+                    ok = mbar_wait_bounded(&sh.acc_full[buf], (uint32_t)(iq / n_acc) & 1u);
+                    tc_fence_after_sync();
+                    if (ok) {
+                        for (int c = cset * 32; c < ng; c += 128) {
+                            uint32_t v[32];
+                            tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * p.NGs + c), v);
+                            tmem_ld_wait();
+                            if (e_valid) {
+                                T* dst = base_m + (size_t)(ci0 + c) * plane;
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) {
-                                if (c + i < ng) {
-                                    const float val = __uint_as_float(v[i]);
+                                for (int i = 0; i < 32; ++i) {
+                                    if (c + i < ng) {
+                                        const float val = __uint_as_float(v[i]);
 #pragma unroll
-                                    for (int dr = 0; dr < R; ++dr) fu_store_rep<R>(dst + (size_t)i * plane + (size_t)dr * p.W, val);
+                                        for (int dr = 0; dr < R; ++dr) fu_store_rep<R>(dst + (size_t)i * plane + (size_t)dr * p.W, val);
+                                    }
                                 }
                             }
                         }
                     }
+                    tc_fence_before_sync();
+                    if (bar_any(1, kFuWork, !ok)) { ok = false; break; }
+                    if (tid == 0) mbar_arrive(&sh.acc_empty[buf]);
                 }
-                tc_fence_before_sync();
-                if (bar_any(2, kFuEpi, !ok)) { ok = false; break; }
-                if (et == 0) mbar_arrive(&sh.acc_empty[buf]);
             }
         }
+        if (tid == 0) bulk_wait_all();
     } else if (warp == kFuRawWarp) {
         // ================= copy engine: g_y slabs =================
+        // A slab: for each piece of the tile's run of pixels, a box of kc_raw channels of the
+        // tile's images.  What a box covers beyond the tensor (channels, images, pixels) arrives
+        // as zeros; pixels of the image's further rows arrive as they are and are masked later.
         if (lane == 0) {
             int rq = 0;
             for (int it = 0; it < n_my && ok; ++it) {
                 const long long tile = first + (long long)it * stride;
                 int n0, a0;
-                fu_tile(p, tile, n0, a0);
+                fu_tile(p.IT, p.RT, p.div_N, tile, n0, a0);
                 const int x0 = a0 * p.r * p.W;
-                for (int g = 0; g < n_pool_groups && ok; ++g)
+                for (int pass = 0; pass < n_pass && ok; ++pass)
                     for (int c = 0; c < p.n_chunks && ok; ++c)
                         for (int sub = 0; sub < p.n_sub && ok; ++sub, ++rq) {
                             const int rs = rq % RS;
                             if (rq >= RS) ok = mbar_wait_bounded(&sh.raw_empty[rs], (uint32_t)(rq / RS - 1) & 1u);
                             if (!ok) break;
                             unsigned char* dst = raw_ring + (size_t)rs * p.raw_stage_bytes;
-                            mbar_expect_tx(&sh.raw_full[rs], (uint32_t)p.raw_tx_bytes);
+                            mbar_expect_tx(&sh.raw_full[rs], (uint32_t)(p.pieces * p.piece_bytes));
                             for (int pc = 0; pc < p.pieces; ++pc)
                                 tma_load_3d(dst + (size_t)pc * p.piece_bytes, &p.tm_gy, x0 + pc * p.PW, c * kTcBK + sub * p.kc_raw, n0,
                                             &sh.raw_full[rs]);
@@ -350,11 +393,11 @@ __global__ void __launch_bounds__(kFuThreads, 1) gyx_fused_kernel(const __grid_c
             for (int it = 0; it < n_my && ok && has_mma; ++it) {
                 const int a_base = aq;
                 for (int g = 0; g < p.n_groups && ok; ++g, ++iq) {
-                    const int buf = iq & 1;
+                    const int buf = iq % n_acc;
                     const int ng16 = (min(p.NG, p.C_in - g * p.NG) + 15) & ~15;
                     const uint32_t idesc = umma_idesc_bf16(128, ng16, /*A MN-major*/ 1, /*B K-major*/ 0);
                     const uint32_t d_tmem = tmem + (uint32_t)(buf * p.NGs);
-                    if (iq >= 2) ok = mbar_wait_bounded(&sh.acc_empty[buf], (uint32_t)((iq >> 1) - 1) & 1u);
+                    if (iq >= n_acc) ok = mbar_wait_bounded(&sh.acc_empty[buf], (uint32_t)(iq / n_acc - 1) & 1u);
                     const bool pooled = (g == 0) || !p.reuse;
                     const bool release = (g == p.n_groups - 1) || !p.reuse;
                     for (int c = 0; c < p.n_chunks && ok; ++c, ++bq) {
@@ -401,25 +444,27 @@ __global__ void __launch_bounds__(kFuThreads, 1) gyx_fused_kernel(const __grid_c
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    if (warp == kFuMmaWarp) tmem_dealloc(tmem, (uint32_t)(2 * p.NGs));
+    if (warp == kFuMmaWarp) tmem_dealloc(tmem, (uint32_t)(n_acc * p.NGs));
 }
 
 // ================================================================== gw_tiled
-constexpr int kGtLoaders = 256;     // 8 loader / epilogue warps + 1 MMA warp
-constexpr int kGtThreads = 288;
+constexpr int kGtWork = 256;        // warps 0-7: stash rows (copy / conversion) and the epilogue
+constexpr int kGtMmaWarp = 8, kGtCopyWarp = 9;
+constexpr int kGtThreads = 320;
 constexpr int kGtStagesMax = 6;
 __host__ __device__ constexpr int gt_stages(int split) { return split == 2 ? 3 : 6; }
 
 struct GwTiledParams {
+    CUtensorMap tm_stash;           // TMAB: the stash as [N][C_in][P], box {64, 128, 1} (bf16: 128-byte swizzle)
     const unsigned char* gbar_t;    // [tile][mb][part][c_o chunk][8 KB]
     const void* stash;              // dense [N][C_in][P] in the layer's dtype
     float* gwu;                     // [C_out][C_in] fp32, zeroed beforehand; every CTA adds its slice
     uint32_t* err_word;
     int N, C_in, C_out, Hp, Wp, P;
-    int IT, RT, tiles_per_img, MB, n_chunks, S;
+    int IT, RT, MB, n_chunks, S;
     int logv;                       // log2 of the stash elements per asynchronous copy piece (pieces of 4, 8 or 16 bytes)
     long long kchunks;              // tiles * MB
-    FastDiv div_tiles_per_img, div_P, div_MB;
+    FastDiv div_N, div_P, div_MB;
 };
 
 struct GtShared {
@@ -434,15 +479,51 @@ __device__ __forceinline__ void cp_async_bytes(uint32_t dst, const void* src, in
     else asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
 
+// fp32 rows [128][64] at `bt` -> the (high, low) bf16 K-major tiles, in place (high at bt,
+// low 16 KB behind it).  Thread t takes the 16-byte pieces t, t + 256, ...: sixteen
+// consecutive lanes read one 256-byte row and write one 128-byte row of each tile, both
+// without bank conflicts.  Every piece is in registers before any is overwritten.
+// Returns false when some thread of the 256 reports a failed wait.
+__device__ __forceinline__ bool gt_split_in_place(unsigned char* bt, int tid, bool ok) {
+    float4 v[8];
+    if (ok) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = reinterpret_cast<const float4*>(bt)[tid + 256 * i];
+    }
+    if (bar_any(1, kGtWork, !ok)) return false;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const uint32_t idx = (uint32_t)(tid + 256 * i), row = idx >> 4, c4 = idx & 15u;
+        const uint32_t off = (row >> 3) * 1024u + (row & 7u) * 128u + ((((c4 >> 1) ^ row) & 7u) << 4) + ((c4 & 1u) << 3);
+        const __nv_bfloat16 h0 = __float2bfloat16_rn(v[i].x), h1 = __float2bfloat16_rn(v[i].y);
+        const __nv_bfloat16 h2 = __float2bfloat16_rn(v[i].z), h3 = __float2bfloat16_rn(v[i].w);
+        const __nv_bfloat162 ha = __halves2bfloat162(h0, h1), hb = __halves2bfloat162(h2, h3);
+        uint2 hi, lo;
+        hi.x = *reinterpret_cast<const uint32_t*>(&ha);
+        hi.y = *reinterpret_cast<const uint32_t*>(&hb);
+        lo.x = pack_bf16x2(v[i].x - __bfloat162float(h0), v[i].y - __bfloat162float(h1));
+        lo.y = pack_bf16x2(v[i].z - __bfloat162float(h2), v[i].w - __bfloat162float(h3));
+        *reinterpret_cast<uint2*>(bt + off) = hi;
+        *reinterpret_cast<uint2*>(bt + 16384 + off) = lo;
+    }
+    return true;
+}
+
 // T: dtype of the stash.  fp32: the rows land as fp32 [128][64] in the stage's B region and are
-// split in place into the (high, low) bf16 tiles; bf16: the pieces land at their swizzled places.
-template <typename T>
-__global__ void __launch_bounds__(kGtThreads) gw_tiled_kernel(const GwTiledParams p) {
+// split in place into the (high, low) bf16 tiles; bf16: they land at their swizzled places.
+// TMAB: the stash rows come by tensor-map copies issued by the copy warp (every 64-patch
+// block starts on a 16-byte boundary; slots of a block that hold no patch of the tile may
+// then carry other patches' sums -- their patch means are exact zeros); otherwise by
+// asynchronous copies of 4-, 8- or 16-byte pieces issued by the workers, with such slots
+// filled with zeros.
+template <typename T, bool TMAB>
+__global__ void __launch_bounds__(kGtThreads) gw_tiled_kernel(const __grid_constant__ GwTiledParams p) {
     constexpr int SPLIT = sizeof(T) == 4 ? 2 : 1;
     constexpr int ST = gt_stages(SPLIT);
     constexpr int kABytes = 128 * kTcBK * 2;                 // 16 KB per part
     constexpr int kBOff = SPLIT * kABytes;                   // stage: [A hi][A lo][B hi][B lo]
     constexpr int kStageBytes = 2 * SPLIT * kABytes;
+    constexpr uint32_t kBBytes = 128u * kTcBK * (uint32_t)sizeof(T);
     constexpr uint32_t kIdesc = umma_idesc_bf16(128, 128, 0, 0);
     extern __shared__ unsigned char dyn_raw[];
     __shared__ GtShared sh;
@@ -456,13 +537,17 @@ __global__ void __launch_bounds__(kGtThreads) gw_tiled_kernel(const GwTiledParam
 
     pdl_launch_dependents();
     if (tid == 0) {
+        // full: the copy engine's bytes (one arrival that announces them) plus, unless the stash
+        // rows come ready-made from the copy engine, one arrival per worker
+        // (asynchronous copies arrive per thread; after the in-place split of fp32 rows one lane per warp arrives)
+        const uint32_t full_count = (TMAB && SPLIT == 1) ? 1u : SPLIT == 2 ? 1u + kGtWork / 32 : 1u + kGtWork;
         for (int s = 0; s < ST; ++s) {
-            mbar_init(&sh.full[s], kGtLoaders + 1); mbar_init(&sh.empty[s], 1); mbar_init(&sh.landed[s], kGtLoaders);
+            mbar_init(&sh.full[s], full_count); mbar_init(&sh.empty[s], 1); mbar_init(&sh.landed[s], TMAB ? 1u : (uint32_t)kGtWork);
         }
         mbar_init(&sh.accum, 1);
         mbar_fence_init();
     }
-    if (warp == 8) { tmem_alloc(&sh.tmem_base, 128); tmem_relinquish(); }
+    if (warp == kGtMmaWarp) { tmem_alloc(&sh.tmem_base, 128); tmem_relinquish(); }
     if (a_blocks < 2)     // rows 64..127 of the A tiles are never loaded: keep them finite
         for (int i = tid; i < ST * SPLIT * 512; i += kGtThreads) {
             const int s = i / (SPLIT * 512), rest = i % (SPLIT * 512);
@@ -475,96 +560,89 @@ __global__ void __launch_bounds__(kGtThreads) gw_tiled_kernel(const GwTiledParam
     const uint32_t tmem = sh.tmem_base;
     pdl_wait();                       // operands come from the previous kernels of the stream
     bool ok = true;
+    // the patch-mean blocks of chunk q: one bulk copy per part, announced on full[s]
+    auto issue_a = [&](int q, unsigned char* stage, uint64_t* bar, uint32_t extra_bytes) {
+        uint32_t tile, mb;
+        p.div_MB.divmod((uint32_t)(kc_begin + q), tile, mb);
+        mbar_expect_tx(bar, (uint32_t)(SPLIT * a_blocks * 8192) + extra_bytes);
+        for (int part = 0; part < SPLIT; ++part)
+            bulk_g2s(stage + part * kABytes, p.gbar_t + ((((size_t)tile * p.MB + mb) * SPLIT + part) * p.n_chunks + co_blk) * 8192,
+                     (uint32_t)(a_blocks * 8192), bar);
+    };
 
-    if (warp < 8) {
-        const int V = 1 << p.logv;                          // elements per piece
-        const int piece_bytes = V * (int)sizeof(T);
-        const int ppr = kTcBK / V;                          // pieces per row
-        const int row_step = kGtLoaders / ppr;
-        const int k_me = (tid % ppr) * V, row0 = tid / ppr;
-        const T* st = static_cast<const T*>(p.stash);
-        // enqueue the copies of chunk q into its stage
-        auto issue = [&](int q) {
-            const int s = q % ST;
-            unsigned char* stage = dyn + (size_t)s * kStageBytes;
-            uint32_t tile, mb;
-            p.div_MB.divmod((uint32_t)(kc_begin + q), tile, mb);
-            if (tid == 0) {                                 // the patch-mean blocks: one bulk copy per part
-                mbar_expect_tx(&sh.full[s], (uint32_t)(SPLIT * a_blocks * 8192));
-                for (int part = 0; part < SPLIT; ++part)
-                    bulk_g2s(stage + part * kABytes,
-                             p.gbar_t + ((((size_t)tile * p.MB + mb) * SPLIT + part) * p.n_chunks + co_blk) * 8192,
-                             (uint32_t)(a_blocks * 8192), &sh.full[s]);
+    if (warp < kGtWork / 32) {
+        if constexpr (!TMAB) {
+            const int V = 1 << p.logv;                          // elements per piece
+            const int piece_bytes = V * (int)sizeof(T);
+            const int ppr = kTcBK / V;                          // pieces per row
+            const int row_step = kGtWork / ppr;
+            const int k_me = (tid % ppr) * V, row0 = tid / ppr;
+            const T* st = static_cast<const T*>(p.stash);
+            // enqueue the copies of chunk q into its stage
+            auto issue = [&](int q) {
+                const int s = q % ST;
+                unsigned char* stage = dyn + (size_t)s * kStageBytes;
+                uint32_t tile, mb;
+                p.div_MB.divmod((uint32_t)(kc_begin + q), tile, mb);
+                if (tid == 0) issue_a(q, stage, &sh.full[s], 0u);
+                // this thread's piece: patches m .. m+V-1 of the tile
+                const int m = (int)mb * 64 + k_me;
+                int n_img, p0, nvalid;
+                if (p.IT > 1) {
+                    uint32_t il, pp;
+                    p.div_P.divmod((uint32_t)m, il, pp);
+                    n_img = (int)tile * p.IT + (int)il;
+                    p0 = (int)pp;
+                    nvalid = ((int)il < p.IT && n_img < p.N) ? V : 0;
+                } else {
+                    int a0;
+                    fu_tile(1, p.RT, p.div_N, tile, n_img, a0);
+                    const int lim = min(p.RT, p.Hp - a0) * p.Wp - m;
+                    p0 = a0 * p.Wp + m;
+                    nvalid = lim < 0 ? 0 : (lim < V ? lim : V);
+                }
+                const T* src0 = st + ((size_t)n_img * p.C_in + ci0 + row0) * p.P + p0;
+                const size_t step = (size_t)row_step * p.P;
+                const uint32_t bdst = smem_u32(stage + kBOff);
+                for (int i = 0, row = row0; row < 128; ++i, row += row_step) {
+                    const bool rv = nvalid > 0 && ci0 + row < p.C_in;
+                    const uint32_t dst = SPLIT == 2 ? bdst + (uint32_t)(row * 256 + k_me * 4) : bdst + kmajor_off((uint32_t)row, (uint32_t)k_me);
+                    cp_async_bytes(dst, rv ? (const void*)(src0 + i * step) : (const void*)st, piece_bytes,
+                                   rv ? (uint32_t)(nvalid * (int)sizeof(T)) : 0u);
+                }
+                if constexpr (SPLIT == 2)
+                    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&sh.landed[s])) : "memory");
+                else
+                    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&sh.full[s])) : "memory");
+            };
+            const int ahead = ST - 1;
+            for (int q = 0; q < ahead && q < n_chunks; ++q) issue(q);
+            for (int q = 0; q < n_chunks && ok; ++q) {
+                const int qa = q + ahead;
+                if (qa < n_chunks) {
+                    if (qa >= ST) ok = mbar_wait_bounded(&sh.empty[qa % ST], (uint32_t)(qa / ST - 1) & 1u);
+                    if (ok) issue(qa);
+                }
+                if constexpr (SPLIT == 2) {
+                    const int s = q % ST;
+                    ok = mbar_wait_bounded(&sh.landed[s], (uint32_t)(q / ST) & 1u);
+                    if (!gt_split_in_place(dyn + (size_t)s * kStageBytes + kBOff, tid, ok)) { ok = false; break; }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sh.full[s]);
+                }
             }
-            // this thread's piece: patches m .. m+V-1 of the tile
-            const int m = (int)mb * 64 + k_me;
-            int n_img, p0, nvalid;
-            if (p.IT > 1) {
-                uint32_t il, pp;
-                p.div_P.divmod((uint32_t)m, il, pp);
-                n_img = (int)tile * p.IT + (int)il;
-                p0 = (int)pp;
-                nvalid = ((int)il < p.IT && n_img < p.N) ? V : 0;
-            } else {
-                uint32_t n, ti;
-                p.div_tiles_per_img.divmod(tile, n, ti);
-                const int a0 = (int)ti * p.RT;
-                const int lim = min(p.RT, p.Hp - a0) * p.Wp - m;
-                n_img = (int)n;
-                p0 = a0 * p.Wp + m;
-                nvalid = lim < 0 ? 0 : (lim < V ? lim : V);
-            }
-            const T* src0 = st + ((size_t)n_img * p.C_in + ci0 + row0) * p.P + p0;
-            const size_t step = (size_t)row_step * p.P;
-            const uint32_t bdst = smem_u32(stage + kBOff);
-            for (int i = 0, row = row0; row < 128; ++i, row += row_step) {
-                const bool rv = nvalid > 0 && ci0 + row < p.C_in;
-                const uint32_t dst = SPLIT == 2 ? bdst + (uint32_t)(row * 256 + k_me * 4) : bdst + kmajor_off((uint32_t)row, (uint32_t)k_me);
-                cp_async_bytes(dst, rv ? (const void*)(src0 + i * step) : (const void*)st, piece_bytes,
-                               rv ? (uint32_t)(nvalid * (int)sizeof(T)) : 0u);
-            }
-            if constexpr (SPLIT == 2)
-                asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&sh.landed[s])) : "memory");
-            else
-                asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&sh.full[s])) : "memory");
-        };
-        const int ahead = ST - 1;
-        for (int q = 0; q < ahead && q < n_chunks; ++q) issue(q);
-        for (int q = 0; q < n_chunks && ok; ++q) {
-            const int qa = q + ahead;
-            if (qa < n_chunks) {
-                if (qa >= ST) ok = mbar_wait_bounded(&sh.empty[qa % ST], (uint32_t)(qa / ST - 1) & 1u);
-                if (ok) issue(qa);
-            }
-            if constexpr (SPLIT == 2) {
-                // fp32 rows -> (high, low) bf16 tiles, in place: thread = (row, half of the row)
+            cp_async_wait_all();
+        } else if constexpr (SPLIT == 2) {
+            for (int q = 0; q < n_chunks && ok; ++q) {
                 const int s = q % ST;
                 ok = mbar_wait_bounded(&sh.landed[s], (uint32_t)(q / ST) & 1u);
-                unsigned char* bt = dyn + (size_t)s * kStageBytes + kBOff;
-                const int row = tid >> 1, hf = tid & 1;
-                float v[32];
-                if (ok) load_span<32>(reinterpret_cast<const float*>(bt + row * 256 + hf * 128), v);
-                // every row is in registers before any is overwritten
-                if (bar_any(1, kGtLoaders, !ok)) { ok = false; break; }
-                uint32_t hi[16], lo[16];
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const __nv_bfloat16 h0 = __float2bfloat16_rn(v[2 * j]), h1 = __float2bfloat16_rn(v[2 * j + 1]);
-                    const __nv_bfloat162 h2 = __halves2bfloat162(h0, h1);
-                    hi[j] = *reinterpret_cast<const uint32_t*>(&h2);
-                    lo[j] = pack_bf16x2(v[2 * j] - __bfloat162float(h0), v[2 * j + 1] - __bfloat162float(h1));
-                }
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const uint32_t off = kmajor_off((uint32_t)row, (uint32_t)(hf * 32 + c * 8));
-                    *reinterpret_cast<uint4*>(bt + off) = make_uint4(hi[4 * c], hi[4 * c + 1], hi[4 * c + 2], hi[4 * c + 3]);
-                    *reinterpret_cast<uint4*>(bt + kABytes + off) = make_uint4(lo[4 * c], lo[4 * c + 1], lo[4 * c + 2], lo[4 * c + 3]);
-                }
+                if (!gt_split_in_place(dyn + (size_t)s * kStageBytes + kBOff, tid, ok)) { ok = false; break; }
                 fence_proxy_async_smem();
-                mbar_arrive(&sh.full[s]);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.full[s]);
             }
         }
-        cp_async_wait_all();
         if (ok && n_chunks > 0) ok = mbar_wait_bounded(&sh.accum, 0);
         tc_fence_after_sync();
         if (ok && n_chunks > 0) {
@@ -589,13 +667,37 @@ __global__ void __launch_bounds__(kGtThreads) gw_tiled_kernel(const GwTiledParam
                 }
             }
         }
-    } else if (lane == 0) {
-        for (int q = 0; q < n_chunks && ok; ++q) {
-            const uint32_t a_addr = smem_u32(dyn + (size_t)(q % ST) * kStageBytes);
-            ok = mma_chunk<ST, SPLIT>(sh.full, sh.empty, q, q == 0, a_addr, a_addr + kABytes, a_addr + kBOff,
-                                      a_addr + kBOff + kABytes, tmem, kIdesc, 32, 16);
+    } else if (warp == kGtMmaWarp) {
+        if (lane == 0) {
+            for (int q = 0; q < n_chunks && ok; ++q) {
+                const uint32_t a_addr = smem_u32(dyn + (size_t)(q % ST) * kStageBytes);
+                ok = mma_chunk<ST, SPLIT>(sh.full, sh.empty, q, q == 0, a_addr, a_addr + kABytes, a_addr + kBOff,
+                                          a_addr + kBOff + kABytes, tmem, kIdesc, 32, 16);
+            }
+            if (ok && n_chunks > 0) umma_commit(&sh.accum);
         }
-        if (ok && n_chunks > 0) umma_commit(&sh.accum);
+    } else if (warp == kGtCopyWarp && TMAB) {
+        // ================= copy engine: both operands =================
+        if (lane == 0) {
+            for (int q = 0; q < n_chunks && ok; ++q) {
+                const int s = q % ST;
+                if (q >= ST) ok = mbar_wait_bounded(&sh.empty[s], (uint32_t)(q / ST - 1) & 1u);
+                if (!ok) break;
+                unsigned char* stage = dyn + (size_t)s * kStageBytes;
+                issue_a(q, stage, &sh.full[s], SPLIT == 1 ? kBBytes : 0u);
+                uint32_t tile, mb;
+                p.div_MB.divmod((uint32_t)(kc_begin + q), tile, mb);
+                int n_img, x;
+                if (p.IT > 1) { n_img = (int)tile * p.IT + (int)mb; x = 0; }            // P == 64: block mb is image mb of the tile
+                else { int a0; fu_tile(1, p.RT, p.div_N, tile, n_img, a0); x = a0 * p.Wp + (int)mb * 64; }
+                if constexpr (SPLIT == 2) {
+                    mbar_expect_tx(&sh.landed[s], kBBytes);
+                    tma_load_3d(stage + kBOff, &p.tm_stash, x, ci0, n_img, &sh.landed[s]);
+                } else {
+                    tma_load_3d(stage + kBOff, &p.tm_stash, x, ci0, n_img, &sh.full[s]);
+                }
+            }
+        }
     }
     if (!ok) {
         atomicOr(p.err_word, 32u);
@@ -605,19 +707,20 @@ __global__ void __launch_bounds__(kGtThreads) gw_tiled_kernel(const GwTiledParam
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    if (warp == 8) tmem_dealloc(tmem, 128);
+    if (warp == kGtMmaWarp) tmem_dealloc(tmem, 128);
 }
 
 // ================================================================== host side
 static int round_up_int(int v, int a) { return (v + a - 1) / a * a; }
+static int gcd_int(int a, int b) { while (b) { const int t = a % b; a = b; b = t; } return a; }
 
 static FusedPlan fused_plan(const Geo& g) {
     FusedPlan f;
     if (!tc_eligible(g)) return f;
     const int r = g.r, e = (int)g.esize;
     if (!(r == 2 || r == 4 || r == 8) || g.H % r != 0 || g.W % r != 0) return f;
-    if (g.Wp > 128 || g.W > 256) return f;
-    if (((long long)g.H * g.W * e) % 16 != 0) return f;                 // plane stride of the g_y tensor map
+    if (g.Wp > 128) return f;
+    if (((long long)g.H * g.W * e) % 16 != 0) return f;                 // every plane of g_y starts on a 16-byte boundary
     f.parts = g.dtype == GF_F32 ? 2 : 1;
     const int P = g.Hp * g.Wp;
     if (P <= 64) {
@@ -626,34 +729,49 @@ static FusedPlan fused_plan(const Geo& g) {
         f.RT = g.Hp;
         f.tiles_per_img = 1;
         f.tiles = ((long long)g.N + f.IT - 1) / f.IT;
+        f.run = g.H * g.W;
+        f.stash_tma = P == 64 && ((long long)P * e) % 16 == 0;
     } else {
         const int rt0 = g.Hp < 128 / g.Wp ? g.Hp : 128 / g.Wp;
         f.tiles_per_img = (g.Hp + rt0 - 1) / rt0;
         f.RT = (g.Hp + f.tiles_per_img - 1) / f.tiles_per_img;          // even tiles
+        // Tiles whose first patch sits on a 16-byte boundary of the stash rows let the g_W
+        // contraction fetch those rows with tensor-map copies: taken when it costs no extra tile.
+        const int q = 16 / gcd_int(16, (g.Wp * e) % 16 == 0 ? 16 : (g.Wp * e) % 16);
+        const int rt_al = rt0 / q * q;
+        if (rt_al >= 1 && ((long long)P * e) % 16 == 0 && (g.Hp + rt_al - 1) / rt_al == f.tiles_per_img) {
+            f.RT = rt_al;
+            f.stash_tma = true;
+        }
         f.tiles_per_img = (g.Hp + f.RT - 1) / f.RT;
         f.IT = 1;
         f.tiles = (long long)g.N * f.tiles_per_img;
-        if (((long long)f.RT * r * g.W * e) % 16 != 0) return f;         // every tile starts on a 16-byte boundary
+        if (((long long)f.RT * r * g.W * e) % 16 != 0) return f;         // every tile starts on a 16-byte boundary of g_y
+        f.run = f.RT * r * g.W;
     }
-    // copy pieces: pr pixel rows (whole patch rows), at most 256 elements, a multiple of 16 bytes;
-    // the least overshoot past the tile's rows first, then the largest piece
-    const int band = f.RT * r;
-    int best_over = 1 << 30;
-    for (int pr = r; pr <= band && pr * g.W <= 256; pr += r) {
-        if ((pr * g.W * e) % 16 != 0) continue;
-        const int pieces = (band + pr - 1) / pr, over = pieces * pr - band;
-        if (over < best_over || (over == best_over && pr > f.pr)) { best_over = over; f.pr = pr; f.pieces = pieces; }
-    }
-    if (f.pr == 0) return f;
-    f.PW = f.pr * g.W;
     f.PT = f.IT * f.RT * g.Wp;
     f.MB = f.PT > 64 ? 2 : 1;
     f.G = g.Wp % 2 == 0 ? 2 : 1;
-    const long long per_ch = (long long)f.pieces * f.IT * f.PW * e;      // bytes of one channel of a raw slab
-    if (per_ch > kFuRawBudget) return f;
-    f.kc_raw = 64;
-    while ((long long)f.kc_raw * per_ch > kFuRawBudget) f.kc_raw >>= 1;
-    f.raw_stage_bytes = (size_t)round_up_int((int)(f.kc_raw * per_ch), 1024);
+    // Pieces of the run: as few boxes as the 256-element limit allows, of equal width, a multiple
+    // of 16 bytes and of the widest shared-memory access of the pooling threads; every box must
+    // land on a 128-byte boundary of the slab, which narrow slabs get from 128-byte-wide pieces.
+    int unit = f.G * r;
+    while ((unit * e) % 16 != 0) unit *= 2;
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        f.pieces = (f.run + 255) / 256;
+        for (;; ++f.pieces) {
+            f.PW = round_up_int((f.run + f.pieces - 1) / f.pieces, unit);
+            if (f.PW <= 256) break;
+        }
+        const long long per_ch = (long long)f.IT * f.pieces * f.PW * e;      // bytes of one channel of a raw slab
+        if (per_ch > kFuRawBudget) return f;
+        f.kc_raw = 64;
+        while ((long long)f.kc_raw * per_ch > kFuRawBudget) f.kc_raw >>= 1;
+        f.raw_stage_bytes = (size_t)round_up_int((int)(f.kc_raw * per_ch), 128);
+        if (((long long)f.IT * f.kc_raw * f.PW * e) % 128 == 0) break;
+        if (attempt == 1) return f;
+        while ((unit * e) % 128 != 0) unit *= 2;
+    }
     f.n_sub = 64 / f.kc_raw;
     f.n_chunks = (g.C_out + 63) / 64;
     const int ng_max = 256 / f.parts;
@@ -699,42 +817,43 @@ gf_status launch_gyx_fused(const void* gy, const __nv_bfloat16* thetaT, long lon
     const FusedPlan f = fused_plan(g);
     if (!f.ok) return GF_ERR_UNSUPPORTED;
     FusedParams p;
-    if (!make_tmap_plain(&p.tm_gy, gy, (int)g.esize, (uint64_t)g.H * g.W, (uint64_t)g.C_out, (uint64_t)g.N,
-                         (uint64_t)g.H * g.W, (uint64_t)g.C_out * g.H * g.W, (uint32_t)f.PW, (uint32_t)f.kc_raw, (uint32_t)f.IT))
-        return GF_ERR_CUDA;
     const uint64_t part_stride = f.parts == 2 ? (uint64_t)theta_lo_off : (uint64_t)g.C_in * g.C_out;
     if (!make_tmap_bf16(&p.tm_theta, thetaT, 3, (uint64_t)g.C_out, (uint64_t)g.C_in, (uint64_t)f.parts, (uint64_t)g.C_out,
                         part_stride, (uint32_t)f.NG))
         return GF_ERR_CUDA;
+    if (!make_tmap_plain(&p.tm_gy, gy, (int)g.esize, (uint64_t)g.H * g.W, (uint64_t)g.C_out, (uint64_t)g.N,
+                         (uint64_t)g.H * g.W, (uint64_t)g.C_out * g.H * g.W, (uint32_t)f.PW, (uint32_t)f.kc_raw, (uint32_t)f.IT))
+        return GF_ERR_CUDA;
     p.gX = gX; p.gbar_t = gbar_t; p.err_word = err_word;
     p.N = g.N; p.C_in = g.C_in; p.C_out = g.C_out; p.H = g.H; p.W = g.W; p.Hp = g.Hp; p.Wp = g.Wp; p.r = g.r;
-    p.IT = f.IT; p.RT = f.RT; p.tiles_per_img = f.tiles_per_img; p.pr = f.pr; p.PW = f.PW; p.pieces = f.pieces;
+    p.IT = f.IT; p.RT = f.RT; p.PW = f.PW; p.pieces = f.pieces;
+    p.piece_bytes = f.IT * f.kc_raw * f.PW * (int)g.esize;
+    p.div_PW = FastDiv((uint32_t)f.PW);
     p.kc_raw = f.kc_raw; p.n_sub = f.n_sub; p.MB = f.MB; p.PT = f.PT; p.PTG = f.PT / f.G; p.NG = f.NG;
     int ngs = 32;
     while (ngs < f.NG) ngs <<= 1;
     p.NGs = ngs;
+    p.n_acc = 512 / ngs < kFuAccMax ? 512 / ngs : kFuAccMax;
+    p.kpar = kFuWork / p.PTG;
     p.n_groups = f.n_groups; p.n_chunks = f.n_chunks; p.reuse = f.reuse ? 1 : 0;
     p.a_stages = f.a_stages; p.raw_stages = f.raw_stages; p.raw_stage_bytes = (int)f.raw_stage_bytes;
-    p.piece_bytes = f.IT * f.kc_raw * f.PW * (int)g.esize;
-    p.raw_tx_bytes = f.pieces * p.piece_bytes;
     p.tiles = f.tiles;
     p.div_PTG = FastDiv((uint32_t)p.PTG);
-    p.div_tiles_per_img = FastDiv((uint32_t)f.tiles_per_img);
+    p.div_N = FastDiv((uint32_t)g.N);
     p.div_RTWp = FastDiv((uint32_t)(f.RT * g.Wp));
     p.div_Wp = FastDiv((uint32_t)g.Wp);
-    p.div_ppr = FastDiv((uint32_t)(f.pr / g.r));
     p.inv_area = 1.0f / ((float)g.r * (float)g.r);
     if (g.dtype == GF_F32) return launch_fused_t<float>(p, f.G, f.smem, s);
     return launch_fused_t<__nv_bfloat16>(p, f.G, f.smem, s);
 }
 
-template <typename T>
+template <typename T, bool TMAB>
 static gf_status launch_gw_tiled_inst(const GwTiledParams& p, dim3 grid, cudaStream_t s) {
     constexpr int SPLIT = sizeof(T) == 4 ? 2 : 1;
     constexpr size_t smem = (size_t)gt_stages(SPLIT) * 2 * SPLIT * 16384 + 1024;
     static size_t configured[kMaxDevices] = {};
-    if (gf_status st = ensure_dyn_smem(gw_tiled_kernel<T>, smem, configured); st != GF_OK) return st;
-    return launch_pdl(gw_tiled_kernel<T>, grid, dim3(kGtThreads), smem, s, p);
+    if (gf_status st = ensure_dyn_smem(gw_tiled_kernel<T, TMAB>, smem, configured); st != GF_OK) return st;
+    return launch_pdl(gw_tiled_kernel<T, TMAB>, grid, dim3(kGtThreads), smem, s, p);
 }
 
 // Widest asynchronous-copy piece (log2 of its elements) with which the stash rows of every
@@ -744,8 +863,7 @@ static int gw_tiled_logv(const Geo& g, const FusedPlan& f) {
     const int P = g.Hp * g.Wp;
     // element offsets a piece may start at are multiples of gcd(P, tile stride in patches, V)
     int unit = P;
-    auto gcd = [](int a, int b) { while (b) { const int t = a % b; a = b; b = t; } return a; };
-    if (f.IT == 1) unit = gcd(unit, f.RT * g.Wp);
+    if (f.IT == 1) unit = gcd_int(unit, f.RT * g.Wp);
     for (int lv = e == 4 ? 2 : 3; lv >= 0; --lv) {
         const int V = 1 << lv;
         if (V * e < 4) break;
@@ -759,6 +877,17 @@ bool fused_path_ok(const Geo& g) {
     return f.ok && gw_tiled_logv(g, f) >= 0 && (g.C_out + 127) / 128 <= 65535 && (g.C_out + 31) / 32 <= 65535;
 }
 
+// Measured on the layer shapes of the benchmark (B200): the fused pair wins when every SM gets
+// a tile and the layer either writes far more g_X than it reads g_y (the separate g_X kernel
+// shares the SMs with the g_W kernel there) or has few channels (one c_i group, short
+// contractions); elsewhere the pooling pass plus the two contractions side by side are faster,
+// because the g_W contraction of the fused pair cannot start before the fused kernel has ended.
+bool fused_path_preferred(const Geo& g) {
+    const FusedPlan f = fused_plan(g);
+    if (!f.ok || f.tiles < sm_count()) return false;
+    return g.C_in >= 3 * g.C_out || (g.C_in <= 128 && g.C_out <= 128);
+}
+
 gf_status launch_gw_tiled(const unsigned char* gbar_t, const void* stash, float* gwu, uint32_t* err_word, const Geo& g,
                           cudaStream_t s) {
     ProfScope prof(K_GW_TILED, s);
@@ -767,23 +896,32 @@ gf_status launch_gw_tiled(const unsigned char* gbar_t, const void* stash, float*
     GwTiledParams p;
     p.gbar_t = gbar_t; p.stash = stash; p.gwu = gwu; p.err_word = err_word;
     p.N = g.N; p.C_in = g.C_in; p.C_out = g.C_out; p.Hp = g.Hp; p.Wp = g.Wp; p.P = g.Hp * g.Wp;
-    p.IT = f.IT; p.RT = f.RT; p.tiles_per_img = f.tiles_per_img; p.MB = f.MB; p.n_chunks = f.n_chunks;
+    p.IT = f.IT; p.RT = f.RT; p.MB = f.MB; p.n_chunks = f.n_chunks;
     p.logv = gw_tiled_logv(g, f);
     if (p.logv < 0) return GF_ERR_UNSUPPORTED;
     p.kchunks = f.tiles * f.MB;
-    p.div_tiles_per_img = FastDiv((uint32_t)f.tiles_per_img);
+    p.div_N = FastDiv((uint32_t)g.N);
     p.div_P = FastDiv((uint32_t)p.P);
     p.div_MB = FastDiv((uint32_t)f.MB);
+    // every CTA resident at once: output tiles times K slices within the SM count
     const int tiles_out = ((g.C_in + 127) / 128) * ((g.C_out + 127) / 128);
-    long long S = (sm_count() + tiles_out - 1) / tiles_out;
+    long long S = sm_count() / tiles_out;
     if (S > p.kchunks) S = p.kchunks;
     if (S < 1) S = 1;
     if (S > 65535) S = 65535;
     p.S = (int)S;
     if ((g.C_out + 127) / 128 > 65535) return GF_ERR_UNSUPPORTED;
     dim3 grid((g.C_in + 127) / 128, (g.C_out + 127) / 128, (unsigned)S);
-    if (g.dtype == GF_F32) return launch_gw_tiled_inst<float>(p, grid, s);
-    return launch_gw_tiled_inst<__nv_bfloat16>(p, grid, s);
+    bool tma_b = f.stash_tma;
+    if (tma_b) {
+        const uint64_t P = (uint64_t)p.P;
+        tma_b = g.dtype == GF_F32
+                    ? make_tmap_plain(&p.tm_stash, stash, 4, P, (uint64_t)g.C_in, (uint64_t)g.N, P, (uint64_t)g.C_in * P, 64, 128, 1)
+                    : make_tmap_bf16(&p.tm_stash, stash, 3, P, (uint64_t)g.C_in, (uint64_t)g.N, P, (uint64_t)g.C_in * P, 128);
+    }
+    if (g.dtype == GF_F32)
+        return tma_b ? launch_gw_tiled_inst<float, true>(p, grid, s) : launch_gw_tiled_inst<float, false>(p, grid, s);
+    return tma_b ? launch_gw_tiled_inst<__nv_bfloat16, true>(p, grid, s) : launch_gw_tiled_inst<__nv_bfloat16, false>(p, grid, s);
 }
 
 }  // namespace gf

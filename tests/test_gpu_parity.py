@@ -14,6 +14,16 @@ from parity_util import TOL, check_layer_full, check_layer_sampled, f64, relerr,
 pytestmark = pytest.mark.gpu
 
 
+@pytest.fixture(params=["auto", "fused"])
+def dense_path(gf, request):
+    """Both ways a dense layer can be computed: the library's own choice per layer, and the fused
+    gradient-filter + g_X kernel forced wherever it can run (layers it cannot take fall back to the
+    separate kernels).  The library's choice is restored afterwards."""
+    gf.gf_set_dense_path(gf.GF_PATH_FUSED if request.param == "fused" else gf.GF_PATH_AUTO)
+    yield request.param
+    gf.gf_set_dense_path(gf.GF_PATH_AUTO)
+
+
 def L(name, N, Cin, Cout, H, W, K, G, r, dtype="f32", x_dist="relu", gy_std=1e-2, idx=0):
     return Layer(name, 0, idx, N, Cin, Cout, H, W, K, G, r, dtype, x_dist, gy_std)
 
@@ -76,7 +86,7 @@ SMALL = [
 
 @pytest.mark.parametrize("layer", SMALL, ids=lambda l: l.name)
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_small_shapes_element_by_element(gf, layer, dtype):
+def test_small_shapes_element_by_element(gf, layer, dtype, dense_path):
     check_layer_full(gf, layer.with_(dtype=dtype))
 
 
@@ -134,6 +144,16 @@ def test_full_size_configs_element_by_element(gf, layer):
     check_layer_full(gf, layer, isolate=False)
 
 
+@pytest.mark.parametrize("layer", workloads.config2() + workloads.config3(2)[::2], ids=lambda l: f"{l.name}_r{l.r}_{l.dtype}")
+def test_full_size_fused_path_element_by_element(gf, layer):
+    """The fused kernels at full size on layers the library would give to the separate kernels."""
+    gf.gf_set_dense_path(gf.GF_PATH_FUSED)
+    try:
+        check_layer_full(gf, layer, isolate=False)
+    finally:
+        gf.gf_set_dense_path(gf.GF_PATH_AUTO)
+
+
 @pytest.mark.parametrize("layer", FULL_SAMPLED, ids=lambda l: f"{l.name}_r{l.r}_{l.dtype}")
 def test_full_size_configs_sampled(gf, layer):
     check_layer_sampled(gf, layer)
@@ -175,7 +195,7 @@ def _integer_inputs(layer, seed):
 
 @pytest.mark.parametrize("layer", EXACT, ids=lambda l: l.name)
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
-def test_exact_arithmetic_bit_for_bit(gf, layer, dtype):
+def test_exact_arithmetic_bit_for_bit(gf, layer, dtype, dense_path):
     layer = layer.with_(dtype=dtype)
     x, gy, w = _integer_inputs(layer, seed=4242)
     stash_ref = oracle.stash_forward(f64(x), layer.r)

@@ -28,8 +28,17 @@ CASES = [
 ]
 
 
+@pytest.fixture(params=["auto", "fused"])
+def dense_path(gf, request):
+    """The library's own choice of kernels for dense layers, and the fused gradient-filter kernel
+    forced wherever it can run: the built-in scratch has to serve both layouts."""
+    gf.gf_set_dense_path(gf.GF_PATH_FUSED if request.param == "fused" else gf.GF_PATH_AUTO)
+    yield request.param
+    gf.gf_set_dense_path(gf.GF_PATH_AUTO)
+
+
 @pytest.mark.parametrize("layer", CASES, ids=lambda l: l.name)
-def test_static_scratch_matches_gf_backward_twice(gf, layer):
+def test_static_scratch_matches_gf_backward_twice(gf, layer, dense_path):
     desc = gf.desc_for(layer)
     assert gf.gf_backward_workspace_bytes(desc) <= gf.GF_STATIC_SCRATCH_BYTES
     dt = workloads.torch_dtype(layer.dtype)
