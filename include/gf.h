@@ -84,6 +84,19 @@ gf_status gf_backward_workspace_bytes(const gf_conv_desc* desc, size_t* bytes);
 gf_status gf_stash_forward(const gf_conv_desc* desc, const void* x, void* stash,
                            void* stream);
 
+/* The forward-side step fused into the producer of x (Section 4.2 books the stash as the
+ * method's forward overhead; the supplement's on-device results show it can vanish): reads
+ * the pre-activation tensor z [N,C_in,H,W] once, writes x = act(z) -- which the layer's
+ * forward convolution consumes -- and the stash of that x, instead of a second pass over x.
+ * act: GF_ACT_NONE, GF_ACT_RELU (max(z,0)) or GF_ACT_RELU6 (min(max(z,0),6)), the
+ * activations of the paper's networks.  x may be z itself (in place); stash as in
+ * gf_stash_forward.  For r in {2,4,8} dividing H and W one streaming kernel does all
+ * three; other shapes run the activation and the pooling as two passes; r == 1 writes act(z)
+ * to both x and stash. */
+typedef enum gf_activation { GF_ACT_NONE = 0, GF_ACT_RELU = 1, GF_ACT_RELU6 = 2 } gf_activation;
+gf_status gf_act_stash_forward(const gf_conv_desc* desc, int32_t act, const void* z, void* x,
+                               void* stash, void* stream);
+
 /* Backward of one layer (Sections 3.3-3.4): from g_y, the stash written by
  * gf_stash_forward and the kernel W, write g_W (fp32, all KH*KW taps of an
  * input/output channel pair carry the same value when r >= 2) and g_X.  Either
@@ -140,6 +153,36 @@ gf_status gf_host_step_arena_bytes(const gf_conv_desc* desc, size_t* bytes);
 gf_status gf_layer_step_host(const gf_conv_desc* desc, const void* h_x, const void* h_gy,
                              const void* h_W, float* h_gW, void* h_gX, void* arena,
                              size_t arena_bytes, void* stream);
+
+/* ---- Error diagnostics of the paper's analysis (Section 4.1) -----------------------------
+ * Not part of a training step: the quantities with which the paper relates patch size, noise
+ * level and accuracy (Figure "SNR", Table of energy ratios).  `energies` is a DEVICE pointer
+ * to two doubles, 8-byte aligned, overwritten with { signal energy, noise energy }; the
+ * signal-to-noise ratio is their quotient (+inf when nothing is lost).  Sums run in fp64;
+ * the order of the block-level additions is not fixed. */
+
+/* First line of Eq. (snr_g3) for any approximate tensor against its reference (by Parseval's
+ * theorem the same number in the spatial and in the frequency domain):
+ * energies = { sum ref^2, sum (ref - approx)^2 } over `count` elements of `dtype`.  With ref =
+ * the exact g_x of a layer (gf_backward with r = 1) and approx = its filtered g_x this is the
+ * SNR of g~_x of Proposition 1. */
+gf_status gf_snr_terms(const void* ref, const void* approx, int64_t count, int32_t dtype,
+                       double* energies, void* stream);
+
+/* The same two terms for the gradient filter itself (Section 3.3), in one pass over
+ * g [planes, H, W] and without forming the filtered map: ref = g, approx = g with every r x r
+ * patch replaced by its average (an edge patch averages over the elements it has). */
+gf_status gf_filter_snr_terms(const void* g, int64_t planes, int32_t H, int32_t W, int32_t r,
+                              int32_t dtype, double* energies, void* stream);
+
+/* Eq. (dcac_ratio), the assumption of Proposition 1: for every kernel W[c_o, c_i] of
+ * W [C_out, C_ig, KH, KW], ratio[c_o * C_ig + c_i] = |Theta[0,0]|^2 / max over the other bins
+ * of |Theta[u,v]|^2, Theta being the dft_h x dft_w DFT of the kernel zero-padded to that
+ * extent (0 = the kernel's own extent; the proof works with the patch's extent r x r).
+ * A one-bin DFT has no AC part: +inf.  `ratio` is a device array of C_out * C_ig floats.
+ * KH, KW <= 31 and dft_h, dft_w <= 64, else GF_ERR_UNSUPPORTED. */
+gf_status gf_dcac_ratio(const void* W, int32_t C_out, int32_t C_ig, int32_t KH, int32_t KW,
+                        int32_t dft_h, int32_t dft_w, int32_t dtype, float* ratio, void* stream);
 
 /* Dense layers with r in {2,4,8} dividing H and W can be computed two ways: the gradient
  * filter (Section 3.3) as a pooling pass of its own followed by the two reduced contractions

@@ -156,6 +156,39 @@ def literal_backward(x, gy, theta, r: int, groups: int = 1,
 # The method, in its own order
 # ---------------------------------------------------------------------------
 
+def activation(z, kind: str) -> np.ndarray:
+    """The producers of x in the paper's networks: "none", "relu" = max(z, 0) (ResNet),
+    "relu6" = min(max(z, 0), 6) (MobileNetV2, MCUNet).  Plain element-wise definitions."""
+    z = _f64(z)
+    out = np.empty_like(z)
+    flat_in, flat_out = z.reshape(-1), out.reshape(-1)
+    for i in range(flat_in.size):
+        v = flat_in[i]
+        if kind == "relu":
+            v = v if v > 0.0 else 0.0
+        elif kind == "relu6":
+            v = 0.0 if v < 0.0 else (6.0 if v > 6.0 else v)
+        elif kind != "none":
+            raise ValueError(kind)
+        flat_out[i] = v
+    return out
+
+
+def activation_fast(z, kind: str) -> np.ndarray:
+    """activation() through numpy's clip, for tensors too large for a Python loop."""
+    z = _f64(z)
+    if kind == "none":
+        return z.copy()
+    return np.clip(z, 0.0, 6.0 if kind == "relu6" else None)
+
+
+def act_stash_forward(z, kind: str, r: int):
+    """Forward-side step fused into the producer of x (Section 4.2): x = act(z) and the stash of
+    that x.  Returns (x, stash)."""
+    x = activation_fast(z, kind)
+    return x, stash_forward(x, r)
+
+
 def stash_forward(x, r: int) -> np.ndarray:
     """What the forward pass keeps instead of x.  r == 1: x itself."""
     if r == 1:

@@ -20,12 +20,14 @@ GF_ERR_WORKSPACE, GF_ERR_ALIGN, GF_ERR_CUDA, GF_ERR_TIMEOUT = 4, 5, 6, 7
 GF_F32, GF_BF16 = 0, 1
 GF_NCHW, GF_NHWC = 0, 1
 GF_PATH_AUTO, GF_PATH_FUSED, GF_PATH_SPLIT = 0, 1, 2
+GF_ACT_NONE, GF_ACT_RELU, GF_ACT_RELU6 = 0, 1, 2
 
 EXPORTS = (
     "gf_stash_dims", "gf_stash_bytes", "gf_backward_workspace_bytes", "gf_stash_forward",
     "gf_backward", "gf_last_async_status", "gf_host_step_arena_bytes", "gf_layer_step_host",
     "gf_kernel_launch_count", "gf_status_string", "gf_profile_configure", "gf_profile_read",
     "gf_kernel_name", "gf_kernel_id_count", "gf_backward_static_scratch", "gf_set_dense_path",
+    "gf_snr_terms", "gf_filter_snr_terms", "gf_dcac_ratio", "gf_act_stash_forward",
 )
 
 
@@ -72,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.gf_stash_bytes.argtypes = [dp, ctypes.POINTER(sz)]
         L.gf_backward_workspace_bytes.argtypes = [dp, ctypes.POINTER(sz)]
         L.gf_stash_forward.argtypes = [dp, vp, vp, vp]
+        L.gf_act_stash_forward.argtypes = [dp, ctypes.c_int32, vp, vp, vp, vp]
+        L.gf_act_stash_forward.restype = ctypes.c_int
         L.gf_backward.argtypes = [dp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.gf_backward_static_scratch.argtypes = [dp, vp, vp, vp, vp, vp, vp]
         L.gf_backward_static_scratch.restype = ctypes.c_int
@@ -90,6 +94,12 @@ def lib() -> ctypes.CDLL:
         L.gf_kernel_id_count.restype = ctypes.c_int32
         L.gf_set_dense_path.argtypes = [ctypes.c_int32]
         L.gf_set_dense_path.restype = ctypes.c_int
+        i32, i64 = ctypes.c_int32, ctypes.c_int64
+        L.gf_snr_terms.argtypes = [vp, vp, i64, i32, vp, vp]
+        L.gf_filter_snr_terms.argtypes = [vp, i64, i32, i32, i32, i32, vp, vp]
+        L.gf_dcac_ratio.argtypes = [vp, i32, i32, i32, i32, i32, i32, i32, vp, vp]
+        for name in ("gf_snr_terms", "gf_filter_snr_terms", "gf_dcac_ratio"):
+            getattr(L, name).restype = ctypes.c_int
         L.gf_status_string.argtypes = [ctypes.c_int]
         L.gf_status_string.restype = ctypes.c_char_p
         for name in ("gf_stash_dims", "gf_stash_bytes", "gf_backward_workspace_bytes", "gf_stash_forward",
@@ -168,6 +178,12 @@ def gf_stash_forward(desc: gf_conv_desc, x, stash, stream=None) -> None:
            "gf_stash_forward")
 
 
+def gf_act_stash_forward(desc: gf_conv_desc, act: int, z, x, stash, stream=None) -> None:
+    """x <- act(z) and stash <- patch sums of x, in one pass over z (x may be z)."""
+    _check(lib().gf_act_stash_forward(ctypes.byref(desc), int(act), _ptr(z), _ptr(x), _ptr(stash), _stream(stream)),
+           "gf_act_stash_forward")
+
+
 def gf_backward(desc: gf_conv_desc, g_y, stash, W, g_W, g_X, workspace, workspace_bytes=None,
                 stream=None) -> None:
     if workspace_bytes is None:
@@ -210,6 +226,33 @@ def gf_layer_step_host(desc: gf_conv_desc, h_x, h_gy, h_W, h_gW, h_gX, arena, ar
 def gf_set_dense_path(path: int) -> None:
     """GF_PATH_AUTO (the library's choice per layer), GF_PATH_FUSED or GF_PATH_SPLIT, process-wide."""
     _check(lib().gf_set_dense_path(int(path)), "gf_set_dense_path")
+
+
+def _gf_dtype(t: torch.Tensor) -> int:
+    return {torch.float32: GF_F32, torch.bfloat16: GF_BF16}[t.dtype]
+
+
+def gf_snr_terms(ref: torch.Tensor, approx: torch.Tensor, energies: torch.Tensor, stream=None) -> None:
+    """energies (2 doubles on the device) <- sum ref^2, sum (ref - approx)^2."""
+    assert ref.dtype == approx.dtype and ref.numel() == approx.numel() and energies.dtype == torch.float64
+    _check(lib().gf_snr_terms(_ptr(ref), _ptr(approx), ctypes.c_int64(ref.numel()), _gf_dtype(ref), _ptr(energies),
+                              _stream(stream)), "gf_snr_terms")
+
+
+def gf_filter_snr_terms(g: torch.Tensor, r: int, energies: torch.Tensor, stream=None) -> None:
+    """The SNR terms of the gradient filter with patch size r on g [..., H, W]."""
+    assert energies.dtype == torch.float64 and g.dim() >= 2
+    H, W = int(g.shape[-2]), int(g.shape[-1])
+    _check(lib().gf_filter_snr_terms(_ptr(g), ctypes.c_int64(g.numel() // (H * W)), H, W, int(r), _gf_dtype(g),
+                                     _ptr(energies), _stream(stream)), "gf_filter_snr_terms")
+
+
+def gf_dcac_ratio(W: torch.Tensor, ratio: torch.Tensor, dft: tuple[int, int] = (0, 0), stream=None) -> None:
+    """ratio [C_out, C_ig] (fp32, device) <- DC / largest AC energy of every kernel of W [C_out, C_ig, KH, KW]."""
+    C_out, C_ig, KH, KW = (int(v) for v in W.shape)
+    assert ratio.dtype == torch.float32 and ratio.numel() == C_out * C_ig
+    _check(lib().gf_dcac_ratio(_ptr(W), C_out, C_ig, KH, KW, int(dft[0]), int(dft[1]), _gf_dtype(W), _ptr(ratio),
+                               _stream(stream)), "gf_dcac_ratio")
 
 
 def gf_kernel_launch_count() -> int:

@@ -259,6 +259,25 @@ gf_status gf_stash_forward(const gf_conv_desc* desc, const void* x, void* stash,
     return launch_pool(K_STASH_POOL, x, g.dtype, stash, nullptr, g.dtype, /*mean=*/false, planes, g.H, g.W, g.r, 0, err, s);
 }
 
+gf_status gf_act_stash_forward(const gf_conv_desc* desc, int32_t act, const void* z, void* x, void* stash, void* stream) {
+    if (!desc || !z || !x || !stash) return GF_ERR_NULL;
+    if (act < GF_ACT_NONE || act > GF_ACT_RELU6) return GF_ERR_BAD_DESC;
+    gf_status st = validate(desc);
+    if (st != GF_OK) return st;
+    if (misaligned(z) || misaligned(x) || misaligned(stash)) return GF_ERR_ALIGN;
+    const Geo g = make_geo(*desc);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int64_t planes = (int64_t)g.N * g.C_in;
+    if (g.r == 1) return launch_act(z, x, stash, (long long)planes * g.H * g.W, g.dtype, act, s);
+    if (act == GF_ACT_NONE) {
+        if (x != z) GF_CUDA_TRY(cudaMemcpyAsync(x, z, (size_t)planes * g.H * g.W * g.esize, cudaMemcpyDeviceToDevice, s));
+        return gf_stash_forward(desc, x, stash, stream);
+    }
+    uint32_t* err = global_err_word();
+    if (!err) return GF_ERR_CUDA;
+    return launch_pool(K_STASH_POOL, z, g.dtype, stash, nullptr, g.dtype, /*mean=*/false, planes, g.H, g.W, g.r, 0, err, s, act, x);
+}
+
 gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* stash, const void* W,
                       float* g_W, void* g_X, void* workspace, size_t workspace_bytes, void* stream) {
     return backward_impl(desc, g_y, stash, W, g_W, g_X, workspace, workspace_bytes, stream, /*may_fork=*/true);

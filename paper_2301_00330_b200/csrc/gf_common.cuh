@@ -184,8 +184,13 @@ gf_status backward_impl(const gf_conv_desc* desc, const void* g_y, const void* s
 // ---- kernel entry points (host launchers) ----------------------------------
 // pool: out[plane, a, b] = sum (or mean) of in[plane] over patch (a,b).  out_lo: bf16 low
 // parts (NULL: none).  out_pitch: elements between output planes, 0 = dense; a gap is zeroed.
+// act != 0: gf_activation applied to every input element first; act(in) is also written to act_out
+// (same dtype; may be `in` itself).
 gf_status launch_pool(int kernel_id, const void* in, int in_dtype, void* out, void* out_lo, int out_dtype, bool mean,
-                      int64_t planes, int H, int W, int r, int out_pitch, uint32_t* err_word, cudaStream_t s);
+                      int64_t planes, int H, int W, int r, int out_pitch, uint32_t* err_word, cudaStream_t s, int act = 0,
+                      void* act_out = nullptr);
+// out (and out2 when given) <- act(in), element by element
+gf_status launch_act(const void* in, void* out, void* out2, long long n, int dtype, int act, cudaStream_t s);
 gf_status launch_copy(const void* in, void* out, size_t bytes, cudaStream_t s);
 
 gf_status launch_ksum(const void* W, const Geo& g, float* tsum, cudaStream_t s);

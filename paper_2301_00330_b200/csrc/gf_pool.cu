@@ -12,6 +12,8 @@
 //  pool_tile_kernel     any r, any alignment: one tile per CTA, staged with
 //                       128-bit loads.
 //  pool_bigpatch_kernel patches too large for a tile: one CTA per output value.
+#include <type_traits>
+
 #include "gf_common.cuh"
 #include "gf_pipe.cuh"
 #include "gf_span.cuh"
@@ -31,6 +33,8 @@ constexpr int kStreamCtasPerSm = 2;
 
 struct PoolParams {
     const void* in;
+    void* act_out;     // fused activation: where act(in) goes (may be `in` itself); NULL otherwise
+    int act;           // gf_activation applied to every input element before pooling (0: none)
     void* out;
     void* out_lo;      // bf16 output only: low parts, out = rn(v), out_lo = rn(v - out); NULL: plain output
     uint32_t* err_word;
@@ -160,6 +164,15 @@ __device__ __forceinline__ int stage_plain(const TIn* __restrict__ in, long long
     return shift;
 }
 
+// ---- activation fused into the pooling pass ----------------------------------------------
+// ACT: 0 none, 1 max(v, 0), 2 min(max(v, 0), 6) -- the producers of x in the paper's networks
+// (ResNet: ReLU; MobileNetV2 / MCUNet: ReLU6).
+template <int ACT> __device__ __forceinline__ float apply_act(float v) {
+    if constexpr (ACT == 1) return fmaxf(v, 0.f);
+    else if constexpr (ACT == 2) return fminf(fmaxf(v, 0.f), 6.f);
+    else return v;
+}
+
 // ---- streamed kernel ------------------------------------------------------------------
 // Requires r in {2,4,8}, r | W and r | H.  Then the whole tensor is a sequence of
 // "strips": strip s is the R image rows [s*R, s*R+R) of the [planes*H, W] matrix,
@@ -167,12 +180,12 @@ __device__ __forceinline__ int stage_plain(const TIn* __restrict__ in, long long
 // A tile is S consecutive strips (plane boundaries do not matter).
 // EXT: the output has a low-part array and/or a padded plane pitch (tensor-core operands);
 // the plain case keeps to one vector store at og0 + o.
-template <typename TIn, typename TOut, int R, int G, bool EXT>
-__device__ __forceinline__ void reduce_item(const PoolParams& p, const TIn* buf, long long og0, uint32_t q) {
+template <typename TIn, typename TOut, int R, int G, bool EXT, int ACT>
+__device__ __forceinline__ void reduce_item(const PoolParams& p, TIn* buf, long long og0, uint32_t q) {
     const uint32_t o = q * G;
     uint32_t A, b;
     p.div_Wp.divmod(o, A, b);
-    const TIn* src = buf + (int)(A * R) * p.W + (int)b * R;
+    TIn* src = buf + (int)(A * R) * p.W + (int)b * R;
     float acc[G];
 #pragma unroll
     for (int k = 0; k < G; ++k) acc[k] = 0.f;
@@ -180,6 +193,11 @@ __device__ __forceinline__ void reduce_item(const PoolParams& p, const TIn* buf,
     for (int i = 0; i < R; ++i) {
         float v[G * R];
         load_span<G * R>(src + i * p.W, v);
+        if constexpr (ACT != 0) {      // the activated values replace the raw ones in the tile, which is then written out
+#pragma unroll
+            for (int k = 0; k < G * R; ++k) v[k] = apply_act<ACT>(v[k]);
+            store_span<G * R>(src + i * p.W, v);
+        }
 #pragma unroll
         for (int k = 0; k < G; ++k) {
             float s = v[k * R];
@@ -230,13 +248,19 @@ struct LinearLane {
 };
 
 // One vector per lane; every lane of a warp takes part (inactive ones add zeros).
-template <typename TIn, typename TOut, int R, bool EXT>
-__device__ __forceinline__ void reduce_linear(const PoolParams& p, const LinearLane<TIn, R>& ln, const TIn* buf,
+template <typename TIn, typename TOut, int R, bool EXT, int ACT>
+__device__ __forceinline__ void reduce_linear(const PoolParams& p, const LinearLane<TIn, R>& ln, TIn* buf,
                                               long long og0, uint32_t v, uint32_t o, bool active) {
     using LL = LinearLane<TIn, R>;
     float val[LL::VE];
-    if (active) load_span<LL::VE>(buf + (size_t)v * LL::VE, val);
-    else {
+    if (active) {
+        load_span<LL::VE>(buf + (size_t)v * LL::VE, val);
+        if constexpr (ACT != 0) {
+#pragma unroll
+            for (int k = 0; k < LL::VE; ++k) val[k] = apply_act<ACT>(val[k]);
+            store_span<LL::VE>(buf + (size_t)v * LL::VE, val);
+        }
+    } else {
 #pragma unroll
         for (int k = 0; k < LL::VE; ++k) val[k] = 0.f;
     }
@@ -272,8 +296,10 @@ __device__ __forceinline__ void reduce_linear(const PoolParams& p, const LinearL
     }
 }
 
-// G == 0 selects the linear mode.
-template <typename TIn, typename TOut, int R, int G, bool EXT>
+// G == 0 selects the linear mode.  ACT != 0: the activation is applied to the tile in shared
+// memory while it is pooled, and the copy engine writes the activated tile to act_out: the
+// producer of x and the stash in one pass over the pre-activation tensor.
+template <typename TIn, typename TOut, int R, int G, bool EXT, int ACT>
 __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) pool_stream_kernel(const PoolParams p) {
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     __shared__ uint64_t full[kStreamStages];
@@ -326,28 +352,47 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) pool_stream_
         }
         if (ok) {
             const long long dst = tile * p.S * p.Wp;      // first output of the tile, flattened over planes
-            const TIn* b = buf(s);
+            TIn* b = buf(s);
             if constexpr (G == 0) {
                 const uint32_t nvec = bytes >> 4, nvec_up = (nvec + 31u) & ~31u;   // whole warps take part
                 uint32_t o = lane_ctx.o0;
 #pragma unroll 2
                 for (uint32_t v = threadIdx.x; v < nvec_up; v += kStreamThreads, o += lane_ctx.o_step)
-                    reduce_linear<TIn, TOut, R, EXT>(p, lane_ctx, b, dst, v, o, v < nvec);
+                    reduce_linear<TIn, TOut, R, EXT, ACT>(p, lane_ctx, b, dst, v, o, v < nvec);
             } else {
                 const uint32_t nitems = (uint32_t)(ns * p.Wp) / (G > 0 ? G : 1);
                 uint32_t q = threadIdx.x;
                 for (; q + kStreamThreads < nitems; q += 2 * kStreamThreads) {   // two independent items in flight
-                    reduce_item<TIn, TOut, R, (G > 0 ? G : 1), EXT>(p, b, dst, q);
-                    reduce_item<TIn, TOut, R, (G > 0 ? G : 1), EXT>(p, b, dst, q + kStreamThreads);
+                    reduce_item<TIn, TOut, R, (G > 0 ? G : 1), EXT, ACT>(p, b, dst, q);
+                    reduce_item<TIn, TOut, R, (G > 0 ? G : 1), EXT, ACT>(p, b, dst, q + kStreamThreads);
                 }
-                if (q < nitems) reduce_item<TIn, TOut, R, (G > 0 ? G : 1), EXT>(p, b, dst, q);
+                if (q < nitems) reduce_item<TIn, TOut, R, (G > 0 ? G : 1), EXT, ACT>(p, b, dst, q);
             }
         }
+        if constexpr (ACT != 0) fence_proxy_async_smem();     // the activated tile is read by the copy engine
         failed = __syncthreads_or(!ok);     // also: every thread is done reading slot s
         done = it + 1;
         if (failed) break;
+        if constexpr (ACT != 0) {
+            if (threadIdx.x == 0) {
+                // activated tile -> act_out (a tile whose byte count is not a multiple of 16 -- only the
+                // tensor's last can be -- is written by the threads below); the slot is refilled
+                // once the copy engine has read it
+                if ((bytes & 15u) == 0) {
+                    bulk_s2g(static_cast<TIn*>(p.act_out) + tile * p.S * strip_elems, buf(s), bytes);
+                    bulk_commit();
+                    bulk_wait_read<0>();
+                }
+            }
+            if ((bytes & 15u) != 0) {
+                TIn* o = static_cast<TIn*>(p.act_out) + tile * p.S * strip_elems;
+                for (int e = threadIdx.x; e < ns * strip_elems; e += kStreamThreads) o[e] = buf(s)[e];
+                __syncthreads();
+            }
+        }
         if (threadIdx.x == 0 && it + kStreamStages < n_my) issue(it + kStreamStages);
     }
+    if constexpr (ACT != 0) { if (threadIdx.x == 0) bulk_wait_all(); }
     if (failed && threadIdx.x == 0) {
         atomicOr(p.err_word, 1u);
         // copies still in flight target this CTA's shared memory: wait for them (bounded)
@@ -464,19 +509,24 @@ static bool plan_stream(PoolParams& p, size_t e) {
     return p.tiles <= 0x7fffffffLL;
 }
 
-template <typename TIn, typename TOut, int R, int G, bool EXT>
+template <typename TIn, typename TOut, int R, int G, bool EXT, int ACT>
 static gf_status launch_stream_ext(const PoolParams& p, cudaStream_t s) {
     constexpr size_t smem = (size_t)kStreamStages * kStreamTileBytes;
     static size_t configured[kMaxDevices] = {};
-    if (gf_status st = ensure_dyn_smem(pool_stream_kernel<TIn, TOut, R, G, EXT>, smem, configured); st != GF_OK) return st;
+    if (gf_status st = ensure_dyn_smem(pool_stream_kernel<TIn, TOut, R, G, EXT, ACT>, smem, configured); st != GF_OK) return st;
     const long long grid = p.tiles < (long long)sm_count() * kStreamCtasPerSm ? p.tiles : (long long)sm_count() * kStreamCtasPerSm;
-    return launch_pdl(pool_stream_kernel<TIn, TOut, R, G, EXT>, dim3((unsigned)grid), dim3(kStreamThreads), smem, s, p);
+    return launch_pdl(pool_stream_kernel<TIn, TOut, R, G, EXT, ACT>, dim3((unsigned)grid), dim3(kStreamThreads), smem, s, p);
 }
 
 template <typename TIn, typename TOut, int R, int G>
 static gf_status launch_stream_inst(const PoolParams& p, cudaStream_t s) {
-    if (p.out_lo || p.out_pitch != p.plane_out) return launch_stream_ext<TIn, TOut, R, G, true>(p, s);
-    return launch_stream_ext<TIn, TOut, R, G, false>(p, s);
+    if constexpr (std::is_same<TIn, TOut>::value) {      // the fused activation keeps the tensor's dtype
+        if (p.act == 1) return launch_stream_ext<TIn, TOut, R, G, false, 1>(p, s);
+        if (p.act == 2) return launch_stream_ext<TIn, TOut, R, G, false, 2>(p, s);
+    }
+    if (p.act != 0) return GF_ERR_UNSUPPORTED;
+    if (p.out_lo || p.out_pitch != p.plane_out) return launch_stream_ext<TIn, TOut, R, G, true, 0>(p, s);
+    return launch_stream_ext<TIn, TOut, R, G, false, 0>(p, s);
 }
 
 template <typename TIn, typename TOut>
@@ -493,9 +543,44 @@ static gf_status launch_stream(const PoolParams& p, cudaStream_t s) {
     return GF_ERR_UNSUPPORTED;
 }
 
+// act(in) -> out, element by element (the fallback of the fused activation, and its r == 1 case:
+// out2, when given, receives the same values)
+template <typename T>
+__global__ void __launch_bounds__(256) act_kernel(const T* __restrict__ in, T* __restrict__ out, T* __restrict__ out2,
+                                                  long long n, int act) {
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+        const float v = to_f32(in[i]);
+        const T o = from_f32<T>(act == 1 ? apply_act<1>(v) : act == 2 ? apply_act<2>(v) : v);
+        out[i] = o;
+        if (out2) out2[i] = o;
+    }
+}
+
+gf_status launch_act(const void* in, void* out, void* out2, long long n, int dtype, int act, cudaStream_t s) {
+    if (n == 0) return GF_OK;
+    long long grid = (n + 255) / 256;
+    const long long cap = (long long)sm_count() * 16;
+    if (grid > cap) grid = cap;
+    if (dtype == GF_F32)
+        act_kernel<float><<<(unsigned)grid, 256, 0, s>>>((const float*)in, (float*)out, (float*)out2, n, act);
+    else
+        act_kernel<__nv_bfloat16><<<(unsigned)grid, 256, 0, s>>>((const __nv_bfloat16*)in, (__nv_bfloat16*)out,
+                                                               (__nv_bfloat16*)out2, n, act);
+    return after_launch();
+}
+
 template <typename TIn, typename TOut>
 static gf_status pool_dispatch(PoolParams& p, size_t e, cudaStream_t s) {
     if (plan_stream(p, e)) return launch_stream<TIn, TOut>(p, s);
+    if (p.act != 0) {
+        // shapes the streamed kernel does not take: the activation as a pass of its own, then the
+        // pooling of its result
+        if (!std::is_same<TIn, TOut>::value) return GF_ERR_UNSUPPORTED;
+        gf_status st = launch_act(p.in, p.act_out, nullptr, p.total_elems, sizeof(TIn) == 4 ? GF_F32 : GF_BF16, p.act, s);
+        if (st != GF_OK) return st;
+        p.in = p.act_out;
+        p.act = 0;
+    }
     const long long plane_bytes = (long long)p.H * p.W * (long long)e;
     const long long band_bytes = (long long)(p.r < p.H ? p.r : p.H) * p.W * (long long)e;   // one patch row
     bool big = false;
@@ -523,9 +608,12 @@ static gf_status pool_dispatch(PoolParams& p, size_t e, cudaStream_t s) {
 }
 
 gf_status launch_pool(int kernel_id, const void* in, int in_dtype, void* out, void* out_lo, int out_dtype, bool mean,
-                      int64_t planes, int H, int W, int r, int out_pitch, uint32_t* err_word, cudaStream_t s) {
+                      int64_t planes, int H, int W, int r, int out_pitch, uint32_t* err_word, cudaStream_t s, int act,
+                      void* act_out) {
     ProfScope prof(kernel_id, s);
     PoolParams p;
+    if (act != 0 && (!act_out || out_lo || out_pitch != 0 || in_dtype != out_dtype)) return GF_ERR_UNSUPPORTED;
+    p.act = act; p.act_out = act_out;
     if (out_lo && out_dtype != GF_BF16) return GF_ERR_UNSUPPORTED;
     p.in = in; p.out = out; p.out_lo = out_lo; p.err_word = err_word; p.planes = planes; p.total_elems = planes * H * W;
     p.H = H; p.W = W; p.r = r; p.mean = mean ? 1 : 0;

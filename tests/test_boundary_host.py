@@ -138,3 +138,15 @@ def test_product_never_imports_the_checker():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 text = open(os.path.join(dirpath, f)).read()
                 assert "oracle" not in text.lower(), os.path.join(dirpath, f)
+
+
+def test_diagnostics_reject_bad_arguments(gf):
+    """Section 4.1 diagnostics: argument checks come before anything touches the device."""
+    L = gf.lib()
+    a = ctypes.c_void_p(0x1000)
+    assert L.gf_snr_terms(None, a, 4, 0, a, None) == gf.GF_ERR_NULL
+    assert L.gf_snr_terms(a, a, -1, 0, a, None) == gf.GF_ERR_BAD_DESC
+    assert L.gf_snr_terms(a, a, 4, 0, ctypes.c_void_p(0x1004), None) == gf.GF_ERR_ALIGN
+    assert L.gf_filter_snr_terms(a, 1, 0, 4, 2, 0, a, None) == gf.GF_ERR_BAD_DESC
+    assert L.gf_dcac_ratio(a, 1, 1, 3, 3, 2, 3, 0, a, None) == gf.GF_ERR_BAD_DESC          # DFT smaller than the kernel
+    assert L.gf_dcac_ratio(a, 1, 1, 3, 3, 128, 3, 0, a, None) == gf.GF_ERR_UNSUPPORTED

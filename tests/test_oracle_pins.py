@@ -290,3 +290,29 @@ def test_kernel_sum_ignores_rotation():
     w = rnd(rng, 3, 2, 3, 3)
     assert rel(oracle.kernel_sum(w), oracle.kernel_sum(w[:, :, ::-1, ::-1])) < 1e-15
     assert rel(oracle.kernel_sum(w), w.sum((2, 3))) < 1e-15
+
+
+# ---- activation + stash (forward-side step fused into the producer of x, Section 4.2) ----
+
+def test_activation_definitions_and_library_clip():
+    z = np.array([-7.5, -0.0, 0.0, 0.25, 5.999, 6.0, 6.5, 100.0]).reshape(1, 1, 2, 4)
+    assert np.array_equal(oracle.activation(z, "none"), z)
+    assert np.array_equal(oracle.activation(z, "relu").ravel(), [0, 0, 0, 0.25, 5.999, 6.0, 6.5, 100.0])
+    assert np.array_equal(oracle.activation(z, "relu6").ravel(), [0, 0, 0, 0.25, 5.999, 6.0, 6.0, 6.0])
+    big = np.random.default_rng(3).normal(scale=4.0, size=(2, 3, 5, 7))
+    for kind in ("none", "relu", "relu6"):
+        assert np.array_equal(oracle.activation(big, kind), oracle.activation_fast(big, kind))
+    assert np.array_equal(oracle.activation_fast(big, "relu"), torch.relu(torch.from_numpy(big)).numpy())
+    assert np.array_equal(oracle.activation_fast(big, "relu6"), torch.nn.functional.relu6(torch.from_numpy(big)).numpy())
+    with pytest.raises(ValueError):
+        oracle.activation(z, "gelu")
+
+
+def test_act_stash_forward_is_the_stash_of_the_activated_map():
+    z = np.random.default_rng(8).normal(scale=3.0, size=(2, 3, 7, 9))
+    for r in (1, 2, 4):
+        x, stash = oracle.act_stash_forward(z, "relu6", r)
+        assert np.array_equal(x, np.clip(z, 0, 6))
+        assert np.array_equal(stash, oracle.stash_forward(np.clip(z, 0, 6), r))
+        if r > 1:   # mass: the stash keeps the sum of the activated map
+            assert stash.sum() == pytest.approx(np.clip(z, 0, 6).sum(), rel=1e-12)
