@@ -7,3 +7,5 @@ from .gf_oracle import (act_stash_forward, activation, activation_fast, backward
                         literal_backward, num_threads, patch_mean, patch_sum,
                         reduced_gw, reduced_gx, stash_forward, stash_num_values)
 from .gf_diagnostics import dcac_ratio, filter_snr_terms, snr_terms, snr_terms_fast  # noqa: F401,E402
+from .gf_strided import (exact_backward_strided, kernel_phase_sums, strided_backward,  # noqa: F401,E402
+                         strided_stash_forward)
