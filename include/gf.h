@@ -22,11 +22,20 @@
  *  - Tensors: x [N,C_in,H,W], g_y [N,C_out,H,W], W [C_out,C_in/groups,KH,KW],
  *    g_X like x, g_W like W but ALWAYS fp32.  x, g_y, W, the stash and g_X have
  *    the descriptor's dtype; all sums are accumulated in fp32.
- *  - Supported geometry: stride 1, odd KH and KW, pad_h = (KH-1)/2,
- *    pad_w = (KW-1)/2 (so g_y has the resolution of x, as Eq. (grad_x)
- *    requires), groups dividing C_in and C_out, any r >= 1 (r need not divide
- *    H or W: there are ceil(H/r) x ceil(W/r) patches and an edge patch averages
- *    over the elements it has).  NCHW only.  Anything else: GF_ERR_UNSUPPORTED.
+ *  - Supported geometry: odd KH and KW, pad_h = (KH-1)/2, pad_w = (KW-1)/2,
+ *    groups dividing C_in and C_out, any r >= 1 (r need not divide the map:
+ *    there are ceil(H_y/r) x ceil(W_y/r) patches and an edge patch averages
+ *    over the elements it has).  Stride 1 (g_y has the resolution of x, as
+ *    Eq. (grad_x) requires) or a stride s that divides H and W: g_y is then
+ *    [N,C_out,H/s,W/s], the gradient filter acts on that map, the stash holds
+ *    the sums of x over the (r s) x (r s) windows the patches see (the grid on
+ *    which the paper's ImageNet table books a stride-2 layer), and
+ *        g~_x[n,c_i,h,w] = sum_{c_o} g~_y[n,c_o,h/s,w/s] theta~'_{h%s,w%s}[c_o,c_i]
+ *        g~_theta        = (1/s^2) sum x~ g~_y
+ *    with theta~'_{p,q} the sum of the taps through which pixel phase (p,q)
+ *    reaches an output.  The paper states its formulas for stride 1 only; this
+ *    is the library's extension of them (same two approximations).  NCHW only.
+ *    Anything else: GF_ERR_UNSUPPORTED.
  *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Work
  *    is enqueued on it and the call returns without synchronising.  Errors that
  *    the host can detect are returned before anything is launched.
@@ -60,7 +69,7 @@ typedef enum gf_layout { GF_NCHW = 0, GF_NHWC = 1 } gf_layout;
 typedef struct gf_conv_desc {
     int32_t N, C_in, C_out, H, W;
     int32_t KH, KW;
-    int32_t stride;         /* must be 1 */
+    int32_t stride;         /* 1, or s >= 2 dividing H and W (g_y is then [H/s, W/s]) */
     int32_t pad_h, pad_w;   /* must be (KH-1)/2, (KW-1)/2 */
     int32_t groups;
     int32_t r;              /* patch size, >= 1; 1 = exact backward */
@@ -68,8 +77,8 @@ typedef struct gf_conv_desc {
     int32_t layout;         /* gf_layout; only GF_NCHW */
 } gf_conv_desc;
 
-/* Logical shape [N, C_in, ceil(H/r), ceil(W/r)] of the stash (Section 3.3: one
- * unique value per patch).  For r == 1 it is the shape of x. */
+/* Logical shape [N, C_in, ceil(H/(r s)), ceil(W/(r s))] of the stash, s the stride
+ * (Section 3.3: one unique value per patch of g_y).  For r == 1 it is the shape of x. */
 gf_status gf_stash_dims(const gf_conv_desc* desc, int64_t dims[4]);
 
 /* Bytes of the stash: product of gf_stash_dims times the element size.  The

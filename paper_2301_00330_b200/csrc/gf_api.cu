@@ -93,7 +93,8 @@ static gf_status validate(const gf_conv_desc* d) {
     if (d->dtype != GF_F32 && d->dtype != GF_BF16) return GF_ERR_BAD_DESC;
     if (d->layout != GF_NCHW && d->layout != GF_NHWC) return GF_ERR_BAD_DESC;
     if (d->layout != GF_NCHW) return GF_ERR_UNSUPPORTED;
-    if (d->stride != 1) return GF_ERR_UNSUPPORTED;
+    // strided layers: the output map is [H / stride, W / stride] (see gf_strided.cu)
+    if (d->stride > 1 && (d->H % d->stride != 0 || d->W % d->stride != 0 || d->stride > 16)) return GF_ERR_UNSUPPORTED;
     if (d->KH % 2 == 0 || d->KW % 2 == 0) return GF_ERR_UNSUPPORTED;
     if (d->pad_h != (d->KH - 1) / 2 || d->pad_w != (d->KW - 1) / 2) return GF_ERR_UNSUPPORTED;
     // index arithmetic inside the kernels is 32-bit per plane and per tile
@@ -161,6 +162,25 @@ static Workspace plan_split(const Geo& g) {
     return w;
 }
 
+// Strided layers: error word | phase kernel sums fp32 [C_out, s*s*C_ig] | G- fp32 [N, C_out, P] |
+// reduced g_X on the patch grid fp32 [N, s*s*C_in, P] | g_W slices fp32 [S, C_out, C_ig]
+struct StridedPlan { size_t off_tph, off_gbar, off_ghat, off_part, total; int splits; Geo gy; };
+static StridedPlan plan_strided(const Geo& g, int stride) {
+    StridedPlan w;
+    w.gy = g;                                   // the geometry of g_y: what the pooling and the g_W contraction see
+    w.gy.H = g.H / stride; w.gy.W = g.W / stride;
+    w.gy.Hp = (w.gy.H + g.r - 1) / g.r; w.gy.Wp = (w.gy.W + g.r - 1) / g.r;
+    const size_t P = (size_t)w.gy.Hp * w.gy.Wp, s2 = (size_t)stride * stride;
+    size_t off = 256;
+    w.off_tph = off; off += align_up((size_t)g.C_out * s2 * g.C_ig * 4, 256);
+    w.off_gbar = off; off += align_up((size_t)g.N * g.C_out * P * 4, 256);
+    w.off_ghat = off; off += align_up((size_t)g.N * s2 * g.C_in * P * 4, 256);
+    w.splits = dense_splits(w.gy);
+    w.off_part = off; off += align_up((size_t)w.splits * g.C_out * g.C_ig * 4, 256);
+    w.total = off;
+    return w;
+}
+
 Workspace plan_workspace(const Geo& g) {
     const Workspace split = plan_split(g);
     if (g.r == 1 || !fused_path_ok(g)) return split;
@@ -222,9 +242,11 @@ gf_status gf_stash_dims(const gf_conv_desc* desc, int64_t dims[4]) {
     if (!dims) return GF_ERR_NULL;
     gf_status st = validate(desc);
     if (st != GF_OK) return st;
+    // one value per channel and per patch of the g_y grid: windows of r * stride pixels of x
+    const int win = desc->r == 1 ? 1 : desc->r * desc->stride;
     dims[0] = desc->N; dims[1] = desc->C_in;
-    dims[2] = (desc->H + desc->r - 1) / desc->r;
-    dims[3] = (desc->W + desc->r - 1) / desc->r;
+    dims[2] = (desc->H + win - 1) / win;
+    dims[3] = (desc->W + win - 1) / win;
     return GF_OK;
 }
 
@@ -241,7 +263,8 @@ gf_status gf_backward_workspace_bytes(const gf_conv_desc* desc, size_t* bytes) {
     if (!bytes) return GF_ERR_NULL;
     gf_status st = validate(desc);
     if (st != GF_OK) return st;
-    *bytes = plan_workspace(make_geo(*desc)).total;
+    const Geo g = make_geo(*desc);
+    *bytes = (desc->stride > 1 && g.r > 1) ? plan_strided(g, desc->stride).total : plan_workspace(g).total;
     return GF_OK;
 }
 
@@ -256,7 +279,8 @@ gf_status gf_stash_forward(const gf_conv_desc* desc, const void* x, void* stash,
     if (g.r == 1) return launch_copy(x, stash, (size_t)planes * g.H * g.W * g.esize, s);
     uint32_t* err = global_err_word();
     if (!err) return GF_ERR_CUDA;
-    return launch_pool(K_STASH_POOL, x, g.dtype, stash, nullptr, g.dtype, /*mean=*/false, planes, g.H, g.W, g.r, 0, err, s);
+    return launch_pool(K_STASH_POOL, x, g.dtype, stash, nullptr, g.dtype, /*mean=*/false, planes, g.H, g.W, g.r * desc->stride, 0,
+                       err, s);
 }
 
 gf_status gf_act_stash_forward(const gf_conv_desc* desc, int32_t act, const void* z, void* x, void* stash, void* stream) {
@@ -275,7 +299,8 @@ gf_status gf_act_stash_forward(const gf_conv_desc* desc, int32_t act, const void
     }
     uint32_t* err = global_err_word();
     if (!err) return GF_ERR_CUDA;
-    return launch_pool(K_STASH_POOL, z, g.dtype, stash, nullptr, g.dtype, /*mean=*/false, planes, g.H, g.W, g.r, 0, err, s, act, x);
+    return launch_pool(K_STASH_POOL, z, g.dtype, stash, nullptr, g.dtype, /*mean=*/false, planes, g.H, g.W, g.r * desc->stride, 0,
+                       err, s, act, x);
 }
 
 gf_status gf_backward(const gf_conv_desc* desc, const void* g_y, const void* stash, const void* W,
@@ -341,10 +366,48 @@ gf_status backward_impl(const gf_conv_desc* desc, const void* g_y, const void* s
         (g_W && misaligned(g_W)) || (g_X && misaligned(g_X)))
         return GF_ERR_ALIGN;
     const Geo g = make_geo(*desc);
-    const Workspace ws = plan_workspace(g);
-    if (workspace_bytes < ws.total) return GF_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     char* base = static_cast<char*>(workspace);
+    if (desc->stride > 1 && g.r > 1) {
+        // strided layer: kernel sums per pixel phase, gradient filter on g_y's own grid, the two
+        // reduced contractions on CUDA cores (g_X against all phases at once, then dealt out to
+        // the pixels of each window; g_W scaled by 1 / stride^2)
+        const int stride = desc->stride, s2 = stride * stride;
+        const StridedPlan sp = plan_strided(g, stride);
+        if (workspace_bytes < sp.total) return GF_ERR_WORKSPACE;
+        if (!g_W && !g_X) return GF_OK;
+        Geo gv = sp.gy;                         // g_X as a layer on the patch grid with s*s*C_in channels, not expanded
+        gv.C_in = s2 * g.C_in; gv.C_ig = s2 * g.C_ig; gv.H = sp.gy.Hp; gv.W = sp.gy.Wp; gv.r = 1; gv.dtype = GF_F32; gv.esize = 4;
+        st = dense_check_limits(sp.gy, sp.splits);
+        if (st == GF_OK) st = dense_check_limits(gv, 1);
+        if (st != GF_OK) return st;
+        uint32_t* err = reinterpret_cast<uint32_t*>(base);
+        GF_CUDA_TRY(cudaMemsetAsync(err, 0, sizeof(uint32_t), s));
+        float* tph = reinterpret_cast<float*>(base + sp.off_tph);
+        float* gbar = reinterpret_cast<float*>(base + sp.off_gbar);
+        float* ghat = reinterpret_cast<float*>(base + sp.off_ghat);
+        float* part = reinterpret_cast<float*>(base + sp.off_part);
+        st = launch_pool(K_GY_POOL, g_y, g.dtype, gbar, nullptr, GF_F32, /*mean=*/true, (int64_t)g.N * g.C_out, sp.gy.H, sp.gy.W, g.r,
+                         0, err, s);
+        if (st != GF_OK) return st;
+        if (g_X) {
+            st = launch_ksum_phase(W, g.dtype, g.C_out, g.C_ig, g.KH, g.KW, stride, tph, s);
+            if (st != GF_OK) return st;
+            st = launch_gx_mix(gbar, tph, ghat, gv, s);
+            if (st != GF_OK) return st;
+            st = launch_expand_phase(ghat, g_X, g.dtype, g.N, g.C_in, g.G, g.H, g.W, stride, g.r, s);
+            if (st != GF_OK) return st;
+        }
+        if (g_W) {
+            st = launch_gw_partial(gbar, stash, part, sp.splits, sp.gy, s);
+            if (st != GF_OK) return st;
+            st = launch_gw_finish(part, sp.splits, g_W, sp.gy, s, 1.0f / (float)s2);
+            if (st != GF_OK) return st;
+        }
+        return GF_OK;
+    }
+    const Workspace ws = plan_workspace(g);
+    if (workspace_bytes < ws.total) return GF_ERR_WORKSPACE;
     uint32_t* err = reinterpret_cast<uint32_t*>(base + ws.off_err);
     if (!g_W && !g_X) return GF_OK;
     // limits of the launch geometry, checked before anything is enqueued
@@ -357,7 +420,7 @@ gf_status backward_impl(const gf_conv_desc* desc, const void* g_y, const void* s
     // The error word is cleared here, ahead of every kernel of the call that may set it.
     GF_CUDA_TRY(cudaMemsetAsync(err, 0, sizeof(uint32_t), s));
 
-    if (g.r == 1) return launch_exact(g_y, stash, W, g_W, g_X, g, s);
+    if (g.r == 1) return launch_exact(g_y, stash, W, g_W, g_X, g, desc->stride, s);
 
     float* tsum = reinterpret_cast<float*>(base + ws.off_tsum);
     float* gbar = reinterpret_cast<float*>(base + ws.off_gbar);
@@ -475,12 +538,13 @@ gf_status plan_arena(const gf_conv_desc* desc, Arena* a) {
     if (st != GF_OK) return st;
     size_t off = 0;
     a->x = off; off += align_up((size_t)g.N * g.C_in * g.H * g.W * g.esize, 256);
-    a->gy = off; off += align_up((size_t)g.N * g.C_out * g.H * g.W * g.esize, 256);
+    a->gy = off; off += align_up((size_t)g.N * g.C_out * (g.H / desc->stride) * (g.W / desc->stride) * g.esize, 256);
     a->w = off; off += align_up((size_t)g.C_out * g.C_ig * g.KH * g.KW * g.esize, 256);
     a->stash = off; off += align_up(stash_bytes, 256);
     a->gw = off; off += align_up((size_t)g.C_out * g.C_ig * g.KH * g.KW * 4, 256);
     a->gx = off; off += align_up((size_t)g.N * g.C_in * g.H * g.W * g.esize, 256);
-    a->ws_bytes = plan_workspace(g).total;
+    st = gf_backward_workspace_bytes(desc, &a->ws_bytes);
+    if (st != GF_OK) return st;
     a->ws = off; off += align_up(a->ws_bytes, 256);
     a->total = off;
     return GF_OK;
@@ -508,7 +572,7 @@ gf_status gf_layer_step_host(const gf_conv_desc* desc, const void* h_x, const vo
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     char* base = static_cast<char*>(arena);
     const size_t x_bytes = (size_t)g.N * g.C_in * g.H * g.W * g.esize;
-    const size_t gy_bytes = (size_t)g.N * g.C_out * g.H * g.W * g.esize;
+    const size_t gy_bytes = (size_t)g.N * g.C_out * (g.H / desc->stride) * (g.W / desc->stride) * g.esize;
     const size_t w_elems = (size_t)g.C_out * g.C_ig * g.KH * g.KW;
     GF_CUDA_TRY(cudaMemcpyAsync(base + a.x, h_x, x_bytes, cudaMemcpyHostToDevice, s));
     GF_CUDA_TRY(cudaMemcpyAsync(base + a.gy, h_gy, gy_bytes, cudaMemcpyHostToDevice, s));

@@ -197,7 +197,8 @@ gf_status launch_ksum(const void* W, const Geo& g, float* tsum, cudaStream_t s);
 gf_status launch_gx_mix(const float* gbar, const float* tsum, void* gX, const Geo& g, cudaStream_t s);
 gf_status launch_gw_partial(const float* gbar, const void* stash, float* part, int splits,
                             const Geo& g, cudaStream_t s);
-gf_status launch_gw_finish(const float* part, int splits, float* gW, const Geo& g, cudaStream_t s);
+// scale: factor applied to every value (1 / stride^2 for strided layers)
+gf_status launch_gw_finish(const float* part, int splits, float* gW, const Geo& g, cudaStream_t s, float scale = 1.0f);
 gf_status dense_check_limits(const Geo& g, int splits);
 gf_status tc_check_limits(const Geo& g);
 gf_status launch_depthwise(const void* gy, const void* stash, const void* W, float* part,
@@ -236,6 +237,11 @@ gf_status launch_gyx_fused(const void* gy, const __nv_bfloat16* thetaT, long lon
 gf_status launch_gw_tiled(const unsigned char* gbar_t, const void* stash, float* gwu, uint32_t* err_word, const Geo& g,
                           cudaStream_t s);
 gf_status launch_exact(const void* gy, const void* x, const void* W, float* gW, void* gX,
-                       const Geo& g, cudaStream_t s);
+                       const Geo& g, int stride, cudaStream_t s);
+// strided layers (gf_strided.cu): per-phase kernel sums, rows of s*s*C_ig values per output channel
+gf_status launch_ksum_phase(const void* W, int dtype, int C_out, int C_ig, int KH, int KW, int stride, float* tph, cudaStream_t s);
+// gX[n, c, h, w] <- ghat[n, (group, phase of (h, w), channel in group), h / (r s), w / (r s)]
+gf_status launch_expand_phase(const float* ghat, void* gX, int dtype, int N, int C_in, int G, int H, int W, int stride, int r,
+                              cudaStream_t s);
 
 }  // namespace gf

@@ -207,7 +207,7 @@ gf_status launch_gw_partial(const float* gbar, const void* stash, float* part, i
 
 // ---------------------------------------------------------------- gw_finish
 __global__ void gw_finish_kernel(const float* __restrict__ part, int S, size_t n_pairs, int taps,
-                                 FastDiv div_taps, float* __restrict__ gW) {
+                                 FastDiv div_taps, float* __restrict__ gW, float scale) {
     pdl_launch_dependents();
     pdl_wait();
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -221,20 +221,20 @@ __global__ void gw_finish_kernel(const float* __restrict__ part, int S, size_t n
         for (int u = 0; u < 8; ++u) acc[u] += part[(size_t)(k + u) * n_pairs + pair];
     }
     for (; k < S; ++k) acc[0] += part[(size_t)k * n_pairs + pair];
-    gW[i] = ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
+    gW[i] = (((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]))) * scale;
 }
 
 // One partial matrix (the tensor-core path accumulates in place): a pure broadcast of
 // every unique value to its taps, four consecutive outputs (one 16-byte store) per thread.
 __global__ void __launch_bounds__(256) gw_broadcast_kernel(const float* __restrict__ part, size_t total, FastDiv div_taps,
-                                                           float* __restrict__ gW) {
+                                                           float* __restrict__ gW, float scale) {
     pdl_launch_dependents();
     pdl_wait();
     const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
     if (i >= total) return;
     float v[4];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) v[k] = i + k < total ? part[div_taps.div((uint32_t)(i + k))] : 0.f;
+    for (int k = 0; k < 4; ++k) v[k] = i + k < total ? part[div_taps.div((uint32_t)(i + k))] * scale : 0.f;
     if (i + 4 <= total) {
         *reinterpret_cast<float4*>(gW + i) = make_float4(v[0], v[1], v[2], v[3]);
     } else {
@@ -245,7 +245,7 @@ __global__ void __launch_bounds__(256) gw_broadcast_kernel(const float* __restri
 // Many partial matrices (S >= 16): 32 pairs per block, the partials dealt to the block's 8
 // warps, every load of a warp independent; the sum order is fixed.
 __global__ void __launch_bounds__(256) gw_finish_wide_kernel(const float* __restrict__ part, int S, size_t n_pairs,
-                                                             int taps, FastDiv div_taps, float* __restrict__ gW) {
+                                                             int taps, FastDiv div_taps, float* __restrict__ gW, float scale) {
     __shared__ float red[8][33];
     pdl_launch_dependents();
     pdl_wait();
@@ -268,11 +268,11 @@ __global__ void __launch_bounds__(256) gw_finish_wide_kernel(const float* __rest
         float v = 0.f;
 #pragma unroll
         for (int w = 0; w < 8; ++w) v += red[w][pl];
-        gW[pair0 * taps + o] = v;
+        gW[pair0 * taps + o] = v * scale;
     }
 }
 
-gf_status launch_gw_finish(const float* part, int splits, float* gW, const Geo& g, cudaStream_t s) {
+gf_status launch_gw_finish(const float* part, int splits, float* gW, const Geo& g, cudaStream_t s, float scale) {
     ProfScope prof(K_GW_FINISH, s);
     const size_t n_pairs = (size_t)g.C_out * g.C_ig;
     const int taps = g.KH * g.KW;
@@ -280,12 +280,12 @@ gf_status launch_gw_finish(const float* part, int splits, float* gW, const Geo& 
     if (total > 0x7fffffffULL) return GF_ERR_UNSUPPORTED;
     if (splits == 1)
         return launch_pdl(gw_broadcast_kernel, dim3((unsigned)((total / 4 + 256) / 256)), dim3(256), 0, s, part, total,
-                          FastDiv(taps), gW);
+                          FastDiv(taps), gW, scale);
     if (splits >= 16)
         return launch_pdl(gw_finish_wide_kernel, dim3((unsigned)((n_pairs + 31) / 32)), dim3(256), 0, s, part, splits,
-                          n_pairs, taps, FastDiv(taps), gW);
+                          n_pairs, taps, FastDiv(taps), gW, scale);
     return launch_pdl(gw_finish_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, s, part, splits, n_pairs,
-                      taps, FastDiv(taps), gW);
+                      taps, FastDiv(taps), gW, scale);
 }
 
 }  // namespace gf

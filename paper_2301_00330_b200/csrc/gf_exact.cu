@@ -1,9 +1,10 @@
 // r == 1: the method is off and the backward is the exact ("vanilla")
-// convolution backward of Section 3.1, stride 1, zero padding.  Plain direct
+// convolution backward of Section 3.1, stride s, zero padding.  Plain direct
 // kernels, not tuned: this path exists so that a patch size of 1 has the
-// meaning the paper gives it.
-//   g_W[c_o,c_l,u,v] = sum_{n,i,j} x[n,c_i,i+u-ph,j+v-pw] g_y[n,c_o,i,j]
-//   g_X[n,c_i,h,w]   = sum_{c_o,u,v} W[c_o,c_l,u,v] g_y[n,c_o,h-u+ph,w-v+pw]
+// meaning the paper gives it.  g_y is [N, C_out, H/s, W/s].
+//   g_W[c_o,c_l,u,v] = sum_{n,i,j} x[n,c_i,s i+u-ph,s j+v-pw] g_y[n,c_o,i,j]
+//   g_X[n,c_i,h,w]   = sum_{c_o,u,v} W[c_o,c_l,u,v] g_y[n,c_o,(h-u+ph)/s,(w-v+pw)/s]
+//                      over the taps for which both quotients are whole numbers
 #include "gf_common.cuh"
 
 namespace gf {
@@ -11,7 +12,7 @@ namespace gf {
 template <typename T>
 __global__ void __launch_bounds__(256) exact_gx_kernel(const T* __restrict__ gy, const T* __restrict__ Wt,
                                                        T* __restrict__ gX, int N, int C_in, int C_out, int G,
-                                                       int H, int W, int KH, int KW) {
+                                                       int H, int W, int KH, int KW, int S) {
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const long long total = (long long)N * C_in * H * W;
     if (idx >= total) return;
@@ -19,16 +20,17 @@ __global__ void __launch_bounds__(256) exact_gx_kernel(const T* __restrict__ gy,
     const int ci = (int)((idx / ((long long)W * H)) % C_in), n = (int)(idx / ((long long)W * H * C_in));
     const int C_ig = C_in / G, C_og = C_out / G, q = ci / C_ig, cl = ci - q * C_ig;
     const int ph = (KH - 1) / 2, pw = (KW - 1) / 2;
+    const int Hy = H / S, Wy = W / S;
     float s = 0.f;
     for (int co = q * C_og; co < (q + 1) * C_og; ++co)
         for (int u = 0; u < KH; ++u) {
-            const int i = h - u + ph;
-            if (i < 0 || i >= H) continue;
+            const int is = h - u + ph;
+            if (is < 0 || is % S != 0 || is / S >= Hy) continue;
             for (int v = 0; v < KW; ++v) {
-                const int j = w - v + pw;
-                if (j < 0 || j >= W) continue;
+                const int js = w - v + pw;
+                if (js < 0 || js % S != 0 || js / S >= Wy) continue;
                 s = fmaf(to_f32(Wt[(((size_t)co * C_ig + cl) * KH + u) * KW + v]),
-                         to_f32(gy[(((size_t)n * C_out + co) * H + i) * W + j]), s);
+                         to_f32(gy[(((size_t)n * C_out + co) * Hy + is / S) * Wy + js / S]), s);
             }
         }
     gX[idx] = from_f32<T>(s);
@@ -38,7 +40,7 @@ __global__ void __launch_bounds__(256) exact_gx_kernel(const T* __restrict__ gy,
 template <typename T>
 __global__ void __launch_bounds__(256) exact_gw_kernel(const T* __restrict__ gy, const T* __restrict__ x,
                                                        float* __restrict__ gW, int N, int C_in, int C_out, int G,
-                                                       int H, int W, int KH, int KW) {
+                                                       int H, int W, int KH, int KW, int S) {
     __shared__ float warp_part[8];
     const int taps = KH * KW;
     const int C_ig = C_in / G, C_og = C_out / G;
@@ -47,15 +49,16 @@ __global__ void __launch_bounds__(256) exact_gw_kernel(const T* __restrict__ gy,
     const int u = t / KW, v = t - u * KW;
     const int ci = (co / C_og) * C_ig + cl;
     const int ph = (KH - 1) / 2, pw = (KW - 1) / 2;
-    const long long per = (long long)H * W, total = (long long)N * per;
+    const int Hy = H / S, Wy = W / S;
+    const long long per = (long long)Hy * Wy, total = (long long)N * per;
     float s = 0.f;
     for (long long e = threadIdx.x; e < total; e += 256) {
         const int n = (int)(e / per), rem = (int)(e - n * per);
-        const int i = rem / W, j = rem - i * W;
-        const int h = i + u - ph, w = j + v - pw;
+        const int i = rem / Wy, j = rem - i * Wy;
+        const int h = S * i + u - ph, w = S * j + v - pw;
         if (h < 0 || h >= H || w < 0 || w >= W) continue;
         s = fmaf(to_f32(x[(((size_t)n * C_in + ci) * H + h) * W + w]),
-                 to_f32(gy[(((size_t)n * C_out + co) * H + i) * W + j]), s);
+                 to_f32(gy[(((size_t)n * C_out + co) * Hy + i) * Wy + j]), s);
     }
     s = warp_sum(s);
     if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = s;
@@ -68,7 +71,7 @@ __global__ void __launch_bounds__(256) exact_gw_kernel(const T* __restrict__ gy,
 }
 
 gf_status launch_exact(const void* gy, const void* x, const void* W, float* gW, void* gX,
-                       const Geo& g, cudaStream_t s) {
+                       const Geo& g, int stride, cudaStream_t s) {
     if (gX) {
         ProfScope prof(K_EXACT_GX, s);
         const long long total = (long long)g.N * g.C_in * g.H * g.W;
@@ -76,11 +79,11 @@ gf_status launch_exact(const void* gy, const void* x, const void* W, float* gW, 
         if (blocks > 0x7fffffffLL) return GF_ERR_UNSUPPORTED;
         if (g.dtype == GF_F32)
             exact_gx_kernel<float><<<(unsigned)blocks, 256, 0, s>>>((const float*)gy, (const float*)W, (float*)gX,
-                                                                     g.N, g.C_in, g.C_out, g.G, g.H, g.W, g.KH, g.KW);
+                                                                     g.N, g.C_in, g.C_out, g.G, g.H, g.W, g.KH, g.KW, stride);
         else
             exact_gx_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, s>>>(
                 (const __nv_bfloat16*)gy, (const __nv_bfloat16*)W, (__nv_bfloat16*)gX, g.N, g.C_in, g.C_out, g.G,
-                g.H, g.W, g.KH, g.KW);
+                g.H, g.W, g.KH, g.KW, stride);
         gf_status st = after_launch();
         if (st != GF_OK) return st;
     }
@@ -90,11 +93,11 @@ gf_status launch_exact(const void* gy, const void* x, const void* W, float* gW, 
         if (blocks > 0x7fffffffLL) return GF_ERR_UNSUPPORTED;
         if (g.dtype == GF_F32)
             exact_gw_kernel<float><<<(unsigned)blocks, 256, 0, s>>>((const float*)gy, (const float*)x, gW, g.N,
-                                                                     g.C_in, g.C_out, g.G, g.H, g.W, g.KH, g.KW);
+                                                                     g.C_in, g.C_out, g.G, g.H, g.W, g.KH, g.KW, stride);
         else
             exact_gw_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, s>>>(
                 (const __nv_bfloat16*)gy, (const __nv_bfloat16*)x, gW, g.N, g.C_in, g.C_out, g.G, g.H, g.W, g.KH,
-                g.KW);
+                g.KW, stride);
         return after_launch();
     }
     return GF_OK;

@@ -95,7 +95,9 @@ def test_descriptor_validation(gf):
     assert st(dtype=7) == gf.GF_ERR_BAD_DESC
     assert st(layout=5) == gf.GF_ERR_BAD_DESC
     assert st(layout=gf.GF_NHWC) == gf.GF_ERR_UNSUPPORTED
-    assert st(stride=2) == gf.GF_ERR_UNSUPPORTED
+    assert st(stride=2) == gf.GF_OK                          # s | H and s | W: g_y is [H/s, W/s]
+    assert st(stride=3) == gf.GF_ERR_UNSUPPORTED             # 3 does not divide 8
+    assert st(stride=0) == gf.GF_ERR_BAD_DESC
     assert st(KH=2) == gf.GF_ERR_UNSUPPORTED
     assert st(pad_h=0) == gf.GF_ERR_UNSUPPORTED
     assert st(KH=3, KW=5, pad_w=1) == gf.GF_ERR_UNSUPPORTED
