@@ -66,8 +66,10 @@ def test_stash_bytes_match_the_papers_mem_column(gf, model, k, ours_kb, shapes):
     """Table "ImageNet classification", column Mem, rows "Ours" (fp32, batch 1, r = 2).
     The stash lives on the grid of g_y, so a layer is described by its g_y map."""
     total = 0
-    for c_in, _, _, hy, wy in shapes:
-        total += gf.gf_stash_bytes(gf.make_desc(1, c_in, c_in, hy, wy, 3, r=2))
+    for c_in, hx, wx, hy, wy in shapes:
+        stride = hx // hy
+        assert hx == hy * stride and wx == wy * stride
+        total += gf.gf_stash_bytes(gf.make_desc(1, c_in, c_in, hx, wx, 3, r=2, stride=stride))
     assert abs(total / 1024 - ours_kb) < 0.005
 
 
