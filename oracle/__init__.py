@@ -9,3 +9,4 @@ from .gf_oracle import (act_stash_forward, activation, activation_fast, backward
 from .gf_diagnostics import dcac_ratio, filter_snr_terms, snr_terms, snr_terms_fast  # noqa: F401,E402
 from .gf_strided import (exact_backward_strided, kernel_phase_sums, strided_backward,  # noqa: F401,E402
                          strided_stash_forward)
+from . import gf_int8 as int8  # noqa: F401,E402
