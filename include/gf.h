@@ -163,6 +163,26 @@ gf_status gf_layer_step_host(const gf_conv_desc* desc, const void* h_x, const vo
                              const void* h_W, float* h_gW, void* h_gX, void* arena,
                              size_t arena_bytes, void* stream);
 
+/* ---- INT8 variant of the two reduced contractions ------------------------------------------
+ * The supplement's section on combining gradient filtering with gradient quantization trains
+ * with feature maps, weights and gradients as INT8 (its CIFAR table); the paper names the
+ * schemes (per-tensor and per-sample) and prints no formulas.  This entry point fixes the
+ * plainest one -- per tensor, symmetric, round to nearest even:
+ *     scale(t) = max|t| / 127 (1 for an all-zero tensor), code(v) = clamp(rint(v / scale), -127, 127)
+ * -- applies it to the stash, to the patch means of g_y (Section 3.3) and to the kernel sums,
+ * and evaluates Eq. (grad_w) and Eq. (grad_x) on the codes with 32-bit integer accumulation:
+ *     g_W = (sum codes_X codes_G) * (scale_X * scale_G),  g_X = (sum codes_G codes_Th) * (scale_G * scale_Th).
+ * Arguments, layouts and nullable outputs as gf_backward; dense layers (groups 1), stride 1,
+ * r >= 2, N * patches per image * 127^2 < 2^31 (else GF_ERR_UNSUPPORTED).  Every floating-point
+ * step that decides a code is fp32 in a fixed order (patch mean: elements row by row, left to
+ * right, times the reciprocal of their count; kernel sum: taps in memory order), so results
+ * are reproducible bit for bit; the integer sums are exact.  The workspace has its own size
+ * query; gf_last_async_status reads its error word like gf_backward's. */
+gf_status gf_backward_int8_workspace_bytes(const gf_conv_desc* desc, size_t* bytes);
+gf_status gf_backward_int8(const gf_conv_desc* desc, const void* g_y, const void* stash,
+                           const void* W, float* g_W, void* g_X, void* workspace,
+                           size_t workspace_bytes, void* stream);
+
 /* ---- Error diagnostics of the paper's analysis (Section 4.1) -----------------------------
  * Not part of a training step: the quantities with which the paper relates patch size, noise
  * level and accuracy (Figure "SNR", Table of energy ratios).  `energies` is a DEVICE pointer

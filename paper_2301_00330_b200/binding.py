@@ -28,6 +28,7 @@ EXPORTS = (
     "gf_kernel_launch_count", "gf_status_string", "gf_profile_configure", "gf_profile_read",
     "gf_kernel_name", "gf_kernel_id_count", "gf_backward_static_scratch", "gf_set_dense_path",
     "gf_snr_terms", "gf_filter_snr_terms", "gf_dcac_ratio", "gf_act_stash_forward",
+    "gf_backward_int8", "gf_backward_int8_workspace_bytes",
 )
 
 
@@ -77,6 +78,10 @@ def lib() -> ctypes.CDLL:
         L.gf_act_stash_forward.argtypes = [dp, ctypes.c_int32, vp, vp, vp, vp]
         L.gf_act_stash_forward.restype = ctypes.c_int
         L.gf_backward.argtypes = [dp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.gf_backward_int8.argtypes = [dp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.gf_backward_int8.restype = ctypes.c_int
+        L.gf_backward_int8_workspace_bytes.argtypes = [dp, ctypes.POINTER(sz)]
+        L.gf_backward_int8_workspace_bytes.restype = ctypes.c_int
         L.gf_backward_static_scratch.argtypes = [dp, vp, vp, vp, vp, vp, vp]
         L.gf_backward_static_scratch.restype = ctypes.c_int
         L.gf_last_async_status.argtypes = [vp, vp]
@@ -191,6 +196,20 @@ def gf_backward(desc: gf_conv_desc, g_y, stash, W, g_W, g_X, workspace, workspac
     _check(lib().gf_backward(ctypes.byref(desc), _ptr(g_y), _ptr(stash), _ptr(W), _ptr(g_W), _ptr(g_X),
                              _ptr(workspace), ctypes.c_size_t(workspace_bytes), _stream(stream)),
            "gf_backward")
+
+
+def gf_backward_int8_workspace_bytes(desc: gf_conv_desc) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().gf_backward_int8_workspace_bytes(ctypes.byref(desc), ctypes.byref(out)), "gf_backward_int8_workspace_bytes")
+    return int(out.value)
+
+
+def gf_backward_int8(desc: gf_conv_desc, g_y, stash, W, g_W, g_X, workspace, workspace_bytes=None, stream=None) -> None:
+    """gf_backward with the operands of the two reduced contractions quantised to INT8."""
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    _check(lib().gf_backward_int8(ctypes.byref(desc), _ptr(g_y), _ptr(stash), _ptr(W), _ptr(g_W), _ptr(g_X), _ptr(workspace),
+                                  ctypes.c_size_t(workspace_bytes), _stream(stream)), "gf_backward_int8")
 
 
 GF_STATIC_SCRATCH_BYTES = 8 << 20

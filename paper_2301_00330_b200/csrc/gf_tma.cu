@@ -44,6 +44,20 @@ bool make_tmap_bf16(CUtensorMap* out, const void* base, int rank, uint64_t d0, u
     return r == CUDA_SUCCESS;
 }
 
+bool make_tmap_u8_2d(CUtensorMap* out, const void* base, uint64_t width, uint64_t rows, uint64_t pitch, uint32_t box_rows) {
+    PFN_cuTensorMapEncodeTiled enc = encoder();
+    if (!enc) return false;
+    if ((reinterpret_cast<uintptr_t>(base) & 15u) != 0 || pitch % 16 != 0 || box_rows < 1 || box_rows > 256) return false;
+    cuuint64_t dims[2] = {width, rows};
+    cuuint64_t strides[1] = {pitch};
+    cuuint32_t box[2] = {128, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    const CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 bool make_tmap_plain(CUtensorMap* out, const void* base, int elem_bytes, uint64_t d0, uint64_t d1, uint64_t d2,
                      uint64_t stride1, uint64_t stride2, uint32_t box0, uint32_t box1, uint32_t box2) {
     PFN_cuTensorMapEncodeTiled enc = encoder();

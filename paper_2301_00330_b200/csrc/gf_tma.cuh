@@ -34,7 +34,18 @@ bool make_tmap_bf16(CUtensorMap* out, const void* base, int rank, uint64_t d0, u
 bool make_tmap_plain(CUtensorMap* out, const void* base, int elem_bytes, uint64_t d0, uint64_t d1, uint64_t d2,
                      uint64_t stride1, uint64_t stride2, uint32_t box0, uint32_t box1, uint32_t box2);
 
+// Byte matrix [rows][pitch] (int8 operands), rows of `width` valid bytes, box = {128 bytes, box_rows},
+// 128-byte swizzle: a box lands as a K-major tile of 128-byte rows.  pitch is a multiple of 16.
+bool make_tmap_u8_2d(CUtensorMap* out, const void* base, uint64_t width, uint64_t rows, uint64_t pitch, uint32_t box_rows);
+
 #ifdef __CUDACC__
+__device__ __forceinline__ void tma_load_2d(void* dst_smem, const CUtensorMap* m, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+            smem_u32(dst_smem)),
+        "l"(reinterpret_cast<uint64_t>(m)), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
 __device__ __forceinline__ void tma_load_3d(void* dst_smem, const CUtensorMap* m, int x, int y, int z, uint64_t* bar) {
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(

@@ -154,3 +154,17 @@ def test_diagnostics_reject_bad_arguments(gf):
     assert L.gf_filter_snr_terms(a, 1, 0, 4, 2, 0, a, None) == gf.GF_ERR_BAD_DESC
     assert L.gf_dcac_ratio(a, 1, 1, 3, 3, 2, 3, 0, a, None) == gf.GF_ERR_BAD_DESC          # DFT smaller than the kernel
     assert L.gf_dcac_ratio(a, 1, 1, 3, 3, 128, 3, 0, a, None) == gf.GF_ERR_UNSUPPORTED
+
+
+def test_int8_entry_point_validates_on_the_host(gf):
+    """gf_backward_int8: dense stride-1 layers with r >= 2 whose integer sums fit 32 bits."""
+    L = gf.lib()
+    size = ctypes.c_size_t(0)
+    ok = gf.make_desc(2, 8, 8, 8, 8, 3, r=2)
+    assert L.gf_backward_int8_workspace_bytes(ctypes.byref(ok), ctypes.byref(size)) == gf.GF_OK and size.value > 0
+    for bad in (gf.make_desc(2, 8, 8, 8, 8, 3, r=1), gf.make_desc(2, 8, 8, 8, 8, 3, r=2, groups=2),
+                gf.make_desc(2, 8, 8, 8, 8, 3, r=2, stride=2), gf.make_desc(4096, 8, 8, 64, 64, 3, r=2)):
+        assert L.gf_backward_int8_workspace_bytes(ctypes.byref(bad), ctypes.byref(size)) == gf.GF_ERR_UNSUPPORTED
+    a = ctypes.c_void_p(0x1000)
+    assert L.gf_backward_int8(ctypes.byref(ok), a, a, a, a, a, a, 16, None) == gf.GF_ERR_WORKSPACE
+    assert L.gf_backward_int8(ctypes.byref(ok), None, a, a, a, a, a, 1 << 30, None) == gf.GF_ERR_NULL
