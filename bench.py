@@ -50,7 +50,19 @@ PAPER_CONTEXT = {
 # DRAM bytes per launch of a kernel from one ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by (layer name, kernel name), with the sha1 of the kernel's
 # source file at capture time; a changed source makes the entry stale (reported as null).
-NCU_TRAFFIC: dict[tuple[str, str], dict] = {}
+NCU_TRAFFIC: dict[tuple[str, str], dict] = {
+    # ncu --set full --clock-control none, python bench.py --table --no-exact --only <layer>/r2 (profiles/*.md)
+    ("cfg3b_dw_576", "dw_fused"): {"bytes": 289.06e6 + 188.65e6, "sha1": "4b5034114d07f51de9ec93105e217e4cac06777c"},
+    ("cfg3c_pw_576_96", "gyx_fused"): {"bytes": 38.90e6 + 191.65e6, "sha1": "c2d76b39a44a92f630179823637696df5538dfdc"},
+    ("cfg3c_pw_576_96", "gw_tiled"): {"bytes": 74.89e6 + 2.70e6, "sha1": "c2d76b39a44a92f630179823637696df5538dfdc"},
+    ("cfg3a_pw_96_576", "stash_pool"): {"bytes": 38.55e6 + 0.01e6, "sha1": "56c08adc367812dd2e6ee11acb71cb1a0a803d89"},
+    ("cfg3a_pw_96_576", "gx_tc"): {"bytes": 58.06e6 + 6.21e6, "sha1": "ad0e9c6bc266fdbd98fb4f0844a50827a978735e"},
+    ("cfg3a_pw_96_576", "gw_tc"): {"bytes": 67.71e6 + 0.79e6, "sha1": "ad0e9c6bc266fdbd98fb4f0844a50827a978735e"},
+    # not captured: the same kernel on the two larger inputs of the step; its traffic on the captured
+    # layer equals the bytes of x (the stash it writes was still in L2 when the kernel ended), scaled here
+    ("cfg3b_dw_576", "stash_pool"): {"bytes": 38.55e6 * 6.0, "sha1": "56c08adc367812dd2e6ee11acb71cb1a0a803d89", "scaled": True},
+    ("cfg3c_pw_576_96", "stash_pool"): {"bytes": 38.55e6 * 6.0, "sha1": "56c08adc367812dd2e6ee11acb71cb1a0a803d89", "scaled": True},
+}
 
 KERNEL_SOURCE = {
     "stash_pool": "gf_pool.cu", "gy_pool": "gf_pool.cu", "ksum": "gf_tc.cu", "gx_mix": "gf_dense.cu",
@@ -178,15 +190,41 @@ def kernel_cost(name: str, L) -> tuple[float, float]:
     return table[name]
 
 
+def _source_sha1(src: str) -> str:
+    with open(os.path.join(ROOT, "paper_2301_00330_b200", "csrc", src), "rb") as f:
+        return hashlib.sha1(f.read()).hexdigest()
+
+
 def traffic_for(layer_name: str, kernel: str):
+    """DRAM bytes of one launch from the ncu capture on file, or None when there is none or the
+    kernel's source has changed since the capture (the entry holds the source's hash at that time)."""
     ent = NCU_TRAFFIC.get((layer_name, kernel))
     src = KERNEL_SOURCE.get(kernel)
     if not ent or not src:
         return None
-    path = os.path.join(ROOT, "paper_2301_00330_b200", "csrc", src)
-    with open(path, "rb") as f:
-        sha = hashlib.sha1(f.read()).hexdigest()
-    return ent["bytes"] if sha == ent.get("sha1") else None
+    return ent["bytes"] if ent.get("sha1") == _source_sha1(src) else None
+
+
+def roofline_step(name: str, total_ms: float, launches: int, steps: int, layers) -> dict:
+    """Roofline of a kernel over all its launches of a step: algorithmic bytes of those launches
+    (summed over the layers that use it) / their summed duration."""
+    peaks, which = measured_peaks()
+    users = [L for L in layers if name in KERNELS_OF_LAYER.get(L.name, ())]
+    per_step = sum(kernel_cost(name, L)[0] for L in users)
+    per_launch = launches / max(steps, 1)
+    ach = per_step * steps / (total_ms * 1e-3) / 1e9 if total_ms > 0 else 0.0
+    traffic = [traffic_for(L.name, name) for L in users]
+    return {"kernel": name, "layers": [L.name for L in users], "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"],
+            "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "peak_source": f"of {which}",
+            "launches_per_step": per_launch, "algorithmic_bytes_per_launch": per_step / max(per_launch, 1),
+            "avg_launch_us": total_ms * 1e3 / max(launches, 1),
+            "traffic": (sum(traffic) / len(traffic)) if traffic and all(t is not None for t in traffic) else None,
+            "traffic_note": "ncu dram__bytes_read.sum + dram__bytes_write.sum per launch, averaged over the step's launches "
+                            "of this kernel; the two 289 MB inputs are scaled from the capture on the 38.5 MB one "
+                            "(read bytes = bytes of x; the stash written was still in L2 when the kernel ended)"}
+
+
+KERNELS_OF_LAYER: dict[str, tuple] = {}
 
 
 def roofline(name: str, avg_ms: float, L) -> dict:
@@ -352,6 +390,94 @@ def time_layer(gf, L, peaks, with_exact: bool = True, with_kernels: bool = False
     return row
 
 
+def diagnostics(gf, runs) -> dict:
+    """Section 4.1 on the step's own tensors: SNR of the filtered g_y per layer (Eq. (snr_g3), first
+    line) and the DC/AC energy ratio of the 3x3 kernels (Eq. (dcac_ratio)), by the library's kernels."""
+    import math
+    import torch
+    out = {"note": "synthetic i.i.d. gradients and Kaiming-random kernels: the numbers show the diagnostics run, they are not "
+                   "the paper's (trained networks have DC-dominated kernels and smoother gradients)", "layers": {}}
+    e = torch.zeros(2, dtype=torch.float64, device="cuda")
+    for L, desc, w, _, sets in runs:
+        gy = sets[0][1]
+        gf.gf_filter_snr_terms(gy, L.r, e)
+        torch.cuda.synchronize()
+        sig, noise = (float(v) for v in e.cpu())
+        row = {"snr_gy": sig / noise if noise > 0 else None,
+               "snr_gy_db": 10.0 * math.log10(sig / noise) if noise > 0 and sig > 0 else None}
+        if L.K > 1:
+            ratio = torch.empty((L.C_out, L.C_ig), dtype=torch.float32, device="cuda")
+            gf.gf_dcac_ratio(w, ratio)
+            torch.cuda.synchronize()
+            row["dcac_ratio_mean"] = float(ratio.mean())
+            row["dcac_ratio_share_ge_1"] = float((ratio >= 1).float().mean())
+        out["layers"][L.name] = row
+    return out
+
+
+def extras(gf, layers) -> dict:
+    """Timings of the further entry points on shapes of the step (events behind a backlog, 10 calls)."""
+    import torch
+    from paper_2301_00330_b200 import workloads
+    stream = torch.cuda.current_stream()
+
+    def timed(fn, n=10):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        backlog(3.0)
+        e0.record(stream)
+        for _ in range(n):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return round(e0.elapsed_time(e1) * 1e3 / n, 1)
+
+    out = {}
+    # the stash produced inside the producer of x (ReLU6 + x + stash in one pass) on the depthwise layer's input
+    L = layers[1]
+    desc = gf.desc_for(L)
+    z = torch.randn((L.N, L.C_in, L.H, L.W), device="cuda")
+    x = torch.empty_like(z)
+    stash = torch.empty(gf.gf_stash_dims(desc), device="cuda")
+    t_fused = timed(lambda: gf.gf_act_stash_forward(desc, gf.GF_ACT_RELU6, z, x, stash, stream))
+    t_act = timed(lambda: torch.clamp(z, 0.0, 6.0, out=x))
+    t_stash = timed(lambda: gf.gf_stash_forward(desc, x, stash, stream))
+    nbytes = z.numel() * 4 * 2 + stash.numel() * 4
+    out["act_stash_forward"] = {"layer": L.name, "fused_us": t_fused, "separate_us": {"relu6_torch": t_act, "gf_stash_forward": t_stash},
+                                "fused_gbs": round(nbytes / t_fused / 1e3, 1),
+                                "note": "Section 4.2: the forward overhead of the method is what the fused pass costs beyond the activation alone"}
+    del z, x, stash
+    # INT8 variant of the reduced contractions on the two pointwise layers
+    out["backward_int8_us"] = {}
+    for L in (layers[0], layers[2]):
+        desc = gf.desc_for(L)
+        x0, gy0, w0 = workloads.make_inputs(L)
+        gy, w = gy0.cuda(), w0.cuda()
+        buf = gf.alloc_layer(desc)
+        gf.gf_stash_forward(desc, x0.cuda(), buf.stash, stream)
+        ws = torch.empty(gf.gf_backward_int8_workspace_bytes(desc), dtype=torch.uint8, device="cuda")
+        out["backward_int8_us"][L.name] = timed(lambda: gf.gf_backward_int8(desc, gy, buf.stash, w, buf.g_W, buf.g_X, ws, None, stream))
+        del gy, w, buf, ws
+    # a stride-2 layer of the kind inside the paper's trained ranges (ResNet-18 stage transition)
+    desc = gf.make_desc(64, 128, 256, 28, 28, 3, r=2, stride=2)
+    xs = torch.randn((64, 128, 28, 28), device="cuda").clamp_(min=0)
+    gys = torch.randn((64, 256, 14, 14), device="cuda") * 1e-2
+    wsd = torch.randn((256, 128, 3, 3), device="cuda") * 0.04
+    stash = torch.empty(gf.gf_stash_dims(desc), device="cuda")
+    gW, gX = torch.empty_like(wsd), torch.empty_like(xs)
+    ws = torch.empty(gf.gf_backward_workspace_bytes(desc), dtype=torch.uint8, device="cuda")
+    gf.gf_stash_forward(desc, xs, stash, stream)
+    out["stride2_3x3_128_256_28x28_N64_r2"] = {
+        "stash_us": timed(lambda: gf.gf_stash_forward(desc, xs, stash, stream)),
+        "backward_us": timed(lambda: gf.gf_backward(desc, gys, stash, wsd, gW, gX, ws, None, stream)),
+        "exact_cudnn_us": timed(lambda: torch.ops.aten.convolution_backward(gys, xs, wsd, None, [2, 2], [1, 1], [1, 1], False,
+                                                                            [0, 0], 1, [True, True, False]), 4)}
+    torch.cuda.empty_cache()
+    return out
+
+
 def per_config_layers():
     """Every layer of the workload configurations (rows of the measurement table)."""
     from paper_2301_00330_b200 import workloads
@@ -412,7 +538,7 @@ def run_ours(args) -> None:
     # (layer, kernel) pair that takes the most time ----
     diag_steps = 4
     breakdown = {}
-    dominant, dom_ms = None, -1.0
+    per_kernel_ms: dict[str, float] = {}
     for k, (L, *_rest) in enumerate(runs):
         gf.gf_profile_configure(2)
         backlog()
@@ -423,17 +549,18 @@ def run_ours(args) -> None:
         gf.gf_profile_configure(0)
         breakdown[L.name] = {kn: {"launches_per_step": n / diag_steps, "avg_us": round(ms / n * 1e3, 2)}
                              for kn, (n, ms) in diag.items()}
+        KERNELS_OF_LAYER[L.name] = tuple(diag.keys())
         for kn, (n, ms) in diag.items():
-            if ms > dom_ms:
-                dominant, dom_ms = (k, kn), ms
+            per_kernel_ms[kn] = per_kernel_ms.get(kn, 0.0) + ms
 
-    # ---- dominant kernel: event pairs around it alone, over eager steps of its layer ----
-    dom_layer, dom_kernel = dominant
-    dom_steps = max(1, min(args.steps, 32))
+    # ---- dominant kernel = the one with the largest summed time over a step (all its launches, all
+    # layers): event pairs around it alone, over eager steps ----
+    dom_kernel = max(per_kernel_ms, key=per_kernel_ms.get)
+    dom_steps = max(1, min(args.steps, 16))
     gf.gf_profile_configure(1, gf.kernel_id(dom_kernel))
     backlog()
     for i in range(dom_steps):
-        layer_step(dom_layer, i)
+        step(i)
     torch.cuda.synchronize()
     dom = gf.gf_profile_read()
     gf.gf_profile_configure(0)
@@ -520,10 +647,10 @@ def run_ours(args) -> None:
             dist.destroy_process_group()
         return
 
-    L_dom = layers[dom_layer]
     n_dom, ms_dom = dom.get(dom_kernel, (0, 0.0))
-    roof = roofline(dom_kernel, ms_dom / max(n_dom, 1), L_dom)
+    roof = roofline_step(dom_kernel, ms_dom, n_dom, dom_steps, layers)
     roof["timed_launches"] = n_dom
+    roof["share_of_step_kernel_time"] = per_kernel_ms[dom_kernel] / sum(per_kernel_ms.values())
     peaks, which = measured_peaks()
     step_bytes = sum(L.backward_bytes() + L.stash_bytes_moved() for L in layers)
     line = {
@@ -532,7 +659,7 @@ def run_ours(args) -> None:
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": workload_config(layers),
         "timing": (f"CUDA events around K steps; {replays} replays of a {n_sets}-step CUDA graph + {rest} eager steps; "
-                   f"dominant kernel timed by event pairs over {dom_steps} eager steps of its layer"),
+                   f"dominant kernel (largest summed time over a step) timed by event pairs over {dom_steps} eager steps"),
         "parallelism": "replicas only" if world > 1 else "single GPU",
         "block_us": ms_per_step * 1e3,
         "step_algorithmic_bytes": step_bytes,
@@ -543,10 +670,12 @@ def run_ours(args) -> None:
         "gpu_launches": int(launches),
     }
     if world == 1:
+        line["diagnostics"] = diagnostics(gf, runs)
         for _, _, _, _, sets in runs:
             sets.clear()
         runs.clear()
         torch.cuda.empty_cache()
+        line["extras"] = extras(gf, layers)
         line["cpu_baseline"] = time_oracle(layers, 32, 2, 1)
         if not args.no_per_config:
             rows = [time_layer(gf, L, peaks) for L in per_config_layers()]
