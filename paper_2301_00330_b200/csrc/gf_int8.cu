@@ -32,8 +32,35 @@ __device__ __forceinline__ void block_absmax(float v, uint32_t* out) {
     if ((threadIdx.x & 31) == 0 && b != 0) atomicMax(out, b);
 }
 
-// Patch means in the fixed order, one thread per patch, and their max|.|.
-template <typename T>
+// R consecutive elements starting at p (aligned to their total size when R * sizeof(T) <= 16, else to 16 bytes)
+template <int R> __device__ __forceinline__ void load_row(const float* p, float (&v)[R]) {
+    if constexpr (R == 2) { const float2 t = __ldcs(reinterpret_cast<const float2*>(p)); v[0] = t.x; v[1] = t.y; }
+    else {
+#pragma unroll
+        for (int k = 0; k < R / 4; ++k) {
+            const float4 t = __ldcs(reinterpret_cast<const float4*>(p) + k);
+            v[4 * k] = t.x; v[4 * k + 1] = t.y; v[4 * k + 2] = t.z; v[4 * k + 3] = t.w;
+        }
+    }
+}
+template <int R> __device__ __forceinline__ void load_row(const __nv_bfloat16* p, float (&v)[R]) {
+    if constexpr (R == 2) { const uint32_t t = __ldcs(reinterpret_cast<const unsigned int*>(p)); v[0] = __uint_as_float(t << 16); v[1] = __uint_as_float(t & 0xffff0000u); }
+    else if constexpr (R == 4) {
+        const uint2 t = __ldcs(reinterpret_cast<const uint2*>(p));
+        v[0] = __uint_as_float(t.x << 16); v[1] = __uint_as_float(t.x & 0xffff0000u);
+        v[2] = __uint_as_float(t.y << 16); v[3] = __uint_as_float(t.y & 0xffff0000u);
+    } else {
+        const uint4 t = __ldcs(reinterpret_cast<const uint4*>(p));
+        const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) { v[2 * k] = __uint_as_float(w[k] << 16); v[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u); }
+    }
+}
+
+// Patch means in the fixed order, one thread per patch, and their max|.|.  R > 0: r == R divides
+// H and W and the rows of a patch can be fetched as vectors (all of them before the first
+// addition, which keeps the loads in flight together; the additions keep their order).
+template <typename T, int R>
 __global__ void __launch_bounds__(kQThreads) q_gbar_kernel(const T* __restrict__ gy, float* __restrict__ gbar, long long patches,
                                                            int H, int W, int r, int Hp, int Wp, FastDiv div_Wp, uint32_t* amax) {
     float worst = 0.f;
@@ -41,8 +68,23 @@ __global__ void __launch_bounds__(kQThreads) q_gbar_kernel(const T* __restrict__
         const long long pl = q / ((long long)Hp * Wp);
         uint32_t a, b;
         div_Wp.divmod((uint32_t)(q - pl * (long long)Hp * Wp), a, b);
-        const int i1 = min((int)(a + 1) * r, H), j1 = min((int)(b + 1) * r, W);
         const T* src = gy + pl * (long long)H * W;
+        if constexpr (R > 0) {
+            float v[R][R];
+            const T* p0 = src + (long long)a * R * W + (long long)b * R;
+#pragma unroll
+            for (int i = 0; i < R; ++i) load_row<R>(p0 + (long long)i * W, v[i]);
+            float sum = 0.f;
+#pragma unroll
+            for (int i = 0; i < R; ++i)
+#pragma unroll
+                for (int j = 0; j < R; ++j) sum = __fadd_rn(sum, v[i][j]);
+            const float mean = __fmul_rn(sum, __fdiv_rn(1.0f, (float)(R * R)));
+            gbar[q] = mean;
+            worst = fmaxf(worst, fabsf(mean));
+            continue;
+        }
+        const int i1 = min((int)(a + 1) * r, H), j1 = min((int)(b + 1) * r, W);
         float sum = 0.f;
         for (int i = (int)a * r; i < i1; ++i)
             for (int j = (int)b * r; j < j1; ++j) sum = __fadd_rn(sum, to_f32(src[(long long)i * W + j]));
@@ -89,6 +131,38 @@ __global__ void __launch_bounds__(kQThreads) quant_planes_kernel(const T* __rest
     }
 }
 
+// The patch means [n][C][P] fp32 -> codes in both layouts, a tile of 64 channels x 64 patches of
+// one image per block through shared memory, so that every global access is a run of 64 bytes or
+// more: K-major rows q_k[c][n P + p ..] and patch-major rows q_t[n P + p][c ..].
+__global__ void __launch_bounds__(kQThreads) quant_gbar_tiled_kernel(const float* __restrict__ src, int C, int P, int p_tiles,
+                                                                     const uint32_t* __restrict__ amax, int8_t* __restrict__ q_k,
+                                                                     long long kp, int8_t* __restrict__ q_t, long long cp) {
+    __shared__ int8_t tile[64][64 + 4];
+    const float scale = scale_of(*amax);
+    const int pt = blockIdx.x % p_tiles, n = blockIdx.x / p_tiles;
+    const int c0 = blockIdx.y * 64, p0 = pt * 64;
+    const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;              // 4 rows of 64 at a time
+    float v[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {                                       // all loads in flight before the first use
+        const int c = c0 + ty + 4 * k, pp = p0 + tx;
+        v[k] = (c < C && pp < P) ? __ldcs(src + ((size_t)n * C + c) * P + pp) : 0.f;
+    }
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+        const int cc = ty + 4 * k, c = c0 + cc, pp = p0 + tx;
+        const int8_t code = (c < C && pp < P) ? code_of(v[k], scale) : (int8_t)0;
+        tile[cc][tx] = code;
+        if (c < C && pp < P) q_k[(long long)c * kp + (long long)n * P + pp] = code;
+    }
+    if (!q_t) return;
+    __syncthreads();
+    for (int pl = ty; pl < 64; pl += 4) {
+        const int pp = p0 + pl, c = c0 + tx;
+        if (pp < P && c < C) q_t[((long long)n * P + pp) * cp + c] = tile[tx][pl];
+    }
+}
+
 // kernel sums [C_out][C_in] fp32 -> codes transposed [C_in][C_out] (pitch cp)
 __global__ void __launch_bounds__(kQThreads) quant_theta_kernel(const float* __restrict__ tsum, int C_out, int C_in,
                                                                 const uint32_t* __restrict__ amax, int8_t* __restrict__ q_t,
@@ -109,8 +183,12 @@ __global__ void __launch_bounds__(kQThreads) quant_theta_kernel(const float* __r
 //                   with integer reductions (slices of K add up exactly in any order).
 //   EPI == 1 (g_X): rows = flattened (image, patch), columns = c_i; every value is scaled and
 //                   written to the r x r pixels of its patch.
-constexpr int kI8Stages = 6;
-constexpr int kI8Threads = 192;          // warps 0-3: epilogue (one thread per accumulator row), 4: copies, 5: MMA
+constexpr int kI8StagesMax = 6;
+// g_W: long K, a deep ring; g_X: K = C_out is a few chunks, two stages, so that three CTAs share an SM
+// and their stores overlap
+__host__ __device__ constexpr int i8_stages(int epi) { return epi == 0 ? 6 : 2; }
+constexpr int kI8EpiWarps = 8;           // warps 0-7: epilogue (lane quarter warp & 3, column half warp >> 2)
+constexpr int kI8Threads = (kI8EpiWarps + 2) * 32;   // + copies, MMA
 constexpr int kI8Stage = 2 * 128 * 128;  // bytes: A tile + B tile
 
 struct I8Params {
@@ -127,13 +205,29 @@ struct I8Params {
 };
 
 struct I8Shared {
-    uint64_t full[kI8Stages], empty[kI8Stages];
+    uint64_t full[kI8StagesMax], empty[kI8StagesMax];
     uint64_t accum;
     uint32_t tmem_base;
 };
 
+// R copies of v at dst (aligned to R elements)
+template <int R> __device__ __forceinline__ void i8_store_rep(float* dst, float v) {
+    if constexpr (R == 2) __stcs(reinterpret_cast<float2*>(dst), make_float2(v, v));
+    else if constexpr (R == 4) __stcs(reinterpret_cast<float4*>(dst), make_float4(v, v, v, v));
+    else { __stcs(reinterpret_cast<float4*>(dst), make_float4(v, v, v, v)); __stcs(reinterpret_cast<float4*>(dst) + 1, make_float4(v, v, v, v)); }
+}
+template <int R> __device__ __forceinline__ void i8_store_rep(__nv_bfloat16* dst, float v) {
+    const __nv_bfloat162 b2 = __float2bfloat162_rn(v);
+    const uint32_t w = *reinterpret_cast<const uint32_t*>(&b2);
+    if constexpr (R == 2) __stcs(reinterpret_cast<unsigned int*>(dst), w);
+    else if constexpr (R == 4) __stcs(reinterpret_cast<uint2*>(dst), make_uint2(w, w));
+    else __stcs(reinterpret_cast<uint4*>(dst), make_uint4(w, w, w, w));
+}
+
 template <int EPI, typename TOut>
 __global__ void __launch_bounds__(kI8Threads) i8_gemm_kernel(const __grid_constant__ I8Params p) {
+    constexpr int kI8Stages = i8_stages(EPI);
+    constexpr int kCopyWarp = kI8EpiWarps, kMmaWarp = kI8EpiWarps + 1;
     extern __shared__ unsigned char dyn_raw[];
     __shared__ I8Shared sh;
     unsigned char* dyn = align1024(dyn_raw);
@@ -147,14 +241,14 @@ __global__ void __launch_bounds__(kI8Threads) i8_gemm_kernel(const __grid_consta
         mbar_init(&sh.accum, 1);
         mbar_fence_init();
     }
-    if (warp == 5) { tmem_alloc(&sh.tmem_base, 128); tmem_relinquish(); }
+    if (warp == kMmaWarp) { tmem_alloc(&sh.tmem_base, 128); tmem_relinquish(); }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = sh.tmem_base;
     bool ok = true;
 
-    if (warp == 4) {
+    if (warp == kCopyWarp) {
         if (lane == 0) {
             for (int q = 0; q < n_chunks && ok; ++q) {
                 const int s = q % kI8Stages;
@@ -166,7 +260,7 @@ __global__ void __launch_bounds__(kI8Threads) i8_gemm_kernel(const __grid_consta
                 tma_load_2d(stage + 128 * 128, &p.tm_b, (kc_begin + q) * 128, n0, &sh.full[s]);
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == kMmaWarp) {
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_s8(128, 128);
             for (int q = 0; q < n_chunks && ok; ++q) {
@@ -187,12 +281,13 @@ __global__ void __launch_bounds__(kI8Threads) i8_gemm_kernel(const __grid_consta
         if (n_chunks > 0) ok = mbar_wait_bounded(&sh.accum, 0);
         tc_fence_after_sync();
         if (ok && n_chunks > 0) {
-            const int m = m0 + warp * 32 + lane;               // accumulator row of this thread
+            const int quarter = warp & 3, c_lo = (warp >> 2) * 64;
+            const int m = m0 + quarter * 32 + lane;            // accumulator row of this thread
             if constexpr (EPI == 0) {
 #pragma unroll 1
-                for (int c = 0; c < 128; c += 32) {
+                for (int c = c_lo; c < c_lo + 64; c += 32) {
                     uint32_t v[32];
-                    tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c, v);
+                    tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c, v);
                     tmem_ld_wait();
                     if (m < p.M) {
                         int32_t* out = p.acc_w + (size_t)m * p.N + n0 + c;
@@ -210,17 +305,30 @@ __global__ void __launch_bounds__(kI8Threads) i8_gemm_kernel(const __grid_consta
                 TOut* gx = static_cast<TOut*>(p.gX);
                 const size_t plane = (size_t)p.H * p.W;
                 TOut* base = gx + (size_t)n * p.C_in * plane + (size_t)a * p.r * p.W + (size_t)b * p.r;
+                // whole patches of 2, 4 or 8 pixels per side on maps they divide: vector stores
+                const bool vec = rows == p.r && cols == p.r && p.W % p.r == 0 && (plane * sizeof(TOut)) % 16 == 0 &&
+                                 (p.r == 2 || p.r == 4 || p.r == 8);
 #pragma unroll 1
-                for (int c = 0; c < 128; c += 32) {
+                for (int c = c_lo; c < c_lo + 64; c += 32) {
                     uint32_t v[32];
-                    tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c, v);
+                    tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c, v);
                     tmem_ld_wait();
                     if (m < p.M) {
-                        for (int i = 0; i < 32 && n0 + c + i < p.N; ++i) {
-                            const TOut o = from_f32<TOut>(__fmul_rn((float)(int32_t)v[i], scale));
+#pragma unroll 4
+                        for (int i = 0; i < 32; ++i) {
+                            if (n0 + c + i >= p.N) break;
+                            const float val = __fmul_rn((float)(int32_t)v[i], scale);
                             TOut* dst = base + (size_t)(n0 + c + i) * plane;
-                            for (int dr = 0; dr < rows; ++dr)
-                                for (int dc = 0; dc < cols; ++dc) dst[(size_t)dr * p.W + dc] = o;
+                            if (vec) {
+                                const float o = to_f32(from_f32<TOut>(val));
+                                if (p.r == 2) { i8_store_rep<2>(dst, o); i8_store_rep<2>(dst + p.W, o); }
+                                else if (p.r == 4) { for (int dr = 0; dr < 4; ++dr) i8_store_rep<4>(dst + (size_t)dr * p.W, o); }
+                                else { for (int dr = 0; dr < 8; ++dr) i8_store_rep<8>(dst + (size_t)dr * p.W, o); }
+                            } else {
+                                const TOut o = from_f32<TOut>(val);
+                                for (int dr = 0; dr < rows; ++dr)
+                                    for (int dc = 0; dc < cols; ++dc) dst[(size_t)dr * p.W + dc] = o;
+                            }
                         }
                     }
                 }
@@ -235,7 +343,7 @@ __global__ void __launch_bounds__(kI8Threads) i8_gemm_kernel(const __grid_consta
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    if (warp == 5) tmem_dealloc(tmem, 128);
+    if (warp == kMmaWarp) tmem_dealloc(tmem, 128);
 }
 
 // g_W[co][ci][tap] = (float)acc * (scale_G * scale_X) for every tap
@@ -299,7 +407,7 @@ unsigned q_grid(long long items) {
 
 template <int EPI, typename TOut>
 gf_status launch_i8_gemm(const I8Params& p, dim3 grid, cudaStream_t s) {
-    constexpr size_t smem = (size_t)kI8Stages * kI8Stage + 1024;
+    constexpr size_t smem = (size_t)i8_stages(EPI) * kI8Stage + 1024;
     static size_t configured[kMaxDevices] = {};
     if (gf_status st = ensure_dyn_smem(i8_gemm_kernel<EPI, TOut>, smem, configured); st != GF_OK) return st;
     i8_gemm_kernel<EPI, TOut><<<grid, kI8Threads, smem, s>>>(p);
@@ -353,16 +461,28 @@ gf_status gf_backward_int8(const gf_conv_desc* desc, const void* g_y, const void
     // the gradient filter in the fixed order, and max|G-|
     const long long patches = w.K * g.C_out;
     const FastDiv div_Wp((uint32_t)g.Wp), div_P((uint32_t)w.P);
-    if (g.dtype == GF_F32)
-        q_gbar_kernel<float><<<q_grid(patches), kQThreads, 0, s>>>((const float*)g_y, gbar, patches, g.H, g.W, g.r, g.Hp, g.Wp,
-                                                                   div_Wp, amax_g);
-    else
-        q_gbar_kernel<__nv_bfloat16><<<q_grid(patches), kQThreads, 0, s>>>((const __nv_bfloat16*)g_y, gbar, patches, g.H, g.W, g.r,
-                                                                           g.Hp, g.Wp, div_Wp, amax_g);
-    if ((st = after_launch()) != GF_OK) return st;
-    quant_planes_kernel<float><<<q_grid(patches), kQThreads, 0, s>>>(gbar, patches, g.C_out, w.P, div_P, FastDiv((uint32_t)g.C_out),
-                                                                    amax_g, qg_k, w.kp, g_X ? qg_t : nullptr, w.cp);
-    if ((st = after_launch()) != GF_OK) return st;
+    {
+        ProfScope prof(K_GY_POOL, s);
+        // vector rows need r | H, r | W and rows that start on a multiple of their size
+        const bool vec = (g.r == 2 || g.r == 4 || g.r == 8) && g.H % g.r == 0 && g.W % g.r == 0 &&
+                         ((long long)g.H * g.W * (long long)g.esize) % 16 == 0;
+        const int R = vec ? g.r : 0;
+        const unsigned grid = q_grid(patches);
+#define GF_QG(TT, RR) q_gbar_kernel<TT, RR><<<grid, kQThreads, 0, s>>>((const TT*)g_y, gbar, patches, g.H, g.W, g.r, g.Hp, g.Wp, div_Wp, amax_g)
+        if (g.dtype == GF_F32) { if (R == 2) GF_QG(float, 2); else if (R == 4) GF_QG(float, 4); else if (R == 8) GF_QG(float, 8); else GF_QG(float, 0); }
+        else { if (R == 2) GF_QG(__nv_bfloat16, 2); else if (R == 4) GF_QG(__nv_bfloat16, 4); else if (R == 8) GF_QG(__nv_bfloat16, 8); else GF_QG(__nv_bfloat16, 0); }
+#undef GF_QG
+        st = after_launch();
+    }
+    if (st != GF_OK) return st;
+    {
+        ProfScope prof(K_SPLIT, s);
+        const int p_tiles = (w.P + 63) / 64;
+        const dim3 grid((unsigned)(g.N * p_tiles), (unsigned)((g.C_out + 63) / 64), 1);
+        if (grid.y > 65535) return GF_ERR_UNSUPPORTED;
+        quant_gbar_tiled_kernel<<<grid, kQThreads, 0, s>>>(gbar, g.C_out, w.P, p_tiles, amax_g, qg_k, w.kp, g_X ? qg_t : nullptr, w.cp);
+        if ((st = after_launch()) != GF_OK) return st;
+    }
 
     I8Params p;
     p.err_word = err; p.C_in = g.C_in; p.H = g.H; p.W = g.W; p.r = g.r; p.Hp = g.Hp; p.Wp = g.Wp; p.P = w.P;
@@ -382,7 +502,10 @@ gf_status gf_backward_int8(const gf_conv_desc* desc, const void* g_y, const void
         p.M = (int)w.K; p.N = g.C_in; p.k_chunks = (int)(w.cp / 128); p.S = 1;
         const dim3 grid((unsigned)(w.cip / 128), (unsigned)(w.mp / 128), 1);
         if (grid.y > 65535) return GF_ERR_UNSUPPORTED;
-        st = g.dtype == GF_F32 ? launch_i8_gemm<1, float>(p, grid, s) : launch_i8_gemm<1, __nv_bfloat16>(p, grid, s);
+        {
+            ProfScope prof(K_GX_TC, s);
+            st = g.dtype == GF_F32 ? launch_i8_gemm<1, float>(p, grid, s) : launch_i8_gemm<1, __nv_bfloat16>(p, grid, s);
+        }
         if (st != GF_OK) return st;
     }
     if (g_W) {
@@ -411,7 +534,11 @@ gf_status gf_backward_int8(const gf_conv_desc* desc, const void* g_y, const void
         p.S = S;
         const dim3 grid((unsigned)(w.cip / 128), (unsigned)(w.cop / 128), (unsigned)S);
         if (grid.y > 65535) return GF_ERR_UNSUPPORTED;
-        if ((st = launch_i8_gemm<0, float>(p, grid, s)) != GF_OK) return st;
+        {
+            ProfScope prof(K_GW_TC, s);
+            st = launch_i8_gemm<0, float>(p, grid, s);
+        }
+        if (st != GF_OK) return st;
         const long long total = (long long)g.C_out * g.C_in * g.KH * g.KW;
         i8_gw_finish_kernel<<<q_grid(total), kQThreads, 0, s>>>(acc, total, g.KH * g.KW, amax_g, amax_x, g_W);
         if ((st = after_launch()) != GF_OK) return st;
