@@ -162,16 +162,53 @@ static Workspace plan_split(const Geo& g) {
     return w;
 }
 
-// Strided layers: error word | phase kernel sums fp32 [C_out, s*s*C_ig] | G- fp32 [N, C_out, P] |
-// reduced g_X on the patch grid fp32 [N, s*s*C_in, P] | g_W slices fp32 [S, C_out, C_ig]
-struct StridedPlan { size_t off_tph, off_gbar, off_ghat, off_part, total; int splits; Geo gy; };
+// Strided layers.  Three ways, by layer kind: depthwise in one kernel per plane; dense layers with
+// C_out a multiple of 8 on the tensor-core contractions (the phases as s*s*C_in "virtual" input
+// channels on the patch grid, dealt out to the pixels afterwards); everything else on the
+// CUDA-core contractions.
+//   generic:  error word | phase kernel sums fp32 [C_out, s*s*C_ig] | G- fp32 [N, C_out, P] |
+//             reduced g_X on the patch grid fp32 [N, s*s*C_in, P] | g_W slices fp32 [S, C_out, C_ig]
+//   tensor:   error word | phase kernel sums bf16 [s*s*C_in, C_out] (+ low parts) | G- bf16 (+ low) in the operand pitch |
+//             reduced g_X on the patch grid in the layer's dtype | g_W unique values | stash as bf16 operand rows
+//   depthwise: error word | per-image shares of g_W fp32 [N, C]
+struct StridedPlan {
+    int kind;                      // 0 generic, 1 tensor cores, 2 depthwise
+    size_t off_tph, off_gbar, off_ghat, off_part, off_split, total;
+    int splits;
+    Geo gy;                        // the geometry of g_y: what the pooling and the g_W contraction see
+};
 static StridedPlan plan_strided(const Geo& g, int stride) {
     StridedPlan w;
-    w.gy = g;                                   // the geometry of g_y: what the pooling and the g_W contraction see
+    w.gy = g;
     w.gy.H = g.H / stride; w.gy.W = g.W / stride;
     w.gy.Hp = (w.gy.H + g.r - 1) / g.r; w.gy.Wp = (w.gy.W + g.r - 1) / g.r;
     const size_t P = (size_t)w.gy.Hp * w.gy.Wp, s2 = (size_t)stride * stride;
     size_t off = 256;
+    w.off_tph = w.off_gbar = w.off_ghat = w.off_part = w.off_split = off;
+    if (dw_strided_ok(w.gy, stride)) {
+        w.kind = 2;
+        w.splits = g.N;
+        w.off_part = off; off += align_up((size_t)g.N * g.C_in * 4, 256);
+        w.total = off;
+        return w;
+    }
+    Geo gv = w.gy;                  // g_X as a layer on the patch grid with s*s*C_in channels
+    gv.C_in = (int)s2 * g.C_in; gv.C_ig = (int)s2 * g.C_ig; gv.H = w.gy.Hp; gv.W = w.gy.Wp; gv.r = 1;
+    if (g.G == 1 && g.C_out % 8 == 0 && tc_check_limits(gv) == GF_OK && tc_check_limits(w.gy) == GF_OK &&
+        tc_pitch(gv) == tc_pitch(w.gy) &&
+        (long long)g.N * ((long long)P + 7) / 8 * 8 < (1LL << 31)) {
+        w.kind = 1;
+        w.splits = 1;
+        const size_t pitch = (size_t)tc_pitch(w.gy);
+        w.off_tph = off; off += align_up(s2 * g.C_in * g.C_out * 4, 256);
+        w.off_gbar = off; off += align_up((size_t)g.N * g.C_out * pitch * 4, 256);
+        w.off_ghat = off; off += align_up((size_t)g.N * s2 * g.C_in * P * g.esize, 256);
+        w.off_part = off; off += align_up((size_t)g.C_out * g.C_in * 4, 256);
+        w.off_split = off; off += 2 * align_up((size_t)g.N * g.C_in * pitch * 2, 256);
+        w.total = off;
+        return w;
+    }
+    w.kind = 0;
     w.off_tph = off; off += align_up((size_t)g.C_out * s2 * g.C_ig * 4, 256);
     w.off_gbar = off; off += align_up((size_t)g.N * g.C_out * P * 4, 256);
     w.off_ghat = off; off += align_up((size_t)g.N * s2 * g.C_in * P * 4, 256);
@@ -369,24 +406,73 @@ gf_status backward_impl(const gf_conv_desc* desc, const void* g_y, const void* s
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     char* base = static_cast<char*>(workspace);
     if (desc->stride > 1 && g.r > 1) {
-        // strided layer: kernel sums per pixel phase, gradient filter on g_y's own grid, the two
-        // reduced contractions on CUDA cores (g_X against all phases at once, then dealt out to
-        // the pixels of each window; g_W scaled by 1 / stride^2)
+        // strided layer: kernel sums per pixel phase, gradient filter on g_y's own grid, g_X against
+        // all phases at once and then dealt out to the pixels of each window, g_W scaled by
+        // 1 / stride^2 (plan_strided picks the kernels by layer kind)
         const int stride = desc->stride, s2 = stride * stride;
         const StridedPlan sp = plan_strided(g, stride);
         if (workspace_bytes < sp.total) return GF_ERR_WORKSPACE;
         if (!g_W && !g_X) return GF_OK;
+        uint32_t* err = reinterpret_cast<uint32_t*>(base);
+        float* part = reinterpret_cast<float*>(base + sp.off_part);
+        const float gw_scale = 1.0f / (float)s2;
+        if (sp.kind == 2) {
+            GF_CUDA_TRY(cudaMemsetAsync(err, 0, sizeof(uint32_t), s));
+            st = launch_dw_strided(g_y, stash, W, g_W ? part : nullptr, g_X, g, stride, sp.gy.Hp, sp.gy.Wp, s);
+            if (st != GF_OK) return st;
+            return g_W ? launch_gw_finish(part, sp.splits, g_W, sp.gy, s, gw_scale) : GF_OK;
+        }
         Geo gv = sp.gy;                         // g_X as a layer on the patch grid with s*s*C_in channels, not expanded
-        gv.C_in = s2 * g.C_in; gv.C_ig = s2 * g.C_ig; gv.H = sp.gy.Hp; gv.W = sp.gy.Wp; gv.r = 1; gv.dtype = GF_F32; gv.esize = 4;
+        gv.C_in = s2 * g.C_in; gv.C_ig = s2 * g.C_ig; gv.H = sp.gy.Hp; gv.W = sp.gy.Wp; gv.r = 1;
+        if (sp.kind == 1) {
+            const bool split = g.dtype == GF_F32;
+            const size_t P = (size_t)sp.gy.Hp * sp.gy.Wp, pitch = (size_t)tc_pitch(sp.gy);
+            const long long theta_lo = split ? (long long)align_up((size_t)s2 * g.C_in * g.C_out, 8) : 0;
+            const long long gbar_lo = split ? (long long)align_up((size_t)g.N * g.C_out * pitch, 8) : 0;
+            const long long stash_lo = split ? (long long)(align_up((size_t)g.N * g.C_in * pitch * 2, 256) / 2) : 0;
+            __nv_bfloat16* thetaT = reinterpret_cast<__nv_bfloat16*>(base + sp.off_tph);
+            __nv_bfloat16* gbar16 = reinterpret_cast<__nv_bfloat16*>(base + sp.off_gbar);
+            void* ghat = base + sp.off_ghat;
+            GF_CUDA_TRY(cudaMemsetAsync(err, 0, sizeof(uint32_t), s));
+            st = launch_pool(K_GY_POOL, g_y, g.dtype, gbar16, split ? gbar16 + gbar_lo : nullptr, GF_BF16, /*mean=*/true,
+                             (int64_t)g.N * g.C_out, sp.gy.H, sp.gy.W, g.r, (int)pitch, err, s);
+            if (st != GF_OK) return st;
+            st = launch_ksum_phase_t(W, g.dtype, g.C_out, g.C_in, g.KH, g.KW, stride, thetaT, split ? thetaT + theta_lo : nullptr,
+                                     g_W ? part : nullptr, s);
+            if (st != GF_OK) return st;
+            if (g_X) {
+                st = launch_gx_tc(gbar16, gbar_lo, thetaT, theta_lo, ghat, 0, err, gv, s);
+                if (st != GF_OK) return st;
+                st = launch_expand_phase(ghat, /*ghat_f32=*/g.dtype == GF_F32, g_X, g.dtype, g.N, g.C_in, g.G, g.H, g.W, stride, g.r, s);
+                if (st != GF_OK) return st;
+            }
+            if (g_W) {
+                const __nv_bfloat16* stash16 = static_cast<const __nv_bfloat16*>(stash);
+                if (split || pitch != P) {
+                    __nv_bfloat16* spl = reinterpret_cast<__nv_bfloat16*>(base + sp.off_split);
+                    if (pitch == P)
+                        st = launch_split_f32(static_cast<const float*>(stash), spl, spl + stash_lo, (size_t)g.N * g.C_in * P, s);
+                    else
+                        st = launch_repack(stash, g.dtype, spl, split ? spl + stash_lo : nullptr, (long long)g.N * g.C_in, (int)P,
+                                           (int)pitch, s);
+                    if (st != GF_OK) return st;
+                    stash16 = spl;
+                }
+                st = launch_gw_tc(gbar16, gbar_lo, stash16, stash_lo, part, tc_gw_splits(sp.gy), err, sp.gy, s);
+                if (st != GF_OK) return st;
+                st = launch_gw_finish(part, 1, g_W, sp.gy, s, gw_scale);
+                if (st != GF_OK) return st;
+            }
+            return GF_OK;
+        }
+        gv.dtype = GF_F32; gv.esize = 4;
         st = dense_check_limits(sp.gy, sp.splits);
         if (st == GF_OK) st = dense_check_limits(gv, 1);
         if (st != GF_OK) return st;
-        uint32_t* err = reinterpret_cast<uint32_t*>(base);
         GF_CUDA_TRY(cudaMemsetAsync(err, 0, sizeof(uint32_t), s));
         float* tph = reinterpret_cast<float*>(base + sp.off_tph);
         float* gbar = reinterpret_cast<float*>(base + sp.off_gbar);
         float* ghat = reinterpret_cast<float*>(base + sp.off_ghat);
-        float* part = reinterpret_cast<float*>(base + sp.off_part);
         st = launch_pool(K_GY_POOL, g_y, g.dtype, gbar, nullptr, GF_F32, /*mean=*/true, (int64_t)g.N * g.C_out, sp.gy.H, sp.gy.W, g.r,
                          0, err, s);
         if (st != GF_OK) return st;
@@ -395,13 +481,13 @@ gf_status backward_impl(const gf_conv_desc* desc, const void* g_y, const void* s
             if (st != GF_OK) return st;
             st = launch_gx_mix(gbar, tph, ghat, gv, s);
             if (st != GF_OK) return st;
-            st = launch_expand_phase(ghat, g_X, g.dtype, g.N, g.C_in, g.G, g.H, g.W, stride, g.r, s);
+            st = launch_expand_phase(ghat, /*ghat_f32=*/true, g_X, g.dtype, g.N, g.C_in, g.G, g.H, g.W, stride, g.r, s);
             if (st != GF_OK) return st;
         }
         if (g_W) {
             st = launch_gw_partial(gbar, stash, part, sp.splits, sp.gy, s);
             if (st != GF_OK) return st;
-            st = launch_gw_finish(part, sp.splits, g_W, sp.gy, s, 1.0f / (float)s2);
+            st = launch_gw_finish(part, sp.splits, g_W, sp.gy, s, gw_scale);
             if (st != GF_OK) return st;
         }
         return GF_OK;

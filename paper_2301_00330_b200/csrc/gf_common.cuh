@@ -241,7 +241,15 @@ gf_status launch_exact(const void* gy, const void* x, const void* W, float* gW, 
 // strided layers (gf_strided.cu): per-phase kernel sums, rows of s*s*C_ig values per output channel
 gf_status launch_ksum_phase(const void* W, int dtype, int C_out, int C_ig, int KH, int KW, int stride, float* tph, cudaStream_t s);
 // gX[n, c, h, w] <- ghat[n, (group, phase of (h, w), channel in group), h / (r s), w / (r s)]
-gf_status launch_expand_phase(const float* ghat, void* gX, int dtype, int N, int C_in, int G, int H, int W, int stride, int r,
-                              cudaStream_t s);
+// (ghat: fp32, or the layer's dtype when it comes from the tensor-core contraction)
+gf_status launch_expand_phase(const void* ghat, bool ghat_f32, void* gX, int dtype, int N, int C_in, int G, int H, int W, int stride,
+                              int r, cudaStream_t s);
+// the same sums transposed as bf16 (high, low) rows [(phase, c_i)][c_o] for the tensor-core contraction; clears gwu
+gf_status launch_ksum_phase_t(const void* W, int dtype, int C_out, int C_in, int KH, int KW, int stride, __nv_bfloat16* thetaT,
+                              __nv_bfloat16* thetaT_lo, float* gwu, cudaStream_t s);
+// depthwise strided layers in one kernel per (image, channel) plane; part: [N][C] per-image shares of g_W
+bool dw_strided_ok(const Geo& gy_geo, int stride);
+gf_status launch_dw_strided(const void* gy, const void* stash, const void* W, float* part, void* gX, const Geo& g, int stride, int Hp,
+                            int Wp, cudaStream_t s);
 
 }  // namespace gf
