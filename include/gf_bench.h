@@ -35,6 +35,17 @@ typedef struct gf_kernel_time {
  * written, or -1 if a CUDA call failed. */
 int32_t gf_profile_read(gf_kernel_time* out, int32_t max_entries);
 
+/* Self-test of the bounded device-side waits (no counterpart in the paper).  Every wait a
+ * kernel of this library makes on an mbarrier gives up after a limit of clocks, sets a bit of
+ * the workspace's error word and lets the kernel return, so that a copy that never lands is
+ * reported (GF_ERR_TIMEOUT from gf_last_async_status) instead of hanging the GPU.  This call
+ * launches one small block that waits, with that same wait and a limit of `limit_cycles`
+ * clocks (1 .. 2e9; about 0.5 ns each), on a barrier that nothing ever arrives on: the wait
+ * runs out, the block records it in the error word at the head of `workspace` (device
+ * memory, >= 256 bytes, 16-byte aligned) and ends normally.  The next gf_backward on that
+ * workspace clears the word again. */
+gf_status gf_selftest_bounded_wait(void* workspace, int64_t limit_cycles, void* stream);
+
 /* Name of a kernel id (ids are 0 .. gf_kernel_id_count()-1), NULL if out of range. */
 const char* gf_kernel_name(int32_t kernel_id);
 int32_t gf_kernel_id_count(void);

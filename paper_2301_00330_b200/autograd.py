@@ -5,8 +5,9 @@ activation stash is taken by gf_stash_forward instead of keeping x (Section 3.4)
 gf_backward gives g_W and g_X from the incoming g_y, the stash and W.  Only marshalling
 happens here; every step of the path runs in the CUDA library.
 
-Geometry: what the library accepts (stride 1, "same" padding, odd kernels, NCHW, fp32 or
-bf16 on a CUDA device); anything else raises GfError from the library call.
+Geometry: what the library accepts (stride 1 or a stride dividing H and W, padding (k-1)/2,
+odd kernels, NCHW, fp32 or bf16 on a CUDA device); anything else raises GfError from the
+library call.
 """
 from __future__ import annotations
 
@@ -17,19 +18,19 @@ from . import binding as B
 
 class _FilteredConv2dFn(torch.autograd.Function):
     @staticmethod
-    def forward(ctx, x, weight, r: int, groups: int):
+    def forward(ctx, x, weight, r: int, groups: int, stride: int = 1):
         if not (x.is_cuda and weight.is_cuda):
             raise RuntimeError("filtered_conv2d needs CUDA tensors: there is no CPU path")
         x = x.contiguous()
         weight = weight.contiguous()
         C_out, _, KH, KW = weight.shape
         N, C_in, H, W = x.shape
-        desc = B.make_desc(N, C_in, C_out, H, W, KH, KW, r=r, groups=groups, dtype=x.dtype)
+        desc = B.make_desc(N, C_in, C_out, H, W, KH, KW, r=r, groups=groups, stride=stride, dtype=x.dtype)
         stash = torch.empty(B.gf_stash_dims(desc), dtype=x.dtype, device=x.device)
         stream = torch.cuda.current_stream(x.device)
         with torch.cuda.device(x.device):
             B.gf_stash_forward(desc, x, stash, stream)
-        y = torch.nn.functional.conv2d(x, weight, None, 1, ((KH - 1) // 2, (KW - 1) // 2), 1, groups)
+        y = torch.nn.functional.conv2d(x, weight, None, stride, ((KH - 1) // 2, (KW - 1) // 2), 1, groups)
         ctx.desc = desc
         ctx.need_gx = x.requires_grad
         ctx.need_gw = weight.requires_grad
@@ -50,28 +51,28 @@ class _FilteredConv2dFn(torch.autograd.Function):
             B.gf_backward(desc, g_y, stash, weight, g_W, g_X, ws, None, stream)
         if g_W is not None and g_W.dtype != weight.dtype:
             g_W = g_W.to(weight.dtype)
-        return g_X, g_W, None, None
+        return g_X, g_W, None, None, None
 
 
-def filtered_conv2d(x: torch.Tensor, weight: torch.Tensor, r: int = 2, groups: int = 1) -> torch.Tensor:
-    """conv2d(x, weight) with stride 1 and "same" padding whose gradients are the filtered
-    ones with patch size r (r = 1: the exact gradients).  The bias, if any, is added by the
-    caller (its gradient is not affected by the method)."""
-    return _FilteredConv2dFn.apply(x, weight, int(r), int(groups))
+def filtered_conv2d(x: torch.Tensor, weight: torch.Tensor, r: int = 2, groups: int = 1, stride: int = 1) -> torch.Tensor:
+    """conv2d(x, weight) with padding (k-1)/2 and the given stride whose gradients are the
+    filtered ones with patch size r (r = 1: the exact gradients).  The bias, if any, is added
+    by the caller (its gradient is not affected by the method)."""
+    return _FilteredConv2dFn.apply(x, weight, int(r), int(groups), int(stride))
 
 
 class FilteredConv2d(torch.nn.Module):
-    """Drop-in for nn.Conv2d(..., stride=1, padding=k//2) in the layers that are fine-tuned."""
+    """Drop-in for nn.Conv2d(..., padding=k//2) in the layers that are fine-tuned."""
 
     def __init__(self, in_channels: int, out_channels: int, kernel_size: int, r: int = 2, groups: int = 1,
-                 bias: bool = True, device=None, dtype=None):
+                 bias: bool = True, device=None, dtype=None, stride: int = 1):
         super().__init__()
-        self.r, self.groups = r, groups
+        self.r, self.groups, self.stride = r, groups, stride
         self.weight = torch.nn.Parameter(torch.empty(out_channels, in_channels // groups, kernel_size, kernel_size,
                                                      device=device, dtype=dtype))
         torch.nn.init.kaiming_normal_(self.weight)
         self.bias = torch.nn.Parameter(torch.zeros(out_channels, device=device, dtype=dtype)) if bias else None
 
     def forward(self, x):
-        y = filtered_conv2d(x, self.weight, self.r, self.groups)
+        y = filtered_conv2d(x, self.weight, self.r, self.groups, self.stride)
         return y if self.bias is None else y + self.bias.view(1, -1, 1, 1)

@@ -28,7 +28,7 @@ EXPORTS = (
     "gf_kernel_launch_count", "gf_status_string", "gf_profile_configure", "gf_profile_read",
     "gf_kernel_name", "gf_kernel_id_count", "gf_backward_static_scratch", "gf_set_dense_path",
     "gf_snr_terms", "gf_filter_snr_terms", "gf_dcac_ratio", "gf_act_stash_forward",
-    "gf_backward_int8", "gf_backward_int8_workspace_bytes",
+    "gf_backward_int8", "gf_backward_int8_workspace_bytes", "gf_selftest_bounded_wait",
 )
 
 
@@ -105,6 +105,8 @@ def lib() -> ctypes.CDLL:
         L.gf_dcac_ratio.argtypes = [vp, i32, i32, i32, i32, i32, i32, i32, vp, vp]
         for name in ("gf_snr_terms", "gf_filter_snr_terms", "gf_dcac_ratio"):
             getattr(L, name).restype = ctypes.c_int
+        L.gf_selftest_bounded_wait.argtypes = [vp, ctypes.c_int64, vp]
+        L.gf_selftest_bounded_wait.restype = ctypes.c_int
         L.gf_status_string.argtypes = [ctypes.c_int]
         L.gf_status_string.restype = ctypes.c_char_p
         for name in ("gf_stash_dims", "gf_stash_bytes", "gf_backward_workspace_bytes", "gf_stash_forward",
@@ -272,6 +274,12 @@ def gf_dcac_ratio(W: torch.Tensor, ratio: torch.Tensor, dft: tuple[int, int] = (
     assert ratio.dtype == torch.float32 and ratio.numel() == C_out * C_ig
     _check(lib().gf_dcac_ratio(_ptr(W), C_out, C_ig, KH, KW, int(dft[0]), int(dft[1]), _gf_dtype(W), _ptr(ratio),
                                _stream(stream)), "gf_dcac_ratio")
+
+
+def gf_selftest_bounded_wait(workspace, limit_cycles: int, stream=None) -> None:
+    """Launches a block whose bounded wait must expire; it records that in the workspace's error word."""
+    _check(lib().gf_selftest_bounded_wait(_ptr(workspace), ctypes.c_int64(int(limit_cycles)), _stream(stream)),
+           "gf_selftest_bounded_wait")
 
 
 def gf_kernel_launch_count() -> int:

@@ -5,6 +5,7 @@
 #include <mutex>
 
 #include "gf_common.cuh"
+#include "gf_pipe.cuh"
 
 namespace gf {
 
@@ -678,6 +679,28 @@ gf_status gf_set_dense_path(int32_t path) {
     if (path < 0 || path > 2) return GF_ERR_BAD_DESC;
     g_dense_path.store(path, std::memory_order_relaxed);
     return GF_OK;
+}
+
+}  // extern "C"
+
+namespace gf {
+// Waits on a barrier that nothing arrives on: the bounded wait has to run out and report.
+__global__ void selftest_wait_kernel(uint32_t* err_word, long long limit) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) { gf::mbar_init(&bar, 1); gf::mbar_fence_init(); }
+    __syncthreads();
+    if (threadIdx.x == 0 && !gf::mbar_wait_bounded(&bar, 0, limit)) atomicOr(err_word, 128u);
+}
+}  // namespace gf
+
+extern "C" {
+
+gf_status gf_selftest_bounded_wait(void* workspace, int64_t limit_cycles, void* stream) {
+    if (!workspace) return GF_ERR_NULL;
+    if (limit_cycles < 1 || limit_cycles > 2000000000LL) return GF_ERR_BAD_DESC;
+    if (misaligned(workspace)) return GF_ERR_ALIGN;
+    selftest_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<uint32_t*>(workspace), (long long)limit_cycles);
+    return after_launch();
 }
 
 gf_status gf_profile_configure(int32_t mode, int32_t kernel_id) {

@@ -38,3 +38,21 @@ def test_module_trains_one_step(gf):
     opt.step()
     assert torch.isfinite(m.weight).all() and not torch.equal(before, m.weight)
     assert m.bias.grad is not None
+
+
+def test_strided_layer_through_autograd(gf):
+    """A stride-2 layer: the output has half the resolution and the gradients are the strided
+    filtered ones (oracle/gf_strided.py)."""
+    g = torch.Generator(device="cpu")
+    g.manual_seed(3)
+    x = torch.randn((2, 8, 16, 16), generator=g)
+    w = torch.randn((16, 8, 3, 3), generator=g) * 0.2
+    gy = torch.randn((2, 16, 8, 8), generator=g)
+    xd, wd = x.cuda().requires_grad_(True), w.cuda().requires_grad_(True)
+    y = gf.filtered_conv2d(xd, wd, r=2, stride=2)
+    assert y.shape == (2, 16, 8, 8)
+    assert torch.allclose(y.detach().cpu(), torch.nn.functional.conv2d(x, w, None, 2, 1), rtol=1e-3, atol=1e-3)
+    y.backward(gy.cuda())
+    torch.cuda.synchronize()
+    gw_ref, gx_ref = oracle.strided_backward(f64(gy), oracle.strided_stash_forward(f64(x), 2, 2), f64(w), 2, 2)
+    assert relerr(f64(xd.grad), gx_ref) <= TOL["f32"] and relerr(f64(wd.grad), gw_ref) <= TOL["f32"]

@@ -228,6 +228,27 @@ def test_error_word_is_reported_and_cleared(gf):
     assert gf.gf_last_async_status(buf.workspace) == gf.GF_OK
 
 
+def test_a_device_wait_that_runs_out_is_reported(gf):
+    """The bounded wait itself, on the GPU: a block waits (a millisecond's worth of clocks) on a barrier
+    that nothing arrives on; the wait gives up, the block ends normally and records it, the host
+    reads GF_ERR_TIMEOUT, and the context stays usable: the next backward on the same workspace
+    clears the word, completes and matches the call made before."""
+    layer = L("wait_runs_out", 2, 24, 40, 14, 14, 3, 1, 2)
+    x, gy, w = workloads.make_inputs(layer)
+    desc = gf.desc_for(layer)
+    buf = gf.alloc_layer(desc)
+    xd, gyd, wd = x.cuda(), gy.cuda(), w.cuda()
+    gf.gf_stash_forward(desc, xd, buf.stash)
+    gf.gf_backward(desc, gyd, buf.stash, wd, buf.g_W, buf.g_X, buf.workspace)
+    assert gf.gf_last_async_status(buf.workspace) == gf.GF_OK
+    gW0, gX0 = buf.g_W.clone(), buf.g_X.clone()
+    gf.gf_selftest_bounded_wait(buf.workspace, 2_000_000)
+    assert gf.gf_last_async_status(buf.workspace) == gf.GF_ERR_TIMEOUT
+    gf.gf_backward(desc, gyd, buf.stash, wd, buf.g_W, buf.g_X, buf.workspace)
+    assert gf.gf_last_async_status(buf.workspace) == gf.GF_OK
+    assert torch.equal(buf.g_X, gX0) and relerr(f64(buf.g_W), f64(gW0)) <= 1e-6
+
+
 def test_ondevice_table_shapes_sampled(gf):
     """The seven layer shapes of the paper's on-device latency table (batch 32,
     3x3, stride 1, pad 1); 14x14 with r = 4 has partial patches."""
