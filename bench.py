@@ -474,6 +474,23 @@ def extras(gf, layers) -> dict:
         "backward_us": timed(lambda: gf.gf_backward(desc, gys, stash, wsd, gW, gX, ws, None, stream)),
         "exact_cudnn_us": timed(lambda: torch.ops.aten.convolution_backward(gys, xs, wsd, None, [2, 2], [1, 1], [1, 1], False,
                                                                             [0, 0], 1, [True, True, False]), 4)}
+    del xs, gys, wsd, stash, gW, gX, ws
+    # the step's layers with channels-last tensors (same bytes, other kernels)
+    out["nhwc_layer_us"] = {}
+    for L in layers:
+        desc = gf.make_desc(L.N, L.C_in, L.C_out, L.H, L.W, L.K, r=L.r, groups=L.groups,
+                            dtype=gf.GF_F32 if L.dtype == "f32" else gf.GF_BF16, layout=gf.GF_NHWC)
+        x0, gy0, w0 = workloads.make_inputs(L)
+        xl, gyl, wl = x0.cuda().permute(0, 2, 3, 1).contiguous(), gy0.cuda().permute(0, 2, 3, 1).contiguous(), w0.cuda()
+        n, c, hp, wp = gf.gf_stash_dims(desc)
+        stash = torch.empty((n, hp, wp, c), dtype=xl.dtype, device="cuda")
+        gW, gX = torch.empty(wl.shape, dtype=torch.float32, device="cuda"), torch.empty_like(xl)
+        ws = torch.empty(gf.gf_backward_workspace_bytes(desc), dtype=torch.uint8, device="cuda")
+        gf.gf_stash_forward(desc, xl, stash, stream)
+        t_s = timed(lambda: gf.gf_stash_forward(desc, xl, stash, stream))
+        t_b = timed(lambda: gf.gf_backward(desc, gyl, stash, wl, gW, gX, ws, None, stream))
+        out["nhwc_layer_us"][L.name] = {"stash_us": t_s, "backward_us": t_b, "layer_us": round(t_s + t_b, 1)}
+        del xl, gyl, wl, stash, gW, gX, ws
     torch.cuda.empty_cache()
     return out
 

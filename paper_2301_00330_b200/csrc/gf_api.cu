@@ -93,7 +93,6 @@ static gf_status validate(const gf_conv_desc* d) {
     if (d->C_in % d->groups != 0 || d->C_out % d->groups != 0) return GF_ERR_BAD_DESC;
     if (d->dtype != GF_F32 && d->dtype != GF_BF16) return GF_ERR_BAD_DESC;
     if (d->layout != GF_NCHW && d->layout != GF_NHWC) return GF_ERR_BAD_DESC;
-    if (d->layout != GF_NCHW) return GF_ERR_UNSUPPORTED;
     // strided layers: the output map is [H / stride, W / stride] (see gf_strided.cu)
     if (d->stride > 1 && (d->H % d->stride != 0 || d->W % d->stride != 0 || d->stride > 16)) return GF_ERR_UNSUPPORTED;
     if (d->KH % 2 == 0 || d->KW % 2 == 0) return GF_ERR_UNSUPPORTED;
@@ -103,6 +102,8 @@ static gf_status validate(const gf_conv_desc* d) {
     if ((int64_t)d->N * d->C_in > (int64_t)1 << 30 || (int64_t)d->N * d->C_out > (int64_t)1 << 30)
         return GF_ERR_UNSUPPORTED;
     if ((int64_t)d->C_out * (d->C_in / d->groups) * d->KH * d->KW > (int64_t)1 << 30) return GF_ERR_UNSUPPORTED;
+    // channels-last: stride 1, r >= 2, channel counts in multiples of 8, dense or depthwise
+    if (d->layout == GF_NHWC && (d->r < 2 || !nhwc_supported(make_geo(*d), d->stride))) return GF_ERR_UNSUPPORTED;
     return GF_OK;
 }
 
@@ -302,6 +303,7 @@ gf_status gf_backward_workspace_bytes(const gf_conv_desc* desc, size_t* bytes) {
     gf_status st = validate(desc);
     if (st != GF_OK) return st;
     const Geo g = make_geo(*desc);
+    if (desc->layout == GF_NHWC) { *bytes = nhwc_workspace_bytes(g); return GF_OK; }
     *bytes = (desc->stride > 1 && g.r > 1) ? plan_strided(g, desc->stride).total : plan_workspace(g).total;
     return GF_OK;
 }
@@ -314,6 +316,7 @@ gf_status gf_stash_forward(const gf_conv_desc* desc, const void* x, void* stash,
     const Geo g = make_geo(*desc);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int64_t planes = (int64_t)g.N * g.C_in;
+    if (desc->layout == GF_NHWC) return launch_nhwc_stash(x, stash, g, s);
     if (g.r == 1) return launch_copy(x, stash, (size_t)planes * g.H * g.W * g.esize, s);
     uint32_t* err = global_err_word();
     if (!err) return GF_ERR_CUDA;
@@ -326,6 +329,7 @@ gf_status gf_act_stash_forward(const gf_conv_desc* desc, int32_t act, const void
     if (act < GF_ACT_NONE || act > GF_ACT_RELU6) return GF_ERR_BAD_DESC;
     gf_status st = validate(desc);
     if (st != GF_OK) return st;
+    if (desc->layout != GF_NCHW) return GF_ERR_UNSUPPORTED;
     if (misaligned(z) || misaligned(x) || misaligned(stash)) return GF_ERR_ALIGN;
     const Geo g = make_geo(*desc);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -406,6 +410,11 @@ gf_status backward_impl(const gf_conv_desc* desc, const void* g_y, const void* s
     const Geo g = make_geo(*desc);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     char* base = static_cast<char*>(workspace);
+    if (desc->layout == GF_NHWC) {
+        if (workspace_bytes < nhwc_workspace_bytes(g)) return GF_ERR_WORKSPACE;
+        if (!g_W && !g_X) return GF_OK;
+        return nhwc_backward(g, g_y, stash, W, g_W, g_X, base, s);
+    }
     if (desc->stride > 1 && g.r > 1) {
         // strided layer: kernel sums per pixel phase, gradient filter on g_y's own grid, g_X against
         // all phases at once and then dealt out to the pixels of each window, g_W scaled by

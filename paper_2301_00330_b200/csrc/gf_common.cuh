@@ -236,6 +236,12 @@ gf_status launch_gyx_fused(const void* gy, const __nv_bfloat16* thetaT, long lon
                            unsigned char* gbar_t, uint32_t* err_word, const Geo& g, cudaStream_t s);
 gf_status launch_gw_tiled(const unsigned char* gbar_t, const void* stash, float* gwu, uint32_t* err_word, const Geo& g,
                           cudaStream_t s);
+// channels-last tensors (gf_nhwc.cu)
+bool nhwc_supported(const Geo& g, int stride);
+size_t nhwc_workspace_bytes(const Geo& g);
+gf_status launch_nhwc_stash(const void* x, void* stash, const Geo& g, cudaStream_t s);
+gf_status nhwc_backward(const Geo& g, const void* g_y, const void* stash, const void* W, float* g_W, void* g_X, char* base,
+                        cudaStream_t s);
 gf_status launch_exact(const void* gy, const void* x, const void* W, float* gW, void* gX,
                        const Geo& g, int stride, cudaStream_t s);
 // strided layers (gf_strided.cu): per-phase kernel sums, rows of s*s*C_ig values per output channel

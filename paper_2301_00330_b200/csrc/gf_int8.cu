@@ -389,7 +389,7 @@ gf_status check_i8(const gf_conv_desc* d) {
     size_t probe = 0;
     const gf_status st = gf_backward_workspace_bytes(d, &probe);      // the descriptor checks of the library
     if (st != GF_OK) return st;
-    if (d->groups != 1 || d->stride != 1 || d->r < 2) return GF_ERR_UNSUPPORTED;
+    if (d->groups != 1 || d->stride != 1 || d->r < 2 || d->layout != GF_NCHW) return GF_ERR_UNSUPPORTED;
     const long long P = (long long)((d->H + d->r - 1) / d->r) * ((d->W + d->r - 1) / d->r);
     const long long K = (long long)d->N * P;
     // 32-bit accumulators: K * 127^2 must stay below 2^31 for the g_W contraction, C_out * 127^2 for g_X

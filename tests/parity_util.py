@@ -90,13 +90,13 @@ def check_layer_full(gf, L: workloads.Layer, isolate: bool = True):
     return errs
 
 
-def check_layer_sampled(gf, L: workloads.Layer, n_ch: int = 6, n_img: int = 2, seed: int = 0):
+def check_layer_sampled(gf, L: workloads.Layer, n_ch: int = 6, n_img: int = 2, seed: int = 0, runner=None):
     """Full-size layer: the stash in full, g_W on sampled channel pairs and g_X on
     sampled (image, channel) planes, each computed by the checker from sliced
     inputs; plus the structural properties that hold at any size."""
     x, gy, w = workloads.make_inputs(L)
     tol = TOL[L.dtype]
-    stash, gW, gX = run_gpu(gf, L, x, gy, w)
+    stash, gW, gX = (runner or run_gpu)(gf, L, x, gy, w)      # a runner returns its tensors in NCHW order
     rng = np.random.default_rng(seed)
     errs = {}
     stash_ref = oracle.stash_forward(f64(x), L.r)
@@ -124,6 +124,6 @@ def check_layer_sampled(gf, L: workloads.Layer, n_ch: int = 6, n_img: int = 2, s
     # properties at any size: all taps equal; g_X constant on every patch
     assert bool((gW == gW[:, :, :1, :1]).all())
     if L.H % L.r == 0 and L.W % L.r == 0:
-        blocks = gX.view(L.N, L.C_in, L.Hp, L.r, L.Wp, L.r)
+        blocks = gX.reshape(L.N, L.C_in, L.Hp, L.r, L.Wp, L.r)
         assert bool((blocks == blocks[:, :, :, :1, :, :1]).all())
     return errs
