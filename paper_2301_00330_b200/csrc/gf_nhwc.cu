@@ -21,6 +21,8 @@
 #include "gf_tc.cuh"
 #include "gf_tma.cuh"
 
+#include <type_traits>
+
 namespace gf {
 
 namespace {
@@ -91,7 +93,8 @@ __global__ void __launch_bounds__(kNpThreads) nhwc_pool_kernel(const T* __restri
 }
 
 // ---------------------------------------------------------------- the two contractions
-constexpr int kNxStages = 3;
+constexpr int kNxStages = 3;          // g_W kernel
+constexpr int kNxMaxStages = 4;       // g_X kernel: 2 to 4, chosen by the launcher
 constexpr int kNxEpiWarps = 8;
 constexpr int kNxThreads = (kNxEpiWarps + 2) * 32;
 
@@ -103,43 +106,65 @@ struct NhwcGemmParams {
     int M;                      // patches
     int C_in, C_out, H, W, r, Hp, Wp;
     int NT;                     // g_x: c_i per CTA (multiple of 16, <= 256)
+    int stages;                 // g_x: ring slots
     int k_chunks, S;            // chunks of 64 along the contraction, slices of them (g_w)
     FastDiv div_Wp, div_Hp;
 };
 
 struct NxShared {
-    uint64_t full[kNxStages], empty[kNxStages];
+    uint64_t full[kNxMaxStages], empty[kNxMaxStages];
     uint64_t accum;
     uint32_t tmem_base;
 };
 
-// 8 consecutive values of one accumulator row to 8 consecutive channels
-__device__ __forceinline__ void put8(float* dst, const uint32_t* v) {
-    __stcs(reinterpret_cast<float4*>(dst), make_float4(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]), __uint_as_float(v[3])));
-    __stcs(reinterpret_cast<float4*>(dst) + 1, make_float4(__uint_as_float(v[4]), __uint_as_float(v[5]), __uint_as_float(v[6]), __uint_as_float(v[7])));
+// Named barrier `id` over `nthreads` threads that also tells every one of them whether any of them
+// passed a true predicate (a wait that ran out): nobody is left alone at a later barrier.
+__device__ __forceinline__ bool nx_bar_any(int id, int nthreads, bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, %2, %3, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "r"((uint32_t)pred), "r"(id), "r"(nthreads)
+        : "memory");
+    return r != 0;
 }
-__device__ __forceinline__ void put8(__nv_bfloat16* dst, const uint32_t* v) {
-    __stcs(reinterpret_cast<uint4*>(dst), make_uint4(pack2(__uint_as_float(v[0]), __uint_as_float(v[1])), pack2(__uint_as_float(v[2]), __uint_as_float(v[3])),
-                                                     pack2(__uint_as_float(v[4]), __uint_as_float(v[5])), pack2(__uint_as_float(v[6]), __uint_as_float(v[7]))));
+
+// 8 consecutive accumulator values of a row as 8 output elements in the staging tile
+__device__ __forceinline__ void stage8(float* dst, const uint32_t* v) {
+    reinterpret_cast<uint4*>(dst)[0] = make_uint4(v[0], v[1], v[2], v[3]);
+    reinterpret_cast<uint4*>(dst)[1] = make_uint4(v[4], v[5], v[6], v[7]);
+}
+__device__ __forceinline__ void stage8(__nv_bfloat16* dst, const uint32_t* v) {
+    *reinterpret_cast<uint4*>(dst) = make_uint4(pack2(__uint_as_float(v[0]), __uint_as_float(v[1])), pack2(__uint_as_float(v[2]), __uint_as_float(v[3])),
+                                                pack2(__uint_as_float(v[4]), __uint_as_float(v[5])), pack2(__uint_as_float(v[6]), __uint_as_float(v[7])));
 }
 
 // SPLIT: 1 = bf16 operands, 2 = fp32 values as (high, low) bf16 pairs (hi*hi + hi*lo + lo*hi).
 template <typename TOut, int SPLIT>
 __global__ void __launch_bounds__(kNxThreads) nhwc_gx_kernel(const __grid_constant__ NhwcGemmParams p) {
     constexpr int kABytes = 128 * 128;                       // [128 patches][64 c_o] bf16
+    constexpr int kVec = 16 / (int)sizeof(TOut);             // output elements per 16-byte store
     extern __shared__ unsigned char dyn_raw[];
     __shared__ NxShared sh;
     unsigned char* dyn = align1024(dyn_raw);
-    const int b_bytes = p.NT * 128;
+    // The parameter block's address is taken (the tensor maps), so its fields are read once here
+    // into registers: reads through it inside the loops would be loads from memory every time.
+    const int NT = p.NT, n_stages = p.stages, k_chunks = p.k_chunks, M = p.M, C_in = p.C_in, H = p.H, W = p.W, r = p.r;
+    const FastDiv div_Wp = p.div_Wp, div_Hp = p.div_Hp;
+    TOut* const gX = static_cast<TOut*>(p.gX);
+    const int b_bytes = NT * 128;
     const int stage_bytes = SPLIT * (kABytes + b_bytes);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int ci0 = blockIdx.x * p.NT, m0 = blockIdx.y * 128;
-    const int ng = min(p.NT, p.C_in - ci0);
+    const int ci0 = blockIdx.x * NT, m0 = blockIdx.y * 128;
+    const int ng = min(NT, C_in - ci0);
     int ncols = 32;
-    while (ncols < p.NT) ncols <<= 1;
+    while (ncols < NT) ncols <<= 1;
 
     if (tid == 0) {
-        for (int s = 0; s < kNxStages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+        for (int s = 0; s < n_stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
         mbar_init(&sh.accum, 1);
         mbar_fence_init();
     }
@@ -153,10 +178,10 @@ __global__ void __launch_bounds__(kNxThreads) nhwc_gx_kernel(const __grid_consta
     bool ok = true;
 
     if (warp == kNxEpiWarps) {
-        if (lane == 0)
-            for (int q = 0; q < p.k_chunks && ok; ++q) {
-                const int s = q % kNxStages;
-                if (q >= kNxStages) ok = mbar_wait_bounded(&sh.empty[s], (uint32_t)(q / kNxStages - 1) & 1u);
+        if (lane == 0) {
+            int s = 0, round = 0;
+            for (int q = 0; q < k_chunks && ok; ++q) {
+                if (round > 0) ok = mbar_wait_bounded(&sh.empty[s], (uint32_t)(round - 1) & 1u);
                 if (!ok) break;
                 unsigned char* stage = dyn + (size_t)s * stage_bytes;
                 mbar_expect_tx(&sh.full[s], (uint32_t)stage_bytes);
@@ -164,13 +189,15 @@ __global__ void __launch_bounds__(kNxThreads) nhwc_gx_kernel(const __grid_consta
                     tma_load_3d(stage + part * kABytes, &p.tm_a, q * kTcBK, m0, part, &sh.full[s]);
                     tma_load_3d(stage + SPLIT * kABytes + part * b_bytes, &p.tm_b, q * kTcBK, ci0, part, &sh.full[s]);
                 }
+                if (++s == n_stages) { s = 0; ++round; }
             }
+        }
     } else if (warp == kNxEpiWarps + 1) {
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_bf16(128, (ng + 15) & ~15, 0, 0);
-            for (int q = 0; q < p.k_chunks && ok; ++q) {
-                const int s = q % kNxStages;
-                ok = mbar_wait_bounded(&sh.full[s], (uint32_t)(q / kNxStages) & 1u);
+            int s = 0, round = 0;
+            for (int q = 0; q < k_chunks && ok; ++q) {
+                ok = mbar_wait_bounded(&sh.full[s], (uint32_t)round & 1u);
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t a_hi = smem_u32(dyn + (size_t)s * stage_bytes), a_lo = a_hi + kABytes;
@@ -185,31 +212,47 @@ __global__ void __launch_bounds__(kNxThreads) nhwc_gx_kernel(const __grid_consta
                     }
                 }
                 umma_commit(&sh.empty[s]);
+                if (++s == n_stages) { s = 0; ++round; }
             }
             if (ok) umma_commit(&sh.accum);
         }
     } else {
+        // The accumulator is complete, so every copy has landed and every MMA has read its operands:
+        // the ring's memory is free and takes the output tile [128 patches][ng channels] (rows 16
+        // bytes longer than the data, so that the 16-byte stores of a warp's 32 rows spread over the
+        // banks).  Then every warp writes whole rows: one patch's channels, contiguous in g_X, to
+        // each of the patch's r x r pixels.
         ok = mbar_wait_bounded(&sh.accum, 0);
         tc_fence_after_sync();
+        const int pitch = NT * (int)sizeof(TOut) + 16;
         if (ok) {
             const int quarter = warp & 3, half = warp >> 2;
-            const int m = m0 + quarter * 32 + lane;
-            uint32_t nb, b, n, a;
-            p.div_Wp.divmod((uint32_t)min(m, p.M - 1), nb, b);
-            p.div_Hp.divmod(nb, n, a);
-            const int rows = min(p.r, p.H - (int)a * p.r), cols = min(p.r, p.W - (int)b * p.r);
-            TOut* base = static_cast<TOut*>(p.gX) + (((size_t)n * p.H + (size_t)a * p.r) * p.W + (size_t)b * p.r) * p.C_in + ci0;
+            unsigned char* row = dyn + (size_t)(quarter * 32 + lane) * pitch;
             for (int c = half * 32; c < ng; c += 64) {
                 uint32_t v[32];
                 tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c, v);
                 tmem_ld_wait();
-                if (m < p.M) {
-                    const int n8 = min(32, ng - c) / 8;              // channel counts are multiples of 8
+                const int n8 = min(32, ng - c) / 8;                  // channel counts are multiples of 8
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    if (k < n8) stage8(reinterpret_cast<TOut*>(row) + c + 8 * k, v + 8 * k);
+            }
+        }
+        const bool bad = nx_bar_any(1, kNxEpiWarps * 32, !ok);
+        if (!bad) {
+            const int m_end = min(128, M - m0);
+            for (int ml = warp; ml < m_end; ml += kNxEpiWarps) {
+                uint32_t nb, b, n, a;
+                div_Wp.divmod((uint32_t)(m0 + ml), nb, b);
+                div_Hp.divmod(nb, n, a);
+                const int rows = min(r, H - (int)a * r), cols = min(r, W - (int)b * r);
+                TOut* base = gX + (((size_t)n * H + (size_t)a * r) * W + (size_t)b * r) * C_in + ci0;
+                const TOut* src = reinterpret_cast<const TOut*>(dyn + (size_t)ml * pitch);
+                for (int c = lane * kVec; c < ng; c += 32 * kVec) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(src + c);
                     for (int dr = 0; dr < rows; ++dr)
-                        for (int dc = 0; dc < cols; ++dc) {
-                            TOut* dst = base + ((size_t)dr * p.W + dc) * p.C_in + c;
-                            for (int k = 0; k < n8; ++k) put8(dst + 8 * k, v + 8 * k);
-                        }
+                        for (int dc = 0; dc < cols; ++dc)
+                            __stcs(reinterpret_cast<uint4*>(base + ((size_t)dr * W + dc) * C_in + c), v);
                 }
             }
         }
@@ -234,6 +277,8 @@ __global__ void __launch_bounds__(kNxThreads) nhwc_gw_kernel(const __grid_consta
     __shared__ NxShared sh;
     unsigned char* dyn = align1024(dyn_raw);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int C_in = p.C_in, C_out = p.C_out;                       // read once: see nhwc_gx_kernel
+    float* const gwu = p.gwu;
     const int ci0 = blockIdx.x * 128, co0 = blockIdx.y * 128, split = blockIdx.z;
     const int kc_begin = (int)((long long)p.k_chunks * split / p.S), kc_end = (int)((long long)p.k_chunks * (split + 1) / p.S);
     const int n_chunks = kc_end - kc_begin;
@@ -295,16 +340,16 @@ __global__ void __launch_bounds__(kNxThreads) nhwc_gw_kernel(const __grid_consta
         if (ok && n_chunks > 0) {
             const int quarter = warp & 3, half = warp >> 2;
             const int co = co0 + quarter * 32 + lane;
-            float* out = p.gwu + (size_t)co * p.C_in + ci0;
+            float* out = gwu + (size_t)co * C_in + ci0;
 #pragma unroll 1
             for (int c = half * 64; c < half * 64 + 64; c += 32) {
                 uint32_t v[32];
                 tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c, v);
                 tmem_ld_wait();
-                if (co < p.C_out) {
+                if (co < C_out) {
 #pragma unroll
                     for (int i = 0; i < 32; i += 4)
-                        if (ci0 + c + i < p.C_in) red_add_v4(out + c + i, v[i], v[i + 1], v[i + 2], v[i + 3]);   // C_in % 8 == 0
+                        if (ci0 + c + i < C_in) red_add_v4(out + c + i, v[i], v[i + 1], v[i + 2], v[i + 3]);   // C_in % 8 == 0
                 }
             }
         }
@@ -322,18 +367,26 @@ __global__ void __launch_bounds__(kNxThreads) nhwc_gw_kernel(const __grid_consta
 
 // ---------------------------------------------------------------- depthwise
 // Thread (v8, lane): 8 channels and every `q_stride`-th patch from `lane` on.  Per patch: mean of the
-// patch of g_y, g_X = mean x kernel sum on the patch's pixels, mean x stash summed in registers;
-// at the end one addition per channel and thread into part [C] (zeroed beforehand).
-template <typename T>
-__global__ void __launch_bounds__(kNpThreads) nhwc_dw_kernel(const T* __restrict__ gy, const T* __restrict__ stash, const T* __restrict__ Wt,
-                                                             float* __restrict__ part, T* __restrict__ gX, long long patches, int C, int H,
-                                                             int W, int r, int Hp, int Wp, int taps, FastDiv div_c8, FastDiv div_Wp,
-                                                             FastDiv div_Hp) {
+// patch of g_y, g_X = mean x kernel sum on the patch's pixels, mean x stash summed in registers.
+// At the end the block adds its threads' sums per channel in shared memory and writes them to its
+// row of part [blocks][C]; the finishing kernel adds the rows.  R: the patch size when it is 2
+// (all loads of a full patch issued before the first use), else 0.
+template <typename T, int R>
+__global__ void __launch_bounds__(kNpThreads, 3) nhwc_dw_kernel(const T* __restrict__ gy, const T* __restrict__ stash,
+                                                                const T* __restrict__ Wt, float* __restrict__ part, T* __restrict__ gX,
+                                                                long long patches, int C, int H, int W, int r_rt, int Hp, int Wp,
+                                                                int taps, FastDiv div_c8, FastDiv div_Wp, FastDiv div_Hp) {
+    extern __shared__ float dw_red[];                               // [C]
+    const int r = R > 0 ? R : r_rt;
     const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;       // the launcher makes the thread count a multiple of C / 8
     uint32_t lane_q, v8;
     div_c8.divmod(t, lane_q, v8);
     const uint32_t q_stride = div_c8.div(gridDim.x * blockDim.x);
     const int c0 = (int)v8 * 8;
+    if (part) {
+        for (int c = threadIdx.x; c < C; c += blockDim.x) dw_red[c] = 0.f;
+        __syncthreads();
+    }
     float ts[8], dot[8];
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
@@ -346,21 +399,34 @@ __global__ void __launch_bounds__(kNpThreads) nhwc_dw_kernel(const T* __restrict
         uint32_t nb, b, n, a;
         div_Wp.divmod((uint32_t)q, nb, b);
         div_Hp.divmod(nb, n, a);
-        const int i1 = min((int)(a + 1) * r, H), j1 = min((int)(b + 1) * r, W);
-        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-        for (int i = (int)a * r; i < i1; ++i)
-            for (int j = (int)b * r; j < j1; ++j) {
-                float v[8];
-                load8(gy + (((size_t)n * H + i) * W + j) * C + c0, v);
+        const int i0 = (int)a * r, j0 = (int)b * r;
+        const int i1 = min(i0 + r, H), j1 = min(j0 + r, W);
+        const size_t pix = (((size_t)n * H + i0) * W + j0) * C + c0;
+        float acc[8], st[8];
+        if (part) load8(stash + (size_t)q * C + c0, st);
+        if (R == 2 && i1 - i0 == 2 && j1 - j0 == 2) {
+            float v0[8], v1[8], v2[8], v3[8];
+            load8(gy + pix, v0);
+            load8(gy + pix + C, v1);
+            load8(gy + pix + (size_t)W * C, v2);
+            load8(gy + pix + (size_t)W * C + C, v3);
 #pragma unroll
-                for (int k = 0; k < 8; ++k) acc[k] += v[k];
-            }
-        const float inv = 1.0f / (float)((i1 - (int)a * r) * (j1 - (int)b * r));
+            for (int k = 0; k < 8; ++k) acc[k] = ((v0[k] + v1[k]) + (v2[k] + v3[k])) * 0.25f;
+        } else {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) acc[k] *= inv;
+            for (int k = 0; k < 8; ++k) acc[k] = 0.f;
+            for (int i = i0; i < i1; ++i)
+                for (int j = j0; j < j1; ++j) {
+                    float v[8];
+                    load8(gy + (((size_t)n * H + i) * W + j) * C + c0, v);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) acc[k] += v[k];
+                }
+            const float inv = 1.0f / (float)((i1 - i0) * (j1 - j0));
+#pragma unroll
+            for (int k = 0; k < 8; ++k) acc[k] *= inv;
+        }
         if (part) {
-            float st[8];
-            load8(stash + (size_t)q * C + c0, st);
 #pragma unroll
             for (int k = 0; k < 8; ++k) dot[k] = fmaf(acc[k], st[k], dot[k]);
         }
@@ -368,14 +434,33 @@ __global__ void __launch_bounds__(kNpThreads) nhwc_dw_kernel(const T* __restrict
             float o[8];
 #pragma unroll
             for (int k = 0; k < 8; ++k) o[k] = acc[k] * ts[k];
-            for (int i = (int)a * r; i < i1; ++i)
-                for (int j = (int)b * r; j < j1; ++j) store8(gX + (((size_t)n * H + i) * W + j) * C + c0, o);
+            for (int i = i0; i < i1; ++i)
+                for (int j = j0; j < j1; ++j) store8(gX + (((size_t)n * H + i) * W + j) * C + c0, o);
         }
     }
     if (part) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) atomicAdd(part + c0 + k, dot[k]);
+        for (int k = 0; k < 8; ++k) atomicAdd(&dw_red[c0 + k], dot[k]);
+        __syncthreads();
+        for (int c = threadIdx.x; c < C; c += blockDim.x) part[(size_t)blockIdx.x * C + c] = dw_red[c];
     }
+}
+
+// blocks of the depthwise kernel: a multiple of `unit` (so that the thread count is a multiple of
+// C / 8), about four per SM, at most kDwMaxBlocks
+constexpr int kDwMaxBlocks = 1024;
+int dw_unit(int C) {
+    const int c8 = C / 8;
+    int gcd = kNpThreads, rem = c8;
+    while (rem) { const int tmp = gcd % rem; gcd = rem; rem = tmp; }
+    return c8 / gcd;
+}
+int dw_blocks(int C) {
+    const int unit = dw_unit(C);
+    int want = sm_count() * 4;
+    if (want > kDwMaxBlocks) want = kDwMaxBlocks;
+    const int blocks = want / unit * unit;
+    return blocks < unit ? unit : blocks;
 }
 
 unsigned np_grid(long long items) {
@@ -391,6 +476,7 @@ bool nhwc_supported(const Geo& g, int stride) {
     if (stride != 1 || g.C_in % 8 != 0 || g.C_out % 8 != 0) return false;
     const bool depthwise = g.G == g.C_in && g.G == g.C_out;
     if (g.G != 1 && !depthwise) return false;
+    if (depthwise && (g.C_in > 12288 || dw_unit(g.C_in) > kDwMaxBlocks)) return false;
     const long long M = (long long)g.N * g.Hp * g.Wp;
     return M * (g.C_in > g.C_out ? g.C_in : g.C_out) / 8 < 0x7fffffffLL && (long long)g.N * g.H < 0x7fffffffLL;
 }
@@ -401,7 +487,7 @@ size_t nhwc_workspace_bytes(const Geo& g) {
     auto up = [](size_t v) { return (v + 255) / 256 * 256; };
     const size_t M = (size_t)g.N * g.Hp * g.Wp;
     if (g.r == 1) return 256;
-    if (g.G != 1) return 256 + up((size_t)g.C_in * 4);
+    if (g.G != 1) return 256 + up((size_t)kDwMaxBlocks * g.C_in * 4);
     size_t off = 256;
     off += up((size_t)g.C_out * g.C_in * 4);
     off += up(M * g.C_out * 4);
@@ -427,7 +513,7 @@ gf_status launch_nhwc_stash(const void* x, void* stash, const Geo& g, cudaStream
 
 template <typename TOut, int SPLIT>
 static gf_status launch_nhwc_gx(const NhwcGemmParams& p, dim3 grid, cudaStream_t s) {
-    const size_t smem = (size_t)kNxStages * SPLIT * (128 * 128 + (size_t)p.NT * 128) + 1024;
+    const size_t smem = (size_t)p.stages * SPLIT * (128 * 128 + (size_t)p.NT * 128) + 1024;
     static size_t configured[kMaxDevices] = {};
     if (gf_status st = ensure_dyn_smem(nhwc_gx_kernel<TOut, SPLIT>, smem, configured); st != GF_OK) return st;
     return launch_pdl(nhwc_gx_kernel<TOut, SPLIT>, grid, dim3(kNxThreads), smem, s, p);
@@ -451,29 +537,26 @@ gf_status nhwc_backward(const Geo& g, const void* g_y, const void* stash, const 
     gf_status st;
     if (g.G != 1) {                                       // depthwise
         float* part = reinterpret_cast<float*>(base + 256);
-        if (g_W) GF_CUDA_TRY(cudaMemsetAsync(part, 0, (size_t)g.C_in * 4, s));
+        const int blocks = dw_blocks(g.C_in);
         {
             ProfScope prof(K_DW_FUSED, s);
-            // a thread count that is a multiple of C / 8, so that a thread keeps its channels over its patches
-            const int c8 = g.C_in / 8;
-            int gcd = 256, rem = c8;
-            while (rem) { const int tmp = gcd % rem; gcd = rem; rem = tmp; }
-            const int unit = c8 / gcd;                                    // blocks per multiple
-            long long blocks = ((long long)sm_count() * 4 / unit) * unit;
-            if (blocks < unit) blocks = unit;
-            const FastDiv d8((uint32_t)c8);
-            if (g.dtype == GF_F32)
-                nhwc_dw_kernel<float><<<(unsigned)blocks, kNpThreads, 0, s>>>((const float*)g_y, (const float*)stash, (const float*)W,
-                                                                              g_W ? part : nullptr, (float*)g_X, M, g.C_in, g.H, g.W, g.r,
-                                                                              g.Hp, g.Wp, g.KH * g.KW, d8, dW, dH);
-            else
-                nhwc_dw_kernel<__nv_bfloat16><<<(unsigned)blocks, kNpThreads, 0, s>>>((const __nv_bfloat16*)g_y, (const __nv_bfloat16*)stash,
-                                                                                      (const __nv_bfloat16*)W, g_W ? part : nullptr,
-                                                                                      (__nv_bfloat16*)g_X, M, g.C_in, g.H, g.W, g.r, g.Hp,
-                                                                                      g.Wp, g.KH * g.KW, d8, dW, dH);
+            const FastDiv d8((uint32_t)(g.C_in / 8));
+            const size_t smem = g_W ? (size_t)g.C_in * 4 : 0;
+            auto go = [&](auto kern, auto* tag) {
+                using T = std::remove_pointer_t<decltype(tag)>;
+                kern<<<(unsigned)blocks, kNpThreads, smem, s>>>((const T*)g_y, (const T*)stash, (const T*)W, g_W ? part : nullptr, (T*)g_X, M,
+                                                               g.C_in, g.H, g.W, g.r, g.Hp, g.Wp, g.KH * g.KW, d8, dW, dH);
+            };
+            if (g.dtype == GF_F32) {
+                if (g.r == 2) go(nhwc_dw_kernel<float, 2>, (float*)nullptr);
+                else go(nhwc_dw_kernel<float, 0>, (float*)nullptr);
+            } else {
+                if (g.r == 2) go(nhwc_dw_kernel<__nv_bfloat16, 2>, (__nv_bfloat16*)nullptr);
+                else go(nhwc_dw_kernel<__nv_bfloat16, 0>, (__nv_bfloat16*)nullptr);
+            }
             if ((st = after_launch()) != GF_OK) return st;
         }
-        return g_W ? launch_gw_finish(part, 1, g_W, g, s) : GF_OK;
+        return g_W ? launch_gw_finish(part, blocks, g_W, g, s) : GF_OK;
     }
     const bool split = g.dtype == GF_F32;
     const int parts = split ? 2 : 1;
@@ -507,8 +590,20 @@ gf_status nhwc_backward(const Geo& g, const void* g_y, const void* stash, const 
     p.div_Wp = dW; p.div_Hp = dH;
     if (g_X) {
         ProfScope prof(K_GX_TC, s);
-        const int nt_max = split ? 128 : 256;
-        p.NT = g.C_in > nt_max ? nt_max : (g.C_in + 15) / 16 * 16;
+        // c_i per CTA: as wide as tensor memory and the ring allow (256), in equal parts.  Measured: the
+        // kernel is bound by its writes, and the longer the run of channels a CTA writes per pixel the
+        // faster they go (576 channels: 3 x 192 beats 5 x 128 and 9 x 64 by a third).
+        const int n_ci = (g.C_in + 255) / 256;
+        p.NT = ((g.C_in + n_ci - 1) / n_ci + 15) / 16 * 16;
+        {
+            const size_t stage = (size_t)parts * (128 * 128 + (size_t)p.NT * 128);
+            const size_t tile = (size_t)128 * ((size_t)p.NT * g.esize + 16);
+            int st_n = (int)((size_t)100 * 1024 / stage);                // two CTAs per SM where two slots fit in that
+            if (st_n < 2) st_n = 2;
+            if (st_n > kNxMaxStages) st_n = kNxMaxStages;
+            while ((size_t)st_n * stage < tile) ++st_n;                  // the output tile reuses the ring
+            p.stages = st_n;
+        }
         p.k_chunks = (g.C_out + kTcBK - 1) / kTcBK; p.S = 1;
         if (!make_tmap_bf16(&p.tm_a, gbar, 3, (uint64_t)g.C_out, (uint64_t)M, (uint64_t)parts, (uint64_t)g.C_out,
                             split ? (uint64_t)gbar_lo : (uint64_t)M * g.C_out, 128) ||
