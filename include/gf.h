@@ -36,6 +36,16 @@
  *    reaches an output.  The paper states its formulas for stride 1 only; this
  *    is the library's extension of them (same two approximations).  NCHW only.
  *    Anything else: GF_ERR_UNSUPPORTED.
+ *  - Layout.  GF_NCHW: the tensors as written above.  GF_NHWC (channels last):
+ *    x [N,H,W,C_in], g_y [N,H,W,C_out], g_X like x and the stash
+ *    [N,ceil(H/r),ceil(W/r),C_in]; W and g_W stay [C_out,C_in/groups,KH,KW].
+ *    The paper's formulas index channels and pixels and fix no memory order;
+ *    the results are those of NCHW, permuted.  Channels-last is supported for
+ *    gf_stash_forward, gf_backward, gf_backward_static_scratch and
+ *    gf_layer_step_host (whose host buffers then have that order too) with r >= 2,
+ *    stride 1, C_in and C_out multiples of 8, and groups == 1 or a depthwise
+ *    layer (groups == C_in == C_out, at most 12288 channels); other channels-last
+ *    descriptors, and every other call given one, return GF_ERR_UNSUPPORTED.
  *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Work
  *    is enqueued on it and the call returns without synchronising.  Errors that
  *    the host can detect are returned before anything is launched.
@@ -74,7 +84,7 @@ typedef struct gf_conv_desc {
     int32_t groups;
     int32_t r;              /* patch size, >= 1; 1 = exact backward */
     int32_t dtype;          /* gf_dtype */
-    int32_t layout;         /* gf_layout; only GF_NCHW */
+    int32_t layout;         /* gf_layout; GF_NHWC within the limits stated above */
 } gf_conv_desc;
 
 /* Logical shape [N, C_in, ceil(H/(r s)), ceil(W/(r s))] of the stash, s the stride
@@ -82,7 +92,8 @@ typedef struct gf_conv_desc {
 gf_status gf_stash_dims(const gf_conv_desc* desc, int64_t dims[4]);
 
 /* Bytes of the stash: product of gf_stash_dims times the element size.  The
- * physical layout is the dense NCHW array of that shape. */
+ * physical layout is the dense NCHW array of that shape, or for GF_NHWC the dense
+ * [N, Hp, Wp, C_in] array with the same four extents. */
 gf_status gf_stash_bytes(const gf_conv_desc* desc, size_t* bytes);
 
 /* Bytes of device scratch gf_backward needs for this descriptor (always > 0). */

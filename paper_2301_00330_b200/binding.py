@@ -145,8 +145,9 @@ def _ptr(t) -> ctypes.c_void_p:
     if t is None:
         return ctypes.c_void_p(0)
     if isinstance(t, torch.Tensor):
-        if not t.is_contiguous():
-            raise ValueError("tensors passed to the gf_* calls must be contiguous")
+        # dense in either order; which one the bytes are in is the descriptor's `layout`
+        if not (t.is_contiguous() or (t.dim() == 4 and t.is_contiguous(memory_format=torch.channels_last))):
+            raise ValueError("tensors passed to the gf_* calls must be dense (contiguous, or channels_last for GF_NHWC)")
         return ctypes.c_void_p(t.data_ptr())
     return ctypes.c_void_p(int(t))
 

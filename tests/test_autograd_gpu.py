@@ -56,3 +56,24 @@ def test_strided_layer_through_autograd(gf):
     torch.cuda.synchronize()
     gw_ref, gx_ref = oracle.strided_backward(f64(gy), oracle.strided_stash_forward(f64(x), 2, 2), f64(w), 2, 2)
     assert relerr(f64(xd.grad), gx_ref) <= TOL["f32"] and relerr(f64(wd.grad), gw_ref) <= TOL["f32"]
+
+
+@pytest.mark.parametrize("groups,c_in,c_out", [(1, 16, 24), (16, 16, 16), (1, 12, 8)])
+def test_channels_last_input_through_autograd(gf, groups, c_in, c_out):
+    """An input in torch's channels_last format: the channels-last kernels where the library has them
+    (the first two cases), a contiguous copy otherwise (12 channels); the gradients are the same
+    filtered ones, and g_X comes back in the input's format when the channels-last kernels ran."""
+    L = workloads.Layer("cl", 0, 0, 2, c_in, c_out, 12, 12, 3, groups, 2, "f32", "normal", 1.0)
+    x, gy, w = workloads.make_inputs(L)
+    xd = x.cuda().contiguous(memory_format=torch.channels_last).requires_grad_(True)
+    wd = w.cuda().requires_grad_(True)
+    launches = gf.gf_kernel_launch_count()
+    y = gf.filtered_conv2d(xd, wd, r=2, groups=groups)
+    y.backward(gy.cuda())
+    torch.cuda.synchronize()
+    assert gf.gf_kernel_launch_count() > launches
+    stash_ref = oracle.stash_forward(f64(x), 2)
+    gw_ref, gx_ref = oracle.backward(f64(gy), stash_ref, f64(w), 2, groups=groups)
+    assert relerr(f64(xd.grad), gx_ref) <= TOL["f32"] and relerr(f64(wd.grad), gw_ref) <= TOL["f32"]
+    if c_in % 8 == 0:
+        assert xd.grad.is_contiguous(memory_format=torch.channels_last)

@@ -139,6 +139,27 @@ def test_nhwc_nullable_outputs(gf):
     assert torch.equal(gx_a, gx_c)
 
 
+def test_nhwc_static_scratch_and_host_step(gf):
+    """The two other entry points that take a channels-last descriptor give the results of gf_backward."""
+    layer = L("other_calls", 2, 24, 40, 14, 14, 3, 1, 2)
+    x, gy, w = workloads.make_inputs(layer)
+    stash, gw_a, gx_a = run_nhwc(gf, layer, x, gy, w)
+    desc = gf.make_desc(layer.N, layer.C_in, layer.C_out, layer.H, layer.W, layer.K, r=layer.r, layout=gf.GF_NHWC)
+    gW = torch.empty_like(gw_a)
+    gX = torch.empty((layer.N, layer.H, layer.W, layer.C_in), device="cuda")
+    gf.gf_backward_static_scratch(desc, nhwc(gy).cuda(), nhwc(stash), w.cuda(), gW, gX)
+    torch.cuda.synchronize()
+    assert relerr(f64(gW), f64(gw_a)) <= 1e-6 and torch.equal(nchw_of(gX), gx_a)
+    # host buffers in, host buffers out
+    h_x, h_gy, h_w = nhwc(x).pin_memory(), nhwc(gy).pin_memory(), w.pin_memory()
+    h_gW = torch.empty(gw_a.shape, dtype=torch.float32).pin_memory()
+    h_gX = torch.empty((layer.N, layer.H, layer.W, layer.C_in)).pin_memory()
+    arena = torch.empty(gf.gf_host_step_arena_bytes(desc), dtype=torch.uint8, device="cuda")
+    gf.gf_layer_step_host(desc, h_x, h_gy, h_w, h_gW, h_gX, arena)
+    torch.cuda.synchronize()
+    assert relerr(f64(h_gW), f64(gw_a)) <= 1e-6 and torch.equal(nchw_of(h_gX), gx_a.cpu())
+
+
 def test_nhwc_unsupported_shapes_are_refused(gf):
     ok = dict(N=2, C_in=16, C_out=16, H=8, W=8, KH=3, r=2, layout=gf.GF_NHWC)
 
