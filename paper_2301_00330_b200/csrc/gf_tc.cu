@@ -694,6 +694,308 @@ __global__ void __launch_bounds__(kGwThreads) gw_tc_kernel(const GwTcParams p) {
     if (warp == 8) tmem_dealloc(tmem, NT);
 }
 
+// ================================================================== gw_tma
+// The same contraction with both operands fetched by the copy engine: possible when the rows of
+// the [N][C][P] arrays start on 16-byte boundaries (pitch % 8 == 0).  A unit of the contraction
+// is 64 consecutive patches of one image (a box never crosses into the next image; what lies
+// past the last patch of the image reads as zero, and MMA steps of 16 patches that hold no
+// patch at all are not issued).  Warps 0-7: epilogue; warp 8: copies; warp 9: MMA issue.
+struct GwTmaParams {
+    CUtensorMap tm_a[2], tm_b[2];   // gbar, stash as [N][C][P] bf16: high parts, low parts (fp32 layers)
+    float* gwu;                     // [C_out][C_in] fp32, zeroed beforehand; every CTA adds its slice
+    uint32_t* err_word;
+    int C_in, C_out, S;
+    int cpi, units_total;           // 64-patch units per image, units in all
+    int P_live;                     // patches per image
+    FastDiv div_cpi;
+};
+constexpr int kGwTmaThreads = 320;
+
+template <int NT, int SPLIT>
+__global__ void __launch_bounds__(kGwTmaThreads) gw_tma_kernel(const __grid_constant__ GwTmaParams p) {
+    constexpr int kStages = gw_stages(SPLIT, NT);
+    constexpr int kABytes = 128 * kTcBK * 2;
+    constexpr int kBBytes = NT * kTcBK * 2;
+    constexpr int kBOff = SPLIT * kABytes;                  // stage: [A hi][A lo][B hi][B lo]
+    constexpr int kStageBytes = SPLIT * (kABytes + kBBytes);
+    constexpr uint32_t kIdesc = umma_idesc_bf16(128, NT, 0, 0);
+    extern __shared__ unsigned char dyn_raw[];
+    __shared__ GwShared sh;
+    unsigned char* dyn = align1024(dyn_raw);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // fields of the parameter block, read once (its address is taken for the tensor maps)
+    const int C_in = p.C_in, C_out = p.C_out, cpi = p.cpi, P_live = p.P_live;
+    const FastDiv div_cpi = p.div_cpi;
+    float* const gwu = p.gwu;
+    const int ci0 = blockIdx.x * NT, co0 = blockIdx.y * 128, split = blockIdx.z;
+    const int u_begin = (int)((long long)p.units_total * split / p.S);
+    const int u_end = (int)((long long)p.units_total * (split + 1) / p.S);
+    const int n_units = u_end - u_begin;
+
+    pdl_launch_dependents();
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+        mbar_init(&sh.accum, 1);
+        mbar_fence_init();
+    }
+    if (warp == 9) { tmem_alloc(&sh.tmem_base, NT); tmem_relinquish(); }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = sh.tmem_base;
+    pdl_wait();                       // operands come from the previous kernels of the stream
+    bool ok = true;
+
+    if (warp == 8) {
+        if (lane == 0) {
+            int s = 0, round = 0;
+            for (int q = 0; q < n_units && ok; ++q) {
+                if (round > 0) ok = mbar_wait_bounded(&sh.empty[s], (uint32_t)(round - 1) & 1u);
+                if (!ok) break;
+                uint32_t n, c;
+                div_cpi.divmod((uint32_t)(u_begin + q), n, c);
+                unsigned char* stage = dyn + (size_t)s * kStageBytes;
+                mbar_expect_tx(&sh.full[s], (uint32_t)kStageBytes);
+#pragma unroll
+                for (int h = 0; h < SPLIT; ++h) {
+                    tma_load_3d(stage + h * kABytes, &p.tm_a[h], (int)c * kTcBK, co0, (int)n, &sh.full[s]);
+                    tma_load_3d(stage + kBOff + h * kBBytes, &p.tm_b[h], (int)c * kTcBK, ci0, (int)n, &sh.full[s]);
+                }
+                if (++s == kStages) { s = 0; ++round; }
+            }
+        }
+    } else if (warp == 9) {
+        if (lane == 0) {
+            int s = 0, round = 0;
+            bool first = true;
+            for (int q = 0; q < n_units && ok; ++q) {
+                ok = mbar_wait_bounded(&sh.full[s], (uint32_t)round & 1u);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t c = (uint32_t)(u_begin + q) - div_cpi.div((uint32_t)(u_begin + q)) * (uint32_t)cpi;
+                const int steps = min(kTcBK / 16, (P_live - (int)c * kTcBK + 15) / 16);   // steps that hold a patch
+                const uint32_t a_hi = smem_u32(dyn + (size_t)s * kStageBytes), a_lo = a_hi + kABytes;
+                const uint32_t b_hi = a_hi + kBOff, b_lo = b_hi + kBBytes;
+                for (int ks = 0; ks < steps; ++ks) {
+                    const uint64_t ad = umma_smem_desc(a_hi + ks * 32, 16, 1024), bd = umma_smem_desc(b_hi + ks * 32, 16, 1024);
+                    umma_bf16(tmem, ad, bd, kIdesc, first ? 0u : 1u);
+                    first = false;
+                    if constexpr (SPLIT == 2) {
+                        umma_bf16(tmem, ad, umma_smem_desc(b_lo + ks * 32, 16, 1024), kIdesc, 1u);
+                        umma_bf16(tmem, umma_smem_desc(a_lo + ks * 32, 16, 1024), bd, kIdesc, 1u);
+                    }
+                }
+                umma_commit(&sh.empty[s]);
+                if (++s == kStages) { s = 0; ++round; }
+            }
+            if (ok && n_units > 0) umma_commit(&sh.accum);
+        }
+    } else {
+        if (n_units > 0) ok = mbar_wait_bounded(&sh.accum, 0);
+        tc_fence_after_sync();
+        if (ok && n_units > 0) {
+            const int co = co0 + (warp & 3) * 32 + lane;
+            const int c_base = (warp >> 2) * (NT / 2);
+            float* out = gwu + (size_t)co * C_in + ci0;
+            const bool vec_ok = (C_in % 4 == 0);
+#pragma unroll 1
+            for (int c = c_base; c < c_base + NT / 2; c += 32) {
+                uint32_t v[32];
+                tmem_ld32(tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)c, v);
+                tmem_ld_wait();
+                if (co < C_out) {
+                    if (vec_ok && ci0 + c + 32 <= C_in) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4) red_add_v4(out + c + i, v[i], v[i + 1], v[i + 2], v[i + 3]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (ci0 + c + i < C_in) atomicAdd(out + c + i, __uint_as_float(v[i]));
+                    }
+                }
+            }
+        }
+    }
+    if (!ok) {
+        atomicOr(p.err_word, 1024u);
+        const long long t0 = clock64();           // copies may still be on their way to this CTA's shared memory
+        while (clock64() - t0 < 2000000LL) {}
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    if (warp == 9) tmem_dealloc(tmem, NT);
+}
+
+// ================================================================== gx_tma
+// Eq. (grad_x) with the patches as the ROWS of the accumulator: D[patch, c_i] = sum_co
+// G-[co, patch] thetaT[c_i, co].  Both operands come through the copy engine (operand rows on
+// 16-byte boundaries): G- as MN-major boxes of 64 patches x 64 c_o of one image, thetaT as K-major
+// boxes of 64 c_o x NT c_i.  A CTA computes 128 patches (two 64-patch units) x NT input channels.
+// A row of the accumulator is a lane of tensor memory, so consecutive lanes hold consecutive
+// patches of a patch row and write neighbouring pixels of a g_X plane: no transposition through
+// shared memory, every warp store covers runs of a pixel row.  Warps 0-7: epilogue; warp 8:
+// copies; warp 9: MMA issue.
+struct GxTmaParams {
+    CUtensorMap tm_g[2];            // gbar [N][C_out][P] bf16: high parts, low parts (fp32 layers)
+    CUtensorMap tm_theta;           // thetaT [part][C_in][C_out] bf16
+    void* gX;
+    uint32_t* err_word;
+    int N, C_in, C_out, H, W, r, Hp, Wp;
+    int P_live, cpi, units_total;   // patches per image, 64-patch units per image and in all
+    int NT, stages;                 // c_i per CTA (multiple of 16, <= 256), ring slots (2..4)
+    FastDiv div_cpi, div_Wp;
+};
+constexpr int kGxTmaThreads = 320;
+constexpr int kGxTmaMaxStages = 4;
+
+struct GxTmaShared {
+    uint64_t full[kGxTmaMaxStages], empty[kGxTmaMaxStages];
+    uint64_t accum;
+    uint32_t tmem_base;
+};
+
+// R: the patch size when every patch is whole and r is 2, 4 or 8 (one vector store per patch and
+// pixel row), else 0 (any r, patches clipped at the right and bottom edges, element-wise stores).
+template <typename TOut, int R, int SPLIT>
+__global__ void __launch_bounds__(kGxTmaThreads) gx_tma_kernel(const __grid_constant__ GxTmaParams p) {
+    constexpr int kABytes = 128 * kTcBK * 2;                // [64 c_o][128 patches] bf16: two 8 KB blocks of 64 patches
+    extern __shared__ unsigned char dyn_raw[];
+    __shared__ GxTmaShared sh;
+    unsigned char* dyn = align1024(dyn_raw);
+    // fields of the parameter block, read once (its address is taken for the tensor maps)
+    const int NT = p.NT, n_stages = p.stages, N = p.N, C_in = p.C_in, H = p.H, W = p.W, r = R > 0 ? R : p.r;
+    const int P_live = p.P_live, units_total = p.units_total;
+    const int k_chunks = (p.C_out + kTcBK - 1) / kTcBK;
+    const FastDiv div_cpi = p.div_cpi, div_Wp = p.div_Wp;
+    TOut* const gX = static_cast<TOut*>(p.gX);
+    const int b_bytes = NT * 128;
+    const int stage_bytes = SPLIT * (kABytes + b_bytes);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int ci0 = blockIdx.x * NT, unit0 = blockIdx.y * 2;
+    const int ng = min(NT, C_in - ci0);
+    int ncols = 32;
+    while (ncols < NT) ncols <<= 1;
+
+    pdl_launch_dependents();
+    if (tid == 0) {
+        for (int s = 0; s < n_stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+        mbar_init(&sh.accum, 1);
+        mbar_fence_init();
+    }
+    if (warp == 9) { tmem_alloc(&sh.tmem_base, (uint32_t)ncols); tmem_relinquish(); }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = sh.tmem_base;
+    pdl_wait();                       // operands come from the previous kernels of the stream
+    bool ok = true;
+
+    if (warp == 8) {
+        if (lane == 0) {
+            // image and first patch of the CTA's two units; a unit past the end reads image N: all zeros
+            int un[2], ux[2];
+#pragma unroll
+            for (int hb = 0; hb < 2; ++hb) {
+                uint32_t n = (uint32_t)N, c = 0;
+                if (unit0 + hb < units_total) div_cpi.divmod((uint32_t)(unit0 + hb), n, c);
+                un[hb] = (int)n;
+                ux[hb] = (int)c * kTcBK;
+            }
+            int s = 0, round = 0;
+            for (int q = 0; q < k_chunks && ok; ++q) {
+                if (round > 0) ok = mbar_wait_bounded(&sh.empty[s], (uint32_t)(round - 1) & 1u);
+                if (!ok) break;
+                unsigned char* stage = dyn + (size_t)s * stage_bytes;
+                mbar_expect_tx(&sh.full[s], (uint32_t)stage_bytes);
+#pragma unroll
+                for (int h = 0; h < SPLIT; ++h) {
+                    tma_load_3d(stage + h * kABytes, &p.tm_g[h], ux[0], q * kTcBK, un[0], &sh.full[s]);
+                    tma_load_3d(stage + h * kABytes + 8192, &p.tm_g[h], ux[1], q * kTcBK, un[1], &sh.full[s]);
+                    tma_load_3d(stage + SPLIT * kABytes + h * b_bytes, &p.tm_theta, q * kTcBK, ci0, h, &sh.full[s]);
+                }
+                if (++s == n_stages) { s = 0; ++round; }
+            }
+        }
+    } else if (warp == 9) {
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_bf16(128, (ng + 15) & ~15, /*A MN-major*/ 1, /*B K-major*/ 0);
+            int s = 0, round = 0;
+            for (int q = 0; q < k_chunks && ok; ++q) {
+                ok = mbar_wait_bounded(&sh.full[s], (uint32_t)round & 1u);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t a_hi = smem_u32(dyn + (size_t)s * stage_bytes), a_lo = a_hi + kABytes;
+                const uint32_t b_hi = a_hi + SPLIT * kABytes, b_lo = b_hi + (uint32_t)b_bytes;
+#pragma unroll
+                for (int ks = 0; ks < kTcBK / 16; ++ks) {
+                    const uint64_t ad = umma_smem_desc(a_hi + ks * 2048, 8192, 1024), bd = umma_smem_desc(b_hi + ks * 32, 16, 1024);
+                    umma_bf16(tmem, ad, bd, idesc, !(q == 0 && ks == 0));
+                    if constexpr (SPLIT == 2) {
+                        umma_bf16(tmem, ad, umma_smem_desc(b_lo + ks * 32, 16, 1024), idesc, 1u);
+                        umma_bf16(tmem, umma_smem_desc(a_lo + ks * 2048, 8192, 1024), bd, idesc, 1u);
+                    }
+                }
+                umma_commit(&sh.empty[s]);
+                if (++s == n_stages) { s = 0; ++round; }
+            }
+            if (ok) umma_commit(&sh.accum);
+        }
+    } else {
+        ok = mbar_wait_bounded(&sh.accum, 0);
+        tc_fence_after_sync();
+        if (ok) {
+            const int quarter = warp & 3, half = warp >> 2;
+            const int row = quarter * 32 + lane;
+            // this lane's patch
+            const int unit = unit0 + (row >> 6);
+            bool live = unit < units_total;
+            uint32_t n = 0, c = 0, a = 0, b = 0;
+            if (live) {
+                div_cpi.divmod((uint32_t)unit, n, c);
+                const int pp = (int)c * kTcBK + (row & 63);
+                live = pp < P_live;
+                if (live) div_Wp.divmod((uint32_t)pp, a, b);
+            }
+            const size_t plane = (size_t)H * W;
+            const int rows = min(r, H - (int)a * r), cols = min(r, W - (int)b * r);
+            TOut* px = gX + ((size_t)n * C_in + ci0) * plane + (size_t)a * r * W + (size_t)b * r;
+            for (int cb = half * 32; cb < ng; cb += 64) {
+                uint32_t v[32];
+                tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)cb, v);
+                tmem_ld_wait();
+                if (live) {
+                    TOut* dst = px + (size_t)cb * plane;
+#pragma unroll
+                    for (int k = 0; k < 32; ++k) {
+                        if (cb + k < ng) {
+                            const float val = __uint_as_float(v[k]);
+                            if constexpr (R > 0) {
+#pragma unroll
+                                for (int dr = 0; dr < R; ++dr) store_rep<R>(dst + (size_t)dr * W, val);
+                            } else {
+                                for (int dr = 0; dr < rows; ++dr)
+                                    for (int dc = 0; dc < cols; ++dc) dst[(size_t)dr * W + dc] = from_f32<TOut>(val);
+                            }
+                        }
+                        dst += plane;
+                    }
+                }
+            }
+        }
+    }
+    if (!ok) {
+        atomicOr(p.err_word, 2048u);
+        const long long t0 = clock64();           // copies may still be on their way to this CTA's shared memory
+        while (clock64() - t0 < 2000000LL) {}
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    if (warp == 9) tmem_dealloc(tmem, (uint32_t)ncols);
+}
+
 // ================================================================== theta sum, transposed bf16
 // thetaT[c_i][c_o] = sum_taps W[c_o][c_i][:], a 32 x 32 tile per block through shared
 // memory so that both the reads (along c_i, taps) and the writes (along c_o) are
@@ -1037,10 +1339,82 @@ static gf_status launch_gx_tc_r(const GxTcParams& p, int R, cudaStream_t s) {
 
 // gbar / thetaT: bf16 arrays; *_lo_off: elements from the high-part to the low-part array
 // (fp32 layers: operands carried as bf16 pairs), 0 for plain bf16 layers.
+// Where the copy-engine pair (gx_tma, gw_tma) replaces the pair with loader warps.  Needed: operand
+// rows on 16-byte boundaries.  Worth it (measured on 16 x 16 ... 128 x 128 maps): long contractions,
+// C_out >= 512, where feeding the tensor cores is what limits the loader-warp kernels (512 -> 2048
+// channels on 8 x 8 patches: 431 -> 343 us fp32, 213 -> 159 us bf16); with short contractions the
+// r x r expansion dominates, and the staged epilogue of gx_tc writes it faster (256 channels, r = 4:
+// 50 against 67 us).  64-patch units must be at least three quarters full: 4 x 4 patches would fill
+// a quarter of a unit, and the kernels would move and multiply mostly zeros.  Both kernels of a
+// layer take the same decision: a persistent kernel beside a non-persistent one starves.
+static bool tma_units_pay(const Geo& g) {
+    const int P_live = g.Hp * g.Wp, cpi = (P_live + kTcBK - 1) / kTcBK;
+    return tc_pitch(g) % 8 == 0 && g.C_out >= 512 && (long long)P_live * 4 >= (long long)cpi * kTcBK * 3;
+}
+
+template <typename TOut, int R, int SPLIT>
+static gf_status launch_gx_tma_inst(const GxTmaParams& p, dim3 grid, cudaStream_t s) {
+    const size_t smem = (size_t)p.stages * SPLIT * (128 * kTcBK * 2 + (size_t)p.NT * 128) + 1024;
+    static size_t configured[kMaxDevices] = {};
+    if (gf_status st = ensure_dyn_smem(gx_tma_kernel<TOut, R, SPLIT>, smem, configured); st != GF_OK) return st;
+    return launch_pdl(gx_tma_kernel<TOut, R, SPLIT>, grid, dim3(kGxTmaThreads), smem, s, p);
+}
+template <typename TOut, int SPLIT>
+static gf_status launch_gx_tma_r(const GxTmaParams& p, int R, dim3 grid, cudaStream_t s) {
+    switch (R) {
+        case 2: return launch_gx_tma_inst<TOut, 2, SPLIT>(p, grid, s);
+        case 4: return launch_gx_tma_inst<TOut, 4, SPLIT>(p, grid, s);
+        case 8: return launch_gx_tma_inst<TOut, 8, SPLIT>(p, grid, s);
+        default: return launch_gx_tma_inst<TOut, 0, SPLIT>(p, grid, s);
+    }
+}
+
+// The copy-engine variant, when the operand rows are 16-byte aligned and the units are well
+// filled.  false: not applicable.
+static bool try_launch_gx_tma(const __nv_bfloat16* gbar, long long gbar_lo_off, const __nv_bfloat16* thetaT,
+                              long long theta_lo_off, void* gX, uint32_t* err_word, const Geo& g, cudaStream_t s,
+                              gf_status* st) {
+    const bool split = g.dtype == GF_F32;
+    const int parts = split ? 2 : 1;
+    if (!tma_units_pay(g) || g.C_out % 8 != 0 || (split && (gbar_lo_off % 8 != 0 || theta_lo_off % 8 != 0))) return false;
+    GxTmaParams p;
+    const int pitch = tc_pitch(g);
+    p.P_live = g.Hp * g.Wp;
+    p.cpi = (p.P_live + kTcBK - 1) / kTcBK;
+    const long long units = (long long)g.N * p.cpi;
+    if ((units + 1) / 2 > 65535) return false;
+    p.units_total = (int)units;
+    // c_i per CTA: as wide as tensor memory and the ring allow (256), in equal parts
+    const int n_ci = (g.C_in + 255) / 256;
+    p.NT = ((g.C_in + n_ci - 1) / n_ci + 15) / 16 * 16;
+    const size_t stage = (size_t)parts * (128 * kTcBK * 2 + (size_t)p.NT * 128);
+    int st_n = (int)((size_t)100 * 1024 / stage);                        // two CTAs per SM where two slots fit in that
+    p.stages = st_n < 2 ? 2 : st_n > kGxTmaMaxStages ? kGxTmaMaxStages : st_n;
+    for (int h = 0; h < parts; ++h)
+        if (!make_tmap_bf16(&p.tm_g[h], gbar + h * gbar_lo_off, 3, (uint64_t)p.P_live, (uint64_t)g.C_out, (uint64_t)g.N,
+                            (uint64_t)pitch, (uint64_t)g.C_out * pitch, 64))
+            return false;
+    if (!split) p.tm_g[1] = p.tm_g[0];
+    if (!make_tmap_bf16(&p.tm_theta, thetaT, 3, (uint64_t)g.C_out, (uint64_t)g.C_in, (uint64_t)parts, (uint64_t)g.C_out,
+                        split ? (uint64_t)theta_lo_off : (uint64_t)g.C_in * g.C_out, (uint32_t)p.NT))
+        return false;
+    p.gX = gX; p.err_word = err_word;
+    p.N = g.N; p.C_in = g.C_in; p.C_out = g.C_out; p.H = g.H; p.W = g.W; p.r = g.r; p.Hp = g.Hp; p.Wp = g.Wp;
+    p.div_cpi = FastDiv((uint32_t)p.cpi);
+    p.div_Wp = FastDiv((uint32_t)g.Wp);
+    const int R = ((g.r == 2 || g.r == 4 || g.r == 8) && g.H % g.r == 0 && g.W % g.r == 0) ? g.r : 0;
+    const dim3 grid((unsigned)((g.C_in + p.NT - 1) / p.NT), (unsigned)((units + 1) / 2), 1);
+    if (split) *st = launch_gx_tma_r<float, 2>(p, R, grid, s);
+    else *st = launch_gx_tma_r<__nv_bfloat16, 1>(p, R, grid, s);
+    return true;
+}
+
 gf_status launch_gx_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const __nv_bfloat16* thetaT,
                        long long theta_lo_off, void* gX, int max_ctas, uint32_t* err_word, const Geo& g,
                        cudaStream_t s) {
     ProfScope prof(K_GX_TC, s);
+    gf_status st_tma = GF_OK;
+    if (try_launch_gx_tma(gbar, gbar_lo_off, thetaT, theta_lo_off, gX, err_word, g, s, &st_tma)) return st_tma;
     GxTcParams p;
     const int P = tc_pitch(g);                      // gbar's plane pitch
     p.P_live = g.Hp * g.Wp;
@@ -1099,10 +1473,59 @@ static gf_status launch_gw_tc_v(const GwTcParams& p, dim3 grid, cudaStream_t s) 
     }
 }
 
+template <int NT, int SPLIT>
+static gf_status launch_gw_tma_inst(const GwTmaParams& p, dim3 grid, cudaStream_t s) {
+    constexpr size_t smem = (size_t)gw_stages(SPLIT, NT) * SPLIT * (128 * kTcBK * 2 + NT * kTcBK * 2) + 1024;
+    static size_t configured[kMaxDevices] = {};
+    if (gf_status st = ensure_dyn_smem(gw_tma_kernel<NT, SPLIT>, smem, configured); st != GF_OK) return st;
+    return launch_pdl(gw_tma_kernel<NT, SPLIT>, grid, dim3(kGwTmaThreads), smem, s, p);
+}
+
+// The copy-engine variant, when the operand rows are 16-byte aligned.  false: not applicable.
+static bool try_launch_gw_tma(const __nv_bfloat16* gbar, long long gbar_lo_off, const __nv_bfloat16* stash,
+                              long long stash_lo_off, float* gwu, int splits, uint32_t* err_word, const Geo& g,
+                              cudaStream_t s, gf_status* st) {
+    const int pitch = tc_pitch(g), NT = gw_tile_n(g);
+    const bool split = g.dtype == GF_F32;
+    if (!tma_units_pay(g) || (split && (gbar_lo_off % 8 != 0 || stash_lo_off % 8 != 0))) return false;
+    GwTmaParams p;
+    const int P_live = g.Hp * g.Wp;
+    for (int h = 0; h < (split ? 2 : 1); ++h) {
+        if (!make_tmap_bf16(&p.tm_a[h], gbar + h * gbar_lo_off, 3, (uint64_t)P_live, (uint64_t)g.C_out, (uint64_t)g.N,
+                            (uint64_t)pitch, (uint64_t)g.C_out * pitch, 128) ||
+            !make_tmap_bf16(&p.tm_b[h], stash + h * stash_lo_off, 3, (uint64_t)P_live, (uint64_t)g.C_in, (uint64_t)g.N,
+                            (uint64_t)pitch, (uint64_t)g.C_in * pitch, (uint32_t)NT))
+            return false;
+    }
+    if (!split) { p.tm_a[1] = p.tm_a[0]; p.tm_b[1] = p.tm_b[0]; }
+    p.gwu = gwu; p.err_word = err_word; p.C_in = g.C_in; p.C_out = g.C_out; p.P_live = P_live;
+    p.cpi = (P_live + kTcBK - 1) / kTcBK;
+    const long long units = (long long)g.N * p.cpi;
+    if (units > 0x7fffffffLL) return false;
+    p.units_total = (int)units;
+    p.div_cpi = FastDiv((uint32_t)p.cpi);
+    // slices of the contraction: enough CTAs for every SM (the kernel shares them with whatever runs
+    // beside it CTA by CTA; it is not a persistent kernel with a share of its own)
+    (void)splits;
+    const int tiles = ((g.C_in + NT - 1) / NT) * ((g.C_out + 127) / 128);
+    int S = (sm_count() + tiles - 1) / tiles;
+    if (S > p.units_total) S = p.units_total;
+    if (S > 65535) S = 65535;
+    p.S = S < 1 ? 1 : S;
+    dim3 grid((g.C_in + NT - 1) / NT, (g.C_out + 127) / 128, p.S);
+    if (split) *st = launch_gw_tma_inst<128, 2>(p, grid, s);
+    else if (NT == 256) *st = launch_gw_tma_inst<256, 1>(p, grid, s);
+    else *st = launch_gw_tma_inst<128, 1>(p, grid, s);
+    return true;
+}
+
 gf_status launch_gw_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const __nv_bfloat16* stash,
                        long long stash_lo_off, float* gwu, int splits, uint32_t* err_word, const Geo& g,
                        cudaStream_t s) {
     ProfScope prof(K_GW_TC, s);
+    if ((g.C_out + 127) / 128 > 65535 || splits > 65535) return GF_ERR_UNSUPPORTED;
+    gf_status st_tma = GF_OK;
+    if (try_launch_gw_tma(gbar, gbar_lo_off, stash, stash_lo_off, gwu, splits, err_word, g, s, &st_tma)) return st_tma;
     const int NT = gw_tile_n(g);
     GwTcParams p;
     const int P = tc_pitch(g);                      // plane pitch of both operands; gaps hold zeros

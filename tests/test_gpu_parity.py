@@ -81,6 +81,14 @@ SMALL = [
     L("pitch_r4_28x28", 2, 24, 16, 28, 28, 1, 1, 4),        # 7x7 patches
     L("pitch_wide_rows", 1, 8, 8, 6, 118, 3, 1, 2),         # 3x59 patches: rows too wide for a row tile
     L("pitch_many_images", 37, 136, 72, 14, 14, 1, 1, 2),   # 7x7 patches, two c_i tiles, many items per CTA
+    # long contractions (C_out >= 512) on patch planes whose rows start on 16-byte boundaries: both
+    # operands of both contractions through the copy engine, 64-patch units
+    L("tma_pair_r2", 3, 72, 520, 16, 24, 1, 1, 2),          # 96 patches: units 3/4 full; ragged contraction tail
+    L("tma_pair_generic_r3", 2, 264, 512, 24, 24, 3, 1, 3), # r = 3: element-wise stores; two c_i tiles
+    L("tma_pair_partial", 2, 16, 512, 15, 31, 1, 1, 2),     # clipped patches at the right and bottom edges
+    L("tma_pair_r8", 2, 24, 512, 64, 64, 1, 1, 8),
+    L("tma_pair_r4_multi_ci", 2, 520, 512, 32, 32, 1, 1, 4),  # three c_i tiles of 176
+    L("tma_pair_odd_units", 5, 40, 640, 16, 16, 3, 1, 2),   # five units: the last CTA's second unit is empty
 ]
 
 
