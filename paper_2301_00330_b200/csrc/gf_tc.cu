@@ -1504,11 +1504,12 @@ static bool try_launch_gw_tma(const __nv_bfloat16* gbar, long long gbar_lo_off, 
     if (units > 0x7fffffffLL) return false;
     p.units_total = (int)units;
     p.div_cpi = FastDiv((uint32_t)p.cpi);
-    // slices of the contraction: enough CTAs for every SM (the kernel shares them with whatever runs
-    // beside it CTA by CTA; it is not a persistent kernel with a share of its own)
+    // slices of the contraction: as many as give every SM at most one CTA (a second, partly filled
+    // round of CTAs costs as much as a full one).  The kernel shares the SMs with whatever runs
+    // beside it CTA by CTA; it is not a persistent kernel with a share of its own.
     (void)splits;
     const int tiles = ((g.C_in + NT - 1) / NT) * ((g.C_out + 127) / 128);
-    int S = (sm_count() + tiles - 1) / tiles;
+    int S = sm_count() / tiles;
     if (S > p.units_total) S = p.units_total;
     if (S > 65535) S = 65535;
     p.S = S < 1 ? 1 : S;
