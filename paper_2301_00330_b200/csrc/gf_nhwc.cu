@@ -478,6 +478,7 @@ bool nhwc_supported(const Geo& g, int stride) {
     if (g.G != 1 && !depthwise) return false;
     if (depthwise && (g.C_in > 12288 || dw_unit(g.C_in) > kDwMaxBlocks)) return false;
     const long long M = (long long)g.N * g.Hp * g.Wp;
+    if (!depthwise && (M + 127) / 128 > 65535) return false;          // row tiles of the g_X kernel: one grid dimension
     return M * (g.C_in > g.C_out ? g.C_in : g.C_out) / 8 < 0x7fffffffLL && (long long)g.N * g.H < 0x7fffffffLL;
 }
 
@@ -611,7 +612,6 @@ gf_status nhwc_backward(const Geo& g, const void* g_y, const void* stash, const 
                             split ? (uint64_t)theta_lo : (uint64_t)g.C_in * g.C_out, (uint32_t)p.NT))
             return GF_ERR_CUDA;
         const dim3 grid((unsigned)((g.C_in + p.NT - 1) / p.NT), (unsigned)((M + 127) / 128), 1);
-        if (grid.y > 65535) return GF_ERR_UNSUPPORTED;
         if (g.dtype == GF_F32) st = launch_nhwc_gx<float, 2>(p, grid, s);
         else st = launch_nhwc_gx<__nv_bfloat16, 1>(p, grid, s);
         if (st != GF_OK) return st;
