@@ -1340,16 +1340,21 @@ static gf_status launch_gx_tc_r(const GxTcParams& p, int R, cudaStream_t s) {
 // gbar / thetaT: bf16 arrays; *_lo_off: elements from the high-part to the low-part array
 // (fp32 layers: operands carried as bf16 pairs), 0 for plain bf16 layers.
 // Where the copy-engine pair (gx_tma, gw_tma) replaces the pair with loader warps.  Needed: operand
-// rows on 16-byte boundaries.  Worth it (measured on 16 x 16 ... 128 x 128 maps): long contractions,
-// C_out >= 512, where feeding the tensor cores is what limits the loader-warp kernels (512 -> 2048
-// channels on 8 x 8 patches: 431 -> 343 us fp32, 213 -> 159 us bf16); with short contractions the
-// r x r expansion dominates, and the staged epilogue of gx_tc writes it faster (256 channels, r = 4:
-// 50 against 67 us).  64-patch units must be at least three quarters full: 4 x 4 patches would fill
-// a quarter of a unit, and the kernels would move and multiply mostly zeros.  Both kernels of a
-// layer take the same decision: a persistent kernel beside a non-persistent one starves.
+// rows on 16-byte boundaries, and 64-patch units at least three quarters full (4 x 4 patches would
+// fill a quarter of a unit: the kernels would move and multiply mostly zeros).  Worth it (measured
+// on 16 x 16 ... 128 x 128 maps): long contractions, C_out >= 512, where feeding the tensor cores is
+// what limits the loader-warp kernels (512 -> 2048 channels on 8 x 8 patches: 431 -> 316 us fp32,
+// 213 -> 146 us bf16); and layers with at least 1.5 row tiles of 128 patches per SM (256 channels
+// on 40 x 30 patches, N = 32: 129 -> 118 us).  With fewer tiles than that and a short contraction
+// the r x r expansion dominates and gx_tc, whose epilogue overlaps the next tile's contraction,
+// is faster (512 -> 256 channels, 32 x 32 patches, N = 8, r = 4: 57 against 69 us).  The rule reads
+// only what the two kernels of a layer see alike (N, patch grid, C_out), so that both take the same
+// decision: a persistent kernel beside a non-persistent one starves.
 static bool tma_units_pay(const Geo& g) {
     const int P_live = g.Hp * g.Wp, cpi = (P_live + kTcBK - 1) / kTcBK;
-    return tc_pitch(g) % 8 == 0 && g.C_out >= 512 && (long long)P_live * 4 >= (long long)cpi * kTcBK * 3;
+    if (tc_pitch(g) % 8 != 0 || (long long)P_live * 4 < (long long)cpi * kTcBK * 3) return false;
+    const long long row_tiles = ((long long)g.N * cpi + 1) / 2;
+    return (g.C_out >= 512 && row_tiles >= 64) || 2 * row_tiles >= 3LL * sm_count();
 }
 
 template <typename TOut, int R, int SPLIT>
