@@ -216,6 +216,9 @@ gf_status launch_repack(const void* in, int in_dtype, __nv_bfloat16* hi, __nv_bf
 // beside_pool: launched right behind the gradient-filter pooling kernel, works next to it
 gf_status launch_ksum_t(const void* W, const Geo& g, __nv_bfloat16* thetaT, __nv_bfloat16* thetaT_lo, float* gwu,
                         bool beside_pool, cudaStream_t s);
+// true: the two contractions of this layer run as the copy-engine pair (non-persistent kernels that
+// share the SMs CTA by CTA), false: as the persistent pair, each on its share of the SMs
+bool tc_copy_engine_pair(const Geo& g);
 gf_status launch_split_f32(const float* in, __nv_bfloat16* hi, __nv_bfloat16* lo, size_t n, cudaStream_t s);
 // max_ctas: CTAs the kernel may use (0: one per SM)
 gf_status launch_gx_tc(const __nv_bfloat16* gbar, long long gbar_lo_off, const __nv_bfloat16* thetaT,

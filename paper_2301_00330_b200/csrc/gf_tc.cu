@@ -1357,6 +1357,8 @@ static bool tma_units_pay(const Geo& g) {
     return (g.C_out >= 512 && row_tiles >= 64) || 2 * row_tiles >= 3LL * sm_count();
 }
 
+bool tc_copy_engine_pair(const Geo& g) { return tma_units_pay(g); }
+
 template <typename TOut, int R, int SPLIT>
 static gf_status launch_gx_tma_inst(const GxTmaParams& p, dim3 grid, cudaStream_t s) {
     const size_t smem = (size_t)p.stages * SPLIT * (128 * kTcBK * 2 + (size_t)p.NT * 128) + 1024;
