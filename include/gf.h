@@ -42,9 +42,10 @@
  *    The paper's formulas index channels and pixels and fix no memory order;
  *    the results are those of NCHW, permuted.  Channels-last is supported for
  *    gf_stash_forward, gf_backward, gf_backward_static_scratch and
- *    gf_layer_step_host (whose host buffers then have that order too) with r >= 2,
+ *    gf_layer_step_host (whose host buffers then have that order too): with
+ *    r == 1 (exact backward) in every geometry NCHW has; with r >= 2 for
  *    stride 1, C_in and C_out multiples of 8, and groups == 1 or a depthwise
- *    layer (groups == C_in == C_out, at most 12288 channels); other channels-last
+ *    layer (groups == C_in == C_out, at most 12288 channels).  Other channels-last
  *    descriptors, and every other call given one, return GF_ERR_UNSUPPORTED.
  *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Work
  *    is enqueued on it and the call returns without synchronising.  Errors that

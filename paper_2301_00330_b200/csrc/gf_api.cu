@@ -102,8 +102,9 @@ static gf_status validate(const gf_conv_desc* d) {
     if ((int64_t)d->N * d->C_in > (int64_t)1 << 30 || (int64_t)d->N * d->C_out > (int64_t)1 << 30)
         return GF_ERR_UNSUPPORTED;
     if ((int64_t)d->C_out * (d->C_in / d->groups) * d->KH * d->KW > (int64_t)1 << 30) return GF_ERR_UNSUPPORTED;
-    // channels-last: stride 1, r >= 2, channel counts in multiples of 8, dense or depthwise
-    if (d->layout == GF_NHWC && (d->r < 2 || !nhwc_supported(make_geo(*d), d->stride))) return GF_ERR_UNSUPPORTED;
+    // channels-last: r == 1 (exact backward) as for NCHW; r >= 2: stride 1, channel counts in multiples of
+    // 8, dense or depthwise
+    if (d->layout == GF_NHWC && d->r >= 2 && !nhwc_supported(make_geo(*d), d->stride)) return GF_ERR_UNSUPPORTED;
     return GF_OK;
 }
 
@@ -303,7 +304,7 @@ gf_status gf_backward_workspace_bytes(const gf_conv_desc* desc, size_t* bytes) {
     gf_status st = validate(desc);
     if (st != GF_OK) return st;
     const Geo g = make_geo(*desc);
-    if (desc->layout == GF_NHWC) { *bytes = nhwc_workspace_bytes(g); return GF_OK; }
+    if (desc->layout == GF_NHWC && g.r > 1) { *bytes = nhwc_workspace_bytes(g); return GF_OK; }
     *bytes = (desc->stride > 1 && g.r > 1) ? plan_strided(g, desc->stride).total : plan_workspace(g).total;
     return GF_OK;
 }
@@ -316,7 +317,7 @@ gf_status gf_stash_forward(const gf_conv_desc* desc, const void* x, void* stash,
     const Geo g = make_geo(*desc);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int64_t planes = (int64_t)g.N * g.C_in;
-    if (desc->layout == GF_NHWC) return launch_nhwc_stash(x, stash, g, s);
+    if (desc->layout == GF_NHWC && g.r > 1) return launch_nhwc_stash(x, stash, g, s);
     if (g.r == 1) return launch_copy(x, stash, (size_t)planes * g.H * g.W * g.esize, s);
     uint32_t* err = global_err_word();
     if (!err) return GF_ERR_CUDA;
@@ -420,7 +421,7 @@ gf_status backward_impl(const gf_conv_desc* desc, const void* g_y, const void* s
     const Geo g = make_geo(*desc);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     char* base = static_cast<char*>(workspace);
-    if (desc->layout == GF_NHWC) {
+    if (desc->layout == GF_NHWC && g.r > 1) {
         if (workspace_bytes < nhwc_workspace_bytes(g)) return GF_ERR_WORKSPACE;
         if (!g_W && !g_X) return GF_OK;
         return nhwc_backward(g, g_y, stash, W, g_W, g_X, base, s);
@@ -526,7 +527,7 @@ gf_status backward_impl(const gf_conv_desc* desc, const void* g_y, const void* s
     // The error word is cleared here, ahead of every kernel of the call that may set it.
     GF_CUDA_TRY(cudaMemsetAsync(err, 0, sizeof(uint32_t), s));
 
-    if (g.r == 1) return launch_exact(g_y, stash, W, g_W, g_X, g, desc->stride, s);
+    if (g.r == 1) return launch_exact(g_y, stash, W, g_W, g_X, g, desc->stride, desc->layout == GF_NHWC, s);
 
     float* tsum = reinterpret_cast<float*>(base + ws.off_tsum);
     float* gbar = reinterpret_cast<float*>(base + ws.off_gbar);

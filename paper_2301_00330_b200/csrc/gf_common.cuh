@@ -245,8 +245,8 @@ size_t nhwc_workspace_bytes(const Geo& g);
 gf_status launch_nhwc_stash(const void* x, void* stash, const Geo& g, cudaStream_t s);
 gf_status nhwc_backward(const Geo& g, const void* g_y, const void* stash, const void* W, float* g_W, void* g_X, char* base,
                         cudaStream_t s);
-gf_status launch_exact(const void* gy, const void* x, const void* W, float* gW, void* gX,
-                       const Geo& g, int stride, cudaStream_t s);
+gf_status launch_exact(const void* gy, const void* x, const void* W, float* gW, void* gX, const Geo& g, int stride,
+                       bool channels_last, cudaStream_t s);
 // strided layers (gf_strided.cu): per-phase kernel sums, rows of s*s*C_ig values per output channel
 gf_status launch_ksum_phase(const void* W, int dtype, int C_out, int C_ig, int KH, int KW, int stride, float* tph, cudaStream_t s);
 // gX[n, c, h, w] <- ghat[n, (group, phase of (h, w), channel in group), h / (r s), w / (r s)]

@@ -96,13 +96,14 @@ def test_descriptor_validation(gf):
     assert st(groups=3) == gf.GF_ERR_BAD_DESC
     assert st(dtype=7) == gf.GF_ERR_BAD_DESC
     assert st(layout=5) == gf.GF_ERR_BAD_DESC
-    # channels-last: stride 1, r >= 2, channel counts in multiples of 8, dense or depthwise
+    # channels-last with r >= 2: stride 1, channel counts in multiples of 8, dense or depthwise
     assert st(layout=gf.GF_NHWC) == gf.GF_OK
     assert st(layout=gf.GF_NHWC, groups=8) == gf.GF_OK
     assert st(layout=gf.GF_NHWC, C_in=12, C_out=12) == gf.GF_ERR_UNSUPPORTED
     assert st(layout=gf.GF_NHWC, groups=2) == gf.GF_ERR_UNSUPPORTED
     assert st(layout=gf.GF_NHWC, stride=2) == gf.GF_ERR_UNSUPPORTED
-    assert st(layout=gf.GF_NHWC, r=1) == gf.GF_ERR_UNSUPPORTED
+    assert st(layout=gf.GF_NHWC, r=1) == gf.GF_OK                  # exact backward: as for NCHW
+    assert st(layout=gf.GF_NHWC, r=1, C_in=12, C_out=12, groups=2) == gf.GF_OK
     assert st(stride=2) == gf.GF_OK                          # s | H and s | W: g_y is [H/s, W/s]
     assert st(stride=3) == gf.GF_ERR_UNSUPPORTED             # 3 does not divide 8
     assert st(stride=0) == gf.GF_ERR_BAD_DESC

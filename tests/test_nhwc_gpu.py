@@ -139,6 +139,38 @@ def test_nhwc_nullable_outputs(gf):
     assert torch.equal(gx_a, gx_c)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shape", [(2, 8, 12, 9, 7, 3, 2, 1), (1, 4, 4, 8, 8, 5, 1, 1), (2, 6, 6, 8, 8, 3, 6, 1),
+                                   (2, 6, 10, 8, 12, 3, 1, 2)], ids=["groups2", "k5", "depthwise", "stride2"])
+def test_nhwc_r1_is_the_exact_backward(gf, shape, dtype):
+    """r = 1 switches the method off (Section 4.2): the exact backward, here on channels-last tensors,
+    any channel count, groups and dividing stride."""
+    N, Cin, Cout, H, W, K, G, stride = shape
+    layer = Layer("nhwc_r1", 0, 0, N, Cin, Cout, H, W, K, G, 1, dtype, "normal", 1.0)
+    x, gy, w = workloads.make_inputs(layer)
+    gy = gy[:, :, ::stride, ::stride].contiguous()
+    desc = gf.make_desc(N, Cin, Cout, H, W, K, r=1, groups=G, stride=stride,
+                        dtype=gf.GF_F32 if dtype == "f32" else gf.GF_BF16, layout=gf.GF_NHWC)
+    dt = workloads.torch_dtype(dtype)
+    stash = Guarded((N, H, W, Cin), dt)
+    gf.gf_stash_forward(desc, nhwc(x).cuda(), stash.t)
+    assert torch.equal(stash.t.cpu(), nhwc(x))                     # the stash is x itself
+    gW = Guarded((Cout, Cin // G, K, K), torch.float32)
+    gX = Guarded((N, H, W, Cin), dt)
+    ws_bytes = gf.gf_backward_workspace_bytes(desc)
+    ws = Guarded((ws_bytes,), torch.uint8)
+    gf.gf_backward(desc, nhwc(gy).cuda(), stash.t, w.cuda(), gW.t, gX.t, ws.t, ws_bytes)
+    assert gf.gf_last_async_status(ws.t) == gf.GF_OK
+    torch.cuda.synchronize()
+    for g in (stash, gW, gX, ws):
+        g.check()
+    if stride == 1:
+        gw_ref, gx_ref = oracle.exact_backward(f64(x), f64(gy), f64(w), groups=G, pad=(K - 1) // 2)
+    else:
+        gw_ref, gx_ref = oracle.exact_backward_strided(f64(x), f64(gy), f64(w), stride, groups=G, pad=(K - 1) // 2)
+    assert relerr(f64(gW.t), gw_ref) <= TOL[dtype] and relerr(f64(nchw_of(gX.t)), gx_ref) <= TOL[dtype]
+
+
 def test_nhwc_static_scratch_and_host_step(gf):
     """The two other entry points that take a channels-last descriptor give the results of gf_backward."""
     layer = L("other_calls", 2, 24, 40, 14, 14, 3, 1, 2)
@@ -176,4 +208,5 @@ def test_nhwc_unsupported_shapes_are_refused(gf):
     assert status(C_out=20) == gf.GF_ERR_UNSUPPORTED
     assert status(groups=2) == gf.GF_ERR_UNSUPPORTED                # dense or depthwise only
     assert status(stride=2) == gf.GF_ERR_UNSUPPORTED
-    assert status(r=1) == gf.GF_ERR_UNSUPPORTED
+    assert status(r=1) == gf.GF_OK                                  # exact backward: as for NCHW
+    assert status(r=1, C_in=12, groups=2, stride=2) == gf.GF_OK
