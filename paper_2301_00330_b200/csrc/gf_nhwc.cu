@@ -117,21 +117,6 @@ struct NxShared {
     uint32_t tmem_base;
 };
 
-// Named barrier `id` over `nthreads` threads that also tells every one of them whether any of them
-// passed a true predicate (a wait that ran out): nobody is left alone at a later barrier.
-__device__ __forceinline__ bool nx_bar_any(int id, int nthreads, bool pred) {
-    uint32_t r;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.u32 q, %1, 0;\n\t"
-        "bar.red.or.pred p, %2, %3, q;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(r)
-        : "r"((uint32_t)pred), "r"(id), "r"(nthreads)
-        : "memory");
-    return r != 0;
-}
-
 // 8 consecutive accumulator values of a row as 8 output elements in the staging tile
 __device__ __forceinline__ void stage8(float* dst, const uint32_t* v) {
     reinterpret_cast<uint4*>(dst)[0] = make_uint4(v[0], v[1], v[2], v[3]);
@@ -238,7 +223,7 @@ __global__ void __launch_bounds__(kNxThreads) nhwc_gx_kernel(const __grid_consta
                     if (k < n8) stage8(reinterpret_cast<TOut*>(row) + c + 8 * k, v + 8 * k);
             }
         }
-        const bool bad = nx_bar_any(1, kNxEpiWarps * 32, !ok);
+        const bool bad = bar_any(1, kNxEpiWarps * 32, !ok);
         if (!bad) {
             const int m_end = min(128, M - m0);
             for (int ml = warp; ml < m_end; ml += kNxEpiWarps) {

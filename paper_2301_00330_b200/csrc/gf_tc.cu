@@ -16,6 +16,13 @@
 // contraction and the stores of consecutive tiles overlap.  gw_tc computes one
 // 128 x 128 tile of one batch slice per CTA and adds it to the unique-value matrix
 // with vector reductions (the order of the additions is not fixed).
+//
+//   gx_tma, gw_tma   the same two contractions with both operands fetched by the copy engine
+//           (tensor maps over the [N][C][P] arrays, units of 64 patches of one image), one
+//           output tile per CTA, for long contractions and for layers with many row tiles
+//           (tma_units_pay states the rule and the measurements behind it).  gx_tma turns
+//           the product around -- D[patch, c_i], the patches as accumulator rows -- so that
+//           consecutive lanes write neighbouring pixels and no transposition is needed.
 // Every wait is bounded: on expiry the CTA sets the error word, frees its tensor memory
 // and returns.
 #include "gf_common.cuh"
