@@ -708,6 +708,10 @@ def run_ours(args) -> None:
     n_dom, ms_dom = dom.get(dom_kernel, (0, 0.0))
     roof = roofline_step(dom_kernel, ms_dom, n_dom, dom_steps, layers)
     roof["timed_launches"] = n_dom
+    if dom_kernel == "stash_pool":
+        roof["cuda_kernel"] = ("pool_stream_kernel: four launches per step, three as the stash pass (this entry) and one as the "
+                               "gradient filter of the 96->576 layer (entry gy_pool of `kernels`); by the ncu launch list the "
+                               "four together are the largest share of the step (profiles/launch_list_bench_step_*.md)")
     roof["timing"] = dom_method
     if dom_pairs[0]:
         roof["avg_launch_us_event_pairs"] = dom_pairs[1] * 1e3 / dom_pairs[0]
@@ -736,7 +740,8 @@ def run_ours(args) -> None:
             sets.clear()
         runs.clear()
         torch.cuda.empty_cache()
-        line["extras"] = extras(gf, layers)
+        if not args.no_extras:
+            line["extras"] = extras(gf, layers)
         line["cpu_baseline"] = time_oracle(layers, 32, 2, 1)
         if not args.no_per_config:
             rows = [time_layer(gf, L, peaks) for L in per_config_layers()]
@@ -790,6 +795,7 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-per-config", action="store_true", help="skip the per_config rows (faster)")
+    ap.add_argument("--no-extras", action="store_true", help="skip the timings of the further entry points")
     ap.add_argument("--table", action="store_true", help="time every layer shape once (diagnostic table)")
     ap.add_argument("--only", default="", help="--table: comma-separated substrings of name/rR/dtype to keep")
     ap.add_argument("--no-exact", action="store_true", help="--table: skip the exact cuDNN backward")
