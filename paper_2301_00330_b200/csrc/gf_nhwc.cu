@@ -135,8 +135,7 @@ __global__ void __launch_bounds__(kNxThreads) nhwc_gx_kernel(const __grid_consta
     extern __shared__ unsigned char dyn_raw[];
     __shared__ NxShared sh;
     unsigned char* dyn = align1024(dyn_raw);
-    // The parameter block's address is taken (the tensor maps), so its fields are read once here
-    // into registers: reads through it inside the loops would be loads from memory every time.
+    // the fields the loops below need, read once
     const int NT = p.NT, n_stages = p.stages, k_chunks = p.k_chunks, M = p.M, C_in = p.C_in, H = p.H, W = p.W, r = p.r;
     const FastDiv div_Wp = p.div_Wp, div_Hp = p.div_Hp;
     TOut* const gX = static_cast<TOut*>(p.gX);
@@ -262,7 +261,7 @@ __global__ void __launch_bounds__(kNxThreads) nhwc_gw_kernel(const __grid_consta
     __shared__ NxShared sh;
     unsigned char* dyn = align1024(dyn_raw);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int C_in = p.C_in, C_out = p.C_out;                       // read once: see nhwc_gx_kernel
+    const int C_in = p.C_in, C_out = p.C_out;
     float* const gwu = p.gwu;
     const int ci0 = blockIdx.x * 128, co0 = blockIdx.y * 128, split = blockIdx.z;
     const int kc_begin = (int)((long long)p.k_chunks * split / p.S), kc_end = (int)((long long)p.k_chunks * (split + 1) / p.S);

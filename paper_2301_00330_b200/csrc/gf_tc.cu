@@ -731,7 +731,7 @@ __global__ void __launch_bounds__(kGwTmaThreads) gw_tma_kernel(const __grid_cons
     unsigned char* dyn = align1024(dyn_raw);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    // fields of the parameter block, read once (its address is taken for the tensor maps)
+    // the fields the loops below need, read once
     const int C_in = p.C_in, C_out = p.C_out, cpi = p.cpi, P_live = p.P_live;
     const FastDiv div_cpi = p.div_cpi;
     float* const gwu = p.gwu;
@@ -871,7 +871,7 @@ __global__ void __launch_bounds__(kGxTmaThreads) gx_tma_kernel(const __grid_cons
     extern __shared__ unsigned char dyn_raw[];
     __shared__ GxTmaShared sh;
     unsigned char* dyn = align1024(dyn_raw);
-    // fields of the parameter block, read once (its address is taken for the tensor maps)
+    // the fields the loops below need, read once
     const int NT = p.NT, n_stages = p.stages, N = p.N, C_in = p.C_in, H = p.H, W = p.W, r = R > 0 ? R : p.r;
     const int P_live = p.P_live, units_total = p.units_total;
     const int k_chunks = (p.C_out + kTcBK - 1) / kTcBK;
