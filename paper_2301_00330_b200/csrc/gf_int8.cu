@@ -314,9 +314,9 @@ __global__ void __launch_bounds__(kI8Threads) i8_gemm_kernel(const __grid_consta
                     tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c, v);
                     tmem_ld_wait();
                     if (m < p.M) {
-#pragma unroll 4
-                        for (int i = 0; i < 32; ++i) {
-                            if (n0 + c + i >= p.N) break;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {            // unrolled in full: v[] stays in registers
+                            if (n0 + c + i >= p.N) continue;
                             const float val = __fmul_rn((float)(int32_t)v[i], scale);
                             TOut* dst = base + (size_t)(n0 + c + i) * plane;
                             if (vec) {
