@@ -672,6 +672,9 @@ def run_ours(args) -> None:
     # one stream per layer: each layer's copies in, kernels and copies out are ordered on its own
     # stream, so the uploads of one layer overlap the downloads of another (the two copy directions
     # use different engines); the timed region opens and closes on the main stream
+    # and the layer with the most to download goes first, so that its download runs under the other
+    # layers' uploads instead of after them
+    e2e_sets.sort(key=lambda t: -(t[4].numel() * t[4].element_size() + t[5].numel() * t[5].element_size()))
     lanes = [torch.cuda.Stream() for _ in e2e_sets]
     lane_done = [torch.cuda.Event() for _ in e2e_sets]
 
@@ -697,7 +700,8 @@ def run_ours(args) -> None:
     e2e = {"value": job_value_us(e2e_ms, e2e_steps, world, n_layers), "unit": UNIT, "h2d_bytes_per_step": h2d,
            "d2h_bytes_per_step": d2h, "steps": e2e_steps,
            "api": "gf_layer_step_host per layer, one stream per layer (pinned host buffers; copies of x, g_y, W in and "
-                  "g_W, g_X out inside the timed region; uploads of one layer overlap downloads of another)"}
+                  "g_W, g_X out inside the timed region; uploads of one layer overlap downloads of another, "
+                  "layers issued in the order of their download sizes, largest first)"}
     del e2e_sets
 
     if rank != 0:
