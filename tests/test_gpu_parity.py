@@ -89,6 +89,8 @@ SMALL = [
     L("tma_pair_r8", 2, 24, 512, 64, 64, 1, 1, 8),
     L("tma_pair_r4_multi_ci", 2, 520, 512, 32, 32, 1, 1, 4),  # three c_i tiles of 176
     L("tma_pair_odd_units", 5, 40, 640, 16, 16, 3, 1, 2),   # five units: the last CTA's second unit is empty
+    L("tma_pair_ragged_ci", 2, 70, 512, 16, 16, 1, 1, 2),   # C_in neither a multiple of 16 nor of 4: scalar additions into g_W
+    L("tma_pair_many_tiles", 56, 24, 64, 40, 48, 3, 1, 2),  # short contraction, 224 row tiles: the second arm of the rule
 ]
 
 
