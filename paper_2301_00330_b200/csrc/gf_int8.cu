@@ -96,11 +96,66 @@ __global__ void __launch_bounds__(kQThreads) q_gbar_kernel(const T* __restrict__
     block_absmax(worst, amax);
 }
 
+// The same means, G = 16 bytes / (R elements) adjacent patches per thread: one 16-byte load per
+// pixel row instead of G narrow ones.  Needs rows that start on 16-byte boundaries (W a multiple
+// of the vector) on top of what q_gbar_kernel<T, R> needs.  The order of the additions inside a
+// patch is the same (row by row, left to right, from zero).
+template <typename T, int R>
+__global__ void __launch_bounds__(kQThreads) q_gbar_wide_kernel(const T* __restrict__ gy, float* __restrict__ gbar, long long items,
+                                                                int H, int W, int Hp, int Wp, FastDiv div_WpG, uint32_t* amax) {
+    constexpr int VE = 16 / (int)sizeof(T), G = VE / R;
+    const int WpG = Wp / G;
+    float worst = 0.f;
+    for (long long it = (long long)blockIdx.x * blockDim.x + threadIdx.x; it < items; it += (long long)gridDim.x * blockDim.x) {
+        const long long pl = it / ((long long)Hp * WpG);
+        uint32_t a, bg;
+        div_WpG.divmod((uint32_t)(it - pl * (long long)Hp * WpG), a, bg);
+        const T* p0 = gy + pl * (long long)H * W + (long long)a * R * W + (long long)bg * VE;
+        float v[R][VE];
+#pragma unroll
+        for (int i = 0; i < R; ++i) load_row<VE>(p0 + (long long)i * W, v[i]);
+        float mean[G];
+#pragma unroll
+        for (int k = 0; k < G; ++k) {
+            float sum = 0.f;
+#pragma unroll
+            for (int i = 0; i < R; ++i)
+#pragma unroll
+                for (int j = 0; j < R; ++j) sum = __fadd_rn(sum, v[i][k * R + j]);
+            mean[k] = __fmul_rn(sum, __fdiv_rn(1.0f, (float)(R * R)));
+            worst = fmaxf(worst, fabsf(mean[k]));
+        }
+        float* out = gbar + (pl * Hp + a) * (long long)Wp + (long long)bg * G;      // a multiple of G: Wp is
+        if constexpr (G == 2) *reinterpret_cast<float2*>(out) = make_float2(mean[0], mean[1]);
+        else *reinterpret_cast<float4*>(out) = make_float4(mean[0], mean[1], mean[2], mean[3]);
+    }
+    block_absmax(worst, amax);
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kQThreads) absmax_kernel(const T* __restrict__ v, long long n, uint32_t* amax) {
     float worst = 0.f;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
         worst = fmaxf(worst, fabsf(to_f32(v[i])));
+    block_absmax(worst, amax);
+}
+
+// four consecutive elements (16-byte / 8-byte aligned)
+__device__ __forceinline__ float4 load4(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
+    const uint2 t = __ldcs(reinterpret_cast<const uint2*>(p));
+    return make_float4(__uint_as_float(t.x << 16), __uint_as_float(t.x & 0xffff0000u), __uint_as_float(t.y << 16),
+                       __uint_as_float(t.y & 0xffff0000u));
+}
+
+// max|.| of n elements, n % 4 == 0, four per load
+template <typename T>
+__global__ void __launch_bounds__(kQThreads) absmax4_kernel(const T* __restrict__ v, long long n4, uint32_t* amax) {
+    float worst = 0.f;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (long long)gridDim.x * blockDim.x) {
+        const float4 t = load4(v + 4 * i);
+        worst = fmaxf(fmaxf(worst, fmaxf(fabsf(t.x), fabsf(t.y))), fmaxf(fabsf(t.z), fabsf(t.w)));
+    }
     block_absmax(worst, amax);
 }
 
@@ -128,6 +183,23 @@ __global__ void __launch_bounds__(kQThreads) quant_planes_kernel(const T* __rest
         const long long k = (long long)n * P + p;
         q_k[(long long)c * kp + k] = code;
         if (q_t) q_t[k * cp + c] = code;
+    }
+}
+
+// K-major codes only, four consecutive patches per thread (P % 4 == 0): src [n][C][P] -> q_k[c][n P + p]
+template <typename T>
+__global__ void __launch_bounds__(kQThreads) quant_planes4_kernel(const T* __restrict__ src, long long total4, int C, int P4,
+                                                                  FastDiv div_P4, FastDiv div_C, const uint32_t* __restrict__ amax,
+                                                                  int8_t* __restrict__ q_k, long long kp) {
+    const float scale = scale_of(*amax);
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total4; i += (long long)gridDim.x * blockDim.x) {
+        uint32_t nc, p4, n, c;
+        div_P4.divmod((uint32_t)i, nc, p4);
+        div_C.divmod(nc, n, c);
+        const float4 t = load4(src + 4 * i);
+        const uint32_t w = (uint32_t)(uint8_t)code_of(t.x, scale) | ((uint32_t)(uint8_t)code_of(t.y, scale) << 8) |
+                           ((uint32_t)(uint8_t)code_of(t.z, scale) << 16) | ((uint32_t)(uint8_t)code_of(t.w, scale) << 24);
+        *reinterpret_cast<uint32_t*>(q_k + (long long)c * kp + ((long long)n * P4 + p4) * 4) = w;
     }
 }
 
@@ -160,6 +232,46 @@ __global__ void __launch_bounds__(kQThreads) quant_gbar_tiled_kernel(const float
     for (int pl = ty; pl < 64; pl += 4) {
         const int pp = p0 + pl, c = c0 + tx;
         if (pp < P && c < C) q_t[((long long)n * P + pp) * cp + c] = tile[tx][pl];
+    }
+}
+
+// The same with four patches (K-major rows) or four channels (patch-major rows) per thread: 16-byte
+// loads and 4-byte stores.  Needs P % 4 == 0 (and C % 4 == 0 for the patch-major rows).
+__device__ __forceinline__ uint32_t pack4(int8_t a, int8_t b, int8_t c, int8_t d) {
+    return (uint32_t)(uint8_t)a | ((uint32_t)(uint8_t)b << 8) | ((uint32_t)(uint8_t)c << 16) | ((uint32_t)(uint8_t)d << 24);
+}
+__global__ void __launch_bounds__(kQThreads) quant_gbar_tiled4_kernel(const float* __restrict__ src, int C, int P, int p_tiles,
+                                                                      const uint32_t* __restrict__ amax, int8_t* __restrict__ q_k,
+                                                                      long long kp, int8_t* __restrict__ q_t, long long cp) {
+    __shared__ __align__(4) int8_t tile[64][64 + 4];
+    const float scale = scale_of(*amax);
+    const int pt = blockIdx.x % p_tiles, n = blockIdx.x / p_tiles;
+    const int c0 = blockIdx.y * 64, p0 = pt * 64;
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;              // 16 rows of 16 x 4 patches at a time
+    const int pp = p0 + 4 * tx;
+    float4 v[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {                                        // all loads in flight before the first use
+        const int c = c0 + ty + 16 * k;
+        v[k] = (c < C && pp < P) ? __ldcs(reinterpret_cast<const float4*>(src + ((size_t)n * C + c) * P + pp)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int cc = ty + 16 * k, c = c0 + cc;
+        const bool in = c < C && pp < P;                                 // P % 4 == 0: all four patches or none
+        const uint32_t w = in ? pack4(code_of(v[k].x, scale), code_of(v[k].y, scale), code_of(v[k].z, scale), code_of(v[k].w, scale)) : 0u;
+        *reinterpret_cast<uint32_t*>(&tile[cc][4 * tx]) = w;
+        if (in) *reinterpret_cast<uint32_t*>(q_k + (long long)c * kp + (long long)n * P + pp) = w;
+    }
+    if (!q_t) return;
+    __syncthreads();
+    const int c = c0 + 4 * tx;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int pl = ty + 16 * k, pq = p0 + pl;
+        if (pq < P && c < C)                                             // C % 4 == 0: all four channels or none
+            *reinterpret_cast<uint32_t*>(q_t + ((long long)n * P + pq) * cp + c) =
+                pack4(tile[4 * tx][pl], tile[4 * tx + 1][pl], tile[4 * tx + 2][pl], tile[4 * tx + 3][pl]);
     }
 }
 
@@ -467,11 +579,23 @@ gf_status gf_backward_int8(const gf_conv_desc* desc, const void* g_y, const void
         const bool vec = (g.r == 2 || g.r == 4 || g.r == 8) && g.H % g.r == 0 && g.W % g.r == 0 &&
                          ((long long)g.H * g.W * (long long)g.esize) % 16 == 0;
         const int R = vec ? g.r : 0;
+        // several patches per thread where a 16-byte vector holds more than one patch row and the rows are aligned
+        const int ve = 16 / (int)g.esize, G = (R > 0 && ve / R >= 2 && g.W % ve == 0) ? ve / R : 1;
+        if (G >= 2) {
+            const long long items = patches / G;
+            const FastDiv div_WpG((uint32_t)(g.Wp / G));
+#define GF_QW(TT, RR) q_gbar_wide_kernel<TT, RR><<<q_grid(items), kQThreads, 0, s>>>((const TT*)g_y, gbar, items, g.H, g.W, g.Hp, g.Wp, div_WpG, amax_g)
+            if (g.dtype == GF_F32) GF_QW(float, 2);
+            else if (R == 2) GF_QW(__nv_bfloat16, 2);
+            else GF_QW(__nv_bfloat16, 4);
+#undef GF_QW
+        } else {
         const unsigned grid = q_grid(patches);
 #define GF_QG(TT, RR) q_gbar_kernel<TT, RR><<<grid, kQThreads, 0, s>>>((const TT*)g_y, gbar, patches, g.H, g.W, g.r, g.Hp, g.Wp, div_Wp, amax_g)
         if (g.dtype == GF_F32) { if (R == 2) GF_QG(float, 2); else if (R == 4) GF_QG(float, 4); else if (R == 8) GF_QG(float, 8); else GF_QG(float, 0); }
         else { if (R == 2) GF_QG(__nv_bfloat16, 2); else if (R == 4) GF_QG(__nv_bfloat16, 4); else if (R == 8) GF_QG(__nv_bfloat16, 8); else GF_QG(__nv_bfloat16, 0); }
 #undef GF_QG
+        }
         st = after_launch();
     }
     if (st != GF_OK) return st;
@@ -480,7 +604,10 @@ gf_status gf_backward_int8(const gf_conv_desc* desc, const void* g_y, const void
         const int p_tiles = (w.P + 63) / 64;
         const dim3 grid((unsigned)(g.N * p_tiles), (unsigned)((g.C_out + 63) / 64), 1);
         if (grid.y > 65535) return GF_ERR_UNSUPPORTED;
-        quant_gbar_tiled_kernel<<<grid, kQThreads, 0, s>>>(gbar, g.C_out, w.P, p_tiles, amax_g, qg_k, w.kp, g_X ? qg_t : nullptr, w.cp);
+        if (w.P % 4 == 0 && g.C_out % 4 == 0)
+            quant_gbar_tiled4_kernel<<<grid, kQThreads, 0, s>>>(gbar, g.C_out, w.P, p_tiles, amax_g, qg_k, w.kp, g_X ? qg_t : nullptr, w.cp);
+        else
+            quant_gbar_tiled_kernel<<<grid, kQThreads, 0, s>>>(gbar, g.C_out, w.P, p_tiles, amax_g, qg_k, w.kp, g_X ? qg_t : nullptr, w.cp);
         if ((st = after_launch()) != GF_OK) return st;
     }
 
@@ -510,18 +637,23 @@ gf_status gf_backward_int8(const gf_conv_desc* desc, const void* g_y, const void
     }
     if (g_W) {
         const long long xs = w.K * g.C_in;
-        if (g.dtype == GF_F32) {
-            absmax_kernel<float><<<q_grid(xs), kQThreads, 0, s>>>((const float*)stash, xs, amax_x);
-            if ((st = after_launch()) != GF_OK) return st;
-            quant_planes_kernel<float><<<q_grid(xs), kQThreads, 0, s>>>((const float*)stash, xs, g.C_in, w.P, div_P,
-                                                                       FastDiv((uint32_t)g.C_in), amax_x, qx_k, w.kp, nullptr, 0);
-        } else {
-            absmax_kernel<__nv_bfloat16><<<q_grid(xs), kQThreads, 0, s>>>((const __nv_bfloat16*)stash, xs, amax_x);
-            if ((st = after_launch()) != GF_OK) return st;
-            quant_planes_kernel<__nv_bfloat16><<<q_grid(xs), kQThreads, 0, s>>>((const __nv_bfloat16*)stash, xs, g.C_in, w.P, div_P,
-                                                                               FastDiv((uint32_t)g.C_in), amax_x, qx_k, w.kp,
-                                                                               nullptr, 0);
-        }
+        const bool four = w.P % 4 == 0 && xs / 4 < 0x7fffffffLL;       // rows of the stash in 4-element pieces
+        const FastDiv div_C((uint32_t)g.C_in), div_P4((uint32_t)(four ? w.P / 4 : 1));
+#define GF_QX(TT)                                                                                                                  \
+        do {                                                                                                                       \
+            if (four) absmax4_kernel<TT><<<q_grid(xs / 4), kQThreads, 0, s>>>((const TT*)stash, xs / 4, amax_x);                   \
+            else absmax_kernel<TT><<<q_grid(xs), kQThreads, 0, s>>>((const TT*)stash, xs, amax_x);                                 \
+            if ((st = after_launch()) != GF_OK) return st;                                                                         \
+            if (four)                                                                                                              \
+                quant_planes4_kernel<TT><<<q_grid(xs / 4), kQThreads, 0, s>>>((const TT*)stash, xs / 4, g.C_in, w.P / 4, div_P4,  \
+                                                                              div_C, amax_x, qx_k, w.kp);                          \
+            else                                                                                                                   \
+                quant_planes_kernel<TT><<<q_grid(xs), kQThreads, 0, s>>>((const TT*)stash, xs, g.C_in, w.P, div_P, div_C, amax_x,  \
+                                                                         qx_k, w.kp, nullptr, 0);                                  \
+        } while (0)
+        if (g.dtype == GF_F32) GF_QX(float);
+        else GF_QX(__nv_bfloat16);
+#undef GF_QX
         if ((st = after_launch()) != GF_OK) return st;
         if (!make_tmap_u8_2d(&p.tm_a, qg_k, (uint64_t)w.kp, (uint64_t)w.cop, (uint64_t)w.kp, 128) ||
             !make_tmap_u8_2d(&p.tm_b, qx_k, (uint64_t)w.kp, (uint64_t)w.cip, (uint64_t)w.kp, 128))
