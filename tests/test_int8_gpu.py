@@ -29,6 +29,8 @@ CASES = [
     L("r8", 4, 32, 48, 32, 32, 3, 8),
     L("r3_odd_map", 2, 16, 16, 13, 10, 3, 3),
     L("wide_co", 2, 40, 600, 8, 8, 1, 2),                       # c_o contraction in 5 chunks
+    L("r4_wide_rows", 2, 16, 24, 16, 32, 3, 4),                 # bf16: two patches per 16-byte row of the gradient filter
+    L("r2_wide_rows", 3, 8, 16, 12, 48, 1, 2),                  # two (fp32) / four (bf16) patches per 16-byte row
 ]
 
 
