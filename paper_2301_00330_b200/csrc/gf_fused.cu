@@ -55,7 +55,9 @@ struct FusedPlan {
     int kc_raw = 0;         // channels per raw slab
     int n_sub = 0;          // raw slabs per chunk of 64 channels
     int MB = 1;             // 64-patch blocks per tile
-    int PT = 0;             // patch slots per tile: IT * RT * Wp
+    int PT = 0;             // patch slots per tile: IT * RT * Wp, or (RT / rpw) * 32 with row-aligned slots
+    int rpw = 0;            // > 0: row-aligned slots -- every 32 slots (the accumulator rows one warp of the
+                            // expansion owns) hold rpw WHOLE patch rows and 32 - rpw * Wp empty slots
     int G = 1;              // adjacent patches pooled by one thread
     int NG = 0, n_groups = 0;   // c_i per accumulator, number of such groups
     int n_chunks = 0;       // ceil(C_out / 64)
@@ -74,6 +76,7 @@ struct FusedParams {
     int N, C_in, C_out, H, W, Hp, Wp, r;
     int IT, RT, PW, pieces, piece_bytes, kc_raw, n_sub, MB, PT, PTG, NG, NGs, n_groups, n_chunks, reuse;
     int a_stages, raw_stages, raw_stage_bytes;
+    int rpw;                // row-aligned slots: whole patch rows per 32 slots (0: slots are the patches in row-major order)
     int kpar;               // channels of a raw slab pooled side by side: kFuWork / PTG
     int n_acc;              // accumulators in tensor memory (a ring): 512 / NGs, at most kFuAccMax
     long long tiles;
@@ -88,6 +91,24 @@ struct FuShared {
     uint64_t acc_full[kFuAccMax], acc_empty[kFuAccMax];
     uint32_t tmem_base;
 };
+
+// Which patch a slot of a tile holds: image of the tile, patch row within the tile, patch of the
+// row; false: an empty slot of the row-aligned order.
+__device__ __forceinline__ bool fu_slot(const FusedParams& p, uint32_t m, uint32_t& img, uint32_t& a, uint32_t& b) {
+    if (p.rpw > 0) {
+        const uint32_t w = m & 31u;
+        const bool real = w < (uint32_t)(p.rpw * p.Wp);
+        uint32_t ar;
+        p.div_Wp.divmod(real ? w : 0u, ar, b);
+        a = (m >> 5) * (uint32_t)p.rpw + ar;
+        img = 0;
+        return real;
+    }
+    uint32_t rem;
+    p.div_RTWp.divmod(m, img, rem);
+    p.div_Wp.divmod(rem, a, b);
+    return true;
+}
 
 // first image and first patch row of tile t
 __device__ __forceinline__ void fu_tile(int IT, int RT, const FastDiv& div_N, long long t, int& n0, int& a0) {
@@ -230,9 +251,8 @@ __global__ void __launch_bounds__(kFuThreads, 1) gyx_fused_kernel(const __grid_c
         uint32_t kl, mg;
         p.div_PTG.divmod((uint32_t)tid, kl, mg);
         const bool pool_active = (int)kl < p.kpar;
-        uint32_t pimg, prem, pa, pb;
-        p.div_RTWp.divmod(mg * G, pimg, prem);
-        p.div_Wp.divmod(prem, pa, pb);
+        uint32_t pimg, pa, pb;
+        const bool pool_real = fu_slot(p, mg * G, pimg, pa, pb);
         // a raw slab is [piece][image of the tile][channel][PW]: where the R pixel rows of the position start
         int roff[R];
 #pragma unroll
@@ -249,16 +269,15 @@ __global__ void __launch_bounds__(kFuThreads, 1) gyx_fused_kernel(const __grid_c
         T* gx = static_cast<T*>(p.gX);
         const size_t plane = (size_t)p.H * p.W;
         const uint32_t m = (uint32_t)(quarter * 32 + lane);
-        uint32_t eimg, erem, ea, eb;
-        p.div_RTWp.divmod(m, eimg, erem);
-        p.div_Wp.divmod(erem, ea, eb);
+        uint32_t eimg, ea, eb;
+        const bool e_real = fu_slot(p, m, eimg, ea, eb);
         int aq = 0, rq = 0, iq = 0;
         for (int it = 0; it < n_my && ok; ++it) {
             const long long tile = first + (long long)it * stride;
             int n0, a0;
             fu_tile(p.IT, p.RT, p.div_N, tile, n0, a0);
-            const bool pool_live = n0 + (int)pimg < p.N && a0 + (int)pa < p.Hp;
-            const bool e_valid = (int)m < p.PT && n0 + (int)eimg < p.N && a0 + (int)ea < p.Hp;
+            const bool pool_live = pool_real && n0 + (int)pimg < p.N && a0 + (int)pa < p.Hp;
+            const bool e_valid = e_real && (int)m < p.PT && n0 + (int)eimg < p.N && a0 + (int)ea < p.Hp;
             T* base_m = gx + ((size_t)(n0 + (int)eimg) * p.C_in) * plane + (size_t)((a0 + (int)ea) * R) * p.W + (size_t)eb * R;
             for (int pass = 0; pass < n_pass && ok; ++pass) {
                 for (int c = 0; c < p.n_chunks && ok; ++c, ++aq) {
@@ -446,6 +465,7 @@ struct GwTiledParams {
     uint32_t* err_word;
     int N, C_in, C_out, Hp, Wp, P;
     int IT, RT, MB, n_chunks, S;
+    int rpw;                        // row-aligned slots (see FusedPlan): a 64-slot block is two boxes of 32 stash values
     int logv;                       // log2 of the stash elements per asynchronous copy piece (pieces of 4, 8 or 16 bytes)
     long long kchunks;              // tiles * MB
     FastDiv div_N, div_P, div_MB;
@@ -468,11 +488,16 @@ __device__ __forceinline__ void cp_async_bytes(uint32_t dst, const void* src, in
 // consecutive lanes read one 256-byte row and write one 128-byte row of each tile, both
 // without bank conflicts.  Every piece is in registers before any is overwritten.
 // Returns false when some thread of the 256 reports a failed wait.
-__device__ __forceinline__ bool gt_split_in_place(unsigned char* bt, int tid, bool ok) {
+// halves: the rows arrived as two boxes [128][32] (the first 16 KB, then the second) instead of one [128][64].
+__device__ __forceinline__ bool gt_split_in_place(unsigned char* bt, int tid, bool ok, bool halves = false) {
     float4 v[8];
     if (ok) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) v[i] = reinterpret_cast<const float4*>(bt)[tid + 256 * i];
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t idx = (uint32_t)(tid + 256 * i);
+            const uint32_t src = halves ? ((idx >> 3) & 1u) * 1024u + (idx >> 4) * 8u + (idx & 7u) : idx;   // in 16-byte pieces
+            v[i] = reinterpret_cast<const float4*>(bt)[src];
+        }
     }
     if (bar_any(1, kGtWork, !ok)) return false;
 #pragma unroll
@@ -621,7 +646,7 @@ __global__ void __launch_bounds__(kGtThreads) gw_tiled_kernel(const __grid_const
             for (int q = 0; q < n_chunks && ok; ++q) {
                 const int s = q % ST;
                 ok = mbar_wait_bounded(&sh.landed[s], (uint32_t)(q / ST) & 1u);
-                if (!gt_split_in_place(dyn + (size_t)s * kStageBytes + kBOff, tid, ok)) { ok = false; break; }
+                if (!gt_split_in_place(dyn + (size_t)s * kStageBytes + kBOff, tid, ok, p.rpw > 0)) { ok = false; break; }
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.full[s]);
@@ -676,7 +701,15 @@ __global__ void __launch_bounds__(kGtThreads) gw_tiled_kernel(const __grid_const
                 else { int a0; fu_tile(1, p.RT, p.div_N, tile, n_img, a0); x = a0 * p.Wp + (int)mb * 64; }
                 if constexpr (SPLIT == 2) {
                     mbar_expect_tx(&sh.landed[s], kBBytes);
-                    tma_load_3d(stage + kBOff, &p.tm_stash, x, ci0, n_img, &sh.landed[s]);
+                    if (p.rpw > 0) {     // row-aligned slots: 32 slots = rpw patch rows, two boxes of 32 values per block
+                        int a0;
+                        fu_tile(1, p.RT, p.div_N, tile, n_img, a0);
+                        for (int h = 0; h < 2; ++h)
+                            tma_load_3d(stage + kBOff + h * (int)(kBBytes / 2), &p.tm_stash, (a0 + (2 * (int)mb + h) * p.rpw) * p.Wp, ci0,
+                                        n_img, &sh.landed[s]);
+                    } else {
+                        tma_load_3d(stage + kBOff, &p.tm_stash, x, ci0, n_img, &sh.landed[s]);
+                    }
                 } else {
                     tma_load_3d(stage + kBOff, &p.tm_stash, x, ci0, n_img, &sh.full[s]);
                 }
@@ -734,6 +767,28 @@ static FusedPlan fused_plan(const Geo& g) {
         f.run = f.RT * r * g.W;
     }
     f.PT = f.IT * f.RT * g.Wp;
+    // Row-aligned slots.  The expansion writes, per warp instruction, the pixels of 32 consecutive
+    // slots of one plane.  With slots = patches in row-major order a warp's patches start and end
+    // in the middle of patch rows, and where a pixel row is not a whole number of 32-byte sectors
+    // (28-wide fp32 maps: 112 bytes) the sectors at those ends are written in halves by different
+    // warps at different times: measured 3.3 TB/s for such stores against 5.5 TB/s when every warp
+    // owns whole patch rows (same bytes, same instructions).  So: rpw = floor(32 / Wp) whole rows per
+    // 32 slots, the rest of the 32 left empty (their patch means are zeros), when that costs no
+    // extra tile.  fp32 layers whose stash rows the g_W contraction fetches by tensor maps only
+    // (the copy-piece variants of that kernel keep the dense order).
+    if (f.IT == 1 && g.dtype == GF_F32 && f.stash_tma && g.Wp < 32 && 32 % g.Wp != 0 && ((long long)g.W * e) % 32 != 0) {
+        const int rpw = 32 / g.Wp;
+        const int q = 16 / gcd_int(16, (g.Wp * e) % 16 == 0 ? 16 : (g.Wp * e) % 16);
+        const int step = rpw / gcd_int(rpw, q) * q;                       // tile heights: multiples of both
+        const int rt = (4 * rpw) / step * step;                           // at most 128 slots
+        if (rt >= 1 && (g.Hp + rt - 1) / rt == f.tiles_per_img && ((long long)rpw * g.Wp * e) % 16 == 0 &&
+            ((long long)rt * r * g.W * e) % 16 == 0) {
+            f.RT = rt;
+            f.rpw = rpw;
+            f.run = f.RT * r * g.W;
+            f.PT = f.RT / rpw * 32;
+        }
+    }
     f.MB = f.PT > 64 ? 2 : 1;
     f.G = g.Wp % 2 == 0 ? 2 : 1;
     // Pieces of the run: as few boxes as the 256-element limit allows, of equal width, a multiple
@@ -814,6 +869,7 @@ gf_status launch_gyx_fused(const void* gy, const __nv_bfloat16* thetaT, long lon
     p.piece_bytes = f.IT * f.kc_raw * f.PW * (int)g.esize;
     p.div_PW = FastDiv((uint32_t)f.PW);
     p.kc_raw = f.kc_raw; p.n_sub = f.n_sub; p.MB = f.MB; p.PT = f.PT; p.PTG = f.PT / f.G; p.NG = f.NG;
+    p.rpw = f.rpw;
     int ngs = 32;
     while (ngs < f.NG) ngs <<= 1;
     p.NGs = ngs;
@@ -880,7 +936,7 @@ gf_status launch_gw_tiled(const unsigned char* gbar_t, const void* stash, float*
     GwTiledParams p;
     p.gbar_t = gbar_t; p.stash = stash; p.gwu = gwu; p.err_word = err_word;
     p.N = g.N; p.C_in = g.C_in; p.C_out = g.C_out; p.Hp = g.Hp; p.Wp = g.Wp; p.P = g.Hp * g.Wp;
-    p.IT = f.IT; p.RT = f.RT; p.MB = f.MB; p.n_chunks = f.n_chunks;
+    p.IT = f.IT; p.RT = f.RT; p.MB = f.MB; p.n_chunks = f.n_chunks; p.rpw = f.rpw;
     p.logv = gw_tiled_logv(g, f);
     if (p.logv < 0) return GF_ERR_UNSUPPORTED;
     p.kchunks = f.tiles * f.MB;
@@ -900,9 +956,11 @@ gf_status launch_gw_tiled(const unsigned char* gbar_t, const void* stash, float*
     if (tma_b) {
         const uint64_t P = (uint64_t)p.P;
         tma_b = g.dtype == GF_F32
-                    ? make_tmap_plain(&p.tm_stash, stash, 4, P, (uint64_t)g.C_in, (uint64_t)g.N, P, (uint64_t)g.C_in * P, 64, 128, 1)
+                    ? make_tmap_plain(&p.tm_stash, stash, 4, P, (uint64_t)g.C_in, (uint64_t)g.N, P, (uint64_t)g.C_in * P,
+                                      f.rpw > 0 ? 32 : 64, 128, 1)
                     : make_tmap_bf16(&p.tm_stash, stash, 3, P, (uint64_t)g.C_in, (uint64_t)g.N, P, (uint64_t)g.C_in * P, 128);
     }
+    if (f.rpw > 0 && !tma_b) return GF_ERR_CUDA;        // the row-aligned order exists for the tensor-map variant only
     if (g.dtype == GF_F32)
         return tma_b ? launch_gw_tiled_inst<float, true>(p, grid, s) : launch_gw_tiled_inst<float, false>(p, grid, s);
     return tma_b ? launch_gw_tiled_inst<__nv_bfloat16, true>(p, grid, s) : launch_gw_tiled_inst<__nv_bfloat16, false>(p, grid, s);

@@ -89,6 +89,11 @@ SMALL = [
     L("tma_pair_r8", 2, 24, 512, 64, 64, 1, 1, 8),
     L("tma_pair_r4_multi_ci", 2, 520, 512, 32, 32, 1, 1, 4),  # three c_i tiles of 176
     L("tma_pair_odd_units", 5, 40, 640, 16, 16, 3, 1, 2),   # five units: the last CTA's second unit is empty
+    # 28-wide fp32 maps at r = 2 (14 patches per row): the fused kernel's row-aligned slot order, two whole patch rows
+    # per 32 accumulator rows; 8-row and 6-row tiles, several c_i groups, a ragged c_o chunk
+    L("row_aligned_slots", 3, 24, 40, 28, 28, 3, 1, 2),
+    L("row_aligned_slots_groups", 2, 300, 72, 28, 28, 1, 1, 2),
+    L("row_aligned_slots_w20", 2, 16, 24, 32, 20, 3, 1, 2),     # 10 patches per row: three rows per 32 slots
     L("tma_pair_ragged_ci", 2, 70, 512, 16, 16, 1, 1, 2),   # C_in neither a multiple of 16 nor of 4: scalar additions into g_W
     L("tma_pair_many_tiles", 56, 24, 64, 40, 48, 3, 1, 2),  # short contraction, 224 row tiles: the second arm of the rule
 ]
