@@ -32,7 +32,9 @@
 
 namespace gf {
 
-constexpr int kFuWork = 512;                 // warps 0-15: workers (pool a tile, then write its part of g_X)
+constexpr int kFuWork = 512;                 // warps 0-15: workers
+constexpr int kFuPool = 256;                 //   warps 0-7 pool the tiles (gradient filter) into the operand tiles
+constexpr int kFuEpi = 256;                  //   warps 8-15 expand the accumulators into g_X, a tile behind the pooling
 constexpr int kFuRawWarp = 16, kFuBWarp = 17, kFuMmaWarp = 18;
 constexpr int kFuThreads = 19 * 32;
 constexpr int kFuRawMax = 4, kFuAMax = 4, kFuAccMax = 8;
@@ -218,7 +220,7 @@ __global__ void __launch_bounds__(kFuThreads, 1) gyx_fused_kernel(const __grid_c
     const int AS = p.a_stages, RS = p.raw_stages;
 
     if (tid == 0) {
-        for (int s = 0; s < kFuRawMax; ++s) { mbar_init(&sh.raw_full[s], 1); mbar_init(&sh.raw_empty[s], kFuWork / 32); }
+        for (int s = 0; s < kFuRawMax; ++s) { mbar_init(&sh.raw_full[s], 1); mbar_init(&sh.raw_empty[s], kFuPool / 32); }
         for (int s = 0; s < kFuAMax; ++s) { mbar_init(&sh.a_full[s], 1); mbar_init(&sh.a_empty[s], 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(&sh.b_full[s], 1); mbar_init(&sh.b_empty[s], 1); }
         for (int s = 0; s < kFuAccMax; ++s) { mbar_init(&sh.acc_full[s], 1); mbar_init(&sh.acc_empty[s], 1); }
@@ -243,11 +245,13 @@ __global__ void __launch_bounds__(kFuThreads, 1) gyx_fused_kernel(const __grid_c
     // group (or no g_X is wanted), else one per c_i group
     const int n_pass = (p.reuse || !has_mma) ? 1 : p.n_groups;
 
-    if (warp < kFuWork / 32) {
-        // ================= workers: pool the tile, then expand its accumulators into g_X =================
-        // Pooling: thread (kl, mg) takes position mg (G adjacent patch slots) of the channels kl,
-        // kl + kpar, ... of every raw slab; where those patches sit inside a slab and inside the
-        // operand tile is the same for every tile.
+    if (warp < kFuPool / 32) {
+        // ================= pooling warps: the gradient filter, tile after tile =================
+        // Thread (kl, mg) takes position mg (G adjacent patch slots) of the channels kl, kl + kpar, ...
+        // of every raw slab; where those patches sit inside a slab and inside the operand tile is
+        // the same for every tile.  The warps run ahead of the expansion as far as the operand
+        // ring and the accumulators allow, so that a tile's pixels of g_y are read and pooled while
+        // the previous tile's part of g_X is still being written.
         uint32_t kl, mg;
         p.div_PTG.divmod((uint32_t)tid, kl, mg);
         const bool pool_active = (int)kl < p.kpar;
@@ -263,22 +267,12 @@ __global__ void __launch_bounds__(kFuThreads, 1) gyx_fused_kernel(const __grid_c
         }
         const uint32_t pj = mg * G;
         const uint32_t pool_dst = (pj >> 6) * 8192u + ((pj & 7u) << 1), pool_jc = (pj & 63u) >> 3;
-        // Expansion: lane quarter warp & 3 of tensor memory = patch slots 32 (warp & 3) + lane;
-        // the four warps of a quarter take interleaved 32-column chunks.
-        const int quarter = warp & 3, cset = warp >> 2;
-        T* gx = static_cast<T*>(p.gX);
-        const size_t plane = (size_t)p.H * p.W;
-        const uint32_t m = (uint32_t)(quarter * 32 + lane);
-        uint32_t eimg, ea, eb;
-        const bool e_real = fu_slot(p, m, eimg, ea, eb);
-        int aq = 0, rq = 0, iq = 0;
+        int aq = 0, rq = 0;
         for (int it = 0; it < n_my && ok; ++it) {
             const long long tile = first + (long long)it * stride;
             int n0, a0;
             fu_tile(p.IT, p.RT, p.div_N, tile, n0, a0);
             const bool pool_live = pool_real && n0 + (int)pimg < p.N && a0 + (int)pa < p.Hp;
-            const bool e_valid = e_real && (int)m < p.PT && n0 + (int)eimg < p.N && a0 + (int)ea < p.Hp;
-            T* base_m = gx + ((size_t)(n0 + (int)eimg) * p.C_in) * plane + (size_t)((a0 + (int)ea) * R) * p.W + (size_t)eb * R;
             for (int pass = 0; pass < n_pass && ok; ++pass) {
                 for (int c = 0; c < p.n_chunks && ok; ++c, ++aq) {
                     const int s = aq % AS, u = aq / AS;
@@ -286,7 +280,7 @@ __global__ void __launch_bounds__(kFuThreads, 1) gyx_fused_kernel(const __grid_c
                     // the copy-out of this stage's previous contents must have finished reading it
                     if (tid == 0) bulk_wait_read<1>();
                     if (u >= 1 && has_mma) ok = mbar_wait_bounded(&sh.a_empty[s], (uint32_t)(u - 1) & 1u);
-                    if (bar_any(1, kFuWork, !ok)) { ok = false; break; }
+                    if (bar_any(1, kFuPool, !ok)) { ok = false; break; }
                     const int k_lim = p.C_out - c * kTcBK;
                     for (int sub = 0; sub < p.n_sub && ok; ++sub, ++rq) {
                         const int rs = rq % RS;
@@ -300,7 +294,7 @@ __global__ void __launch_bounds__(kFuThreads, 1) gyx_fused_kernel(const __grid_c
                         if (lane == 0) mbar_arrive(&sh.raw_empty[rs]);
                     }
                     fence_proxy_async_smem();     // the tile is read by the tensor core and the copy engine
-                    if (bar_any(1, kFuWork, !ok)) { ok = false; break; }
+                    if (bar_any(1, kFuPool, !ok)) { ok = false; break; }
                     if (tid == 0) {
                         if (p.gbar_t && pass == 0) {
                             for (int part = 0; part < SPLIT; ++part)
@@ -313,40 +307,56 @@ __global__ void __launch_bounds__(kFuThreads, 1) gyx_fused_kernel(const __grid_c
                         mbar_arrive(&sh.a_full[s]);
                     }
                 }
-                if (!has_mma || !ok) continue;
-                // the c_i groups this pass has fed
-                const int g_lo = p.reuse ? 0 : pass, g_hi = p.reuse ? p.n_groups : pass + 1;
-                for (int g = g_lo; g < g_hi && ok; ++g, ++iq) {
-                    const int buf = iq % n_acc;
-                    const int ci0 = g * p.NG;
-                    const int ng = min(p.NG, p.C_in - ci0);
-                    ok = mbar_wait_bounded(&sh.acc_full[buf], (uint32_t)(iq / n_acc) & 1u);
-                    tc_fence_after_sync();
-                    if (ok) {
-                        for (int c = cset * 32; c < ng; c += 128) {
-                            uint32_t v[32];
-                            tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * p.NGs + c), v);
-                            tmem_ld_wait();
-                            if (e_valid) {
-                                T* dst = base_m + (size_t)(ci0 + c) * plane;
+            }
+        }
+        if (tid == 0) bulk_wait_all();
+    } else if (warp < kFuWork / 32) {
+        // ================= expansion warps: the accumulators of a tile to its pixels of g_X =================
+        // Lane quarter warp & 3 of tensor memory = patch slots 32 (warp & 3) + lane; the two warps of
+        // a quarter take interleaved 32-column chunks.
+        const int ew = warp - kFuPool / 32;
+        const int quarter = ew & 3, cset = ew >> 2;
+        T* gx = static_cast<T*>(p.gX);
+        const size_t plane = (size_t)p.H * p.W;
+        const uint32_t m = (uint32_t)(quarter * 32 + lane);
+        uint32_t eimg, ea, eb;
+        const bool e_real = fu_slot(p, m, eimg, ea, eb);
+        int iq = 0;
+        for (int it = 0; it < n_my && ok && has_mma; ++it) {
+            const long long tile = first + (long long)it * stride;
+            int n0, a0;
+            fu_tile(p.IT, p.RT, p.div_N, tile, n0, a0);
+            const bool e_valid = e_real && (int)m < p.PT && n0 + (int)eimg < p.N && a0 + (int)ea < p.Hp;
+            T* base_m = gx + ((size_t)(n0 + (int)eimg) * p.C_in) * plane + (size_t)((a0 + (int)ea) * R) * p.W + (size_t)eb * R;
+            for (int g = 0; g < p.n_groups && ok; ++g, ++iq) {
+                const int buf = iq % n_acc;
+                const int ci0 = g * p.NG;
+                const int ng = min(p.NG, p.C_in - ci0);
+                ok = mbar_wait_bounded(&sh.acc_full[buf], (uint32_t)(iq / n_acc) & 1u);
+                tc_fence_after_sync();
+                if (ok) {
+                    for (int c = cset * 32; c < ng; c += 64) {
+                        uint32_t v[32];
+                        tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * p.NGs + c), v);
+                        tmem_ld_wait();
+                        if (e_valid) {
+                            T* dst = base_m + (size_t)(ci0 + c) * plane;
 #pragma unroll
-                                for (int i = 0; i < 32; ++i) {
-                                    if (c + i < ng) {
-                                        const float val = __uint_as_float(v[i]);
+                            for (int i = 0; i < 32; ++i) {
+                                if (c + i < ng) {
+                                    const float val = __uint_as_float(v[i]);
 #pragma unroll
-                                        for (int dr = 0; dr < R; ++dr) fu_store_rep<R>(dst + (size_t)i * plane + (size_t)dr * p.W, val);
-                                    }
+                                    for (int dr = 0; dr < R; ++dr) fu_store_rep<R>(dst + (size_t)i * plane + (size_t)dr * p.W, val);
                                 }
                             }
                         }
                     }
-                    tc_fence_before_sync();
-                    if (bar_any(1, kFuWork, !ok)) { ok = false; break; }
-                    if (tid == 0) mbar_arrive(&sh.acc_empty[buf]);
                 }
+                tc_fence_before_sync();
+                if (bar_any(2, kFuEpi, !ok)) { ok = false; break; }
+                if (tid == kFuPool) mbar_arrive(&sh.acc_empty[buf]);
             }
         }
-        if (tid == 0) bulk_wait_all();
     } else if (warp == kFuRawWarp) {
         // ================= copy engine: g_y slabs =================
         // A slab: for each piece of the tile's run of pixels, a box of kc_raw channels of the
@@ -874,7 +884,7 @@ gf_status launch_gyx_fused(const void* gy, const __nv_bfloat16* thetaT, long lon
     while (ngs < f.NG) ngs <<= 1;
     p.NGs = ngs;
     p.n_acc = 512 / ngs < kFuAccMax ? 512 / ngs : kFuAccMax;
-    p.kpar = kFuWork / p.PTG;
+    p.kpar = kFuPool / p.PTG;
     p.n_groups = f.n_groups; p.n_chunks = f.n_chunks; p.reuse = f.reuse ? 1 : 0;
     p.a_stages = f.a_stages; p.raw_stages = f.raw_stages; p.raw_stage_bytes = (int)f.raw_stage_bytes;
     p.tiles = f.tiles;
@@ -917,15 +927,18 @@ bool fused_path_ok(const Geo& g) {
     return f.ok && gw_tiled_logv(g, f) >= 0 && (g.C_out + 127) / 128 <= 65535 && (g.C_out + 31) / 32 <= 65535;
 }
 
-// Measured on the layer shapes of the benchmark (B200): the fused pair wins when every SM gets
-// a tile and the layer either writes far more g_X than it reads g_y (the separate g_X kernel
-// shares the SMs with the g_W kernel there) or has few channels (one c_i group, short
-// contractions); elsewhere the pooling pass plus the two contractions side by side are faster,
-// because the g_W contraction of the fused pair cannot start before the fused kernel has ended.
+// Measured on the layer shapes of the benchmark (B200): the fused pair wins when every SM gets a
+// tile and the layer writes far more g_X than it reads g_y (576 -> 96 channels at 28 x 28: 95 against
+// 121 us; the separate g_X kernel shares the SMs with the g_W kernel there), or has few channels on
+// large maps at r = 2 (128 channels at 160 x 120: 171 against 207 us).  Elsewhere the pooling pass plus
+// the two contractions side by side are faster, because the g_W contraction of the fused pair cannot
+// start before the fused kernel has ended (128 channels at 160 x 120, r = 4: 156 against 147 us;
+// 64 channels at 56 x 56: 32 against 28 us at r = 2, 36 against 22 us at r = 4).
 bool fused_path_preferred(const Geo& g) {
     const FusedPlan f = fused_plan(g);
     if (!f.ok || f.tiles < sm_count()) return false;
-    return g.C_in >= 3 * g.C_out || (g.C_in <= 128 && g.C_out <= 128);
+    if (g.C_in >= 3 * g.C_out) return true;
+    return g.C_in <= 128 && g.C_out <= 128 && g.r == 2 && f.tiles >= 4LL * sm_count();
 }
 
 gf_status launch_gw_tiled(const unsigned char* gbar_t, const void* stash, float* gwu, uint32_t* err_word, const Geo& g,
