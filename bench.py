@@ -53,8 +53,8 @@ PAPER_CONTEXT = {
 NCU_TRAFFIC: dict[tuple[str, str], dict] = {
     # ncu --set full --clock-control none, python bench.py --table --no-exact --only <layer>/r2 (profiles/*.md)
     ("cfg3b_dw_576", "dw_fused"): {"bytes": 289.06e6 + 188.65e6, "sha1": "4b5034114d07f51de9ec93105e217e4cac06777c"},
-    ("cfg3c_pw_576_96", "gyx_fused"): {"bytes": 38.89e6 + 192.70e6, "sha1": "02cc7a9f26229de04b757b7c160b7050e2396203"},
-    ("cfg3c_pw_576_96", "gw_tiled"): {"bytes": 74.89e6 + 2.16e6, "sha1": "02cc7a9f26229de04b757b7c160b7050e2396203"},
+    ("cfg3c_pw_576_96", "gyx_fused"): {"bytes": 38.89e6 + 192.70e6, "sha1": "6ed5190bb4d910ada562260c71fe702d5e2f90dc"},
+    ("cfg3c_pw_576_96", "gw_tiled"): {"bytes": 74.89e6 + 2.16e6, "sha1": "6ed5190bb4d910ada562260c71fe702d5e2f90dc"},
     ("cfg3a_pw_96_576", "stash_pool"): {"bytes": 38.55e6 + 0.01e6, "sha1": "56c08adc367812dd2e6ee11acb71cb1a0a803d89"},
     ("cfg3a_pw_96_576", "gx_tc"): {"bytes": 58.06e6 + 5.71e6, "sha1": "a17659264f21416ec34cfc79629bea8d8d9c06de"},
     ("cfg3a_pw_96_576", "gw_tc"): {"bytes": 67.71e6 + 0.76e6, "sha1": "a17659264f21416ec34cfc79629bea8d8d9c06de"},

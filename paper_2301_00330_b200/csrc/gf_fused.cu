@@ -12,7 +12,10 @@
 //                               A[c_o][patch] the tensor core reads;
 //                 one thread    tcgen05.mma  D[patch, c_i] += A^T[patch, c_o] thetaT[c_i, c_o]
 //                               (thetaT tiles by the copy engine), accumulators in tensor memory;
-//                 epilogue      tcgen05.ld -> every value stored to its r x r pixels of g_X.
+//                 expansion     tcgen05.ld -> every value stored to its r x r pixels of g_X.
+//               warps           The pooling warps (0-7) and the expansion warps (8-15) work on
+//                               consecutive tiles at the same time: a tile is read and pooled
+//                               while the one before it is still being written.
 //               g_y is read from HBM once and g_X written once.  The operand tile is also
 //               copied out (bulk shared -> global) as-is: the patch means in exactly the
 //               layout the g_W contraction wants for its own operand, 8 KB blocks of
